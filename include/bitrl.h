@@ -1,0 +1,150 @@
+/*
+ * bitrl.h - C ABI of the BitLinear W1.58A8 hot path of the BitRL frozen backbone, for NVIDIA B200 (sm_100a).
+ *
+ * The layer (paper: Sec. III-A, Eq. 2 and the paragraph after Eq. 3; Sec. V, edge-deployment paragraph):
+ *   weights are ternary {-1,0,+1}, Q(W) = sign(W) * 1[|W| > tau] (Eq. 2), inference is integer arithmetic
+ *   without floating multiply-accumulate, ternary products being additions and subtractions.
+ * The paper leaves tau, the activation format and the scales open; this library takes the W1.58A8 layer of the
+ * BitNet b1.58 architecture the paper's backbone follows:
+ *   gamma = mean|W| (per matrix),  W_q = clip(rint(W / (gamma + 1e-5)), -1, 1)     [= Eq. 2, tau = (gamma+1e-5)/2]
+ *   a_m   = max(max_k |x[m,k]|, 1e-5),  x_q[m,k] = clip(rint(x[m,k] * (127 / a_m)), -128, 127)
+ *   acc[m,n] = sum_k x_q[m,k] * W_q[n,k]                                   (int32, exact)
+ *   y[m,n]   = (float)acc[m,n] * (gamma * (a_m / 127))                     (fp32, then bf16 RNE if asked)
+ * rint is round-to-nearest, ties-to-even; each fp32 step is one IEEE operation in the order written.
+ *
+ * Conventions
+ *   - Every pointer marked "dev" is device memory on the current CUDA device; "host" is host memory.
+ *   - Matrices are row-major.  W is [N, K] (out x in), x is [M, K], y is [M, N]:  y = x * W^T.
+ *   - K and N must be multiples of 128; device pointers must be 16-byte aligned.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Calls are asynchronous on `stream`.  Argument errors are returned at once; a device-side wait that gave
+ *     up (every wait in the kernels is bounded) is reported by bitrl_poll_status.
+ *   - The caller owns every buffer it passes, including workspaces.  The library owns what *_create returns.
+ *   - No entry point allocates device memory except the *_create functions.  Nothing throws, aborts or traps.
+ */
+#ifndef BITRL_H_
+#define BITRL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define BITRL_API __attribute__((visibility("default")))
+#else
+#define BITRL_API
+#endif
+
+typedef int32_t bitrl_status;
+#define BITRL_OK 0
+#define BITRL_ERR_NULL (-1)      /* a required pointer is NULL */
+#define BITRL_ERR_SHAPE (-2)     /* M < 1, K or N not a multiple of 128, shape does not match the handle */
+#define BITRL_ERR_ALIGN (-3)     /* a device pointer is not 16-byte aligned */
+#define BITRL_ERR_ARCH (-4)      /* current device is not compute capability 10.0 */
+#define BITRL_ERR_CUDA (-5)      /* a CUDA call failed; code in bitrl_last_cuda_error() */
+#define BITRL_ERR_TIMEOUT (-6)   /* a bounded device-side wait expired (see bitrl_poll_status) */
+#define BITRL_ERR_WORKSPACE (-7) /* workspace missing or smaller than the *_workspace_bytes query */
+#define BITRL_ERR_DTYPE (-8)     /* unknown out_dtype */
+
+#define BITRL_OUT_F32 0
+#define BITRL_OUT_BF16 1
+
+/* Largest M served by the streaming (GEMV) kernel; larger M runs the tcgen05 GEMM kernel. */
+#define BITRL_GEMV_MAX_M 16
+
+typedef struct bitrl_linear bitrl_linear_t;   /* packed ternary weights in kernel layout + gamma + N, K */
+typedef struct bitrl_encoder bitrl_encoder_t; /* a stack of blocks of four bitrl_linear_t each */
+
+/* ---- a0: ternarize + pack (offline, once per matrix; the backbone is frozen - Sec. III-A) ---------------
+ * Eq. 2 with tau = (gamma+1e-5)/2.  W: dev fp32 [N,K].  packed: dev [N, K/4] bytes, canonical format:
+ * code c = W_q + 1 in {0,1,2}; byte j of row n holds k = 4j..4j+3, code of k in bits [2(k%4)+1 : 2(k%4)].
+ * gamma: dev fp32 [1].  |W| is summed in fp64 (fixed tree order, deterministic) and rounded once to fp32.
+ * workspace: dev, at least bitrl_pack_workspace_bytes(N, K) bytes. */
+BITRL_API size_t bitrl_pack_workspace_bytes(int32_t N, int32_t K);
+BITRL_API bitrl_status bitrl_pack_ternary(const float* W, int32_t N, int32_t K, uint8_t* packed, float* gamma,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
+/* Builds the weight handle from the canonical packed bytes and gamma (both dev).  The library keeps its own
+ * re-tiled copy (N*K/4 bytes); the inputs may be freed once `stream` has run past this call. */
+BITRL_API bitrl_status bitrl_linear_create(const uint8_t* packed, const float* gamma, int32_t N, int32_t K,
+                                 bitrl_linear_t** out, void* stream);
+BITRL_API bitrl_status bitrl_linear_destroy(bitrl_linear_t* w);
+
+/* ---- a1: per-token absmax int8 activation quantization (Q = 127) ---------------------------------------
+ * x: dev bf16 [M,K].  xq: dev int8 [M,K].  absmax: dev fp32 [M] (the clamped a_m).
+ * rowsum: dev int32 [M] = sum_k x_q[m,k], or NULL.  (The GEMM feeds weight codes W_q+1 as unsigned bytes
+ * and repays sum_k x_q once per output; the row sum is that correction.) */
+BITRL_API bitrl_status bitrl_quant_act(const void* x, int32_t M, int32_t K, int8_t* xq, float* absmax, int32_t* rowsum,
+                             void* stream);
+
+/* ---- a1..a3: the whole layer  y = BitLinear(x) --------------------------------------------------------
+ * x: dev bf16 [M,K]; y: dev [M,N] fp32 (BITRL_OUT_F32) or bf16 (BITRL_OUT_BF16).  K, N must equal the
+ * handle's.  M <= BITRL_GEMV_MAX_M: one streaming kernel (quantization in its prologue, rescale in its
+ * epilogue; no workspace needed).  Larger M: quantization kernel into the workspace, then the tcgen05 GEMM.
+ * workspace: dev, >= bitrl_workspace_bytes(M,K,N) (0 for M <= 16, then NULL is accepted). */
+BITRL_API size_t bitrl_workspace_bytes(int32_t M, int32_t K, int32_t N);
+BITRL_API bitrl_status bitrl_bitlinear_forward(const bitrl_linear_t* w, const void* x, int32_t M, int32_t K, int32_t N,
+                                     void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes,
+                                     void* stream);
+
+/* Same, and additionally writes the integer stages: xq_out dev int8 [M,K], absmax_out dev fp32 [M],
+ * acc_out dev int32 [M,N] (any may be NULL).  Needs the workspace for every M. */
+BITRL_API bitrl_status bitrl_bitlinear_forward_debug(const bitrl_linear_t* w, const void* x, int32_t M, int32_t K,
+                                           int32_t N, void* y, int32_t out_dtype, void* workspace,
+                                           size_t workspace_bytes, int8_t* xq_out, float* absmax_out,
+                                           int32_t* acc_out, void* stream);
+
+/* a2 + a3 on an already quantized input (what a fused producer hands over).
+ * xq dev int8 [M,K], absmax dev fp32 [M], rowsum dev int32 [M] (all required).
+ * residual: NULL, or dev bf16 [M,N]; then y = bf16( fp32(residual) + fp32(bf16(acc*scale)) ), out_dtype must be
+ * BITRL_OUT_BF16, and y may alias residual.  acc_out: NULL or dev int32 [M,N]. */
+BITRL_API bitrl_status bitrl_bitlinear_forward_q(const bitrl_linear_t* w, const int8_t* xq, const float* absmax,
+                                       const int32_t* rowsum, int32_t M, void* y, int32_t out_dtype,
+                                       const void* residual, int32_t* acc_out, void* stream);
+
+/* ---- a4: fused producers of the encoder block (the architecture is cited, not spelled out, by the paper:
+ * Sec. III-B takes the backbone architecture from the BitNet papers by reference; gain 1, eps 1e-5) -------
+ * Each computes u = bf16( v / sqrt(mean_k v^2 + 1e-5) ) in fp32 for its row vector v and then quantizes u
+ * exactly like bitrl_quant_act.  u_out: NULL or dev bf16 [T, K_out] (the value that was quantized).
+ *   rmsnorm_quant:            v = h[t, :]                                   h: dev bf16 [T,K]
+ *   vrepeat_rmsnorm_quant:    v = V of qkv[t], each kv head repeated n_heads/n_kv_heads times ("identity
+ *                             attention": one key per query, so softmax = 1)  qkv: dev bf16 [T,(n_heads+2 n_kv)*hd]
+ *   relu2gate_rmsnorm_quant:  v = max(g,0)^2 * up, gu = [g | up]              gu: dev bf16 [T, 2F] */
+BITRL_API bitrl_status bitrl_rmsnorm_quant(const void* h, int32_t T, int32_t K, int8_t* xq, float* absmax,
+                                 int32_t* rowsum, void* u_out, void* stream);
+BITRL_API bitrl_status bitrl_vrepeat_rmsnorm_quant(const void* qkv, int32_t T, int32_t n_heads, int32_t n_kv_heads,
+                                         int32_t head_dim, int8_t* xq, float* absmax, int32_t* rowsum,
+                                         void* u_out, void* stream);
+BITRL_API bitrl_status bitrl_relu2gate_rmsnorm_quant(const void* gu, int32_t T, int32_t F, int8_t* xq, float* absmax,
+                                           int32_t* rowsum, void* u_out, void* stream);
+
+/* ---- frozen encoder f_theta* (Eq. 3): L blocks of {qkv, out, gate/up, down} ----------------------------
+ * layers: host array of 4*L handles ordered qkv, out, gateup, down per block; the handles must outlive the
+ * encoder.  d = n_heads*head_dim; qkv has N = d + 2*n_kv_heads*head_dim, gateup N = 2*d_ff, down K = d_ff.
+ * Block:  h += out(RMSNorm(repeat(V(qkv(RMSNorm(h))))));  h += down(RMSNorm(relu(g)^2 * up)), [g|up] = gateup(RMSNorm(h)).
+ * h_in, h_out: dev bf16 [T,d] (may alias).  workspace >= bitrl_encoder_workspace_bytes(enc, T). */
+BITRL_API bitrl_status bitrl_encoder_create(const bitrl_linear_t* const* layers, int32_t L, int32_t d, int32_t d_ff,
+                                  int32_t n_heads, int32_t n_kv_heads, bitrl_encoder_t** enc);
+BITRL_API bitrl_status bitrl_encoder_destroy(bitrl_encoder_t* enc);
+BITRL_API size_t bitrl_encoder_workspace_bytes(const bitrl_encoder_t* enc, int32_t T);
+BITRL_API bitrl_status bitrl_encoder_forward(const bitrl_encoder_t* enc, const void* h_in, int32_t T, void* h_out,
+                                   void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---- status ----------------------------------------------------------------------------------------- */
+/* Synchronizes `stream`, then reads and clears the device status word.  BITRL_OK, BITRL_ERR_TIMEOUT (a kernel
+ * wait expired; results of that launch are invalid) or BITRL_ERR_CUDA. */
+BITRL_API bitrl_status bitrl_poll_status(void* stream);
+/* After BITRL_ERR_TIMEOUT: which wait gave up (kernel-specific stage id), else 0. */
+BITRL_API int32_t bitrl_last_timeout_stage(void);
+BITRL_API int32_t bitrl_last_cuda_error(void);
+BITRL_API const char* bitrl_status_string(bitrl_status s);
+/* Number of kernels this library has launched since load (all streams). */
+BITRL_API uint64_t bitrl_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BITRL_H_ */

@@ -201,8 +201,8 @@ void oracle_bitlinear(const uint16_t* x, const int8_t* Wq, float gamma, int64_t 
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Encoder glue (not in the paper beyond "the architecture from Wang et al."; the readings are: gain 1,
-// eps 1e-5, statistics in fp64, result rounded once to fp32 and then to bf16).
+// Encoder glue (the paper only points to the BitNet papers for the block architecture, Sec. III-B; the
+// readings are: gain 1, eps 1e-5, statistics in fp64, result rounded once to fp32 and then to bf16).
 
 // u = x / sqrt(mean_k(x^2) + 1e-5), x given as fp32 [T,K]; output bf16.
 void oracle_rmsnorm_f32(const float* x, int64_t T, int64_t K, uint16_t* u) {

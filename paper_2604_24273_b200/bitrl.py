@@ -1,0 +1,295 @@
+"""Thin ctypes binding of ``libbitrl.so`` (declared in ``include/bitrl.h``).
+
+Argument marshalling only: every step of the layer runs in the library's CUDA kernels.  PyTorch is used for
+device memory and streams.  There is no CPU fallback: if the library is missing or a call fails, an
+exception is raised.
+
+The functions mirror the C names without the ``bitrl_`` prefix:
+``pack_ternary``, ``Linear`` (create/destroy), ``quant_act``, ``bitlinear_forward``, ``bitlinear_forward_debug``,
+``bitlinear_forward_q``, ``rmsnorm_quant``, ``vrepeat_rmsnorm_quant``, ``relu2gate_rmsnorm_quant``, ``Encoder``,
+``poll_status``.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_HERE = Path(__file__).resolve().parent
+LIB_PATH = _HERE / "libbitrl.so"
+
+OK = 0
+ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT, ERR_WORKSPACE, ERR_DTYPE = range(-1, -9, -1)
+OUT_F32, OUT_BF16 = 0, 1
+GEMV_MAX_M = 16
+
+_vp = ctypes.c_void_p
+_i32 = ctypes.c_int32
+_sz = ctypes.c_size_t
+
+EXPORTS = {
+    "bitrl_pack_workspace_bytes": (_sz, [_i32, _i32]),
+    "bitrl_pack_ternary": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp, _sz, _vp]),
+    "bitrl_linear_create": (_i32, [_vp, _vp, _i32, _i32, ctypes.POINTER(_vp), _vp]),
+    "bitrl_linear_destroy": (_i32, [_vp]),
+    "bitrl_quant_act": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp, _vp]),
+    "bitrl_workspace_bytes": (_sz, [_i32, _i32, _i32]),
+    "bitrl_bitlinear_forward": (_i32, [_vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp]),
+    "bitrl_bitlinear_forward_debug": (_i32, [_vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp, _vp, _vp, _vp]),
+    "bitrl_bitlinear_forward_q": (_i32, [_vp, _vp, _vp, _vp, _i32, _vp, _i32, _vp, _vp, _vp]),
+    "bitrl_rmsnorm_quant": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp]),
+    "bitrl_vrepeat_rmsnorm_quant": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]),
+    "bitrl_relu2gate_rmsnorm_quant": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp]),
+    "bitrl_encoder_create": (_i32, [ctypes.POINTER(_vp), _i32, _i32, _i32, _i32, _i32, ctypes.POINTER(_vp)]),
+    "bitrl_encoder_destroy": (_i32, [_vp]),
+    "bitrl_encoder_workspace_bytes": (_sz, [_vp, _i32]),
+    "bitrl_encoder_forward": (_i32, [_vp, _vp, _i32, _vp, _vp, _sz, _vp]),
+    "bitrl_poll_status": (_i32, [_vp]),
+    "bitrl_last_timeout_stage": (_i32, []),
+    "bitrl_last_cuda_error": (_i32, []),
+    "bitrl_status_string": (ctypes.c_char_p, [_i32]),
+    "bitrl_launch_count": (ctypes.c_uint64, []),
+}
+
+
+class BitrlError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().bitrl_status_string(status).decode()
+        extra = f" (cuda error {lib().bitrl_last_cuda_error()})" if status == ERR_CUDA else ""
+        super().__init__(f"{where}: {msg}{extra} [{status}]")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the library; fails loudly when it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2604_24273_b200.build` "
+                              "(or __graft_entry__.build()); there is no CPU fallback")
+        L = ctypes.CDLL(str(LIB_PATH))
+        for name, (res, args) in EXPORTS.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise BitrlError(status, where)
+
+
+def _ptr(t):
+    return None if t is None else _vp(t.data_ptr())
+
+
+def _stream():
+    return _vp(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of dtype {dtype}")
+    return t
+
+
+def launch_count() -> int:
+    return int(lib().bitrl_launch_count())
+
+
+def poll_status() -> None:
+    """Synchronizes the current stream and raises if a device-side wait expired."""
+    _check(lib().bitrl_poll_status(_stream()), "bitrl_poll_status")
+
+
+def pack_ternary(W: torch.Tensor):
+    """W: CUDA fp32 [N,K].  Returns (packed uint8 [N,K/4] canonical, gamma fp32 [1])."""
+    _dev(W, torch.float32, "W")
+    N, K = W.shape
+    packed = torch.empty((N, K // 4), dtype=torch.uint8, device=W.device)
+    gamma = torch.empty((1,), dtype=torch.float32, device=W.device)
+    nbytes = lib().bitrl_pack_workspace_bytes(N, K)
+    ws = torch.empty((nbytes,), dtype=torch.uint8, device=W.device)
+    _check(lib().bitrl_pack_ternary(_ptr(W), N, K, _ptr(packed), _ptr(gamma), _ptr(ws), nbytes, _stream()),
+           "bitrl_pack_ternary")
+    return packed, gamma
+
+
+class Linear:
+    """Owns a ``bitrl_linear_t`` (kernel-layout ternary weights + gamma)."""
+
+    def __init__(self, packed: torch.Tensor, gamma: torch.Tensor, N: int, K: int):
+        _dev(packed, torch.uint8, "packed")
+        _dev(gamma, torch.float32, "gamma")
+        self.N, self.K = int(N), int(K)
+        self.device = packed.device
+        h = _vp()
+        _check(lib().bitrl_linear_create(_ptr(packed), _ptr(gamma), self.N, self.K, ctypes.byref(h), _stream()),
+               "bitrl_linear_create")
+        self.handle = h
+
+    @classmethod
+    def from_master(cls, W: torch.Tensor) -> "Linear":
+        packed, gamma = pack_ternary(W)
+        return cls(packed, gamma, W.shape[0], W.shape[1])
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().bitrl_linear_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def quant_act(x: torch.Tensor, want_rowsum: bool = True):
+    """x: CUDA bf16 [M,K] -> (x_q int8 [M,K], absmax fp32 [M], rowsum int32 [M] or None)."""
+    _dev(x, torch.bfloat16, "x")
+    M, K = x.shape
+    xq = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    a = torch.empty((M,), dtype=torch.float32, device=x.device)
+    rs = torch.empty((M,), dtype=torch.int32, device=x.device) if want_rowsum else None
+    _check(lib().bitrl_quant_act(_ptr(x), M, K, _ptr(xq), _ptr(a), _ptr(rs), _stream()), "bitrl_quant_act")
+    return xq, a, rs
+
+
+def workspace_bytes(M: int, K: int, N: int) -> int:
+    return int(lib().bitrl_workspace_bytes(M, K, N))
+
+
+def _out(M, N, out_dtype, device):
+    return torch.empty((M, N), dtype=torch.float32 if out_dtype == OUT_F32 else torch.bfloat16, device=device)
+
+
+def bitlinear_forward(w: Linear, x: torch.Tensor, out_dtype: int = OUT_BF16, y: torch.Tensor | None = None,
+                      workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """y = BitLinear(x): x CUDA bf16 [M,K] -> y [M,N]."""
+    _dev(x, torch.bfloat16, "x")
+    M, K = x.shape
+    if y is None:
+        y = _out(M, w.N, out_dtype, x.device)
+    need = workspace_bytes(M, K, w.N)
+    if workspace is None and need:
+        workspace = torch.empty((need,), dtype=torch.uint8, device=x.device)
+    nbytes = 0 if workspace is None else workspace.numel()
+    _check(lib().bitrl_bitlinear_forward(w.handle, _ptr(x), M, K, w.N, _ptr(y), out_dtype, _ptr(workspace), nbytes,
+                                         _stream()), "bitrl_bitlinear_forward")
+    return y
+
+
+def bitlinear_forward_debug(w: Linear, x: torch.Tensor, out_dtype: int = OUT_BF16):
+    """Returns (y, x_q int8 [M,K], absmax fp32 [M], acc int32 [M,N])."""
+    _dev(x, torch.bfloat16, "x")
+    M, K = x.shape
+    y = _out(M, w.N, out_dtype, x.device)
+    xq = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    a = torch.empty((M,), dtype=torch.float32, device=x.device)
+    acc = torch.empty((M, w.N), dtype=torch.int32, device=x.device)
+    need = workspace_bytes(M, K, w.N)
+    ws = torch.empty((max(need, 16),), dtype=torch.uint8, device=x.device)
+    _check(lib().bitrl_bitlinear_forward_debug(w.handle, _ptr(x), M, K, w.N, _ptr(y), out_dtype, _ptr(ws), ws.numel(),
+                                               _ptr(xq), _ptr(a), _ptr(acc), _stream()),
+           "bitrl_bitlinear_forward_debug")
+    return y, xq, a, acc
+
+
+def bitlinear_forward_q(w: Linear, xq: torch.Tensor, absmax: torch.Tensor, rowsum: torch.Tensor,
+                        out_dtype: int = OUT_BF16, residual: torch.Tensor | None = None, y: torch.Tensor | None = None,
+                        want_acc: bool = False):
+    _dev(xq, torch.int8, "xq")
+    _dev(absmax, torch.float32, "absmax")
+    _dev(rowsum, torch.int32, "rowsum")
+    M = xq.shape[0]
+    if y is None:
+        y = _out(M, w.N, out_dtype, xq.device)
+    acc = torch.empty((M, w.N), dtype=torch.int32, device=xq.device) if want_acc else None
+    if residual is not None:
+        _dev(residual, torch.bfloat16, "residual")
+    _check(lib().bitrl_bitlinear_forward_q(w.handle, _ptr(xq), _ptr(absmax), _ptr(rowsum), M, _ptr(y), out_dtype,
+                                           _ptr(residual), _ptr(acc), _stream()), "bitrl_bitlinear_forward_q")
+    return (y, acc) if want_acc else y
+
+
+def _producer_out(T, K, device, want_u):
+    xq = torch.empty((T, K), dtype=torch.int8, device=device)
+    a = torch.empty((T,), dtype=torch.float32, device=device)
+    rs = torch.empty((T,), dtype=torch.int32, device=device)
+    u = torch.empty((T, K), dtype=torch.bfloat16, device=device) if want_u else None
+    return xq, a, rs, u
+
+
+def rmsnorm_quant(h: torch.Tensor, want_u: bool = False):
+    _dev(h, torch.bfloat16, "h")
+    T, K = h.shape
+    xq, a, rs, u = _producer_out(T, K, h.device, want_u)
+    _check(lib().bitrl_rmsnorm_quant(_ptr(h), T, K, _ptr(xq), _ptr(a), _ptr(rs), _ptr(u), _stream()),
+           "bitrl_rmsnorm_quant")
+    return xq, a, rs, u
+
+
+def vrepeat_rmsnorm_quant(qkv: torch.Tensor, n_heads: int, n_kv_heads: int, head_dim: int, want_u: bool = False):
+    _dev(qkv, torch.bfloat16, "qkv")
+    T = qkv.shape[0]
+    assert qkv.shape[1] == (n_heads + 2 * n_kv_heads) * head_dim
+    xq, a, rs, u = _producer_out(T, n_heads * head_dim, qkv.device, want_u)
+    _check(lib().bitrl_vrepeat_rmsnorm_quant(_ptr(qkv), T, n_heads, n_kv_heads, head_dim, _ptr(xq), _ptr(a), _ptr(rs),
+                                             _ptr(u), _stream()), "bitrl_vrepeat_rmsnorm_quant")
+    return xq, a, rs, u
+
+
+def relu2gate_rmsnorm_quant(gu: torch.Tensor, want_u: bool = False):
+    _dev(gu, torch.bfloat16, "gu")
+    T, F2 = gu.shape
+    xq, a, rs, u = _producer_out(T, F2 // 2, gu.device, want_u)
+    _check(lib().bitrl_relu2gate_rmsnorm_quant(_ptr(gu), T, F2 // 2, _ptr(xq), _ptr(a), _ptr(rs), _ptr(u), _stream()),
+           "bitrl_relu2gate_rmsnorm_quant")
+    return xq, a, rs, u
+
+
+class Encoder:
+    """Owns a ``bitrl_encoder_t`` over ``layers`` = list of (qkv, out, gateup, down) ``Linear`` tuples."""
+
+    def __init__(self, layers, d: int, d_ff: int, n_heads: int, n_kv_heads: int):
+        self.layers = [tuple(l) for l in layers]  # keeps the handles alive
+        flat = [w.handle for l in self.layers for w in l]
+        arr = (_vp * len(flat))(*flat)
+        h = _vp()
+        _check(lib().bitrl_encoder_create(arr, len(self.layers), d, d_ff, n_heads, n_kv_heads, ctypes.byref(h)),
+               "bitrl_encoder_create")
+        self.handle = h
+        self.d, self.d_ff, self.n_heads, self.n_kv_heads = d, d_ff, n_heads, n_kv_heads
+
+    def workspace_bytes(self, T: int) -> int:
+        return int(lib().bitrl_encoder_workspace_bytes(self.handle, T))
+
+    def forward(self, h_in: torch.Tensor, h_out: torch.Tensor | None = None,
+                workspace: torch.Tensor | None = None) -> torch.Tensor:
+        _dev(h_in, torch.bfloat16, "h_in")
+        T = h_in.shape[0]
+        if h_out is None:
+            h_out = torch.empty_like(h_in)
+        if workspace is None:
+            workspace = torch.empty((self.workspace_bytes(T),), dtype=torch.uint8, device=h_in.device)
+        _check(lib().bitrl_encoder_forward(self.handle, _ptr(h_in), T, _ptr(h_out), _ptr(workspace), workspace.numel(),
+                                           _stream()), "bitrl_encoder_forward")
+        return h_out
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().bitrl_encoder_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,397 @@
+// C-ABI entry points of the bitrl library (declared and documented in include/bitrl.h).  Host code here only
+// validates arguments, carves workspaces and launches the kernels of pack.cuh / quant.cuh / gemv.cuh / gemm.cuh.
+#include <atomic>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+namespace bitrl {
+static std::atomic<uint64_t> g_launches{0};
+static std::atomic<int> g_last_cuda{0};
+static std::atomic<int> g_last_stage{0};
+
+void count_launch(int n) { g_launches.fetch_add(static_cast<uint64_t>(n), std::memory_order_relaxed); }
+bitrl_status cuda_fail(cudaError_t e) {
+  g_last_cuda.store(static_cast<int>(e));
+  (void)cudaGetLastError();
+  return BITRL_ERR_CUDA;
+}
+
+int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+// The kernels are compiled for sm_100a only; any other device cannot run them.
+static bitrl_status check_arch() {
+  static int ok[64] = {0};
+  int dev = 0;
+  BITRL_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return BITRL_ERR_ARCH;
+  if (ok[dev] == 0) {
+    int major = 0, minor = 0;
+    BITRL_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    BITRL_CUDA(cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev));
+    ok[dev] = (major == 10 && minor == 0) ? 1 : -1;
+  }
+  return ok[dev] == 1 ? BITRL_OK : BITRL_ERR_ARCH;
+}
+}  // namespace bitrl
+
+#include "pack.cuh"
+#include "quant.cuh"
+#include "gemv.cuh"
+#include "gemm.cuh"
+
+using namespace bitrl;
+
+struct bitrl_linear {
+  Linear l;
+};
+
+struct bitrl_encoder {
+  std::vector<const bitrl_linear*> layers;  // 4 per block: qkv, out, gateup, down
+  int L, d, d_ff, n_heads, n_kv_heads, head_dim;
+};
+
+namespace {
+
+inline bool shape_ok(int N, int K) { return N >= 128 && K >= 128 && N % 128 == 0 && K % 128 == 0; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Workspace of the M > 16 path: x_q [M,K] int8, absmax [M] f32, rowsum [M] i32.
+struct FwdWs {
+  int8_t* xq;
+  float* absmax;
+  int32_t* rowsum;
+  size_t bytes;
+};
+inline FwdWs carve_fwd(void* ws, int M, int K) {
+  FwdWs f;
+  size_t off = 0;
+  unsigned char* b = static_cast<unsigned char*>(ws);
+  f.xq = reinterpret_cast<int8_t*>(b + off);
+  off += align_up(static_cast<size_t>(M) * K, 256);
+  f.absmax = reinterpret_cast<float*>(b + off);
+  off += align_up(static_cast<size_t>(M) * 4, 256);
+  f.rowsum = reinterpret_cast<int32_t*>(b + off);
+  off += align_up(static_cast<size_t>(M) * 4, 256);
+  f.bytes = off;
+  return f;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t bitrl_pack_workspace_bytes(int32_t N, int32_t K) {
+  (void)N; (void)K;
+  return ABSSUM_MAX_BLOCKS * sizeof(double);
+}
+
+bitrl_status bitrl_pack_ternary(const float* W, int32_t N, int32_t K, uint8_t* packed, float* gamma,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+  if (!W || !packed || !gamma) return BITRL_ERR_NULL;
+  if (!shape_ok(N, K)) return BITRL_ERR_SHAPE;
+  if (!aligned16(W) || !aligned16(packed) || !aligned16(workspace)) return BITRL_ERR_ALIGN;
+  if (!workspace || workspace_bytes < bitrl_pack_workspace_bytes(N, K)) return BITRL_ERR_WORKSPACE;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  return launch_pack(W, N, K, packed, gamma, workspace, static_cast<cudaStream_t>(stream));
+}
+
+bitrl_status bitrl_linear_create(const uint8_t* packed, const float* gamma, int32_t N, int32_t K,
+                                 bitrl_linear_t** out, void* stream) {
+  if (!packed || !gamma || !out) return BITRL_ERR_NULL;
+  if (!shape_ok(N, K)) return BITRL_ERR_SHAPE;
+  if (!aligned16(packed)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  bitrl_linear* w = new (std::nothrow) bitrl_linear();
+  if (!w) return BITRL_ERR_CUDA;
+  w->l.N = N;
+  w->l.K = K;
+  w->l.tiles = nullptr;
+  w->l.gamma = nullptr;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMalloc(&w->l.tiles, static_cast<size_t>(N) * K / 4);
+  if (e == cudaSuccess) e = cudaMalloc(&w->l.gamma, 256);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(w->l.gamma, gamma, sizeof(float), cudaMemcpyDeviceToDevice, st);
+  if (e != cudaSuccess) {
+    cudaFree(w->l.tiles);
+    cudaFree(w->l.gamma);
+    delete w;
+    return cuda_fail(e);
+  }
+  s = launch_retile(packed, N, K, w->l.tiles, st);
+  if (s != BITRL_OK) {
+    cudaFree(w->l.tiles);
+    cudaFree(w->l.gamma);
+    delete w;
+    return s;
+  }
+  *out = w;
+  return BITRL_OK;
+}
+
+bitrl_status bitrl_linear_destroy(bitrl_linear_t* w) {
+  if (!w) return BITRL_OK;
+  cudaFree(w->l.tiles);
+  cudaFree(w->l.gamma);
+  delete w;
+  return BITRL_OK;
+}
+
+bitrl_status bitrl_quant_act(const void* x, int32_t M, int32_t K, int8_t* xq, float* absmax, int32_t* rowsum,
+                             void* stream) {
+  if (!x || !xq || !absmax) return BITRL_ERR_NULL;
+  if (M < 1 || K < 128 || K % 128 != 0) return BITRL_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(xq)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  return launch_quant_act(x, M, K, xq, absmax, rowsum, static_cast<cudaStream_t>(stream));
+}
+
+size_t bitrl_workspace_bytes(int32_t M, int32_t K, int32_t N) {
+  (void)N;
+  if (M < 1 || K < 1) return 0;
+  if (gemv_fits(M, K)) return 0;
+  return carve_fwd(nullptr, M, K).bytes;
+}
+
+static bitrl_status forward_impl(const bitrl_linear_t* w, const void* x, int32_t M, int32_t K, int32_t N, void* y,
+                                 int32_t out_dtype, void* workspace, size_t workspace_bytes, int8_t* xq_out,
+                                 float* absmax_out, int32_t* acc_out, bool debug, void* stream) {
+  if (!w || !x || !y) return BITRL_ERR_NULL;
+  if (M < 1 || K != w->l.K || N != w->l.N) return BITRL_ERR_SHAPE;
+  if (out_dtype != BITRL_OUT_F32 && out_dtype != BITRL_OUT_BF16) return BITRL_ERR_DTYPE;
+  if (!aligned16(x) || !aligned16(y)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (gemv_fits(M, K))
+    return launch_gemv(&w->l, x, nullptr, nullptr, M, y, out_dtype, nullptr, xq_out, absmax_out, acc_out, st);
+  const size_t need = carve_fwd(nullptr, M, K).bytes;
+  if (!workspace || workspace_bytes < need) return BITRL_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return BITRL_ERR_ALIGN;
+  FwdWs f = carve_fwd(workspace, M, K);
+  s = launch_quant_act(x, M, K, f.xq, f.absmax, f.rowsum, st);
+  if (s != BITRL_OK) return s;
+  s = launch_gemm(&w->l, f.xq, f.absmax, f.rowsum, M, y, out_dtype, nullptr, acc_out, st);
+  if (s != BITRL_OK) return s;
+  if (debug) {
+    if (xq_out) BITRL_CUDA(cudaMemcpyAsync(xq_out, f.xq, static_cast<size_t>(M) * K, cudaMemcpyDeviceToDevice, st));
+    if (absmax_out)
+      BITRL_CUDA(cudaMemcpyAsync(absmax_out, f.absmax, static_cast<size_t>(M) * 4, cudaMemcpyDeviceToDevice, st));
+  }
+  return BITRL_OK;
+}
+
+bitrl_status bitrl_bitlinear_forward(const bitrl_linear_t* w, const void* x, int32_t M, int32_t K, int32_t N,
+                                     void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes,
+                                     void* stream) {
+  return forward_impl(w, x, M, K, N, y, out_dtype, workspace, workspace_bytes, nullptr, nullptr, nullptr, false,
+                      stream);
+}
+
+bitrl_status bitrl_bitlinear_forward_debug(const bitrl_linear_t* w, const void* x, int32_t M, int32_t K,
+                                           int32_t N, void* y, int32_t out_dtype, void* workspace,
+                                           size_t workspace_bytes, int8_t* xq_out, float* absmax_out,
+                                           int32_t* acc_out, void* stream) {
+  return forward_impl(w, x, M, K, N, y, out_dtype, workspace, workspace_bytes, xq_out, absmax_out, acc_out, true,
+                      stream);
+}
+
+bitrl_status bitrl_bitlinear_forward_q(const bitrl_linear_t* w, const int8_t* xq, const float* absmax,
+                                       const int32_t* rowsum, int32_t M, void* y, int32_t out_dtype,
+                                       const void* residual, int32_t* acc_out, void* stream) {
+  if (!w || !xq || !absmax || !rowsum || !y) return BITRL_ERR_NULL;
+  if (M < 1) return BITRL_ERR_SHAPE;
+  if (out_dtype != BITRL_OUT_F32 && out_dtype != BITRL_OUT_BF16) return BITRL_ERR_DTYPE;
+  if (residual && out_dtype != BITRL_OUT_BF16) return BITRL_ERR_DTYPE;
+  if (!aligned16(xq) || !aligned16(y) || !aligned16(residual)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (gemv_fits(M, w->l.K))
+    return launch_gemv(&w->l, nullptr, xq, absmax, M, y, out_dtype, residual, nullptr, nullptr, acc_out, st);
+  return launch_gemm(&w->l, xq, absmax, rowsum, M, y, out_dtype, residual, acc_out, st);
+}
+
+bitrl_status bitrl_rmsnorm_quant(const void* h, int32_t T, int32_t K, int8_t* xq, float* absmax,
+                                 int32_t* rowsum, void* u_out, void* stream) {
+  if (!h || !xq || !absmax) return BITRL_ERR_NULL;
+  if (T < 1 || K < 128 || K % 128 != 0 || K > 49152) return BITRL_ERR_SHAPE;
+  if (!aligned16(h) || !aligned16(xq) || !aligned16(u_out)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  return launch_rmsnorm_quant(h, T, K, xq, absmax, rowsum, u_out, static_cast<cudaStream_t>(stream));
+}
+
+bitrl_status bitrl_vrepeat_rmsnorm_quant(const void* qkv, int32_t T, int32_t n_heads, int32_t n_kv_heads,
+                                         int32_t head_dim, int8_t* xq, float* absmax, int32_t* rowsum,
+                                         void* u_out, void* stream) {
+  if (!qkv || !xq || !absmax) return BITRL_ERR_NULL;
+  if (T < 1 || n_heads < 1 || n_kv_heads < 1 || n_heads % n_kv_heads != 0 || head_dim < 8 || head_dim % 8 != 0 ||
+      (n_kv_heads * head_dim) % 128 != 0 || (n_heads * head_dim) % 128 != 0)
+    return BITRL_ERR_SHAPE;
+  if (!aligned16(qkv) || !aligned16(xq) || !aligned16(u_out)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  return launch_vrepeat_rmsnorm_quant(qkv, T, n_heads, n_kv_heads, head_dim, xq, absmax, rowsum, u_out,
+                                      static_cast<cudaStream_t>(stream));
+}
+
+bitrl_status bitrl_relu2gate_rmsnorm_quant(const void* gu, int32_t T, int32_t F, int8_t* xq, float* absmax,
+                                           int32_t* rowsum, void* u_out, void* stream) {
+  if (!gu || !xq || !absmax) return BITRL_ERR_NULL;
+  if (T < 1 || F < 128 || F % 128 != 0 || F > 49152) return BITRL_ERR_SHAPE;
+  if (!aligned16(gu) || !aligned16(xq) || !aligned16(u_out)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  return launch_relu2gate_rmsnorm_quant(gu, T, F, xq, absmax, rowsum, u_out, static_cast<cudaStream_t>(stream));
+}
+
+// ---- encoder ------------------------------------------------------------------------------------------
+
+bitrl_status bitrl_encoder_create(const bitrl_linear_t* const* layers, int32_t L, int32_t d, int32_t d_ff,
+                                  int32_t n_heads, int32_t n_kv_heads, bitrl_encoder_t** enc) {
+  if (!layers || !enc) return BITRL_ERR_NULL;
+  if (L < 1 || n_heads < 1 || n_kv_heads < 1 || n_heads % n_kv_heads != 0 || d % n_heads != 0) return BITRL_ERR_SHAPE;
+  const int hd = d / n_heads;
+  const int n_qkv = d + 2 * n_kv_heads * hd;
+  if (!shape_ok(d, d_ff) || n_qkv % 128 != 0 || (n_kv_heads * hd) % 128 != 0 || hd % 8 != 0) return BITRL_ERR_SHAPE;
+  for (int l = 0; l < L; ++l) {
+    const bitrl_linear_t* const* q = layers + 4 * l;
+    for (int j = 0; j < 4; ++j)
+      if (!q[j]) return BITRL_ERR_NULL;
+    if (q[0]->l.K != d || q[0]->l.N != n_qkv) return BITRL_ERR_SHAPE;
+    if (q[1]->l.K != d || q[1]->l.N != d) return BITRL_ERR_SHAPE;
+    if (q[2]->l.K != d || q[2]->l.N != 2 * d_ff) return BITRL_ERR_SHAPE;
+    if (q[3]->l.K != d_ff || q[3]->l.N != d) return BITRL_ERR_SHAPE;
+  }
+  bitrl_encoder* e = new (std::nothrow) bitrl_encoder();
+  if (!e) return BITRL_ERR_CUDA;
+  e->layers.assign(layers, layers + 4 * L);
+  e->L = L; e->d = d; e->d_ff = d_ff; e->n_heads = n_heads; e->n_kv_heads = n_kv_heads; e->head_dim = hd;
+  *enc = e;
+  return BITRL_OK;
+}
+
+bitrl_status bitrl_encoder_destroy(bitrl_encoder_t* enc) {
+  delete enc;
+  return BITRL_OK;
+}
+
+namespace {
+struct EncWs {
+  int8_t* xq;       // [T, max(d, d_ff)]
+  float* absmax;    // [T]
+  int32_t* rowsum;  // [T]
+  unsigned short* wide;  // [T, max(n_qkv, 2 d_ff)] bf16: qkv, then gate/up
+  size_t bytes;
+};
+EncWs carve_enc(void* ws, const bitrl_encoder* e, int T) {
+  EncWs w;
+  size_t off = 0;
+  unsigned char* b = static_cast<unsigned char*>(ws);
+  const int kmax = e->d > e->d_ff ? e->d : e->d_ff;
+  const int n_qkv = e->d + 2 * e->n_kv_heads * e->head_dim;
+  const int wmax = n_qkv > 2 * e->d_ff ? n_qkv : 2 * e->d_ff;
+  w.xq = reinterpret_cast<int8_t*>(b + off);
+  off += align_up(static_cast<size_t>(T) * kmax, 256);
+  w.absmax = reinterpret_cast<float*>(b + off);
+  off += align_up(static_cast<size_t>(T) * 4, 256);
+  w.rowsum = reinterpret_cast<int32_t*>(b + off);
+  off += align_up(static_cast<size_t>(T) * 4, 256);
+  w.wide = reinterpret_cast<unsigned short*>(b + off);
+  off += align_up(static_cast<size_t>(T) * wmax * 2, 256);
+  w.bytes = off;
+  return w;
+}
+}  // namespace
+
+size_t bitrl_encoder_workspace_bytes(const bitrl_encoder_t* enc, int32_t T) {
+  if (!enc || T < 1) return 0;
+  return carve_enc(nullptr, enc, T).bytes;
+}
+
+bitrl_status bitrl_encoder_forward(const bitrl_encoder_t* enc, const void* h_in, int32_t T, void* h_out,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+  if (!enc || !h_in || !h_out) return BITRL_ERR_NULL;
+  if (T < 1) return BITRL_ERR_SHAPE;
+  if (!workspace || workspace_bytes < bitrl_encoder_workspace_bytes(enc, T)) return BITRL_ERR_WORKSPACE;
+  if (!aligned16(h_in) || !aligned16(h_out) || !aligned16(workspace)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  EncWs w = carve_enc(workspace, enc, T);
+  const int d = enc->d, F = enc->d_ff;
+  if (h_out != h_in)
+    BITRL_CUDA(cudaMemcpyAsync(h_out, h_in, static_cast<size_t>(T) * d * 2, cudaMemcpyDeviceToDevice, st));
+  auto linear = [&](const bitrl_linear* lin, void* y, const void* residual) -> bitrl_status {
+    if (gemv_fits(T, lin->l.K))
+      return launch_gemv(&lin->l, nullptr, w.xq, w.absmax, T, y, BITRL_OUT_BF16, residual, nullptr, nullptr, nullptr, st);
+    return launch_gemm(&lin->l, w.xq, w.absmax, w.rowsum, T, y, BITRL_OUT_BF16, residual, nullptr, st);
+  };
+  for (int l = 0; l < enc->L; ++l) {
+    const bitrl_linear* const* q = enc->layers.data() + 4 * l;
+    if ((s = launch_rmsnorm_quant(h_out, T, d, w.xq, w.absmax, w.rowsum, nullptr, st)) != BITRL_OK) return s;
+    if ((s = linear(q[0], w.wide, nullptr)) != BITRL_OK) return s;
+    if ((s = launch_vrepeat_rmsnorm_quant(w.wide, T, enc->n_heads, enc->n_kv_heads, enc->head_dim, w.xq, w.absmax,
+                                          w.rowsum, nullptr, st)) != BITRL_OK) return s;
+    if ((s = linear(q[1], h_out, h_out)) != BITRL_OK) return s;
+    if ((s = launch_rmsnorm_quant(h_out, T, d, w.xq, w.absmax, w.rowsum, nullptr, st)) != BITRL_OK) return s;
+    if ((s = linear(q[2], w.wide, nullptr)) != BITRL_OK) return s;
+    if ((s = launch_relu2gate_rmsnorm_quant(w.wide, T, F, w.xq, w.absmax, w.rowsum, nullptr, st)) != BITRL_OK) return s;
+    if ((s = linear(q[3], h_out, h_out)) != BITRL_OK) return s;
+  }
+  return BITRL_OK;
+}
+
+// ---- status -------------------------------------------------------------------------------------------
+
+bitrl_status bitrl_poll_status(void* stream) {
+  cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(e);
+  int h[4] = {0, 0, 0, 0};
+  e = cudaMemcpyFromSymbol(h, g_status, sizeof(h));
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (h[0] != 0) {
+    g_last_stage.store(h[1]);
+    const int z[4] = {0, 0, 0, 0};
+    e = cudaMemcpyToSymbol(g_status, z, sizeof(z));
+    if (e != cudaSuccess) return cuda_fail(e);
+    return h[0];
+  }
+  return BITRL_OK;
+}
+
+int32_t bitrl_last_timeout_stage(void) { return g_last_stage.load(); }
+int32_t bitrl_last_cuda_error(void) { return g_last_cuda.load(); }
+uint64_t bitrl_launch_count(void) { return g_launches.load(); }
+
+const char* bitrl_status_string(bitrl_status s) {
+  switch (s) {
+    case BITRL_OK: return "ok";
+    case BITRL_ERR_NULL: return "null pointer";
+    case BITRL_ERR_SHAPE: return "bad shape";
+    case BITRL_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case BITRL_ERR_ARCH: return "device is not compute capability 10.0";
+    case BITRL_ERR_CUDA: return "CUDA error";
+    case BITRL_ERR_TIMEOUT: return "device-side wait timed out";
+    case BITRL_ERR_WORKSPACE: return "workspace missing or too small";
+    case BITRL_ERR_DTYPE: return "bad output dtype";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,287 @@
+// a2+a3 for batched states (M > 16 tokens): the tensor-core kernel.
+//
+// The product is formed transposed, D[n, m] = sum_k C[n,k] * x_q[m,k], so that the ternary weights are the
+// 128-row A operand and the tokens the (up to) 256-wide B operand of one tcgen05.mma: the 2-bit -> int8
+// expansion, the only non-tensor work in the main loop, is then spent on the narrow side of the tile.
+// C = W_q + 1 in {0,1,2} is fed as UNSIGNED bytes (decode = shift + mask), x_q as signed bytes; the surplus
+// sum_k x_q[m,k] is subtracted in the epilogue.  All integer, exact.
+//
+// One persistent CTA per SM, 10 warps:
+//   warp 0      producer : TMA tile of x_q (128-byte swizzle) + bulk copy of the 4 KB packed weight piece
+//   warp 1      MMA      : one thread issues tcgen05.mma kind::i8 (4 per stage, K = 32 each) into TMEM
+//   warps 2-5   expand   : packed piece -> int8 codes in the swizzled K-major layout the MMA reads
+//   warps 6-9   epilogue : TMEM -> registers -> (acc - rowsum) * gamma*a_m/127 -> y (+ residual)
+// Two 256-column accumulators in TMEM let the epilogue of tile i overlap the main loop of tile i+1.
+// Every mbarrier wait is bounded; on expiry the CTA records a status word and leaves through the normal exit.
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace bitrl {
+
+constexpr int GM_ROWS = 128;  // weight rows per tile  (MMA M)
+constexpr int GM_TOK = 256;   // tokens per tile       (MMA N)
+constexpr int GM_BK = 128;    // k per pipeline stage  (one 128-byte swizzle row of int8)
+constexpr int GM_STAGES = 4;
+constexpr int GM_THREADS = 320;
+
+constexpr uint32_t GM_X_BYTES = GM_TOK * GM_BK;     // 32768
+constexpr uint32_t GM_W_BYTES = GM_ROWS * GM_BK;    // 16384
+constexpr uint32_t GM_P_BYTES = TILE_BYTES;         // 4096
+constexpr uint32_t GM_OFF_X = 0;
+constexpr uint32_t GM_OFF_W = GM_OFF_X + GM_STAGES * GM_X_BYTES;
+constexpr uint32_t GM_OFF_P = GM_OFF_W + GM_STAGES * GM_W_BYTES;
+constexpr uint32_t GM_OFF_TOK = GM_OFF_P + GM_STAGES * GM_P_BYTES;  // scale[2][256] f32, rowsum[2][256] i32
+constexpr uint32_t GM_OFF_BAR = GM_OFF_TOK + 2 * GM_TOK * 8;
+constexpr uint32_t GM_NUM_BARS = 3 * GM_STAGES + 4;
+constexpr uint32_t GM_OFF_MISC = GM_OFF_BAR + GM_NUM_BARS * 8;
+constexpr uint32_t GM_SMEM_BYTES = GM_OFF_MISC + 16 + 1024;  // + slack to align the base to 1024
+
+// stage ids reported with BITRL_ERR_TIMEOUT
+enum { GM_WAIT_EMPTY = 1, GM_WAIT_FULL_EXPAND = 2, GM_WAIT_TMEM_EMPTY = 3, GM_WAIT_FULL_MMA = 4,
+       GM_WAIT_EXPANDED = 5, GM_WAIT_TMEM_FULL = 6 };
+
+struct GemmArgs {
+  const uint8_t* tiles;
+  const float* gamma;
+  const float* absmax;
+  const int32_t* rowsum;
+  int M, N, K;
+  void* y;
+  int out_dtype;
+  const unsigned short* residual;
+  int32_t* acc_out;
+  int tiles_n, tiles_total;
+};
+
+__global__ void __launch_bounds__(GM_THREADS, 1)
+gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
+  extern __shared__ unsigned char gm_smem_raw[];
+  const uint32_t raw_addr = ptx::smem_u32(gm_smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  unsigned char* base_ptr = gm_smem_raw + (base - raw_addr);
+
+  const uint32_t bar_full = base + GM_OFF_BAR;                   // [GM_STAGES]
+  const uint32_t bar_expanded = bar_full + 8 * GM_STAGES;        // [GM_STAGES]
+  const uint32_t bar_empty = bar_expanded + 8 * GM_STAGES;       // [GM_STAGES]
+  const uint32_t bar_tmem_full = bar_empty + 8 * GM_STAGES;      // [2]
+  const uint32_t bar_tmem_empty = bar_tmem_full + 16;            // [2]
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + GM_OFF_MISC);
+  float* tok_scale = reinterpret_cast<float*>(base_ptr + GM_OFF_TOK);               // [2][256]
+  int* tok_rowsum = reinterpret_cast<int*>(base_ptr + GM_OFF_TOK + 2 * GM_TOK * 4); // [2][256]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kblocks = a.K / GM_BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < GM_STAGES; ++s) {
+      ptx::mbar_init(bar_full + 8 * s, 1);
+      ptx::mbar_init(bar_expanded + 8 * s, 4);
+      ptx::mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(bar_tmem_full + 8 * b, 1);
+      ptx::mbar_init(bar_tmem_empty + 8 * b, 4);
+    }
+    ptx::mbar_init_fence();
+    ptx::tma_prefetch_desc(&tmap_x);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(base + GM_OFF_MISC, 512);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x) {
+        const int tn = tile % a.tiles_n, tm = tile / a.tiles_n;
+        const uint8_t* wsrc = a.tiles + static_cast<size_t>(tn) * kblocks * TILE_BYTES;
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const uint32_t s = it % GM_STAGES, ph = (it / GM_STAGES) & 1u;
+          if (!ptx::mbar_wait(bar_empty + 8 * s, ph ^ 1u)) { report_timeout(GM_WAIT_EMPTY); ok = false; break; }
+          const uint32_t full = bar_full + 8 * s;
+          ptx::mbar_arrive_expect_tx(full, GM_X_BYTES + GM_P_BYTES);
+          ptx::tma_load_2d(base + GM_OFF_X + s * GM_X_BYTES, &tmap_x, kb * GM_BK, tm * GM_TOK, full);
+          ptx::bulk_g2s(base + GM_OFF_P + s * GM_P_BYTES, wsrc + static_cast<size_t>(kb) * TILE_BYTES, GM_P_BYTES, full);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = ptx::idesc_i8(GM_ROWS, GM_TOK, /*a_signed=*/false, /*b_signed=*/true);
+      uint32_t it = 0, lt = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x, ++lt) {
+        const uint32_t buf = lt & 1u;
+        if (!ptx::mbar_wait(bar_tmem_empty + 8 * buf, ((lt >> 1) & 1u) ^ 1u)) {
+          report_timeout(GM_WAIT_TMEM_EMPTY); ok = false; break;
+        }
+        ptx::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + buf * GM_TOK;
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const uint32_t s = it % GM_STAGES, ph = (it / GM_STAGES) & 1u;
+          if (!ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(GM_WAIT_FULL_MMA); ok = false; break; }
+          if (!ptx::mbar_wait(bar_expanded + 8 * s, ph)) { report_timeout(GM_WAIT_EXPANDED); ok = false; break; }
+          ptx::tc_fence_after_sync();
+          const uint64_t adesc = ptx::smem_desc_sw128(base + GM_OFF_W + s * GM_W_BYTES);
+          const uint64_t bdesc = ptx::smem_desc_sw128(base + GM_OFF_X + s * GM_X_BYTES);
+#pragma unroll
+          for (int k4 = 0; k4 < GM_BK / 32; ++k4)
+            ptx::mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+          ptx::mma_commit(bar_empty + 8 * s);
+        }
+        if (ok) ptx::mma_commit(bar_tmem_full + 8 * buf);
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------------ expanders (one weight row each)
+    const int r = threadIdx.x - 64;
+    const uint32_t row_off = static_cast<uint32_t>(r >> 3) * 1024u + static_cast<uint32_t>(r & 7) * 128u;
+    const uint32_t sw = static_cast<uint32_t>(r & 7);
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x) {
+      for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        const uint32_t s = it % GM_STAGES, ph = (it / GM_STAGES) & 1u;
+        if (!ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(GM_WAIT_FULL_EXPAND); ok = false; break; }
+        const uint4* p = reinterpret_cast<const uint4*>(base_ptr + GM_OFF_P + s * GM_P_BYTES + r * TILE_ROW_BYTES);
+        const uint4 p0 = p[0], p1 = p[1];
+        const uint32_t wd[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+        unsigned char* wrow = base_ptr + GM_OFF_W + s * GM_W_BYTES + row_off;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          uint4 c;
+          c.x = wd[j] & 0x03030303u;
+          c.y = (wd[j] >> 2) & 0x03030303u;
+          c.z = (wd[j] >> 4) & 0x03030303u;
+          c.w = (wd[j] >> 6) & 0x03030303u;
+          *reinterpret_cast<uint4*>(wrow + ((static_cast<uint32_t>(j) ^ sw) << 4)) = c;
+        }
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar_expanded + 8 * s);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int q = warp & 3;            // TMEM lane quarter this warp may read
+    const int ep = threadIdx.x - 192;  // 0..127
+    const float gamma = *a.gamma;
+    uint32_t lt = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x, ++lt) {
+      const int tn = tile % a.tiles_n, tm = tile / a.tiles_n;
+      const uint32_t buf = lt & 1u;
+      float* sc = tok_scale + buf * GM_TOK;
+      int* rsum = tok_rowsum + buf * GM_TOK;
+      for (int j = ep; j < GM_TOK; j += 128) {
+        const int tok = tm * GM_TOK + j;
+        sc[j] = tok < a.M ? out_scale(gamma, a.absmax[tok]) : 0.0f;
+        rsum[j] = tok < a.M ? a.rowsum[tok] : 0;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (!ptx::mbar_wait(bar_tmem_full + 8 * buf, (lt >> 1) & 1u)) { report_timeout(GM_WAIT_TMEM_FULL); ok = false; break; }
+      ptx::tc_fence_after_sync();
+      const int n = tn * GM_ROWS + q * 32 + lane;
+      const int tok_hi = min(GM_TOK, a.M - tm * GM_TOK);
+      for (int c = 0; c < GM_TOK / 32; ++c) {
+        if (c * 32 >= tok_hi) break;  // warp-uniform
+        uint32_t v[32];
+        ptx::tmem_ld_32x32b_x32(tmem_base + buf * GM_TOK + c * 32 + (static_cast<uint32_t>(q * 32) << 16), v);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const int jj = c * 32 + j;
+          if (jj < tok_hi) {
+            const int acc = static_cast<int>(v[j]) - rsum[jj];
+            const size_t o = static_cast<size_t>(tm * GM_TOK + jj) * a.N + n;
+            if (a.acc_out) a.acc_out[o] = acc;
+            const float yv = __fmul_rn(static_cast<float>(acc), sc[jj]);
+            if (a.out_dtype == BITRL_OUT_F32) {
+              static_cast<float*>(a.y)[o] = yv;
+            } else {
+              unsigned short yb = float_to_bf16_bits(yv);
+              if (a.residual)
+                yb = float_to_bf16_bits(__fadd_rn(bf16_bits_to_float(a.residual[o]), bf16_bits_to_float(yb)));
+              static_cast<unsigned short*>(a.y)[o] = yb;
+            }
+          }
+        }
+      }
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar_tmem_empty + 8 * buf);
+    }
+  }
+
+  // ---- teardown: every role leaves through here, also after a timeout ----
+  __syncwarp();
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// cuTensorMapEncodeTiled, resolved through the runtime so the library does not link against libcuda.
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline encode_tiled_fn get_encode_tiled() {
+  static encode_tiled_fn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<encode_tiled_fn>(p);
+  }
+  return fn;
+}
+
+int sm_count();
+
+bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax, const int32_t* rowsum, int M,
+                         void* y, int out_dtype, const void* residual, int32_t* acc_out, cudaStream_t st) {
+  encode_tiled_fn encode = get_encode_tiled();
+  if (!encode) return cuda_fail(cudaErrorSymbolNotFound);
+  CUtensorMap tmap;
+  const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(w->K), static_cast<cuuint64_t>(M)};
+  const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(w->K)};
+  const cuuint32_t box[2] = {GM_BK, GM_TOK};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(xq), gdim, gstride, box,
+                            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
+
+  GemmArgs a{w->tiles, w->gamma, absmax, rowsum, M, w->N, w->K, y, out_dtype,
+             static_cast<const unsigned short*>(residual), acc_out, w->N / GM_ROWS, 0};
+  const int tiles_m = (M + GM_TOK - 1) / GM_TOK;
+  a.tiles_total = a.tiles_n * tiles_m;
+  static bool attr_set = false;
+  if (!attr_set) {
+    BITRL_CUDA(cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM_BYTES));
+    attr_set = true;
+  }
+  const int grid = a.tiles_total < sm_count() ? a.tiles_total : sm_count();
+  gemm_i8_kernel<<<grid, GM_THREADS, GM_SMEM_BYTES, st>>>(tmap, a);
+  count_launch(1);
+  BITRL_CUDA(cudaGetLastError());
+  return BITRL_OK;
+}
+
+}  // namespace bitrl

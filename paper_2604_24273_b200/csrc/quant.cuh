@@ -1,0 +1,189 @@
+// a1 and a4: per-token absmax int8 quantization, alone and fused behind the encoder's row producers
+// (RMSNorm, V-repeat + RMSNorm, ReLU^2 gate + RMSNorm).  One CTA per token row; the row lives in shared memory
+// as fp32 between the passes, so every activation tensor is read from HBM once and the codes written once.
+#pragma once
+
+#include "common.cuh"
+
+namespace bitrl {
+
+constexpr int ROW_THREADS = 256;
+
+enum RowMode { ROW_PLAIN = 0, ROW_RMS = 1, ROW_VREPEAT = 2, ROW_RELU2 = 3 };
+
+struct RowArgs {
+  const unsigned short* in;  // bf16 bits
+  long long in_stride;       // elements between consecutive rows of `in`
+  int in_offset;             // first element of the row vector inside a row of `in`
+  int gate_offset;           // ROW_RELU2: offset of `up` relative to g (= F)
+  int Kv;                    // length of the row vector v that is normalized / quantized
+  int rep;                   // ROW_VREPEAT: copies of each head; 1 otherwise
+  int head_dim;              // ROW_VREPEAT: head width
+  int Kout;                  // row length of xq / u_out (= Kv * rep)
+  int8_t* xq;
+  float* absmax;
+  int32_t* rowsum;
+  unsigned short* u_out;
+};
+
+__device__ __forceinline__ float block_sum(float v, float* red) {
+  v = warp_sum(v);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float t = 0.0f;
+#pragma unroll
+  for (int i = 0; i < ROW_THREADS / 32; ++i) t += red[i];
+  return t;
+}
+__device__ __forceinline__ float block_max(float v, float* red) {
+  v = warp_max(v);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float t = 0.0f;
+#pragma unroll
+  for (int i = 0; i < ROW_THREADS / 32; ++i) t = fmaxf(t, red[i]);
+  return t;
+}
+__device__ __forceinline__ int block_sum_i(int v, int* red) {
+  v = warp_sum_i(v);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  int t = 0;
+#pragma unroll
+  for (int i = 0; i < ROW_THREADS / 32; ++i) t += red[i];
+  return t;
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(ROW_THREADS) row_quant_kernel(RowArgs a) {
+  extern __shared__ __align__(16) float vrow[];  // Kv floats
+  __shared__ float redf[ROW_THREADS / 32];
+  __shared__ int redi[ROW_THREADS / 32];
+
+  const long long row = blockIdx.x;
+  const unsigned short* src = a.in + row * a.in_stride + a.in_offset;
+  const int nvec = a.Kv >> 2;  // groups of 4 elements (Kv is a multiple of 128)
+
+  // pass 1: load, form v, keep it in shared memory, sum of squares in fp32
+  float ss = 0.0f;
+  for (int i = threadIdx.x; i < nvec; i += ROW_THREADS) {
+    const uint2 raw = *reinterpret_cast<const uint2*>(src + 4 * i);
+    float v0 = __uint_as_float(raw.x << 16), v1 = __uint_as_float(raw.x & 0xffff0000u);
+    float v2 = __uint_as_float(raw.y << 16), v3 = __uint_as_float(raw.y & 0xffff0000u);
+    if (MODE == ROW_RELU2) {
+      const uint2 rawu = *reinterpret_cast<const uint2*>(src + a.gate_offset + 4 * i);
+      const float u0 = __uint_as_float(rawu.x << 16), u1 = __uint_as_float(rawu.x & 0xffff0000u);
+      const float u2 = __uint_as_float(rawu.y << 16), u3 = __uint_as_float(rawu.y & 0xffff0000u);
+      v0 = fmaxf(v0, 0.0f); v1 = fmaxf(v1, 0.0f); v2 = fmaxf(v2, 0.0f); v3 = fmaxf(v3, 0.0f);
+      v0 = __fmul_rn(__fmul_rn(v0, v0), u0);
+      v1 = __fmul_rn(__fmul_rn(v1, v1), u1);
+      v2 = __fmul_rn(__fmul_rn(v2, v2), u2);
+      v3 = __fmul_rn(__fmul_rn(v3, v3), u3);
+    }
+    if (MODE != ROW_PLAIN) ss += v0 * v0 + v1 * v1 + v2 * v2 + v3 * v3;
+    *reinterpret_cast<float4*>(vrow + 4 * i) = make_float4(v0, v1, v2, v3);
+  }
+
+  // pass 2: u = bf16(v * rstd); absmax of u
+  float amax = 0.0f;
+  if (MODE != ROW_PLAIN) {
+    ss = block_sum(ss, redf);
+    const float rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(ss, static_cast<float>(a.Kv)), 1e-5f)));
+    for (int i = threadIdx.x; i < nvec; i += ROW_THREADS) {
+      float4 v = *reinterpret_cast<float4*>(vrow + 4 * i);
+      v.x = bf16_bits_to_float(float_to_bf16_bits(__fmul_rn(v.x, rstd)));
+      v.y = bf16_bits_to_float(float_to_bf16_bits(__fmul_rn(v.y, rstd)));
+      v.z = bf16_bits_to_float(float_to_bf16_bits(__fmul_rn(v.z, rstd)));
+      v.w = bf16_bits_to_float(float_to_bf16_bits(__fmul_rn(v.w, rstd)));
+      amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+      *reinterpret_cast<float4*>(vrow + 4 * i) = v;
+    }
+  } else {
+    for (int i = threadIdx.x; i < nvec; i += ROW_THREADS) {
+      const float4 v = *reinterpret_cast<float4*>(vrow + 4 * i);
+      amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+    }
+  }
+  amax = fmaxf(block_max(amax, redf), 1e-5f);
+  const float inv = __fdiv_rn(127.0f, amax);
+
+  // pass 3: codes (and the optional bf16 copy of u), written `rep` times for the V-repeat producer
+  int rs = 0;
+  int8_t* xq = a.xq + row * a.Kout;
+  unsigned short* uo = a.u_out ? a.u_out + row * a.Kout : nullptr;
+  for (int i = threadIdx.x; i < nvec; i += ROW_THREADS) {
+    const float4 v = *reinterpret_cast<float4*>(vrow + 4 * i);
+    const int q0 = quant_code(v.x, inv), q1 = quant_code(v.y, inv), q2 = quant_code(v.z, inv),
+              q3 = quant_code(v.w, inv);
+    rs += q0 + q1 + q2 + q3;
+    const uint32_t word = (q0 & 0xff) | ((q1 & 0xff) << 8) | ((q2 & 0xff) << 16) | (static_cast<uint32_t>(q3) << 24);
+    uint2 ub;
+    if (uo) {
+      ub.x = static_cast<uint32_t>(float_to_bf16_bits(v.x)) | (static_cast<uint32_t>(float_to_bf16_bits(v.y)) << 16);
+      ub.y = static_cast<uint32_t>(float_to_bf16_bits(v.z)) | (static_cast<uint32_t>(float_to_bf16_bits(v.w)) << 16);
+    }
+    if (MODE == ROW_VREPEAT) {
+      const int k = 4 * i;
+      const int kvh = k / a.head_dim, e = k - kvh * a.head_dim;
+      for (int r = 0; r < a.rep; ++r) {
+        const int ko = (kvh * a.rep + r) * a.head_dim + e;
+        *reinterpret_cast<uint32_t*>(xq + ko) = word;
+        if (uo) *reinterpret_cast<uint2*>(uo + ko) = ub;
+      }
+    } else {
+      *reinterpret_cast<uint32_t*>(xq + 4 * i) = word;
+      if (uo) *reinterpret_cast<uint2*>(uo + 4 * i) = ub;
+    }
+  }
+  rs = block_sum_i(rs, redi);
+  if (threadIdx.x == 0) {
+    a.absmax[row] = amax;
+    if (a.rowsum) a.rowsum[row] = rs * a.rep;
+  }
+}
+
+template <int MODE>
+bitrl_status launch_row(const RowArgs& a, int T, cudaStream_t st) {
+  const size_t smem = static_cast<size_t>(a.Kv) * sizeof(float);
+  if (smem > 40 * 1024) {
+    BITRL_CUDA(cudaFuncSetAttribute(row_quant_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    static_cast<int>(smem)));
+  }
+  row_quant_kernel<MODE><<<T, ROW_THREADS, smem, st>>>(a);
+  count_launch(1);
+  BITRL_CUDA(cudaGetLastError());
+  return BITRL_OK;
+}
+
+bitrl_status launch_quant_act(const void* x, int M, int K, int8_t* xq, float* absmax, int32_t* rowsum,
+                              cudaStream_t st) {
+  RowArgs a{static_cast<const unsigned short*>(x), K, 0, 0, K, 1, K, K, xq, absmax, rowsum, nullptr};
+  return launch_row<ROW_PLAIN>(a, M, st);
+}
+
+bitrl_status launch_rmsnorm_quant(const void* h, int T, int K, int8_t* xq, float* absmax, int32_t* rowsum,
+                                  void* u_out, cudaStream_t st) {
+  RowArgs a{static_cast<const unsigned short*>(h), K, 0, 0, K, 1, K, K, xq, absmax, rowsum,
+            static_cast<unsigned short*>(u_out)};
+  return launch_row<ROW_RMS>(a, T, st);
+}
+
+bitrl_status launch_vrepeat_rmsnorm_quant(const void* qkv, int T, int n_heads, int n_kv, int hd, int8_t* xq,
+                                          float* absmax, int32_t* rowsum, void* u_out, cudaStream_t st) {
+  const int d = n_heads * hd, dkv = n_kv * hd;
+  RowArgs a{static_cast<const unsigned short*>(qkv), d + 2 * dkv, d + dkv, 0, dkv, n_heads / n_kv, hd, d,
+            xq, absmax, rowsum, static_cast<unsigned short*>(u_out)};
+  return launch_row<ROW_VREPEAT>(a, T, st);
+}
+
+bitrl_status launch_relu2gate_rmsnorm_quant(const void* gu, int T, int F, int8_t* xq, float* absmax,
+                                            int32_t* rowsum, void* u_out, cudaStream_t st) {
+  RowArgs a{static_cast<const unsigned short*>(gu), 2LL * F, 0, F, F, 1, F, F, xq, absmax, rowsum,
+            static_cast<unsigned short*>(u_out)};
+  return launch_row<ROW_RELU2>(a, T, st);
+}
+
+}  // namespace bitrl
