@@ -1,0 +1,409 @@
+#!/usr/bin/env python
+"""Benchmark of the BitLinear W1.58A8 hot path on B200.
+
+Headline (the line's `value`): packed-weight GB/s of the M=1 streaming kernel over a whole ~2B-parameter
+backbone - one step = one decode pass over 30 blocks x {qkv, out, gate/up, down} = 120 launches streaming
+521 MB of packed ternary weights (4x the 126 MB L2, so every launch reads cold weights).
+Secondary figures in the same JSON line (`extra`): M=8 decode, the M=4096 tcgen05 GEMM (int8 TOPS), the
+30-block encoder forward (states/s); plus the CPU oracle timed on the host cores and the roofline fraction of
+the dominant kernel.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--layers L] [--sections ...]
+
+Under torchrun (N > 1) every rank runs the same step on its own replica of the weights and its own states
+(no collective on the data path); rank 0 prints the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2604_24273_b200 import inputs  # noqa: E402
+
+METRIC = "BitLinear GB/s (M=1) and int8 TOPS (M=4096) on 1 B200 as % of roofline"
+BLOCK = [("qkv", 2560, 3840), ("out", 2560, 2560), ("gateup", 2560, 13824), ("down", 6912, 2560)]  # (name, K, N)
+FULL_LAYERS = 30
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+INT8_OVER_BF16 = 2.0  # nominal dense int8 : bf16 tensor throughput on B200 (4.5 : 2.25 PFLOP/s)
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def packed_bytes_per_layer():
+    return sum(k * n // 4 for _, k, n in BLOCK)
+
+
+# ----------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.1)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0]))
+                smax.append(float(r[1]))
+            except ValueError:
+                continue
+            for nme, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(nme)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------- helpers
+def dist_env():
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def barrier_sync(world):
+    torch.cuda.synchronize()
+    if world > 1:
+        torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+
+def max_over_ranks(ms: float, world: int) -> float:
+    if world == 1:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def time_graph(graph, steps, warmup, world):
+    """W warm-up replays, then K timed replays between CUDA events on the launching stream; max over ranks (ms)."""
+    for _ in range(warmup):
+        graph.replay()
+    barrier_sync(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        graph.replay()
+    e1.record()
+    barrier_sync(world)
+    return max_over_ranks(e0.elapsed_time(e1), world)
+
+
+def capture(fn):
+    """Runs fn once eagerly, then captures it into a CUDA graph (the library launches on the current stream).
+    Returns (graph, number of library kernel launches inside the graph)."""
+    from paper_2604_24273_b200 import bitrl
+
+    fn()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    n0 = bitrl.launch_count()
+    with torch.cuda.graph(g):
+        fn()
+    launches = bitrl.launch_count() - n0
+    torch.cuda.synchronize()
+    return g, launches
+
+
+def build_backbone(bitrl, n_layers, seed=5000):
+    """Blocks of ternary weights.  Master weights are drawn on the GPU (N(0, 0.02), seeded per matrix) to keep
+    set-up short, packed by the library and dropped; only the packed handles stay (17.4 MB per block)."""
+    layers = []
+    gen = torch.Generator(device="cuda")
+    for l in range(n_layers):
+        blk = []
+        for j, (_, k, n) in enumerate(BLOCK):
+            gen.manual_seed(seed + 4 * l + j)
+            W = torch.randn(n, k, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W
+            blk.append(bitrl.Linear.from_master(W))
+            del W
+        layers.append(tuple(blk))
+    torch.cuda.synchronize()
+    return layers
+
+
+# ------------------------------------------------------------------------------------------ oracle legs
+def oracle_block0():
+    import oracle
+
+    mats = []
+    for j, (_, k, n) in enumerate(BLOCK):
+        W = inputs.master_weights(n, k, 5000 + j)
+        Wq, g = oracle.ternarize(W.numpy())
+        mats.append((Wq, g, inputs.bf16_bits(inputs.activations(1, k, 2001))))
+
+    def step():
+        for Wq, g, x in mats:
+            oracle.bitlinear(x, Wq, g)
+    return step
+
+
+def oracle_decode_sample(min_seconds=10.0):
+    """The CPU oracle, as it stands, on the M=1 decode workload: block 0's four matrices (69.5 M weights,
+    17.4 MB packed), quant -> contract -> rescale, repeated for about `min_seconds` of CPU work."""
+    step = oracle_block0()
+    nbytes = packed_bytes_per_layer()
+    reps, t0 = 0, time.perf_counter()
+    while True:
+        step()
+        reps += 1
+        dt = time.perf_counter() - t0
+        if dt >= min_seconds:
+            break
+    return {"value": reps * nbytes / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "sample": f"block 0 (qkv, out, gate/up, down; 17.4 MB packed) at M=1, {reps} passes in {dt:.1f} s; the "
+                      "oracle threads over token rows, so M=1 runs on one core"}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the same metric/config, each step a bounded sample."""
+    rank, _, _ = dist_env()
+    if rank != 0:
+        return
+    step = oracle_block0()
+    nbytes = packed_bytes_per_layer()
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    gbs = args.steps * nbytes / dt / 1e9
+    sample = "each step = block 0 of the backbone (4 matrices, 17.4 MB packed) at M=1 on one host core"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8 x ternary(2-bit) -> int32", "data": "synthetic",
+        "config": {"workload": "configs[1]: decode GEMV sweep, M=1, shapes of a ~2B BitNet b1.58 block",
+                   "sample": sample},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ------------------------------------------------------------------------------------------------ ours
+def run_ours(args):
+    from paper_2604_24273_b200 import bitrl
+
+    rank, world, local = dist_env()
+    torch.cuda.set_device(local)
+    if world > 1:
+        torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local))
+    bitrl.lib()
+    peaks, peak_src = load_peaks()
+    dev = torch.device("cuda", local)
+    n_layers = args.layers
+    sections = set(s for s in args.sections.split(",") if s)
+    sub_steps = max(3, args.steps // 4)
+
+    layers = build_backbone(bitrl, n_layers)
+    bytes_step = n_layers * packed_bytes_per_layer()
+
+    # ---------------- headline: decode pass, M = 1, whole backbone, one CUDA graph of 4 * n_layers launches
+    def decode_setup(M):
+        xs = {k: inputs.activations(M, k, 2000 + M).to(dev) for k in (2560, 6912)}
+        ys = [[torch.empty((M, n), dtype=torch.bfloat16, device=dev) for _, _, n in BLOCK] for _ in range(n_layers)]
+
+        def step():
+            for l in range(n_layers):
+                for j, (_, k, n) in enumerate(BLOCK):
+                    bitrl.bitlinear_forward(layers[l][j], xs[k], bitrl.OUT_BF16, y=ys[l][j])
+        return xs, ys, step
+
+    xs1, ys1, step1 = decode_setup(1)
+    g1, launches1 = capture(step1)
+    sampler = ClockSampler(local).start() if rank == 0 else None
+    ms1 = time_graph(g1, args.steps, args.warmup, world)
+    gbs1 = world * bytes_step * args.steps / (ms1 * 1e-3) / 1e9
+    us_per_launch = ms1 * 1e3 / (args.steps * launches1)
+
+    # end to end: pinned host x -> device, the same graph, last block's outputs back to pinned host memory
+    host_x = {k: inputs.activations(1, k, 2001).pin_memory() for k in (2560, 6912)}
+    host_y = [torch.empty((1, n), dtype=torch.bfloat16).pin_memory() for _, _, n in BLOCK]
+    h2d = sum(t.numel() * 2 for t in host_x.values())
+    d2h = sum(t.numel() * 2 for t in host_y)
+
+    def e2e_step():
+        for k in (2560, 6912):
+            xs1[k].copy_(host_x[k], non_blocking=True)
+        g1.replay()
+        for j in range(len(BLOCK)):
+            host_y[j].copy_(ys1[n_layers - 1][j], non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    for _ in range(args.warmup):
+        e2e_step()
+    barrier_sync(world)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        e2e_step()
+    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3, world)
+    e2e_gbs = world * bytes_step * args.steps / (e2e_ms * 1e-3) / 1e9
+    clocks = sampler.stop() if sampler else None
+
+    extra, cpu = {}, None
+    if rank == 0 and "decode8" in sections:
+        _, _, step8 = decode_setup(8)
+        g8, _ = capture(step8)
+        ms8 = time_graph(g8, args.steps, args.warmup, 1)
+        gb8 = bytes_step * args.steps / (ms8 * 1e-3) / 1e9
+        extra["decode_m8"] = {"GBps": gb8, "ms_per_step": ms8 / args.steps, "frac_of_hbm_peak": gb8 / peaks["hbm_gbs"]}
+        del g8
+
+    if rank == 0 and "gemm" in sections:
+        # M = 4096 GEMM, both judged shapes; weights rotate over several matrices, inputs over four buffers
+        i8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
+        M = 4096
+        gen = torch.Generator(device="cuda")
+        up_only = []  # eight 2560 -> 6912 matrices (the block itself only has the fused 2560 -> 13824 one)
+        for i in range(8):
+            gen.manual_seed(1005 + 100 * i)
+            up_only.append(bitrl.Linear.from_master(
+                torch.randn(6912, 2560, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W))
+        for name, K, N in (("gemm_m4096_k2560_n6912", 2560, 6912), ("gemm_m4096_k6912_n2560", 6912, 2560)):
+            mats = up_only if N == 6912 else [layers[l][3] for l in range(n_layers)]
+            xs = [inputs.activations(M, K, 2400 + i).to(dev) for i in range(4)]
+            y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            ws = torch.empty((bitrl.workspace_bytes(M, K, N),), dtype=torch.uint8, device=dev)
+            q = [bitrl.quant_act(x) for x in xs]
+            reps = 12
+
+            def full():
+                for i in range(reps):
+                    bitrl.bitlinear_forward(mats[i % len(mats)], xs[i % 4], bitrl.OUT_BF16, y=y, workspace=ws)
+
+            def kernel_only():
+                for i in range(reps):
+                    bitrl.bitlinear_forward_q(mats[i % len(mats)], *q[i % 4], bitrl.OUT_BF16, y=y)
+
+            ops = 2.0 * M * N * K * reps
+            res = {}
+            for label, fn in (("layer", full), ("gemm_kernel", kernel_only)):
+                g, _ = capture(fn)
+                ms = time_graph(g, sub_steps, args.warmup, 1)
+                tops = ops * sub_steps / (ms * 1e-3) / 1e12
+                res[label] = {"TOPS": tops, "us": ms * 1e3 / (sub_steps * reps), "frac_of_int8_peak": tops / i8_peak,
+                              "frac_of_nominal_4500": tops / 4500.0}
+                del g
+            res["int8_peak"] = f"{i8_peak:.0f} TOPS = 2 x bf16 burst peak (of {peak_src})"
+            extra[name] = res
+            del xs, y, ws, q
+
+    if rank == 0 and "encoder" in sections:
+        T = 4096  # 128 states x 32 tokens
+        enc = bitrl.Encoder(layers, 2560, 6912, 20, 5)
+        h0 = inputs.activations(T, 2560, 6000).to(dev)
+        h1 = torch.empty_like(h0)
+        ews = torch.empty((enc.workspace_bytes(T),), dtype=torch.uint8, device=dev)
+        ge, le = capture(lambda: enc.forward(h0, h_out=h1, workspace=ews))
+        mse = time_graph(ge, sub_steps, args.warmup, 1) / sub_steps
+        enc_ops = 2.0 * T * sum(k * n for _, k, n in BLOCK) * n_layers
+        i8_sus = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
+        extra[f"encoder_{n_layers}_blocks_T4096"] = {
+            "states_per_s": 128.0 / (mse * 1e-3), "ms": mse, "TOPS": enc_ops / (mse * 1e-3) / 1e12,
+            "frac_of_int8_peak_sustained": enc_ops / (mse * 1e-3) / 1e12 / i8_sus, "launches": le}
+        del ge
+    bitrl.poll_status()
+    if rank == 0 and "cpu" in sections:
+        cpu = oracle_decode_sample()
+
+    if rank == 0:
+        achieved = gbs1 / world
+        line = {
+            "metric": METRIC, "value": gbs1, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms1 / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8 x ternary(2-bit) -> int32", "data": "synthetic",
+            "config": {"workload": f"configs[1]: decode GEMV sweep at M=1 over {n_layers} blocks x (2560->3840, "
+                                   "2560->2560, 2560->13824, 6912->2560) of a ~2B BitNet b1.58 backbone",
+                       "launches_per_step": launches1, "packed_bytes_per_step": bytes_step,
+                       "l2": f"{bytes_step / 1e6:.0f} MB of distinct weights per step against a 126 MB L2: inputs "
+                             "larger than L2, no flush needed",
+                       "timing": "CUDA graph of one step, CUDA events on the launching stream",
+                       "parallelism": f"replicas x{world}, no collective"},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": f"of {peak_src}",
+                         "kernel": "gemv_kernel<1>", "us_per_launch": us_per_launch,
+                         "algorithmic_bytes_per_launch": bytes_step / launches1},
+            "cpu_baseline": cpu,
+            "e2e": {"value": e2e_gbs, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_ms / args.steps},
+            "gpu_launches": launches1 * args.steps,
+            "clocks": clocks,
+            "extra": extra,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=FULL_LAYERS, help="blocks in the backbone (30 = full model)")
+    ap.add_argument("--sections", default="decode8,gemm,encoder,cpu",
+                    help="secondary measurements besides the M=1 headline (comma list; empty = none)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        args.warmup = max(args.warmup, 3)
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
