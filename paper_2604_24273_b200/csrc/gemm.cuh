@@ -6,11 +6,13 @@
 // C = W_q + 1 in {0,1,2} is fed as UNSIGNED bytes (decode = shift + mask), x_q as signed bytes; the surplus
 // sum_k x_q[m,k] is subtracted in the epilogue.  All integer, exact.
 //
-// One persistent CTA per SM, 10 warps:
-//   warp 0      producer : TMA tile of x_q (128-byte swizzle) + bulk copy of the 4 KB packed weight piece
-//   warp 1      MMA      : one thread issues tcgen05.mma kind::i8 (4 per stage, K = 32 each) into TMEM
-//   warps 2-5   expand   : packed piece -> int8 codes in the swizzled K-major layout the MMA reads
-//   warps 6-9   epilogue : TMEM -> registers -> (acc - rowsum) * gamma*a_m/127 -> y (+ residual)
+// One persistent CTA per SM, 11 warps, three decoupled rings in shared memory:
+//   warp 0      X producer : TMA tile of x_q (256 tokens x 128 k, 128-byte swizzle)        ring of 4 x 32 KB
+//   warp 2      P producer : bulk copy of the 4 KB packed weight piece (128 rows x 128 k)    ring of 8 x 4 KB
+//   warps 3-6   expand     : packed piece -> int8 codes in the swizzled K-major layout       ring of 3 x 16 KB
+//   warp 1      MMA        : one thread issues tcgen05.mma kind::i8 (4 per k block, K = 32 each) into TMEM
+//   warps 7-10  epilogue   : TMEM -> registers -> (acc - rowsum) * gamma*a_m/127 -> bf16/fp32, transposed through
+//                            a per-warp shared-memory tile so that global stores are 16 bytes per lane
 // Two 256-column accumulators in TMEM let the epilogue of tile i overlap the main loop of tile i+1.
 // Every mbarrier wait is bounded; on expiry the CTA records a status word and leaves through the normal exit.
 #pragma once
@@ -25,24 +27,31 @@ namespace bitrl {
 constexpr int GM_ROWS = 128;  // weight rows per tile  (MMA M)
 constexpr int GM_TOK = 256;   // tokens per tile       (MMA N)
 constexpr int GM_BK = 128;    // k per pipeline stage  (one 128-byte swizzle row of int8)
-constexpr int GM_STAGES = 4;
-constexpr int GM_THREADS = 320;
+constexpr int GM_XS = 4;      // x_q ring depth
+constexpr int GM_PS = 8;      // packed-weight ring depth
+constexpr int GM_WS = 3;      // expanded-weight ring depth
+constexpr int GM_THREADS = 352;
+constexpr int GM_EXPAND_WARP0 = 3;
+constexpr int GM_EPI_WARP0 = 7;
 
-constexpr uint32_t GM_X_BYTES = GM_TOK * GM_BK;     // 32768
-constexpr uint32_t GM_W_BYTES = GM_ROWS * GM_BK;    // 16384
-constexpr uint32_t GM_P_BYTES = TILE_BYTES;         // 4096
+constexpr uint32_t GM_X_BYTES = GM_TOK * GM_BK;   // 32768
+constexpr uint32_t GM_W_BYTES = GM_ROWS * GM_BK;  // 16384
+constexpr uint32_t GM_P_BYTES = TILE_BYTES;       // 4096
+constexpr uint32_t GM_STAGE_BYTES = 2048;         // per epilogue warp: 32 tokens x 32 rows bf16 (or 16 x 32 fp32)
 constexpr uint32_t GM_OFF_X = 0;
-constexpr uint32_t GM_OFF_W = GM_OFF_X + GM_STAGES * GM_X_BYTES;
-constexpr uint32_t GM_OFF_P = GM_OFF_W + GM_STAGES * GM_W_BYTES;
-constexpr uint32_t GM_OFF_TOK = GM_OFF_P + GM_STAGES * GM_P_BYTES;  // scale[2][256] f32, rowsum[2][256] i32
+constexpr uint32_t GM_OFF_W = GM_OFF_X + GM_XS * GM_X_BYTES;
+constexpr uint32_t GM_OFF_P = GM_OFF_W + GM_WS * GM_W_BYTES;
+constexpr uint32_t GM_OFF_STAGE = GM_OFF_P + GM_PS * GM_P_BYTES;
+constexpr uint32_t GM_OFF_TOK = GM_OFF_STAGE + 4 * GM_STAGE_BYTES;  // scale[2][256] f32, rowsum[2][256] i32
 constexpr uint32_t GM_OFF_BAR = GM_OFF_TOK + 2 * GM_TOK * 8;
-constexpr uint32_t GM_NUM_BARS = 3 * GM_STAGES + 4;
+constexpr uint32_t GM_NUM_BARS = 2 * GM_XS + 2 * GM_PS + 2 * GM_WS + 4;
 constexpr uint32_t GM_OFF_MISC = GM_OFF_BAR + GM_NUM_BARS * 8;
 constexpr uint32_t GM_SMEM_BYTES = GM_OFF_MISC + 16 + 1024;  // + slack to align the base to 1024
+static_assert(GM_SMEM_BYTES <= 232448, "shared memory budget of one CTA");
 
 // stage ids reported with BITRL_ERR_TIMEOUT
-enum { GM_WAIT_EMPTY = 1, GM_WAIT_FULL_EXPAND = 2, GM_WAIT_TMEM_EMPTY = 3, GM_WAIT_FULL_MMA = 4,
-       GM_WAIT_EXPANDED = 5, GM_WAIT_TMEM_FULL = 6 };
+enum { GM_WAIT_X_EMPTY = 1, GM_WAIT_P_EMPTY = 2, GM_WAIT_P_FULL = 3, GM_WAIT_W_EMPTY = 4, GM_WAIT_TMEM_EMPTY = 5,
+       GM_WAIT_X_FULL = 6, GM_WAIT_W_FULL = 7, GM_WAIT_TMEM_FULL = 8 };
 
 struct GemmArgs {
   const uint8_t* tiles;
@@ -64,28 +73,24 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   const uint32_t base = (raw_addr + 1023u) & ~1023u;
   unsigned char* base_ptr = gm_smem_raw + (base - raw_addr);
 
-  const uint32_t bar_full = base + GM_OFF_BAR;                   // [GM_STAGES]
-  const uint32_t bar_expanded = bar_full + 8 * GM_STAGES;        // [GM_STAGES]
-  const uint32_t bar_empty = bar_expanded + 8 * GM_STAGES;       // [GM_STAGES]
-  const uint32_t bar_tmem_full = bar_empty + 8 * GM_STAGES;      // [2]
-  const uint32_t bar_tmem_empty = bar_tmem_full + 16;            // [2]
+  const uint32_t bar_x_full = base + GM_OFF_BAR;
+  const uint32_t bar_x_empty = bar_x_full + 8 * GM_XS;
+  const uint32_t bar_p_full = bar_x_empty + 8 * GM_XS;
+  const uint32_t bar_p_empty = bar_p_full + 8 * GM_PS;
+  const uint32_t bar_w_full = bar_p_empty + 8 * GM_PS;
+  const uint32_t bar_w_empty = bar_w_full + 8 * GM_WS;
+  const uint32_t bar_tmem_full = bar_w_empty + 8 * GM_WS;  // [2]
+  const uint32_t bar_tmem_empty = bar_tmem_full + 16;      // [2]
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + GM_OFF_MISC);
-  float* tok_scale = reinterpret_cast<float*>(base_ptr + GM_OFF_TOK);               // [2][256]
-  int* tok_rowsum = reinterpret_cast<int*>(base_ptr + GM_OFF_TOK + 2 * GM_TOK * 4); // [2][256]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kblocks = a.K / GM_BK;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < GM_STAGES; ++s) {
-      ptx::mbar_init(bar_full + 8 * s, 1);
-      ptx::mbar_init(bar_expanded + 8 * s, 4);
-      ptx::mbar_init(bar_empty + 8 * s, 1);
-    }
-    for (int b = 0; b < 2; ++b) {
-      ptx::mbar_init(bar_tmem_full + 8 * b, 1);
-      ptx::mbar_init(bar_tmem_empty + 8 * b, 4);
-    }
+    for (int s = 0; s < GM_XS; ++s) { ptx::mbar_init(bar_x_full + 8 * s, 1); ptx::mbar_init(bar_x_empty + 8 * s, 1); }
+    for (int s = 0; s < GM_PS; ++s) { ptx::mbar_init(bar_p_full + 8 * s, 1); ptx::mbar_init(bar_p_empty + 8 * s, 4); }
+    for (int s = 0; s < GM_WS; ++s) { ptx::mbar_init(bar_w_full + 8 * s, 4); ptx::mbar_init(bar_w_empty + 8 * s, 1); }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(bar_tmem_full + 8 * b, 1); ptx::mbar_init(bar_tmem_empty + 8 * b, 4); }
     ptx::mbar_init_fence();
     ptx::tma_prefetch_desc(&tmap_x);
   }
@@ -99,20 +104,34 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ producer
+    // ------------------------------------------------------------------ X producer
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x) {
-        const int tn = tile % a.tiles_n, tm = tile / a.tiles_n;
+        const int tm = tile / a.tiles_n;
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const uint32_t s = it % GM_XS, ph = (it / GM_XS) & 1u;
+          if (!ptx::mbar_wait(bar_x_empty + 8 * s, ph ^ 1u)) { report_timeout(GM_WAIT_X_EMPTY); ok = false; break; }
+          ptx::mbar_arrive_expect_tx(bar_x_full + 8 * s, GM_X_BYTES);
+          ptx::tma_load_2d(base + GM_OFF_X + s * GM_X_BYTES, &tmap_x, kb * GM_BK, tm * GM_TOK, bar_x_full + 8 * s);
+        }
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ P producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x) {
+        const int tn = tile % a.tiles_n;
         const uint8_t* wsrc = a.tiles + static_cast<size_t>(tn) * kblocks * TILE_BYTES;
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
-          const uint32_t s = it % GM_STAGES, ph = (it / GM_STAGES) & 1u;
-          if (!ptx::mbar_wait(bar_empty + 8 * s, ph ^ 1u)) { report_timeout(GM_WAIT_EMPTY); ok = false; break; }
-          const uint32_t full = bar_full + 8 * s;
-          ptx::mbar_arrive_expect_tx(full, GM_X_BYTES + GM_P_BYTES);
-          ptx::tma_load_2d(base + GM_OFF_X + s * GM_X_BYTES, &tmap_x, kb * GM_BK, tm * GM_TOK, full);
-          ptx::bulk_g2s(base + GM_OFF_P + s * GM_P_BYTES, wsrc + static_cast<size_t>(kb) * TILE_BYTES, GM_P_BYTES, full);
+          const uint32_t s = it % GM_PS, ph = (it / GM_PS) & 1u;
+          if (!ptx::mbar_wait(bar_p_empty + 8 * s, ph ^ 1u)) { report_timeout(GM_WAIT_P_EMPTY); ok = false; break; }
+          ptx::mbar_arrive_expect_tx(bar_p_full + 8 * s, GM_P_BYTES);
+          ptx::bulk_g2s(base + GM_OFF_P + s * GM_P_BYTES, wsrc + static_cast<size_t>(kb) * TILE_BYTES, GM_P_BYTES,
+                        bar_p_full + 8 * s);
         }
       }
     }
@@ -130,35 +149,39 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + buf * GM_TOK;
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
-          const uint32_t s = it % GM_STAGES, ph = (it / GM_STAGES) & 1u;
-          if (!ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(GM_WAIT_FULL_MMA); ok = false; break; }
-          if (!ptx::mbar_wait(bar_expanded + 8 * s, ph)) { report_timeout(GM_WAIT_EXPANDED); ok = false; break; }
+          const uint32_t xs = it % GM_XS, xph = (it / GM_XS) & 1u;
+          const uint32_t ws = it % GM_WS, wph = (it / GM_WS) & 1u;
+          if (!ptx::mbar_wait(bar_w_full + 8 * ws, wph)) { report_timeout(GM_WAIT_W_FULL); ok = false; break; }
+          if (!ptx::mbar_wait(bar_x_full + 8 * xs, xph)) { report_timeout(GM_WAIT_X_FULL); ok = false; break; }
           ptx::tc_fence_after_sync();
-          const uint64_t adesc = ptx::smem_desc_sw128(base + GM_OFF_W + s * GM_W_BYTES);
-          const uint64_t bdesc = ptx::smem_desc_sw128(base + GM_OFF_X + s * GM_X_BYTES);
+          const uint64_t adesc = ptx::smem_desc_sw128(base + GM_OFF_W + ws * GM_W_BYTES);
+          const uint64_t bdesc = ptx::smem_desc_sw128(base + GM_OFF_X + xs * GM_X_BYTES);
 #pragma unroll
           for (int k4 = 0; k4 < GM_BK / 32; ++k4)
             ptx::mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
-          ptx::mma_commit(bar_empty + 8 * s);
+          ptx::mma_commit(bar_x_empty + 8 * xs);
+          ptx::mma_commit(bar_w_empty + 8 * ws);
         }
         if (ok) ptx::mma_commit(bar_tmem_full + 8 * buf);
       }
     }
-  } else if (warp < 6) {
+  } else if (warp < GM_EPI_WARP0) {
     // ------------------------------------------------------------------ expanders (one weight row each)
-    const int r = threadIdx.x - 64;
+    const int r = threadIdx.x - GM_EXPAND_WARP0 * 32;
     const uint32_t row_off = static_cast<uint32_t>(r >> 3) * 1024u + static_cast<uint32_t>(r & 7) * 128u;
     const uint32_t sw = static_cast<uint32_t>(r & 7);
     uint32_t it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x) {
       for (int kb = 0; kb < kblocks; ++kb, ++it) {
-        const uint32_t s = it % GM_STAGES, ph = (it / GM_STAGES) & 1u;
-        if (!ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(GM_WAIT_FULL_EXPAND); ok = false; break; }
-        const uint4* p = reinterpret_cast<const uint4*>(base_ptr + GM_OFF_P + s * GM_P_BYTES + r * TILE_ROW_BYTES);
-        const uint4 p0 = p[0], p1 = p[1];
+        const uint32_t ps = it % GM_PS, pph = (it / GM_PS) & 1u;
+        const uint32_t ws = it % GM_WS, wph = (it / GM_WS) & 1u;
+        if (!ptx::mbar_wait(bar_p_full + 8 * ps, pph)) { report_timeout(GM_WAIT_P_FULL); ok = false; break; }
+        const uint32_t paddr = base + GM_OFF_P + ps * GM_P_BYTES + r * TILE_ROW_BYTES;
+        const uint4 p0 = ptx::lds128(paddr), p1 = ptx::lds128(paddr + 16);
+        if (!ptx::mbar_wait(bar_w_empty + 8 * ws, wph ^ 1u)) { report_timeout(GM_WAIT_W_EMPTY); ok = false; break; }
         const uint32_t wd[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
-        unsigned char* wrow = base_ptr + GM_OFF_W + s * GM_W_BYTES + row_off;
+        const uint32_t wrow = base + GM_OFF_W + ws * GM_W_BYTES + row_off;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           uint4 c;
@@ -166,56 +189,111 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
           c.y = (wd[j] >> 2) & 0x03030303u;
           c.z = (wd[j] >> 4) & 0x03030303u;
           c.w = (wd[j] >> 6) & 0x03030303u;
-          *reinterpret_cast<uint4*>(wrow + ((static_cast<uint32_t>(j) ^ sw) << 4)) = c;
+          ptx::sts128(wrow + ((static_cast<uint32_t>(j) ^ sw) << 4), c);
         }
         ptx::fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(bar_expanded + 8 * s);
+        if (lane == 0) {
+          ptx::mbar_arrive(bar_w_full + 8 * ws);
+          ptx::mbar_arrive(bar_p_empty + 8 * ps);
+        }
       }
     }
   } else {
     // ------------------------------------------------------------------ epilogue
-    const int q = warp & 3;            // TMEM lane quarter this warp may read
-    const int ep = threadIdx.x - 192;  // 0..127
+    const int q = warp & 3;                           // TMEM lane quarter this warp may read
+    const int ep = threadIdx.x - GM_EPI_WARP0 * 32;   // 0..127
+    const int ew = warp - GM_EPI_WARP0;               // staging buffer index
+    const uint32_t stage = base + GM_OFF_STAGE + ew * GM_STAGE_BYTES;
     const float gamma = *a.gamma;
+    const bool f32 = a.out_dtype == BITRL_OUT_F32;
     uint32_t lt = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x, ++lt) {
       const int tn = tile % a.tiles_n, tm = tile / a.tiles_n;
       const uint32_t buf = lt & 1u;
-      float* sc = tok_scale + buf * GM_TOK;
-      int* rsum = tok_rowsum + buf * GM_TOK;
+      const uint32_t sc_addr = base + GM_OFF_TOK + buf * GM_TOK * 4;
+      const uint32_t rs_addr = base + GM_OFF_TOK + 2 * GM_TOK * 4 + buf * GM_TOK * 4;
       for (int j = ep; j < GM_TOK; j += 128) {
         const int tok = tm * GM_TOK + j;
-        sc[j] = tok < a.M ? out_scale(gamma, a.absmax[tok]) : 0.0f;
-        rsum[j] = tok < a.M ? a.rowsum[tok] : 0;
+        ptx::sts32(sc_addr + 4 * j, __float_as_uint(tok < a.M ? out_scale(gamma, a.absmax[tok]) : 0.0f));
+        ptx::sts32(rs_addr + 4 * j, static_cast<uint32_t>(tok < a.M ? a.rowsum[tok] : 0));
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (!ptx::mbar_wait(bar_tmem_full + 8 * buf, (lt >> 1) & 1u)) { report_timeout(GM_WAIT_TMEM_FULL); ok = false; break; }
       ptx::tc_fence_after_sync();
-      const int n = tn * GM_ROWS + q * 32 + lane;
-      const int tok_hi = min(GM_TOK, a.M - tm * GM_TOK);
+      const int nbase = tn * GM_ROWS + q * 32;  // first output column of this warp
+      const int tok0 = tm * GM_TOK;
+      const int tok_hi = min(GM_TOK, a.M - tok0);
       for (int c = 0; c < GM_TOK / 32; ++c) {
         if (c * 32 >= tok_hi) break;  // warp-uniform
         uint32_t v[32];
         ptx::tmem_ld_32x32b_x32(tmem_base + buf * GM_TOK + c * 32 + (static_cast<uint32_t>(q * 32) << 16), v);
         ptx::tmem_ld_wait();
+        // acc = D - rowsum (exact int32), y = acc * scale
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const int jj = c * 32 + j;
-          if (jj < tok_hi) {
-            const int acc = static_cast<int>(v[j]) - rsum[jj];
-            const size_t o = static_cast<size_t>(tm * GM_TOK + jj) * a.N + n;
-            if (a.acc_out) a.acc_out[o] = acc;
-            const float yv = __fmul_rn(static_cast<float>(acc), sc[jj]);
-            if (a.out_dtype == BITRL_OUT_F32) {
-              static_cast<float*>(a.y)[o] = yv;
-            } else {
-              unsigned short yb = float_to_bf16_bits(yv);
-              if (a.residual)
-                yb = float_to_bf16_bits(__fadd_rn(bf16_bits_to_float(a.residual[o]), bf16_bits_to_float(yb)));
-              static_cast<unsigned short*>(a.y)[o] = yb;
+        for (int g = 0; g < 8; ++g) {
+          const uint4 rs4 = ptx::lds128(rs_addr + (c * 32 + 4 * g) * 4);
+          v[4 * g + 0] -= rs4.x; v[4 * g + 1] -= rs4.y; v[4 * g + 2] -= rs4.z; v[4 * g + 3] -= rs4.w;
+        }
+        if (a.acc_out) {  // debug tap, plain stores
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (c * 32 + j < tok_hi)
+              a.acc_out[static_cast<size_t>(tok0 + c * 32 + j) * a.N + nbase + lane] = static_cast<int>(v[j]);
+        }
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          const uint4 sc4 = ptx::lds128(sc_addr + (c * 32 + 4 * g) * 4);
+          v[4 * g + 0] = __float_as_uint(__fmul_rn(static_cast<float>(static_cast<int>(v[4 * g + 0])), __uint_as_float(sc4.x)));
+          v[4 * g + 1] = __float_as_uint(__fmul_rn(static_cast<float>(static_cast<int>(v[4 * g + 1])), __uint_as_float(sc4.y)));
+          v[4 * g + 2] = __float_as_uint(__fmul_rn(static_cast<float>(static_cast<int>(v[4 * g + 2])), __uint_as_float(sc4.z)));
+          v[4 * g + 3] = __float_as_uint(__fmul_rn(static_cast<float>(static_cast<int>(v[4 * g + 3])), __uint_as_float(sc4.w)));
+        }
+        if (!f32) {
+          // transpose 32 tokens x 32 columns of bf16 through shared memory: row = token (64 bytes)
+#pragma unroll
+          for (int j = 0; j < 32; ++j) ptx::sts16(stage + j * 64 + lane * 2, float_to_bf16_bits(__uint_as_float(v[j])));
+          __syncwarp();
+          unsigned short* yb = static_cast<unsigned short*>(a.y);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int t = i * 8 + (lane >> 2), part = lane & 3;
+            uint4 o = ptx::lds128(stage + i * 512 + lane * 16);
+            if (c * 32 + t < tok_hi) {
+              const size_t off = static_cast<size_t>(tok0 + c * 32 + t) * a.N + nbase + part * 8;
+              if (a.residual) {
+                const uint4 rr = *reinterpret_cast<const uint4*>(a.residual + off);
+                const uint32_t ov[4] = {o.x, o.y, o.z, o.w}, rv[4] = {rr.x, rr.y, rr.z, rr.w};
+                uint32_t res[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const float lo = __fadd_rn(__uint_as_float(rv[e] << 16), __uint_as_float(ov[e] << 16));
+                  const float hi = __fadd_rn(__uint_as_float(rv[e] & 0xffff0000u), __uint_as_float(ov[e] & 0xffff0000u));
+                  res[e] = static_cast<uint32_t>(float_to_bf16_bits(lo)) | (static_cast<uint32_t>(float_to_bf16_bits(hi)) << 16);
+                }
+                o = make_uint4(res[0], res[1], res[2], res[3]);
+              }
+              *reinterpret_cast<uint4*>(yb + off) = o;
             }
+          }
+          __syncwarp();
+        } else {
+          // fp32: two passes of 16 tokens x 32 columns (row = token, 128 bytes)
+          float* yf = static_cast<float*>(a.y);
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) ptx::sts32(stage + j * 128 + lane * 4, v[h * 16 + j]);
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int t = h * 16 + i * 4 + (lane >> 3), part = lane & 7;
+              const uint4 o = ptx::lds128(stage + i * 512 + lane * 16);
+              if (c * 32 + t < tok_hi)
+                *reinterpret_cast<uint4*>(yf + static_cast<size_t>(tok0 + c * 32 + t) * a.N + nbase + part * 4) = o;
+            }
+            __syncwarp();
           }
         }
       }
@@ -272,11 +350,7 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
              static_cast<const unsigned short*>(residual), acc_out, w->N / GM_ROWS, 0};
   const int tiles_m = (M + GM_TOK - 1) / GM_TOK;
   a.tiles_total = a.tiles_n * tiles_m;
-  static bool attr_set = false;
-  if (!attr_set) {
-    BITRL_CUDA(cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM_BYTES));
-    attr_set = true;
-  }
+  BITRL_CUDA(cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM_BYTES));
   const int grid = a.tiles_total < sm_count() ? a.tiles_total : sm_count();
   gemm_i8_kernel<<<grid, GM_THREADS, GM_SMEM_BYTES, st>>>(tmap, a);
   count_launch(1);
