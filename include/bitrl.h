@@ -48,6 +48,7 @@ typedef int32_t bitrl_status;
 #define BITRL_ERR_TIMEOUT (-6)   /* a bounded device-side wait expired (see bitrl_poll_status) */
 #define BITRL_ERR_WORKSPACE (-7) /* workspace missing or smaller than the *_workspace_bytes query */
 #define BITRL_ERR_DTYPE (-8)     /* unknown out_dtype */
+#define BITRL_ERR_LIMIT (-9)     /* size beyond the fixed maximum of an entry point that cannot allocate */
 
 #define BITRL_OUT_F32 0
 #define BITRL_OUT_BF16 1
@@ -66,6 +67,21 @@ typedef struct bitrl_encoder bitrl_encoder_t; /* a stack of blocks of four bitrl
 BITRL_API size_t bitrl_pack_workspace_bytes(int32_t N, int32_t K);
 BITRL_API bitrl_status bitrl_pack_ternary(const float* W, int32_t N, int32_t K, uint8_t* packed, float* gamma,
                                 void* workspace, size_t workspace_bytes, void* stream);
+
+/* Same result as bitrl_pack_ternary, for callers that have no device memory to spare for a workspace and are not
+ * allowed to obtain any: code that runs inside a memory pool it must not grow, inside a stream-ordered region
+ * where cudaMalloc would serialize the device, or in a process whose allocator is owned by another framework.
+ * (The paper has no counterpart; this is a convenience of this library.)  The fp64 partial sums of |W| live in a
+ * fixed 8 KB array that is part of the library image on every GPU that loads it, for the life of the process.
+ *  - Limit: N*K <= BITRL_PACK_STATIC_MAX_WEIGHTS; larger matrices return BITRL_ERR_LIMIT and nothing is launched.
+ *  - Calls no allocator of any kind.  The first call on a device looks up the array's device address (once per
+ *    device, with that device current); make that first call outside any stream capture.
+ *  - All calls share the array and it keeps the previous call's contents.  Nothing in it has to start at zero:
+ *    every slot that a call reads is written earlier in the same call.  Two calls that overlap on the GPU (different
+ *    streams, or threads) race on it and may both produce a wrong gamma; serialize them. */
+#define BITRL_PACK_STATIC_MAX_WEIGHTS (1LL << 28)
+BITRL_API bitrl_status bitrl_pack_ternary_static(const float* W, int32_t N, int32_t K, uint8_t* packed, float* gamma,
+                                                 void* stream);
 
 /* Builds the weight handle from the canonical packed bytes and gamma (both dev).  The library keeps its own
  * re-tiled copy (N*K/4 bytes); the inputs may be freed once `stream` has run past this call. */

@@ -20,7 +20,8 @@ _HERE = Path(__file__).resolve().parent
 LIB_PATH = _HERE / "libbitrl.so"
 
 OK = 0
-ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT, ERR_WORKSPACE, ERR_DTYPE = range(-1, -9, -1)
+ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT, ERR_WORKSPACE, ERR_DTYPE, ERR_LIMIT = range(-1, -10, -1)
+PACK_STATIC_MAX_WEIGHTS = 1 << 28
 OUT_F32, OUT_BF16 = 0, 1
 GEMV_MAX_M = 16
 
@@ -31,6 +32,7 @@ _sz = ctypes.c_size_t
 EXPORTS = {
     "bitrl_pack_workspace_bytes": (_sz, [_i32, _i32]),
     "bitrl_pack_ternary": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp, _sz, _vp]),
+    "bitrl_pack_ternary_static": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp]),
     "bitrl_linear_create": (_i32, [_vp, _vp, _i32, _i32, ctypes.POINTER(_vp), _vp]),
     "bitrl_linear_destroy": (_i32, [_vp]),
     "bitrl_quant_act": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp, _vp]),
@@ -119,6 +121,20 @@ def pack_ternary(W: torch.Tensor):
     _check(lib().bitrl_pack_ternary(_ptr(W), N, K, _ptr(packed), _ptr(gamma), _ptr(ws), nbytes, _stream()),
            "bitrl_pack_ternary")
     return packed, gamma
+
+
+def pack_ternary_static(W: torch.Tensor, packed: torch.Tensor, gamma: torch.Tensor) -> None:
+    """``bitrl_pack_ternary_static``: packs into caller-provided ``packed`` / ``gamma`` and allocates nothing, for
+    callers that may not touch the device allocator.  At most ``PACK_STATIC_MAX_WEIGHTS`` weights; calls must not
+    overlap on the GPU (they share one fixed scratch array inside the library)."""
+    _dev(W, torch.float32, "W")
+    _dev(packed, torch.uint8, "packed")
+    _dev(gamma, torch.float32, "gamma")
+    N, K = W.shape
+    if packed.numel() != N * K // 4 or gamma.numel() < 1:
+        raise ValueError("packed must hold N*K/4 bytes and gamma one float")
+    _check(lib().bitrl_pack_ternary_static(_ptr(W), N, K, _ptr(packed), _ptr(gamma), _stream()),
+           "bitrl_pack_ternary_static")
 
 
 class Linear:

@@ -108,6 +108,39 @@ bitrl_status bitrl_pack_ternary(const float* W, int32_t N, int32_t K, uint8_t* p
   return launch_pack(W, N, K, packed, gamma, workspace, static_cast<cudaStream_t>(stream));
 }
 
+}  // extern "C"
+
+// Scratch of bitrl_pack_ternary_static: one fp64 partial sum per reduction block.  It is part of the library
+// image, so every GPU that loads the library holds these 8 KB until the process exits.  In host code the name
+// below is only a handle for cudaGetSymbolAddress, never a pointer a kernel could use.
+static __device__ __align__(256) double g_pack_static_scratch[ABSSUM_MAX_BLOCKS];
+
+extern "C" {
+
+bitrl_status bitrl_pack_ternary_static(const float* W, int32_t N, int32_t K, uint8_t* packed, float* gamma,
+                                       void* stream) {
+  if (!W || !packed || !gamma) return BITRL_ERR_NULL;
+  if (!shape_ok(N, K)) return BITRL_ERR_SHAPE;
+  if (static_cast<long long>(N) * K > BITRL_PACK_STATIC_MAX_WEIGHTS) return BITRL_ERR_LIMIT;
+  if (!aligned16(W) || !aligned16(packed)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  // Device address of the scratch array, looked up once per device with that device current.
+  static double* scratch_addr[64] = {nullptr};
+  int dev = 0;
+  BITRL_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return BITRL_ERR_ARCH;
+  if (!scratch_addr[dev]) {
+    double* p = nullptr;
+    BITRL_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_pack_static_scratch));
+    if (!p) return BITRL_ERR_CUDA;
+    scratch_addr[dev] = p;
+  }
+  // The reduction writes partial[0 .. blocks) before its last stage reads exactly those slots, so stale
+  // contents from an earlier call are never observed and nothing needs clearing.
+  return launch_pack(W, N, K, packed, gamma, scratch_addr[dev], static_cast<cudaStream_t>(stream));
+}
+
 bitrl_status bitrl_linear_create(const uint8_t* packed, const float* gamma, int32_t N, int32_t K,
                                  bitrl_linear_t** out, void* stream) {
   if (!packed || !gamma || !out) return BITRL_ERR_NULL;
@@ -390,6 +423,7 @@ const char* bitrl_status_string(bitrl_status s) {
     case BITRL_ERR_TIMEOUT: return "device-side wait timed out";
     case BITRL_ERR_WORKSPACE: return "workspace missing or too small";
     case BITRL_ERR_DTYPE: return "bad output dtype";
+    case BITRL_ERR_LIMIT: return "size beyond the fixed maximum of this entry point";
     default: return "unknown status";
   }
 }
