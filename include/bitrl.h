@@ -106,6 +106,17 @@ BITRL_API bitrl_status bitrl_bitlinear_forward(const bitrl_linear_t* w, const vo
                                      void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes,
                                      void* stream);
 
+/* `count` independent layers in one launch, for M <= BITRL_GEMV_MAX_M: y[i] = BitLinear_{w[i]}(x[i]).  One decode-size
+ * matrix is only a few MB, so a launch per matrix is bound by launch latency; when the calls do not depend on one
+ * another (a sweep over matrices, several projections of the same input) this entry point streams all their packed
+ * weights back to back at HBM speed with one persistent kernel.  w, x, y: HOST arrays of `count` entries; x[i] dev
+ * bf16 [M, K_i] (entries may repeat), y[i] dev [M, N_i], all distinct.  1 <= count <= BITRL_MULTI_MAX_JOBS.  No workspace.
+ * Results are bit-identical to `count` separate bitrl_bitlinear_forward calls. */
+#define BITRL_MULTI_MAX_JOBS 128
+BITRL_API bitrl_status bitrl_bitlinear_forward_multi(int32_t count, const bitrl_linear_t* const* w,
+                                                     const void* const* x, void* const* y, int32_t M,
+                                                     int32_t out_dtype, void* stream);
+
 /* Same, and additionally writes the integer stages: xq_out dev int8 [M,K], absmax_out dev fp32 [M],
  * acc_out dev int32 [M,N] (any may be NULL).  Needs the workspace for every M. */
 BITRL_API bitrl_status bitrl_bitlinear_forward_debug(const bitrl_linear_t* w, const void* x, int32_t M, int32_t K,

@@ -38,6 +38,8 @@ EXPORTS = {
     "bitrl_quant_act": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp, _vp]),
     "bitrl_workspace_bytes": (_sz, [_i32, _i32, _i32]),
     "bitrl_bitlinear_forward": (_i32, [_vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp]),
+    "bitrl_bitlinear_forward_multi": (_i32, [_i32, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp), _i32,
+                                             _i32, _vp]),
     "bitrl_bitlinear_forward_debug": (_i32, [_vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp, _vp, _vp, _vp]),
     "bitrl_bitlinear_forward_q": (_i32, [_vp, _vp, _vp, _vp, _i32, _vp, _i32, _vp, _vp, _vp]),
     "bitrl_rmsnorm_quant": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp]),
@@ -200,6 +202,32 @@ def bitlinear_forward(w: Linear, x: torch.Tensor, out_dtype: int = OUT_BF16, y: 
     _check(lib().bitrl_bitlinear_forward(w.handle, _ptr(x), M, K, w.N, _ptr(y), out_dtype, _ptr(workspace), nbytes,
                                          _stream()), "bitrl_bitlinear_forward")
     return y
+
+
+class MultiCall:
+    """Argument block of ``bitrl_bitlinear_forward_multi``: ``count`` independent layers, one launch.
+
+    The three host pointer arrays are built once; ``run()`` only makes the C call (cheap enough to sit in a
+    CUDA-graph capture or a hot loop)."""
+
+    def __init__(self, ws, xs, ys, out_dtype: int = OUT_BF16):
+        assert len(ws) == len(xs) == len(ys) >= 1
+        self.M = xs[0].shape[0]
+        for w, x, y in zip(ws, xs, ys):
+            _dev(x, torch.bfloat16, "x")
+            assert x.shape == (self.M, w.K) and tuple(y.shape) == (self.M, w.N) and y.is_cuda and y.is_contiguous()
+            assert y.dtype == (torch.float32 if out_dtype == OUT_F32 else torch.bfloat16)
+        self.keep = (list(ws), list(xs), list(ys))
+        n = len(ws)
+        self.count, self.out_dtype = n, out_dtype
+        self.w = (_vp * n)(*[w.handle for w in ws])
+        self.x = (_vp * n)(*[x.data_ptr() for x in xs])
+        self.y = (_vp * n)(*[y.data_ptr() for y in ys])
+
+    def run(self):
+        _check(lib().bitrl_bitlinear_forward_multi(self.count, self.w, self.x, self.y, self.M, self.out_dtype,
+                                                   _stream()), "bitrl_bitlinear_forward_multi")
+        return self.keep[2]
 
 
 def bitlinear_forward_debug(w: Linear, x: torch.Tensor, out_dtype: int = OUT_BF16):

@@ -49,6 +49,7 @@ static bitrl_status check_arch() {
 #include "pack.cuh"
 #include "quant.cuh"
 #include "gemv.cuh"
+#include "gemv_multi.cuh"
 #include "gemm.cuh"
 
 using namespace bitrl;
@@ -233,6 +234,22 @@ bitrl_status bitrl_bitlinear_forward(const bitrl_linear_t* w, const void* x, int
                                      void* stream) {
   return forward_impl(w, x, M, K, N, y, out_dtype, workspace, workspace_bytes, nullptr, nullptr, nullptr, false,
                       stream);
+}
+
+bitrl_status bitrl_bitlinear_forward_multi(int32_t count, const bitrl_linear_t* const* w, const void* const* x,
+                                           void* const* y, int32_t M, int32_t out_dtype, void* stream) {
+  if (!w || !x || !y) return BITRL_ERR_NULL;
+  if (count < 1 || count > BITRL_MULTI_MAX_JOBS || M < 1 || M > BITRL_GEMV_MAX_M) return BITRL_ERR_SHAPE;
+  if (out_dtype != BITRL_OUT_F32 && out_dtype != BITRL_OUT_BF16) return BITRL_ERR_DTYPE;
+  const Linear* lins[BITRL_MULTI_MAX_JOBS];
+  for (int i = 0; i < count; ++i) {
+    if (!w[i] || !x[i] || !y[i]) return BITRL_ERR_NULL;
+    if (!aligned16(x[i]) || !aligned16(y[i])) return BITRL_ERR_ALIGN;
+    lins[i] = &w[i]->l;
+  }
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  return launch_gemv_multi(count, lins, x, y, M, out_dtype, static_cast<cudaStream_t>(stream));
 }
 
 bitrl_status bitrl_bitlinear_forward_debug(const bitrl_linear_t* w, const void* x, int32_t M, int32_t K,

@@ -1,0 +1,553 @@
+// Grouped streaming kernel: several independent BitLinear calls with M <= 16 in ONE launch.
+//
+// A single decode-size matrix is only 2-9 MB: one launch per matrix is bound by launch and dependency latency,
+// not by HBM.  When several such calls are independent (a sweep over matrices, or the heads of one layer), this
+// kernel streams all of their packed weights back to back at HBM speed.
+//
+// One persistent CTA per SM.  The work list is the concatenation of all jobs' row tiles (128 rows x all K, one
+// contiguous K/4*128-byte region of the tile layout); every CTA owns a contiguous, byte-balanced range of it.
+//   warp 8      producer: bulk copies (cp.async.bulk) of four consecutive 4 KB (row tile, k block) pieces into a ring of
+//               up to 8 slots of 16 KB - up to 128 KB in flight per SM, independent of the activations, so it runs ahead across jobs
+//   warps 0-7   consumers: warp w owns rows 16w..16w+15 of the row tile for the whole K.  The 2-bit codes are
+//               decoded by shift+mask straight into the A fragments of a warp-level integer MMA
+//               (mma.sync m16n8k32, A = unsigned codes, B = signed int8 activations of 8 tokens, int32 accumulate):
+//               the same instruction count serves 1 to 8 tokens (two MMAs per k step for 9 to 16), so the kernel
+//               stays memory-bound where a dp4a loop would be ALU-bound from M = 4 on.  No cross-warp reduction.
+// The activations of a job are quantized into shared memory by the consumer warps when the job's x differs from the
+// cached one.  All mbarrier waits are bounded; after an expiry a warp keeps walking its work list (skipping waits and
+// stores) so that the consumer-wide named barriers stay matched, and the CTA exits normally.
+#pragma once
+
+#include "common.cuh"
+#include "gemv.cuh"
+#include "ptx.cuh"
+
+namespace bitrl {
+
+constexpr int GVM_MAX_JOBS = 128;
+constexpr int GVM_MAX_CTAS = 192;
+constexpr int GVM_CONSUMERS = 8;
+constexpr int GVM_THREADS = (GVM_CONSUMERS + 1) * 32;
+constexpr int GVM_SMEM_BUDGET = 220 * 1024;
+constexpr int GVM_UNROLL = 4;  // 4 KB pieces per ring slot: one bulk copy, one barrier, one consumer loop iteration
+constexpr int GVM_SLOT_BYTES = GVM_UNROLL * TILE_BYTES;
+constexpr int GVM_XPAD = 16;  // bytes added to each activation row so that the 8 token rows hit different banks
+
+enum { GVM_WAIT_EMPTY = 21, GVM_WAIT_FULL = 22 };
+
+struct GvmJob {
+  const uint8_t* tiles;
+  const float* gamma;
+  const unsigned short* x;
+  void* y;
+  int N, K;
+  int unit_begin;  // index of this job's first row tile in the global work list
+  int pad;
+};
+
+struct GvmArgs {
+  GvmJob jobs[GVM_MAX_JOBS];
+  int unit_start[GVM_MAX_CTAS + 1];  // work-list range of each CTA
+  int njobs, M, out_dtype, depth_log2, kmax;
+};
+
+// D(16x8, int32) += A(16x32, unsigned 8-bit, row) * B(32x8, signed 8-bit, col).
+__device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Fragment mapping used below.  Lane (g = lane/4, t = lane%4) holds weight rows g and g+8 of its warp's 16 rows.
+// Word j of a row covers k = 16j..16j+15 and (word >> 2t) & 0x03030303 are its codes k = 16j+4t..16j+4t+3: exactly
+// the bytes the A fragment wants from this lane (a0/a2: row g, k = 4t.. and 16+4t..; a1/a3: row g+8).  Activations
+// are stored so that the eight words k = 16q+4t.. (q = 0..7) of one token and one 128-k block are contiguous:
+// two 128-bit loads give the B fragments (b0, b1) of the block's four k steps.
+template <int NT>
+__global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid_constant__ GvmArgs a) {
+  extern __shared__ __align__(128) unsigned char gvm_smem[];
+  const int depth = 1 << a.depth_log2;
+  const uint32_t ring = ptx::smem_u32(gvm_smem);
+  unsigned char* xq_s = gvm_smem + depth * GVM_SLOT_BYTES;  // [NT][K + GVM_XPAD], word-permuted per 128-k block
+  const uint32_t xq_addr = ptx::smem_u32(xq_s);
+  unsigned char* tail = xq_s + static_cast<size_t>(NT) * (a.kmax + GVM_XPAD);
+  const uint32_t bar_full = ptx::smem_u32(tail);    // [depth]
+  const uint32_t bar_empty = bar_full + 8 * depth;  // [depth]
+  float* absmax_s = reinterpret_cast<float*>(tail + 16 * depth);  // [NT]
+  int* rowsum_s = reinterpret_cast<int*>(absmax_s + NT);          // [NT]
+  float* redf = reinterpret_cast<float*>(rowsum_s + NT);          // [8]
+  int* redi = reinterpret_cast<int*>(redf + GVM_CONSUMERS);       // [8]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int u_begin = a.unit_start[blockIdx.x], u_end = a.unit_start[blockIdx.x + 1];
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < depth; ++s) {
+      ptx::mbar_init(bar_full + 8 * s, 1);
+      ptx::mbar_init(bar_empty + 8 * s, GVM_CONSUMERS);
+    }
+    ptx::mbar_init_fence();
+  }
+  __syncthreads();
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+  if (warp == GVM_CONSUMERS) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      uint32_t pc = 0;
+      int j = 0;
+      bool ok = true;
+      for (int u = u_begin; ok && u < u_end; ++u) {
+        while (j + 1 < a.njobs && a.jobs[j + 1].unit_begin <= u) ++j;
+        const int kblocks = a.jobs[j].K / TILE_K;
+        const uint8_t* src = a.jobs[j].tiles + static_cast<size_t>(u - a.jobs[j].unit_begin) * kblocks * TILE_BYTES;
+        for (int kb = 0; kb < kblocks; kb += GVM_UNROLL, ++pc) {
+          const uint32_t bytes = static_cast<uint32_t>(min(GVM_UNROLL, kblocks - kb)) * TILE_BYTES;
+          const uint32_t s = pc & (depth - 1), ph = (pc >> a.depth_log2) & 1u;
+          if (!ptx::mbar_wait(bar_empty + 8 * s, ph ^ 1u)) { report_timeout(GVM_WAIT_EMPTY); ok = false; break; }
+          ptx::mbar_arrive_expect_tx(bar_full + 8 * s, bytes);
+          ptx::bulk_g2s(ring + s * GVM_SLOT_BYTES, src + static_cast<size_t>(kb) * TILE_BYTES, bytes, bar_full + 8 * s);
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ consumers
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // x may be produced by the preceding kernel
+    const int g = lane >> 2, t = lane & 3;
+    const int sh = 2 * t;
+    const unsigned short* cached_x = nullptr;
+    int cached_k = 0;
+    uint32_t pc = 0;
+    int j = 0;
+    bool ok = true;
+    for (int u = u_begin; u < u_end; ++u) {
+      while (j + 1 < a.njobs && a.jobs[j + 1].unit_begin <= u) ++j;
+      const GvmJob& job = a.jobs[j];
+      const int K = job.K, kblocks = K / TILE_K;
+      const int xstride = K + GVM_XPAD;
+      if (job.x != cached_x || K != cached_k) {
+        // ---- quantize this job's activations (all consumer warps; the ring keeps filling meanwhile) ----
+        asm volatile("bar.sync 2, 256;" ::: "memory");  // everyone is done with the previous contents
+        const int nvec8 = K >> 3;
+        for (int m = 0; m < NT; ++m) {
+          unsigned char* row = xq_s + static_cast<size_t>(m) * xstride;
+          if (m >= a.M) {
+            for (int i = threadIdx.x; i < (xstride >> 2); i += 256) reinterpret_cast<uint32_t*>(row)[i] = 0u;
+            continue;
+          }
+          const uint4* xr = reinterpret_cast<const uint4*>(job.x + static_cast<size_t>(m) * K);
+          float mx = 0.0f;
+          for (int i = threadIdx.x; i < nvec8; i += 256) mx = fmaxf(mx, absmax8(xr[i]));
+          mx = warp_max(mx);
+          if (lane == 0) redf[warp] = mx;
+          asm volatile("bar.sync 2, 256;" ::: "memory");
+#pragma unroll
+          for (int i = 0; i < GVM_CONSUMERS; ++i) mx = fmaxf(mx, redf[i]);
+          const float amax = fmaxf(mx, 1e-5f);
+          const float inv = __fdiv_rn(127.0f, amax);
+          int rs = 0;
+          for (int i = threadIdx.x; i < nvec8; i += 256) {
+            const uint4 raw = xr[i];
+            const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+            int q[8];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              q[2 * e] = quant_code(__uint_as_float(rw[e] << 16), inv);
+              q[2 * e + 1] = quant_code(__uint_as_float(rw[e] & 0xffff0000u), inv);
+            }
+            const uint32_t lo = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | (static_cast<uint32_t>(q[3]) << 24);
+            const uint32_t hi = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | (static_cast<uint32_t>(q[7]) << 24);
+            rs += q[0] + q[1] + q[2] + q[3] + q[4] + q[5] + q[6] + q[7];
+            // word w = 4q+t of a 128-k block is stored at word position t*8+q of that block
+            const int kb = i >> 4, w = (i & 15) * 2;
+            uint32_t* blk = reinterpret_cast<uint32_t*>(row + kb * TILE_K);
+            blk[(w & 3) * 8 + (w >> 2)] = lo;
+            blk[((w + 1) & 3) * 8 + ((w + 1) >> 2)] = hi;
+          }
+          rs = warp_sum_i(rs);
+          if (lane == 0) redi[warp] = rs;
+          asm volatile("bar.sync 2, 256;" ::: "memory");
+          if (threadIdx.x == 0) {
+            int tsum = 0;
+#pragma unroll
+            for (int i = 0; i < GVM_CONSUMERS; ++i) tsum += redi[i];
+            rowsum_s[m] = tsum;
+            absmax_s[m] = amax;
+          }
+        }
+        asm volatile("bar.sync 2, 256;" ::: "memory");
+        cached_x = job.x;
+        cached_k = K;
+      }
+
+      // ---- one row tile: this warp's 16 rows over the whole K ----
+      // The GVM_UNROLL pieces of a slot are fetched from shared memory together and feed independent accumulator
+      // chains, so that neither the loads nor the MMAs of one piece wait for those of another.
+      constexpr int CH = NT == 8 ? 16 : 8;  // independent accumulator chains (the warp MMA has a long latency)
+      int acc[CH][NT / 8][4];
+#pragma unroll
+      for (int c = 0; c < CH; ++c)
+#pragma unroll
+        for (int h = 0; h < NT / 8; ++h)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc[c][h][e] = 0;
+      const uint32_t xlane = xq_addr + g * xstride + t * 32;
+      for (int kb = 0; kb < kblocks; kb += GVM_UNROLL) {
+        const int np = min(GVM_UNROLL, kblocks - kb);
+        uint4 wr[GVM_UNROLL][4];
+        const uint32_t s = pc & (depth - 1), ph = (pc >> a.depth_log2) & 1u;
+        if (ok && !ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(GVM_WAIT_FULL); ok = false; }
+        if (ok) {
+#pragma unroll
+          for (int p = 0; p < GVM_UNROLL; ++p) {
+            if (p < np) {
+              const uint32_t wslice = ring + s * GVM_SLOT_BYTES + p * TILE_BYTES + warp * 512;
+              wr[p][0] = ptx::lds128(wslice + g * 32);
+              wr[p][1] = ptx::lds128(wslice + g * 32 + 16);
+              wr[p][2] = ptx::lds128(wslice + (g + 8) * 32);
+              wr[p][3] = ptx::lds128(wslice + (g + 8) * 32 + 16);
+            }
+          }
+        }
+        if (ok) {
+#pragma unroll
+          for (int p = 0; p < GVM_UNROLL; ++p) {
+            if (p < np) {
+              const uint32_t w0[8] = {wr[p][0].x, wr[p][0].y, wr[p][0].z, wr[p][0].w, wr[p][1].x, wr[p][1].y, wr[p][1].z, wr[p][1].w};
+              const uint32_t w1[8] = {wr[p][2].x, wr[p][2].y, wr[p][2].z, wr[p][2].w, wr[p][3].x, wr[p][3].y, wr[p][3].z, wr[p][3].w};
+#pragma unroll
+              for (int h = 0; h < NT / 8; ++h) {
+                const uint32_t xa_addr = xlane + h * 8 * xstride + (kb + p) * TILE_K;
+                const uint4 xa = ptx::lds128(xa_addr), xb = ptx::lds128(xa_addr + 16);
+                const uint32_t xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                  mma_u8s8(acc[(p * 4 + ks) % CH][h], (w0[2 * ks] >> sh) & 0x03030303u, (w1[2 * ks] >> sh) & 0x03030303u,
+                           (w0[2 * ks + 1] >> sh) & 0x03030303u, (w1[2 * ks + 1] >> sh) & 0x03030303u, xv[2 * ks],
+                           xv[2 * ks + 1]);
+              }
+            }
+          }
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(bar_empty + 8 * s);
+        }
+        ++pc;
+      }
+#pragma unroll
+      for (int c = 1; c < CH; ++c)
+#pragma unroll
+        for (int h = 0; h < NT / 8; ++h)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc[0][h][e] += acc[c][h][e];
+      if (ok) {
+        // C fragment: acc[h][0..1] = (row g, tokens 8h+2t, +1), acc[h][2..3] = (row g+8, same tokens)
+        const float gamma = *job.gamma;
+        const int n0 = (u - job.unit_begin) * TILE_ROWS + warp * 16 + g;
+#pragma unroll
+        for (int h = 0; h < NT / 8; ++h)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int m = 8 * h + 2 * t + (e & 1);
+            if (m < a.M) {
+              const int tv = acc[0][h][e] - rowsum_s[m];
+              const float yv = __fmul_rn(static_cast<float>(tv), out_scale(gamma, absmax_s[m]));
+              const size_t o = static_cast<size_t>(m) * job.N + n0 + (e >> 1) * 8;
+              if (a.out_dtype == BITRL_OUT_F32) static_cast<float*>(job.y)[o] = yv;
+              else static_cast<unsigned short*>(job.y)[o] = float_to_bf16_bits(yv);
+            }
+          }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// M <= 2 variant: dp4a instead of the warp MMA (cheaper when only one or two tokens use the weights), and 16
+// consumer warps in two groups: group 0 takes the even pieces of every slot, group 1 the odd ones; their partial
+// sums meet in shared memory once per row tile.  Lane = 2*row + k half, as in the single-matrix kernel.
+constexpr int GVD_CONSUMERS = 16;
+constexpr int GVD_THREADS = (GVD_CONSUMERS + 1) * 32;
+
+template <int MT>
+__global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const __grid_constant__ GvmArgs a) {
+  extern __shared__ __align__(128) unsigned char gvm_smem[];
+  const int depth = 1 << a.depth_log2;
+  const uint32_t ring = ptx::smem_u32(gvm_smem);
+  int8_t* xq_s = reinterpret_cast<int8_t*>(gvm_smem + depth * GVM_SLOT_BYTES);  // [MT][K]
+  unsigned char* tail = gvm_smem + depth * GVM_SLOT_BYTES + static_cast<size_t>(MT) * a.kmax;
+  const uint32_t bar_full = ptx::smem_u32(tail);    // [depth]
+  const uint32_t bar_empty = bar_full + 8 * depth;  // [depth]
+  float* absmax_s = reinterpret_cast<float*>(tail + 16 * depth);  // [MT]
+  int* rowsum_s = reinterpret_cast<int*>(absmax_s + MT);          // [MT]
+  float* redf = reinterpret_cast<float*>(rowsum_s + MT);          // [16]
+  int* redi = reinterpret_cast<int*>(redf + GVD_CONSUMERS);       // [16]
+  int* comb = redi + GVD_CONSUMERS;                               // [2][8 warps][16 rows][MT]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int u_begin = a.unit_start[blockIdx.x], u_end = a.unit_start[blockIdx.x + 1];
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < depth; ++s) {
+      ptx::mbar_init(bar_full + 8 * s, 1);
+      ptx::mbar_init(bar_empty + 8 * s, GVD_CONSUMERS);
+    }
+    ptx::mbar_init_fence();
+  }
+  __syncthreads();
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+  if (warp == GVD_CONSUMERS) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      uint32_t pc = 0;
+      int j = 0;
+      bool ok = true;
+      for (int u = u_begin; ok && u < u_end; ++u) {
+        while (j + 1 < a.njobs && a.jobs[j + 1].unit_begin <= u) ++j;
+        const int kblocks = a.jobs[j].K / TILE_K;
+        const uint8_t* src = a.jobs[j].tiles + static_cast<size_t>(u - a.jobs[j].unit_begin) * kblocks * TILE_BYTES;
+        for (int kb = 0; kb < kblocks; kb += GVM_UNROLL, ++pc) {
+          const uint32_t bytes = static_cast<uint32_t>(min(GVM_UNROLL, kblocks - kb)) * TILE_BYTES;
+          const uint32_t s = pc & (depth - 1), ph = (pc >> a.depth_log2) & 1u;
+          if (!ptx::mbar_wait(bar_empty + 8 * s, ph ^ 1u)) { report_timeout(GVM_WAIT_EMPTY); ok = false; break; }
+          ptx::mbar_arrive_expect_tx(bar_full + 8 * s, bytes);
+          ptx::bulk_g2s(ring + s * GVM_SLOT_BYTES, src + static_cast<size_t>(kb) * TILE_BYTES, bytes, bar_full + 8 * s);
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ consumers
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // x may be produced by the preceding kernel
+    const int half = lane & 1, grp = warp >> 3, rw = warp & 7;
+    const unsigned short* cached_x = nullptr;
+    int cached_k = 0;
+    uint32_t pc = 0, tile_no = 0;
+    int j = 0;
+    bool ok = true;
+    for (int u = u_begin; u < u_end; ++u, ++tile_no) {
+      while (j + 1 < a.njobs && a.jobs[j + 1].unit_begin <= u) ++j;
+      const GvmJob& job = a.jobs[j];
+      const int K = job.K, kblocks = K / TILE_K;
+      if (job.x != cached_x || K != cached_k) {
+        asm volatile("bar.sync 2, 512;" ::: "memory");  // everyone is done with the previous contents
+        const int nvec8 = K >> 3;
+        for (int m = 0; m < MT; ++m) {
+          uint2* dst = reinterpret_cast<uint2*>(xq_s + m * K);
+          if (m >= a.M) {
+            for (int i = threadIdx.x; i < nvec8; i += 512) dst[i] = make_uint2(0u, 0u);
+            continue;
+          }
+          const uint4* xr = reinterpret_cast<const uint4*>(job.x + static_cast<size_t>(m) * K);
+          float mx = 0.0f;
+          for (int i = threadIdx.x; i < nvec8; i += 512) mx = fmaxf(mx, absmax8(xr[i]));
+          mx = warp_max(mx);
+          if (lane == 0) redf[warp] = mx;
+          asm volatile("bar.sync 2, 512;" ::: "memory");
+#pragma unroll
+          for (int i = 0; i < GVD_CONSUMERS; ++i) mx = fmaxf(mx, redf[i]);
+          const float amax = fmaxf(mx, 1e-5f);
+          const float inv = __fdiv_rn(127.0f, amax);
+          int rs = 0;
+          for (int i = threadIdx.x; i < nvec8; i += 512) {
+            const uint4 raw = xr[i];
+            const uint32_t rwd[4] = {raw.x, raw.y, raw.z, raw.w};
+            int q[8];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              q[2 * e] = quant_code(__uint_as_float(rwd[e] << 16), inv);
+              q[2 * e + 1] = quant_code(__uint_as_float(rwd[e] & 0xffff0000u), inv);
+            }
+            uint2 wd;
+            wd.x = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | (static_cast<uint32_t>(q[3]) << 24);
+            wd.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | (static_cast<uint32_t>(q[7]) << 24);
+            rs += q[0] + q[1] + q[2] + q[3] + q[4] + q[5] + q[6] + q[7];
+            dst[i] = wd;
+          }
+          rs = warp_sum_i(rs);
+          if (lane == 0) redi[warp] = rs;
+          asm volatile("bar.sync 2, 512;" ::: "memory");
+          if (threadIdx.x == 0) {
+            int tsum = 0;
+#pragma unroll
+            for (int i = 0; i < GVD_CONSUMERS; ++i) tsum += redi[i];
+            rowsum_s[m] = tsum;
+            absmax_s[m] = amax;
+          }
+        }
+        asm volatile("bar.sync 2, 512;" ::: "memory");
+        cached_x = job.x;
+        cached_k = K;
+      }
+
+      // ---- one row tile: this warp's 16 rows, every second piece ----
+      int acc[MT][4];
+#pragma unroll
+      for (int m = 0; m < MT; ++m)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[m][c] = 0;
+      for (int kb = 0; kb < kblocks; kb += GVM_UNROLL, ++pc) {
+        const int np = min(GVM_UNROLL, kblocks - kb);
+        const uint32_t s = pc & (depth - 1), ph = (pc >> a.depth_log2) & 1u;
+        if (ok && !ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(GVM_WAIT_FULL); ok = false; }
+        if (ok) {
+          uint4 wv[GVM_UNROLL / 2];
+#pragma unroll
+          for (int pp = 0; pp < GVM_UNROLL / 2; ++pp) {
+            const int pidx = 2 * pp + grp;
+            if (pidx < np) wv[pp] = ptx::lds128(ring + s * GVM_SLOT_BYTES + pidx * TILE_BYTES + rw * 512 + lane * 16);
+          }
+#pragma unroll
+          for (int pp = 0; pp < GVM_UNROLL / 2; ++pp) {
+            const int pidx = 2 * pp + grp;
+            if (pidx < np) {
+              const uint32_t wword[4] = {wv[pp].x, wv[pp].y, wv[pp].z, wv[pp].w};
+              const int k0 = (kb + pidx) * TILE_K + half * 64;
+#pragma unroll
+              for (int jw = 0; jw < 4; ++jw) {
+                const uint32_t c0 = wword[jw] & 0x03030303u;
+                const uint32_t c1 = (wword[jw] >> 2) & 0x03030303u;
+                const uint32_t c2 = (wword[jw] >> 4) & 0x03030303u;
+                const uint32_t c3 = (wword[jw] >> 6) & 0x03030303u;
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                  const int4 xv = *reinterpret_cast<const int4*>(xq_s + m * K + k0 + 16 * jw);
+                  acc[m][0] = dp4a_u8s8(c0, xv.x, acc[m][0]);
+                  acc[m][1] = dp4a_u8s8(c1, xv.y, acc[m][1]);
+                  acc[m][2] = dp4a_u8s8(c2, xv.z, acc[m][2]);
+                  acc[m][3] = dp4a_u8s8(c3, xv.w, acc[m][3]);
+                }
+              }
+            }
+          }
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(bar_empty + 8 * s);
+        }
+      }
+      // ---- combine: k halves by shuffle, the two warp groups through shared memory ----
+      int* cb = comb + (tile_no & 1u) * (8 * 16 * MT) + (rw * 16 + (lane >> 1)) * MT;
+      int tot[MT];
+#pragma unroll
+      for (int m = 0; m < MT; ++m) {
+        tot[m] = acc[m][0] + acc[m][1] + acc[m][2] + acc[m][3];
+        tot[m] += __shfl_xor_sync(0xffffffffu, tot[m], 1);
+        if (grp == 1 && half == 0) cb[m] = tot[m];
+      }
+      asm volatile("bar.sync 3, 512;" ::: "memory");
+      if (grp == 0 && half == 0 && ok) {
+        const float gamma = *job.gamma;
+        const int n = (u - job.unit_begin) * TILE_ROWS + rw * 16 + (lane >> 1);
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+          if (m < a.M) {
+            const int tv = tot[m] + cb[m] - rowsum_s[m];
+            const float yv = __fmul_rn(static_cast<float>(tv), out_scale(gamma, absmax_s[m]));
+            const size_t o = static_cast<size_t>(m) * job.N + n;
+            if (a.out_dtype == BITRL_OUT_F32) static_cast<float*>(job.y)[o] = yv;
+            else static_cast<unsigned short*>(job.y)[o] = float_to_bf16_bits(yv);
+          }
+        }
+      }
+    }
+  }
+}
+
+// Host side: builds the work list split and launches.  `w`, `x`, `y` are host arrays of `count` entries.
+template <int NT>
+bitrl_status launch_gemv_multi_t(const GvmArgs& a, int grid, size_t smem, cudaStream_t st) {
+  BITRL_CUDA(cudaFuncSetAttribute(gemv_multi_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  static_cast<int>(smem)));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(GVM_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  BITRL_CUDA(cudaLaunchKernelEx(&cfg, gemv_multi_kernel<NT>, a));
+  count_launch(1);
+  return BITRL_OK;
+}
+
+template <int MT>
+bitrl_status launch_gemv_multi_dp4a_t(const GvmArgs& a, int grid, size_t smem, cudaStream_t st) {
+  BITRL_CUDA(cudaFuncSetAttribute(gemv_multi_dp4a_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  static_cast<int>(smem)));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(GVD_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  BITRL_CUDA(cudaLaunchKernelEx(&cfg, gemv_multi_dp4a_kernel<MT>, a));
+  count_launch(1);
+  return BITRL_OK;
+}
+
+inline int gvm_nt(int M) { return M <= 8 ? 8 : 16; }
+// Shared memory beside the ring: activations (+ barriers, reduction scratch, the group-combine buffer).
+inline size_t gvm_fixed_bytes(int M, int kmax) {
+  if (M <= 2) return static_cast<size_t>(M) * kmax + 1024 + 2 * 8 * 16 * 2 * sizeof(int);
+  return static_cast<size_t>(gvm_nt(M)) * (kmax + GVM_XPAD) + 1024;
+}
+
+// Ring depth (log2) that fits beside the activations, or -1.
+inline int gvm_depth_log2(int M, int kmax) {
+  for (int d = 3; d >= 1; --d)
+    if (gvm_fixed_bytes(M, kmax) + (static_cast<size_t>(GVM_SLOT_BYTES) + 16) * (1u << d) <= GVM_SMEM_BUDGET) return d;
+  return -1;
+}
+
+bitrl_status launch_gemv_multi(int count, const Linear* const* w, const void* const* x, void* const* y, int M,
+                               int out_dtype, cudaStream_t st) {
+  static thread_local GvmArgs a;  // 7 KB, kept off the stack
+  int kmax = 0, units = 0;
+  long long pieces = 0;
+  for (int j = 0; j < count; ++j) {
+    a.jobs[j] = GvmJob{w[j]->tiles, w[j]->gamma, static_cast<const unsigned short*>(x[j]), y[j], w[j]->N, w[j]->K,
+                       units, 0};
+    units += w[j]->N / TILE_ROWS;
+    pieces += static_cast<long long>(w[j]->N / TILE_ROWS) * (w[j]->K / TILE_K);
+    if (w[j]->K > kmax) kmax = w[j]->K;
+  }
+  const int dlog = gvm_depth_log2(M, kmax);
+  if (dlog < 0) return BITRL_ERR_SHAPE;
+  int grid = sm_count();
+  if (grid > GVM_MAX_CTAS) grid = GVM_MAX_CTAS;
+  if (grid > units) grid = units;
+  // Contiguous ranges of row tiles with about pieces/grid 4 KB pieces each.
+  {
+    int j = 0, u = 0;
+    long long done = 0;
+    a.unit_start[0] = 0;
+    for (int c = 0; c < grid; ++c) {
+      const long long target = pieces * (c + 1) / grid;
+      while (u < units && done < target) {
+        while (j + 1 < count && a.jobs[j + 1].unit_begin <= u) ++j;
+        done += a.jobs[j].K / TILE_K;
+        ++u;
+      }
+      a.unit_start[c + 1] = u;
+    }
+    a.unit_start[grid] = units;
+  }
+  a.njobs = count;
+  a.M = M;
+  a.out_dtype = out_dtype;
+  a.depth_log2 = dlog;
+  a.kmax = kmax;
+  const size_t smem = static_cast<size_t>(GVM_SLOT_BYTES + 16) * (1u << dlog) + gvm_fixed_bytes(M, kmax);
+  if (M == 1) return launch_gemv_multi_dp4a_t<1>(a, grid, smem, st);
+  if (M == 2) return launch_gemv_multi_dp4a_t<2>(a, grid, smem, st);
+  return gvm_nt(M) == 8 ? launch_gemv_multi_t<8>(a, grid, smem, st) : launch_gemv_multi_t<16>(a, grid, smem, st);
+}
+
+}  // namespace bitrl

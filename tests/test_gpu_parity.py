@@ -345,3 +345,50 @@ def test_argument_errors(oracle_mod, B):
     assert L.bitrl_quant_act(x.data_ptr(), 4, 200, x.data_ptr(), x.data_ptr(), None, st) == B.ERR_SHAPE
     B.poll_status()
     assert B.launch_count() > 0
+
+
+# ------------------------------------------------------------------------------ grouped streaming launch
+
+@pytest.mark.parametrize("M,out_dtype", [(1, 1), (2, 0), (3, 1), (8, 0), (16, 1)])
+def test_forward_multi_matches_oracle_and_single_calls(oracle_mod, B, M, out_dtype):
+    """Several independent layers in one launch: bit-identical to the oracle and to separate calls."""
+    specs = [(3840, 2560, 1001), (384, 256, 7), (2560, 6912, 1004), (128, 128, 6), (2560, 2560, 1002), (384, 256, 7)]
+    xs_cpu = {K: inputs.activations(M, K, 3100 + K + M) for K in {k for _, k, _ in specs}}
+    xs_gpu = {K: v.cuda() for K, v in xs_cpu.items()}
+    ws, xs, ys, refs = [], [], [], []
+    for N, K, seed in specs:
+        _, Wq, g, _, _, lin = layer(oracle_mod, B, N, K, seed)
+        ws.append(lin)
+        xs.append(xs_gpu[K])
+        ys.append(torch.full((M, N), 7.0, dtype=torch.float32 if out_dtype == 0 else torch.bfloat16, device="cuda"))
+        refs.append(oracle_mod.bitlinear(inputs.bf16_bits(xs_cpu[K]), Wq, g))
+    call = B.MultiCall(ws, xs, ys, out_dtype)
+    call.run()
+    call.run()
+    B.poll_status()
+    for lin, x, y, ref in zip(ws, xs, ys, refs):
+        single = B.bitlinear_forward(lin, x, out_dtype)
+        assert torch.equal(single, y)
+        if out_dtype == 0:
+            assert np.array_equal(y.cpu().numpy(), ref["y32"])
+            assert max_rel_err(y.cpu().numpy(), ref["y64"]) <= TOL_F32
+        else:
+            yb = gpu_bf16_bits(y)
+            assert np.array_equal(yb, ref["ybf16"])
+            assert max_rel_err(bits_to_f64(yb), ref["y64"]) <= TOL_BF16
+
+
+def test_forward_multi_argument_errors(oracle_mod, B):
+    import ctypes
+    L = B.lib()
+    _, _, _, _, _, lin = layer(oracle_mod, B, 384, 256, 7)
+    x = inputs.activations(2, 256, 1).cuda()
+    y = torch.empty(2, 384, dtype=torch.bfloat16, device="cuda")
+    vp = ctypes.c_void_p
+    w1, x1, y1 = (vp * 1)(lin.handle), (vp * 1)(x.data_ptr()), (vp * 1)(y.data_ptr())
+    assert L.bitrl_bitlinear_forward_multi(0, w1, x1, y1, 2, 1, None) == B.ERR_SHAPE
+    assert L.bitrl_bitlinear_forward_multi(1, w1, x1, y1, 17, 1, None) == B.ERR_SHAPE
+    assert L.bitrl_bitlinear_forward_multi(1, w1, x1, y1, 2, 9, None) == B.ERR_DTYPE
+    assert L.bitrl_bitlinear_forward_multi(1, w1, (vp * 1)(None), y1, 2, 1, None) == B.ERR_NULL
+    assert L.bitrl_bitlinear_forward_multi(1, w1, x1, y1, 2, 1, None) == B.OK
+    B.poll_status()
