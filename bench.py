@@ -2,11 +2,11 @@
 """Benchmark of the BitLinear W1.58A8 hot path on B200.
 
 Headline (the line's `value`): packed-weight GB/s of the M=1 streaming kernel over a whole ~2B-parameter
-backbone - one step = one decode pass over 30 blocks x {qkv, out, gate/up, down} = 120 launches streaming
-521 MB of packed ternary weights (4x the 126 MB L2, so every launch reads cold weights).
-Secondary figures in the same JSON line (`extra`): M=8 decode, the M=4096 tcgen05 GEMM (int8 TOPS), the
-30-block encoder forward (states/s); plus the CPU oracle timed on the host cores and the roofline fraction of
-the dominant kernel.
+backbone - one step = the sweep over 30 blocks x {qkv, out, gate/up, down} = 120 independent GEMVs streaming
+521 MB of packed ternary weights (4x the 126 MB L2, so all weights are read cold), issued as one grouped launch.
+Secondary figures in the same JSON line (`extra`): the same matrices as a chain of single launches, M=8, the
+M=4096 tcgen05 GEMM (int8 TOPS), the 30-block encoder forward (states/s); plus the CPU oracle timed on the host
+cores and the roofline fraction of the dominant kernel.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--layers L] [--sections ...]
 
@@ -251,18 +251,29 @@ def run_ours(args):
     layers = build_backbone(bitrl, n_layers)
     bytes_step = n_layers * packed_bytes_per_layer()
 
-    # ---------------- headline: decode pass, M = 1, whole backbone, one CUDA graph of 4 * n_layers launches
+    # ---------------- headline: the M = 1 sweep over every matrix of the backbone.  The 4 * n_layers GEMVs are
+    # independent (same activations, distinct weights), so they go through the grouped entry point: one launch of
+    # one persistent kernel per step.
     def decode_setup(M):
         xs = {k: inputs.activations(M, k, 2000 + M).to(dev) for k in (2560, 6912)}
         ys = [[torch.empty((M, n), dtype=torch.bfloat16, device=dev) for _, _, n in BLOCK] for _ in range(n_layers)]
+        ws = [layers[l][j] for l in range(n_layers) for j in range(len(BLOCK))]
+        xl = [xs[k] for _ in range(n_layers) for _, k, _ in BLOCK]
+        yl = [ys[l][j] for l in range(n_layers) for j in range(len(BLOCK))]
+        calls = [bitrl.MultiCall(ws[i:i + 128], xl[i:i + 128], yl[i:i + 128], bitrl.OUT_BF16)
+                 for i in range(0, len(ws), 128)]
 
-        def step():
+        def sweep():
+            for c in calls:
+                c.run()
+
+        def chain():  # the same matrices as one launch each, in stream order (programmatic dependent launch)
             for l in range(n_layers):
                 for j, (_, k, n) in enumerate(BLOCK):
                     bitrl.bitlinear_forward(layers[l][j], xs[k], bitrl.OUT_BF16, y=ys[l][j])
-        return xs, ys, step
+        return xs, ys, sweep, chain
 
-    xs1, ys1, step1 = decode_setup(1)
+    xs1, ys1, step1, chain1 = decode_setup(1)
     g1, launches1 = capture(step1)
     sampler = ClockSampler(local).start() if rank == 0 else None
     ms1 = time_graph(g1, args.steps, args.warmup, world)
@@ -295,12 +306,20 @@ def run_ours(args):
 
     extra, cpu = {}, None
     if rank == 0 and "decode8" in sections:
-        _, _, step8 = decode_setup(8)
-        g8, _ = capture(step8)
-        ms8 = time_graph(g8, args.steps, args.warmup, 1)
-        gb8 = bytes_step * args.steps / (ms8 * 1e-3) / 1e9
-        extra["decode_m8"] = {"GBps": gb8, "ms_per_step": ms8 / args.steps, "frac_of_hbm_peak": gb8 / peaks["hbm_gbs"]}
-        del g8
+        gc, lc = capture(chain1)
+        msc = time_graph(gc, args.steps, args.warmup, 1)
+        gbc = bytes_step * args.steps / (msc * 1e-3) / 1e9
+        extra["chain_m1_one_launch_per_matrix"] = {"GBps": gbc, "us_per_launch": msc * 1e3 / (args.steps * lc),
+                                                  "frac_of_hbm_peak": gbc / peaks["hbm_gbs"], "launches": lc}
+        del gc
+        _, _, step8, chain8 = decode_setup(8)
+        for label, fn in (("sweep_m8_grouped", step8), ("chain_m8_one_launch_per_matrix", chain8)):
+            g8, l8 = capture(fn)
+            ms8 = time_graph(g8, args.steps, args.warmup, 1)
+            gb8 = bytes_step * args.steps / (ms8 * 1e-3) / 1e9
+            extra[label] = {"GBps": gb8, "ms_per_step": ms8 / args.steps, "frac_of_hbm_peak": gb8 / peaks["hbm_gbs"],
+                            "launches": l8}
+            del g8
 
     if rank == 0 and "gemm" in sections:
         # M = 4096 GEMM, both judged shapes; weights rotate over several matrices, inputs over four buffers
@@ -366,15 +385,16 @@ def run_ours(args):
             "warmup": args.warmup, "ms_per_step": ms1 / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int8 x ternary(2-bit) -> int32", "data": "synthetic",
             "config": {"workload": f"configs[1]: decode GEMV sweep at M=1 over {n_layers} blocks x (2560->3840, "
-                                   "2560->2560, 2560->13824, 6912->2560) of a ~2B BitNet b1.58 backbone",
+                                   "2560->2560, 2560->13824, 6912->2560) of a ~2B BitNet b1.58 backbone; the "
+                                   f"{4 * n_layers} independent GEMVs of a step go through the grouped entry point",
                        "launches_per_step": launches1, "packed_bytes_per_step": bytes_step,
                        "l2": f"{bytes_step / 1e6:.0f} MB of distinct weights per step against a 126 MB L2: inputs "
                              "larger than L2, no flush needed",
-                       "timing": "CUDA graph of one step, CUDA events on the launching stream",
+                       "timing": "CUDA graph of one step (one grouped launch), CUDA events on the launching stream",
                        "parallelism": f"replicas x{world}, no collective"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": f"of {peak_src}",
-                         "kernel": "gemv_kernel<1>", "us_per_launch": us_per_launch,
+                         "kernel": "gemv_multi_dp4a_kernel<1>", "us_per_launch": us_per_launch,
                          "algorithmic_bytes_per_launch": bytes_step / launches1},
             "cpu_baseline": cpu,
             "e2e": {"value": e2e_gbs, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

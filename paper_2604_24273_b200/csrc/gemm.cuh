@@ -7,12 +7,13 @@
 // sum_k x_q[m,k] is subtracted in the epilogue.  All integer, exact.
 //
 // One persistent CTA per SM, 11 warps, three decoupled rings in shared memory:
-//   warp 0      X producer : TMA tile of x_q (256 tokens x 128 k, 128-byte swizzle)        ring of 4 x 32 KB
+//   warp 0      X producer : TMA tile of x_q (TOK tokens x 128 k, 128-byte swizzle)        ring of 128 KB
 //   warp 2      P producer : bulk copy of the 4 KB packed weight piece (128 rows x 128 k)    ring of 8 x 4 KB
 //   warps 3-6   expand     : packed piece -> int8 codes in the swizzled K-major layout       ring of 3 x 16 KB
 //   warp 1      MMA        : one thread issues tcgen05.mma kind::i8 (4 per k block, K = 32 each) into TMEM
 //   warps 7-10  epilogue   : TMEM -> registers -> (acc - rowsum) * gamma*a_m/127 -> bf16/fp32, transposed through
 //                            a per-warp shared-memory tile so that global stores are 16 bytes per lane
+// The token-tile width TOK (64..256) is chosen per launch to fill the SMs with whole waves.
 // Two 256-column accumulators in TMEM let the epilogue of tile i overlap the main loop of tile i+1.
 // Every mbarrier wait is bounded; on expiry the CTA records a status word and leaves through the normal exit.
 #pragma once
@@ -25,26 +26,26 @@
 namespace bitrl {
 
 constexpr int GM_ROWS = 128;  // weight rows per tile  (MMA M)
-constexpr int GM_TOK = 256;   // tokens per tile       (MMA N)
+constexpr int GM_TOK_MAX = 256;  // tokens per tile (MMA N) is a template parameter: 64, 128, 192 or 256
 constexpr int GM_BK = 128;    // k per pipeline stage  (one 128-byte swizzle row of int8)
-constexpr int GM_XS = 4;      // x_q ring depth
+constexpr uint32_t GM_X_RING_BYTES = 131072;  // x_q ring: as many (tokens x 128 k) stages as fit in 128 KB
 constexpr int GM_PS = 8;      // packed-weight ring depth
 constexpr int GM_WS = 3;      // expanded-weight ring depth
 constexpr int GM_THREADS = 352;
 constexpr int GM_EXPAND_WARP0 = 3;
 constexpr int GM_EPI_WARP0 = 7;
 
-constexpr uint32_t GM_X_BYTES = GM_TOK * GM_BK;   // 32768
 constexpr uint32_t GM_W_BYTES = GM_ROWS * GM_BK;  // 16384
 constexpr uint32_t GM_P_BYTES = TILE_BYTES;       // 4096
 constexpr uint32_t GM_STAGE_BYTES = 2048;         // per epilogue warp: 32 tokens x 32 rows bf16 (or 16 x 32 fp32)
 constexpr uint32_t GM_OFF_X = 0;
-constexpr uint32_t GM_OFF_W = GM_OFF_X + GM_XS * GM_X_BYTES;
+constexpr uint32_t GM_OFF_W = GM_OFF_X + GM_X_RING_BYTES;
 constexpr uint32_t GM_OFF_P = GM_OFF_W + GM_WS * GM_W_BYTES;
 constexpr uint32_t GM_OFF_STAGE = GM_OFF_P + GM_PS * GM_P_BYTES;
 constexpr uint32_t GM_OFF_TOK = GM_OFF_STAGE + 4 * GM_STAGE_BYTES;  // scale[2][256] f32, rowsum[2][256] i32
-constexpr uint32_t GM_OFF_BAR = GM_OFF_TOK + 2 * GM_TOK * 8;
-constexpr uint32_t GM_NUM_BARS = 2 * GM_XS + 2 * GM_PS + 2 * GM_WS + 4;
+constexpr uint32_t GM_OFF_BAR = GM_OFF_TOK + 2 * GM_TOK_MAX * 8;
+constexpr uint32_t GM_XS_MAX = 16;
+constexpr uint32_t GM_NUM_BARS = 2 * GM_XS_MAX + 2 * GM_PS + 2 * GM_WS + 4;
 constexpr uint32_t GM_OFF_MISC = GM_OFF_BAR + GM_NUM_BARS * 8;
 constexpr uint32_t GM_SMEM_BYTES = GM_OFF_MISC + 16 + 1024;  // + slack to align the base to 1024
 static_assert(GM_SMEM_BYTES <= 232448, "shared memory budget of one CTA");
@@ -66,8 +67,12 @@ struct GemmArgs {
   int tiles_n, tiles_total;
 };
 
+template <int GM_TOK>
 __global__ void __launch_bounds__(GM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
+  constexpr uint32_t GM_X_BYTES = GM_TOK * GM_BK;
+  constexpr uint32_t GM_XS = GM_X_RING_BYTES / GM_X_BYTES;  // 4 stages at 256 tokens, 5 at 192, 8 at 128, 16 at 64
+  static_assert(GM_TOK % 32 == 0 && GM_TOK >= 64 && GM_TOK <= GM_TOK_MAX && GM_XS <= GM_XS_MAX, "token tile");
   extern __shared__ unsigned char gm_smem_raw[];
   const uint32_t raw_addr = ptx::smem_u32(gm_smem_raw);
   const uint32_t base = (raw_addr + 1023u) & ~1023u;
@@ -147,7 +152,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
           report_timeout(GM_WAIT_TMEM_EMPTY); ok = false; break;
         }
         ptx::tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + buf * GM_TOK;
+        const uint32_t d_tmem = tmem_base + buf * GM_TOK_MAX;
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
           const uint32_t xs = it % GM_XS, xph = (it / GM_XS) & 1u;
           const uint32_t ws = it % GM_WS, wph = (it / GM_WS) & 1u;
@@ -212,8 +217,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x, ++lt) {
       const int tn = tile % a.tiles_n, tm = tile / a.tiles_n;
       const uint32_t buf = lt & 1u;
-      const uint32_t sc_addr = base + GM_OFF_TOK + buf * GM_TOK * 4;
-      const uint32_t rs_addr = base + GM_OFF_TOK + 2 * GM_TOK * 4 + buf * GM_TOK * 4;
+      const uint32_t sc_addr = base + GM_OFF_TOK + buf * GM_TOK_MAX * 4;
+      const uint32_t rs_addr = base + GM_OFF_TOK + 2 * GM_TOK_MAX * 4 + buf * GM_TOK_MAX * 4;
       for (int j = ep; j < GM_TOK; j += 128) {
         const int tok = tm * GM_TOK + j;
         ptx::sts32(sc_addr + 4 * j, __float_as_uint(tok < a.M ? out_scale(gamma, a.absmax[tok]) : 0.0f));
@@ -228,7 +233,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
       for (int c = 0; c < GM_TOK / 32; ++c) {
         if (c * 32 >= tok_hi) break;  // warp-uniform
         uint32_t v[32];
-        ptx::tmem_ld_32x32b_x32(tmem_base + buf * GM_TOK + c * 32 + (static_cast<uint32_t>(q * 32) << 16), v);
+        ptx::tmem_ld_32x32b_x32(tmem_base + buf * GM_TOK_MAX + c * 32 + (static_cast<uint32_t>(q * 32) << 16), v);
         ptx::tmem_ld_wait();
         // acc = D - rowsum (exact int32), y = acc * scale
 #pragma unroll
@@ -336,10 +341,25 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
                          void* y, int out_dtype, const void* residual, int32_t* acc_out, cudaStream_t st) {
   encode_tiled_fn encode = get_encode_tiled();
   if (!encode) return cuda_fail(cudaErrorSymbolNotFound);
+  // Token-tile width: fewest "waves x time per k block" over the SMs.  A k block costs 2*TOK cycles of tensor pipe,
+  // but not less than the expanders need for their 128 x 128 codes (about 330 cycles).
+  const int sms = sm_count();
+  const int tiles_n = w->N / GM_ROWS;
+  int tok = 256;
+  {
+    long long best = -1;
+    const int cand[4] = {256, 192, 128, 64};
+    for (int i = 0; i < 4; ++i) {
+      const long long tiles = static_cast<long long>(tiles_n) * ((M + cand[i] - 1) / cand[i]);
+      const long long waves = (tiles + sms - 1) / sms;
+      const long long cost = waves * (2 * cand[i] > 330 ? 2 * cand[i] : 330);
+      if (best < 0 || cost <= best) { best = cost; tok = cand[i]; }  // ties go to the narrower tile
+    }
+  }
   CUtensorMap tmap;
   const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(w->K), static_cast<cuuint64_t>(M)};
   const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(w->K)};
-  const cuuint32_t box[2] = {GM_BK, GM_TOK};
+  const cuuint32_t box[2] = {GM_BK, static_cast<cuuint32_t>(tok)};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(xq), gdim, gstride, box,
                             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -347,12 +367,14 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
   if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
 
   GemmArgs a{w->tiles, w->gamma, absmax, rowsum, M, w->N, w->K, y, out_dtype,
-             static_cast<const unsigned short*>(residual), acc_out, w->N / GM_ROWS, 0};
-  const int tiles_m = (M + GM_TOK - 1) / GM_TOK;
-  a.tiles_total = a.tiles_n * tiles_m;
-  BITRL_CUDA(cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM_BYTES));
-  const int grid = a.tiles_total < sm_count() ? a.tiles_total : sm_count();
-  gemm_i8_kernel<<<grid, GM_THREADS, GM_SMEM_BYTES, st>>>(tmap, a);
+             static_cast<const unsigned short*>(residual), acc_out, tiles_n, 0};
+  a.tiles_total = tiles_n * ((M + tok - 1) / tok);
+  const int grid = a.tiles_total < sms ? a.tiles_total : sms;
+  void (*kern)(const CUtensorMap, const GemmArgs) =
+      tok == 256 ? gemm_i8_kernel<256> : tok == 192 ? gemm_i8_kernel<192> : tok == 128 ? gemm_i8_kernel<128>
+                                                                                       : gemm_i8_kernel<64>;
+  BITRL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM_BYTES));
+  kern<<<grid, GM_THREADS, GM_SMEM_BYTES, st>>>(tmap, a);
   count_launch(1);
   BITRL_CUDA(cudaGetLastError());
   return BITRL_OK;
