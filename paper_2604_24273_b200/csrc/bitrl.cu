@@ -1,6 +1,7 @@
 // C-ABI entry points of the bitrl library (declared and documented in include/bitrl.h).  Host code here only
 // validates arguments, carves workspaces and launches the kernels of pack.cuh / quant.cuh / gemv.cuh / gemm.cuh.
 #include <atomic>
+#include <cstdlib>
 #include <new>
 #include <vector>
 
@@ -16,6 +17,16 @@ bitrl_status cuda_fail(cudaError_t e) {
   g_last_cuda.store(static_cast<int>(e));
   (void)cudaGetLastError();
   return BITRL_ERR_CUDA;
+}
+
+// Which operand path the GEMM uses for the expanded weights; BITRL_GEMM_A=smem selects the shared-memory one.
+bool gemm_a_in_tmem() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("BITRL_GEMM_A");
+    v = (e && e[0] == 's') ? 0 : 1;
+  }
+  return v == 1;
 }
 
 int sm_count() {

@@ -67,12 +67,16 @@ struct GemmArgs {
   int tiles_n, tiles_total;
 };
 
-template <int GM_TOK>
+template <int GM_TOK, bool A_TMEM>
 __global__ void __launch_bounds__(GM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   constexpr uint32_t GM_X_BYTES = GM_TOK * GM_BK;
   constexpr uint32_t GM_XS = GM_X_RING_BYTES / GM_X_BYTES;  // 4 stages at 256 tokens, 5 at 192, 8 at 128, 16 at 64
   static_assert(GM_TOK % 32 == 0 && GM_TOK >= 64 && GM_TOK <= GM_TOK_MAX && GM_XS <= GM_XS_MAX, "token tile");
+  // With the A operand in tensor memory the two accumulators sit at columns [0,TOK) and [256,256+TOK) and the ring
+  // of expanded weight slots (32 columns each) uses the columns they leave free: 192, 224, 448 (TOK <= 192).
+  static_assert(!A_TMEM || (GM_TOK <= 192 && GM_WS <= 3), "tensor-memory column budget");
+  static_assert(GM_WS <= GM_XS, "the expanders watch the x_q ring GM_WS steps behind");
   extern __shared__ unsigned char gm_smem_raw[];
   const uint32_t raw_addr = ptx::smem_u32(gm_smem_raw);
   const uint32_t base = (raw_addr + 1023u) & ~1023u;
@@ -92,9 +96,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   const int kblocks = a.K / GM_BK;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < GM_XS; ++s) { ptx::mbar_init(bar_x_full + 8 * s, 1); ptx::mbar_init(bar_x_empty + 8 * s, 1); }
+    for (int s = 0; s < GM_XS; ++s) { ptx::mbar_init(bar_x_full + 8 * s, 1 + 4); ptx::mbar_init(bar_x_empty + 8 * s, 1); }
     for (int s = 0; s < GM_PS; ++s) { ptx::mbar_init(bar_p_full + 8 * s, 1); ptx::mbar_init(bar_p_empty + 8 * s, 4); }
-    for (int s = 0; s < GM_WS; ++s) { ptx::mbar_init(bar_w_full + 8 * s, 4); ptx::mbar_init(bar_w_empty + 8 * s, 1); }
     for (int b = 0; b < 2; ++b) { ptx::mbar_init(bar_tmem_full + 8 * b, 1); ptx::mbar_init(bar_tmem_empty + 8 * b, 4); }
     ptx::mbar_init_fence();
     ptx::tma_prefetch_desc(&tmap_x);
@@ -144,64 +147,97 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = ptx::idesc_i8(GM_ROWS, GM_TOK, /*a_signed=*/false, /*b_signed=*/true);
-      uint32_t it = 0, lt = 0;
+      uint32_t lt = 0;
+      uint32_t xs = 0, xph = 0, ws = 0;  // ring slots and phase, advanced without divisions
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x, ++lt) {
         const uint32_t buf = lt & 1u;
         if (!ptx::mbar_wait(bar_tmem_empty + 8 * buf, ((lt >> 1) & 1u) ^ 1u)) {
           report_timeout(GM_WAIT_TMEM_EMPTY); ok = false; break;
         }
-        ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + buf * GM_TOK_MAX;
-        for (int kb = 0; kb < kblocks; ++kb, ++it) {
-          const uint32_t xs = it % GM_XS, xph = (it / GM_XS) & 1u;
-          const uint32_t ws = it % GM_WS, wph = (it / GM_WS) & 1u;
-          if (!ptx::mbar_wait(bar_w_full + 8 * ws, wph)) { report_timeout(GM_WAIT_W_FULL); ok = false; break; }
+        for (int kb = 0; kb < kblocks; ++kb) {
           if (!ptx::mbar_wait(bar_x_full + 8 * xs, xph)) { report_timeout(GM_WAIT_X_FULL); ok = false; break; }
           ptx::tc_fence_after_sync();
-          const uint64_t adesc = ptx::smem_desc_sw128(base + GM_OFF_W + ws * GM_W_BYTES);
           const uint64_t bdesc = ptx::smem_desc_sw128(base + GM_OFF_X + xs * GM_X_BYTES);
+          if (A_TMEM) {
+            const uint32_t a_tmem = tmem_base + (ws < 2 ? 192u + 32u * ws : 448u);
 #pragma unroll
-          for (int k4 = 0; k4 < GM_BK / 32; ++k4)
-            ptx::mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
-          ptx::mma_commit(bar_x_empty + 8 * xs);
-          ptx::mma_commit(bar_w_empty + 8 * ws);
+            for (int k4 = 0; k4 < GM_BK / 32; ++k4)
+              ptx::mma_i8_ts(d_tmem, a_tmem + 8 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+          } else {
+            const uint64_t adesc = ptx::smem_desc_sw128(base + GM_OFF_W + ws * GM_W_BYTES);
+#pragma unroll
+            for (int k4 = 0; k4 < GM_BK / 32; ++k4)
+              ptx::mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+          }
+          ptx::mma_commit(bar_x_empty + 8 * xs);  // frees the x_q slot and the weight slot of this k block
+          if (++xs == GM_XS) { xs = 0; xph ^= 1u; }
+          if (++ws == GM_WS) ws = 0;
         }
         if (ok) ptx::mma_commit(bar_tmem_full + 8 * buf);
       }
     }
   } else if (warp < GM_EPI_WARP0) {
     // ------------------------------------------------------------------ expanders (one weight row each)
-    const int r = threadIdx.x - GM_EXPAND_WARP0 * 32;
+    // Shared-memory A: any thread may expand any row.  Tensor-memory A: a warp can only write its own lane quarter
+    // (warp id mod 4), so its 32 lanes take the 32 rows of that quarter.
+    const int r = A_TMEM ? (warp & 3) * 32 + lane : threadIdx.x - GM_EXPAND_WARP0 * 32;
     const uint32_t row_off = static_cast<uint32_t>(r >> 3) * 1024u + static_cast<uint32_t>(r & 7) * 128u;
     const uint32_t sw = static_cast<uint32_t>(r & 7);
+    // The weight slot of k block `it` was last used by k block it - GM_WS; that MMA's completion is the arrival on
+    // x_empty of ITS x_q slot, so the expanders watch the x_q ring GM_WS steps behind (GM_WS <= GM_XS keeps the
+    // watched barrier at most one phase ahead).  Their "ready" arrival goes to x_full of the current x_q slot, which
+    // therefore completes when both the TMA bytes and the four expander warps are in: one wait per k block for the MMA.
     uint32_t it = 0;
+    uint32_t ps = 0, pph = 0, ws = 0, xs = 0, xs_old = 0, xph_old = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x) {
       for (int kb = 0; kb < kblocks; ++kb, ++it) {
-        const uint32_t ps = it % GM_PS, pph = (it / GM_PS) & 1u;
-        const uint32_t ws = it % GM_WS, wph = (it / GM_WS) & 1u;
         if (!ptx::mbar_wait(bar_p_full + 8 * ps, pph)) { report_timeout(GM_WAIT_P_FULL); ok = false; break; }
         const uint32_t paddr = base + GM_OFF_P + ps * GM_P_BYTES + r * TILE_ROW_BYTES;
         const uint4 p0 = ptx::lds128(paddr), p1 = ptx::lds128(paddr + 16);
-        if (!ptx::mbar_wait(bar_w_empty + 8 * ws, wph ^ 1u)) { report_timeout(GM_WAIT_W_EMPTY); ok = false; break; }
-        const uint32_t wd[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
-        const uint32_t wrow = base + GM_OFF_W + ws * GM_W_BYTES + row_off;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          uint4 c;
-          c.x = wd[j] & 0x03030303u;
-          c.y = (wd[j] >> 2) & 0x03030303u;
-          c.z = (wd[j] >> 4) & 0x03030303u;
-          c.w = (wd[j] >> 6) & 0x03030303u;
-          ptx::sts128(wrow + ((static_cast<uint32_t>(j) ^ sw) << 4), c);
+        if (it >= GM_WS) {
+          if (!ptx::mbar_wait(bar_x_empty + 8 * xs_old, xph_old)) { report_timeout(GM_WAIT_W_EMPTY); ok = false; break; }
+          if (++xs_old == GM_XS) { xs_old = 0; xph_old ^= 1u; }
         }
-        ptx::fence_proxy_async_smem();
+        if (A_TMEM) ptx::tc_fence_after_sync();
+        const uint32_t wd[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+        if (A_TMEM) {
+          // row r, k = 4c..4c+3 -> 32-bit column c of TMEM lane r: the whole 128-k slice is one 32-column store
+          uint32_t cols[32];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            cols[4 * j + 0] = wd[j] & 0x03030303u;
+            cols[4 * j + 1] = (wd[j] >> 2) & 0x03030303u;
+            cols[4 * j + 2] = (wd[j] >> 4) & 0x03030303u;
+            cols[4 * j + 3] = (wd[j] >> 6) & 0x03030303u;
+          }
+          ptx::tmem_st_32x32b_x32(tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) +
+                                      (ws < 2 ? 192u + 32u * ws : 448u), cols);
+          ptx::tmem_st_wait();
+          ptx::tc_fence_before_sync();
+        } else {
+          const uint32_t wrow = base + GM_OFF_W + ws * GM_W_BYTES + row_off;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            uint4 c;
+            c.x = wd[j] & 0x03030303u;
+            c.y = (wd[j] >> 2) & 0x03030303u;
+            c.z = (wd[j] >> 4) & 0x03030303u;
+            c.w = (wd[j] >> 6) & 0x03030303u;
+            ptx::sts128(wrow + ((static_cast<uint32_t>(j) ^ sw) << 4), c);
+          }
+          ptx::fence_proxy_async_smem();
+        }
         __syncwarp();
         if (lane == 0) {
-          ptx::mbar_arrive(bar_w_full + 8 * ws);
+          ptx::mbar_arrive(bar_x_full + 8 * xs);
           ptx::mbar_arrive(bar_p_empty + 8 * ps);
         }
+        if (++ps == GM_PS) { ps = 0; pph ^= 1u; }
+        if (++ws == GM_WS) ws = 0;
+        if (++xs == GM_XS) xs = 0;
       }
     }
   } else {
@@ -336,6 +372,7 @@ inline encode_tiled_fn get_encode_tiled() {
 }
 
 int sm_count();
+bool gemm_a_in_tmem();  // expanded weights through tensor memory (default) or through shared memory
 
 bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax, const int32_t* rowsum, int M,
                          void* y, int out_dtype, const void* residual, int32_t* acc_out, cudaStream_t st) {
@@ -370,9 +407,12 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
              static_cast<const unsigned short*>(residual), acc_out, tiles_n, 0};
   a.tiles_total = tiles_n * ((M + tok - 1) / tok);
   const int grid = a.tiles_total < sms ? a.tiles_total : sms;
+  const bool a_tmem = gemm_a_in_tmem() && tok <= 192;
   void (*kern)(const CUtensorMap, const GemmArgs) =
-      tok == 256 ? gemm_i8_kernel<256> : tok == 192 ? gemm_i8_kernel<192> : tok == 128 ? gemm_i8_kernel<128>
-                                                                                       : gemm_i8_kernel<64>;
+      tok == 256 ? gemm_i8_kernel<256, false>
+      : tok == 192 ? (a_tmem ? gemm_i8_kernel<192, true> : gemm_i8_kernel<192, false>)
+      : tok == 128 ? (a_tmem ? gemm_i8_kernel<128, true> : gemm_i8_kernel<128, false>)
+                   : (a_tmem ? gemm_i8_kernel<64, true> : gemm_i8_kernel<64, false>);
   BITRL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM_BYTES));
   kern<<<grid, GM_THREADS, GM_SMEM_BYTES, st>>>(tmap, a);
   count_launch(1);
