@@ -164,6 +164,10 @@ BITRL_API bitrl_status bitrl_encoder_forward(const bitrl_encoder_t* enc, const v
 /* Synchronizes `stream`, then reads and clears the device status word.  BITRL_OK, BITRL_ERR_TIMEOUT (a kernel
  * wait expired; results of that launch are invalid) or BITRL_ERR_CUDA. */
 BITRL_API bitrl_status bitrl_poll_status(void* stream);
+/* Self-test of the failure path: launches a one-thread kernel that waits (for at most `limit_cycles` SM cycles,
+ * clamped to [1e3, 1e9]) on a barrier that nothing ever signals, so the bounded wait expires and records stage 99.
+ * The next bitrl_poll_status returns BITRL_ERR_TIMEOUT; the context stays usable.  No GPU fault is involved. */
+BITRL_API bitrl_status bitrl_selftest_wait_timeout(int64_t limit_cycles, void* stream);
 /* After BITRL_ERR_TIMEOUT: which wait gave up (kernel-specific stage id), else 0. */
 BITRL_API int32_t bitrl_last_timeout_stage(void);
 BITRL_API int32_t bitrl_last_cuda_error(void);

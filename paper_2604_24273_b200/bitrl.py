@@ -49,6 +49,7 @@ EXPORTS = {
     "bitrl_encoder_destroy": (_i32, [_vp]),
     "bitrl_encoder_workspace_bytes": (_sz, [_vp, _i32]),
     "bitrl_encoder_forward": (_i32, [_vp, _vp, _i32, _vp, _vp, _sz, _vp]),
+    "bitrl_selftest_wait_timeout": (_i32, [ctypes.c_int64, _vp]),
     "bitrl_poll_status": (_i32, [_vp]),
     "bitrl_last_timeout_stage": (_i32, []),
     "bitrl_last_cuda_error": (_i32, []),

@@ -418,6 +418,29 @@ bitrl_status bitrl_encoder_forward(const bitrl_encoder_t* enc, const void* h_in,
   return BITRL_OK;
 }
 
+// ---- self-test of the bounded-wait / status-word path ----
+}  // extern "C"
+namespace {
+__global__ void selftest_wait_kernel(long long limit_cycles) {
+  __shared__ __align__(8) unsigned long long bar;
+  const uint32_t b = ptx::smem_u32(&bar);
+  ptx::mbar_init(b, 1);
+  ptx::mbar_init_fence();
+  if (!ptx::mbar_wait(b, 0, limit_cycles)) report_timeout(99);  // nobody arrives: the wait must give up
+}
+}  // namespace
+extern "C" {
+
+bitrl_status bitrl_selftest_wait_timeout(int64_t limit_cycles, void* stream) {
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  long long lim = limit_cycles < 1000 ? 1000 : (limit_cycles > 1000000000LL ? 1000000000LL : limit_cycles);
+  selftest_wait_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(lim);
+  count_launch(1);
+  BITRL_CUDA(cudaGetLastError());
+  return BITRL_OK;
+}
+
 // ---- status -------------------------------------------------------------------------------------------
 
 bitrl_status bitrl_poll_status(void* stream) {

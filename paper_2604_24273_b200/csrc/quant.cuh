@@ -145,8 +145,158 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_kernel(RowArgs a) {
   }
 }
 
+// Register-resident variant: WPR warps share one row and every lane keeps its (up to) 7 groups of 8 values in
+// registers across the three passes, so the row is read from global memory exactly once and no pass goes through
+// shared memory; only the three scalar reductions cross warps.  8 / WPR rows per CTA.
+constexpr int ROWQ_MAXG = 7;
+
+template <int MODE, int WPR>
+__global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, int T) {
+  __shared__ float red_ss[ROW_THREADS / 32];
+  __shared__ float red_mx[ROW_THREADS / 32];
+  __shared__ int red_rs[ROW_THREADS / 32];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int sub = warp % WPR, grp = warp / WPR;
+  const long long row = static_cast<long long>(blockIdx.x) * (ROW_THREADS / 32 / WPR) + grp;
+  const bool live = row < T;
+  const int nvec8 = a.Kv >> 3;
+  const unsigned short* src = a.in + (live ? row : 0) * a.in_stride + a.in_offset;
+
+  float v[ROWQ_MAXG][8];
+  float ss = 0.0f;
+#pragma unroll
+  for (int gi = 0; gi < ROWQ_MAXG; ++gi) {
+    const int i = (gi * WPR + sub) * 32 + lane;
+    if (live && i < nvec8) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(src + 8 * i);
+      const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        v[gi][2 * e] = __uint_as_float(rw[e] << 16);
+        v[gi][2 * e + 1] = __uint_as_float(rw[e] & 0xffff0000u);
+      }
+      if (MODE == ROW_RELU2) {
+        const uint4 rawu = *reinterpret_cast<const uint4*>(src + a.gate_offset + 8 * i);
+        const uint32_t ru[4] = {rawu.x, rawu.y, rawu.z, rawu.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float g0 = fmaxf(v[gi][2 * e], 0.0f), g1 = fmaxf(v[gi][2 * e + 1], 0.0f);
+          v[gi][2 * e] = __fmul_rn(__fmul_rn(g0, g0), __uint_as_float(ru[e] << 16));
+          v[gi][2 * e + 1] = __fmul_rn(__fmul_rn(g1, g1), __uint_as_float(ru[e] & 0xffff0000u));
+        }
+      }
+      if (MODE != ROW_PLAIN) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) ss += v[gi][e] * v[gi][e];
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[gi][e] = 0.0f;
+    }
+  }
+
+  float amax = 0.0f;
+  if (MODE != ROW_PLAIN) {
+    ss = warp_sum(ss);
+    if (WPR > 1) {
+      if (lane == 0) red_ss[warp] = ss;
+      __syncthreads();
+      ss = 0.0f;
+#pragma unroll
+      for (int i = 0; i < WPR; ++i) ss += red_ss[grp * WPR + i];
+    }
+    const float rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(ss, static_cast<float>(a.Kv)), 1e-5f)));
+#pragma unroll
+    for (int gi = 0; gi < ROWQ_MAXG; ++gi)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        v[gi][e] = bf16_bits_to_float(float_to_bf16_bits(__fmul_rn(v[gi][e], rstd)));
+        amax = fmaxf(amax, fabsf(v[gi][e]));
+      }
+  } else {
+#pragma unroll
+    for (int gi = 0; gi < ROWQ_MAXG; ++gi)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(v[gi][e]));
+  }
+  amax = warp_max(amax);
+  if (WPR > 1) {
+    if (lane == 0) red_mx[warp] = amax;
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < WPR; ++i) amax = fmaxf(amax, red_mx[grp * WPR + i]);
+  }
+  amax = fmaxf(amax, 1e-5f);
+  const float inv = __fdiv_rn(127.0f, amax);
+
+  int rs = 0;
+  int8_t* xq = a.xq + (live ? row : 0) * a.Kout;
+  unsigned short* uo = a.u_out ? a.u_out + (live ? row : 0) * a.Kout : nullptr;
+#pragma unroll
+  for (int gi = 0; gi < ROWQ_MAXG; ++gi) {
+    const int i = (gi * WPR + sub) * 32 + lane;
+    if (live && i < nvec8) {
+      int q[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) { q[e] = quant_code(v[gi][e], inv); rs += q[e]; }
+      uint2 wd;
+      wd.x = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | (static_cast<uint32_t>(q[3]) << 24);
+      wd.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | (static_cast<uint32_t>(q[7]) << 24);
+      uint4 ub;
+      if (uo) {
+        ub.x = static_cast<uint32_t>(float_to_bf16_bits(v[gi][0])) | (static_cast<uint32_t>(float_to_bf16_bits(v[gi][1])) << 16);
+        ub.y = static_cast<uint32_t>(float_to_bf16_bits(v[gi][2])) | (static_cast<uint32_t>(float_to_bf16_bits(v[gi][3])) << 16);
+        ub.z = static_cast<uint32_t>(float_to_bf16_bits(v[gi][4])) | (static_cast<uint32_t>(float_to_bf16_bits(v[gi][5])) << 16);
+        ub.w = static_cast<uint32_t>(float_to_bf16_bits(v[gi][6])) | (static_cast<uint32_t>(float_to_bf16_bits(v[gi][7])) << 16);
+      }
+      if (MODE == ROW_VREPEAT) {
+        const int k = 8 * i;
+        const int kvh = k / a.head_dim, e0 = k - kvh * a.head_dim;
+        for (int r = 0; r < a.rep; ++r) {
+          const int ko = (kvh * a.rep + r) * a.head_dim + e0;
+          *reinterpret_cast<uint2*>(xq + ko) = wd;
+          if (uo) *reinterpret_cast<uint4*>(uo + ko) = ub;
+        }
+      } else {
+        *reinterpret_cast<uint2*>(xq + 8 * i) = wd;
+        if (uo) *reinterpret_cast<uint4*>(uo + 8 * i) = ub;
+      }
+    }
+  }
+  rs = warp_sum_i(rs);
+  if (WPR > 1) {
+    if (lane == 0) red_rs[warp] = rs;
+    __syncthreads();
+    rs = 0;
+#pragma unroll
+    for (int i = 0; i < WPR; ++i) rs += red_rs[grp * WPR + i];
+  }
+  if (live && sub == 0 && lane == 0) {
+    a.absmax[row] = amax;
+    if (a.rowsum) a.rowsum[row] = rs * a.rep;
+  }
+}
+
+template <int MODE, int WPR>
+bitrl_status launch_row_reg(const RowArgs& a, int T, cudaStream_t st) {
+  const int rows_per_cta = ROW_THREADS / 32 / WPR;
+  row_quant_reg_kernel<MODE, WPR><<<(T + rows_per_cta - 1) / rows_per_cta, ROW_THREADS, 0, st>>>(a, T);
+  count_launch(1);
+  BITRL_CUDA(cudaGetLastError());
+  return BITRL_OK;
+}
+
 template <int MODE>
 bitrl_status launch_row(const RowArgs& a, int T, cudaStream_t st) {
+  // Rows of up to 8 * 32 * 7 * 8 = 14336 values fit the register-resident kernel (head_dim a multiple of 8 keeps
+  // the 8-value groups of the V-repeat producer inside one head).
+  const int nvec8 = a.Kv >> 3;
+  if (a.Kv % 8 == 0 && a.head_dim % 8 == 0) {
+    if (nvec8 <= 32 * ROWQ_MAXG) return launch_row_reg<MODE, 1>(a, T, st);
+    if (nvec8 <= 64 * ROWQ_MAXG) return launch_row_reg<MODE, 2>(a, T, st);
+    if (nvec8 <= 128 * ROWQ_MAXG) return launch_row_reg<MODE, 4>(a, T, st);
+    if (nvec8 <= 256 * ROWQ_MAXG) return launch_row_reg<MODE, 8>(a, T, st);
+  }
   const size_t smem = static_cast<size_t>(a.Kv) * sizeof(float);
   if (smem > 40 * 1024) {
     BITRL_CUDA(cudaFuncSetAttribute(row_quant_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -392,3 +392,16 @@ def test_forward_multi_argument_errors(oracle_mod, B):
     assert L.bitrl_bitlinear_forward_multi(1, w1, (vp * 1)(None), y1, 2, 1, None) == B.ERR_NULL
     assert L.bitrl_bitlinear_forward_multi(1, w1, x1, y1, 2, 1, None) == B.OK
     B.poll_status()
+
+
+def test_bounded_wait_reports_timeout_and_context_survives(oracle_mod, B):
+    """A device-side wait that nothing satisfies gives up after its limit, the host reads BITRL_ERR_TIMEOUT with the
+    stage id, the status word is cleared, and the next real call works (no trap, no hang, no fault)."""
+    L = B.lib()
+    B.poll_status()
+    assert L.bitrl_selftest_wait_timeout(200000, None) == B.OK
+    with pytest.raises(B.BitrlError) as e:
+        B.poll_status()
+    assert e.value.status == B.ERR_TIMEOUT and L.bitrl_last_timeout_stage() == 99
+    B.poll_status()  # cleared
+    check_layer(oracle_mod, B, 2, 256, 384, 7, 2999, 1)
