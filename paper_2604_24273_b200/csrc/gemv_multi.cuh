@@ -406,10 +406,13 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
               const int k0 = (kb + pidx) * TILE_K + half * 64;
 #pragma unroll
               for (int jw = 0; jw < 4; ++jw) {
+                // The codes are left at their bit positions (c1 * 4, c2 * 16, c3 * 64 still fit an unsigned byte):
+                // four masks and no shifts.  Accumulator i then holds 4^i times its share of the dot product and is
+                // scaled back by an exact shift once per row tile.
                 const uint32_t c0 = wword[jw] & 0x03030303u;
-                const uint32_t c1 = (wword[jw] >> 2) & 0x03030303u;
-                const uint32_t c2 = (wword[jw] >> 4) & 0x03030303u;
-                const uint32_t c3 = (wword[jw] >> 6) & 0x03030303u;
+                const uint32_t c1 = wword[jw] & 0x0c0c0c0cu;
+                const uint32_t c2 = wword[jw] & 0x30303030u;
+                const uint32_t c3 = wword[jw] & 0xc0c0c0c0u;
 #pragma unroll
                 for (int m = 0; m < MT; ++m) {
                   const int4 xv = *reinterpret_cast<const int4*>(xq_s + m * K + k0 + 16 * jw);
@@ -430,7 +433,7 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
       int tot[MT];
 #pragma unroll
       for (int m = 0; m < MT; ++m) {
-        tot[m] = acc[m][0] + acc[m][1] + acc[m][2] + acc[m][3];
+        tot[m] = acc[m][0] + (acc[m][1] >> 2) + (acc[m][2] >> 4) + (acc[m][3] >> 6);  // exact: multiples of 4^i
         tot[m] += __shfl_xor_sync(0xffffffffu, tot[m], 1);
         if (grp == 1 && half == 0) cb[m] = tot[m];
       }
