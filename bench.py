@@ -37,6 +37,10 @@ BLOCK = [("qkv", 2560, 3840), ("out", 2560, 2560), ("gateup", 2560, 13824), ("do
 FULL_LAYERS = 30
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 INT8_OVER_BF16 = 2.0  # nominal dense int8 : bf16 tensor throughput on B200 (4.5 : 2.25 PFLOP/s)
+# DRAM bytes (read + write) of one gemv_multi_dp4a_kernel<1> launch per backbone block, from the ncu capture summarised
+# in profiles/gemv_multi_dp4a_m1_8blocks.md (8 blocks: 138.995 MB read + 4.238 MB written); every weight byte is read
+# exactly once, so traffic scales with the number of blocks.  Set to None whenever that kernel changes.
+HEADLINE_TRAFFIC_PER_BLOCK = (138.995456e6 + 4.237568e6) / 8
 
 
 def load_peaks():
@@ -393,7 +397,8 @@ def run_ours(args):
                        "timing": "CUDA graph of one step (one grouped launch), CUDA events on the launching stream",
                        "parallelism": f"replicas x{world}, no collective"},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": f"of {peak_src}",
+                         "frac": achieved / peaks["hbm_gbs"],
+                         "traffic": None if HEADLINE_TRAFFIC_PER_BLOCK is None else HEADLINE_TRAFFIC_PER_BLOCK * n_layers, "peak_source": f"of {peak_src}",
                          "kernel": "gemv_multi_dp4a_kernel<1>", "us_per_launch": us_per_launch,
                          "algorithmic_bytes_per_launch": bytes_step / launches1},
             "cpu_baseline": cpu,
