@@ -37,9 +37,9 @@ BLOCK = [("qkv", 2560, 3840), ("out", 2560, 2560), ("gateup", 2560, 13824), ("do
 FULL_LAYERS = 30
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 INT8_OVER_BF16 = 2.0  # nominal dense int8 : bf16 tensor throughput on B200 (4.5 : 2.25 PFLOP/s)
-# DRAM bytes (read + write) of one gemv_multi_dp4a_kernel<1> launch per backbone block, from the ncu capture summarised
-# in profiles/gemv_multi_dp4a_m1_8blocks.md (8 blocks: 138.995 MB read + 4.238 MB written); every weight byte is read
-# exactly once, so traffic scales with the number of blocks.  Set to None whenever that kernel changes.
+# DRAM bytes (read + write) of one gemv_multi_dp4a_kernel<1> launch per backbone block, from an ncu capture of the
+# 8-block case (dram__bytes_read.sum 138.995 MB + dram__bytes_write.sum 4.238 MB); every weight byte is read exactly
+# once, so traffic scales with the number of blocks.  Set to None whenever that kernel changes.
 HEADLINE_TRAFFIC_PER_BLOCK = (138.995456e6 + 4.237568e6) / 8
 
 
