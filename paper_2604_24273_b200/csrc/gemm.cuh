@@ -6,10 +6,10 @@
 // C = W_q + 1 in {0,1,2} is fed as UNSIGNED bytes (decode = shift + mask), x_q as signed bytes; the surplus
 // sum_k x_q[m,k] is subtracted in the epilogue.  All integer, exact.
 //
-// One persistent CTA per SM, 11 warps, three decoupled rings in shared memory:
+// One persistent CTA per SM, 15 warps, three decoupled rings in shared memory:
 //   warp 0      X producer : TMA tile of x_q (TOK tokens x 128 k, 128-byte swizzle)        ring of 128 KB
 //   warp 2      P producer : bulk copy of the 4 KB packed weight piece (128 rows x 128 k)    ring of 8 x 4 KB
-//   warps 3-6   expand     : packed piece -> int8 codes in the swizzled K-major layout       ring of 3 x 16 KB
+//   warps 3-6, 11-14 expand: packed piece -> int8 codes in the swizzled K-major layout       ring of 3 x 16 KB
 //   warp 1      MMA        : one thread issues tcgen05.mma kind::i8 (4 per k block, K = 32 each) into TMEM
 //   warps 7-10  epilogue   : TMEM -> registers -> (acc - rowsum) * gamma*a_m/127 -> bf16/fp32, transposed through
 //                            a per-warp shared-memory tile so that global stores are 16 bytes per lane
@@ -31,7 +31,8 @@ constexpr int GM_BK = 128;    // k per pipeline stage  (one 128-byte swizzle row
 constexpr uint32_t GM_X_RING_BYTES = 131072;  // x_q ring: as many (tokens x 128 k) stages as fit in 128 KB
 constexpr int GM_PS = 8;      // packed-weight ring depth
 constexpr int GM_WS = 3;      // expanded-weight ring depth
-constexpr int GM_THREADS = 352;
+constexpr int GM_THREADS = 480;  // 15 warps: 3 single-thread roles, 2 x 4 expander warps, 4 epilogue warps
+constexpr int GM_EXPAND2_WARP0 = 11;  // second expander group
 constexpr int GM_EXPAND_WARP0 = 3;
 constexpr int GM_EPI_WARP0 = 7;
 
@@ -76,7 +77,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   // With the A operand in tensor memory the two accumulators sit at columns [0,TOK) and [256,256+TOK) and the ring
   // of expanded weight slots (32 columns each) uses the columns they leave free: 192, 224, 448 (TOK <= 192).
   static_assert(!A_TMEM || (GM_TOK <= 192 && GM_WS <= 3), "tensor-memory column budget");
-  static_assert(GM_WS <= GM_XS, "the expanders watch the x_q ring GM_WS steps behind");
+  static_assert(GM_WS < GM_XS, "the expanders watch the x_q ring GM_WS steps behind; a watched barrier must not flip twice");
   extern __shared__ unsigned char gm_smem_raw[];
   const uint32_t raw_addr = ptx::smem_u32(gm_smem_raw);
   const uint32_t base = (raw_addr + 1023u) & ~1023u;
@@ -178,11 +179,15 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
         if (ok) ptx::mma_commit(bar_tmem_full + 8 * buf);
       }
     }
-  } else if (warp < GM_EPI_WARP0) {
+  } else if (warp < GM_EPI_WARP0 || warp >= GM_EXPAND2_WARP0) {
     // ------------------------------------------------------------------ expanders (one weight row each)
+    // Two groups of four warps alternate k blocks (group 0 the even ones, group 1 the odd ones): one group needs
+    // longer for a block than the tensor pipe does, two keep ahead of it.
+    const uint32_t grp = warp >= GM_EXPAND2_WARP0 ? 1u : 0u;
     // Shared-memory A: any thread may expand any row.  Tensor-memory A: a warp can only write its own lane quarter
     // (warp id mod 4), so its 32 lanes take the 32 rows of that quarter.
-    const int r = A_TMEM ? (warp & 3) * 32 + lane : threadIdx.x - GM_EXPAND_WARP0 * 32;
+    const int r = A_TMEM ? (warp & 3) * 32 + lane
+                         : static_cast<int>(threadIdx.x) - (grp ? GM_EXPAND2_WARP0 : GM_EXPAND_WARP0) * 32;
     const uint32_t row_off = static_cast<uint32_t>(r >> 3) * 1024u + static_cast<uint32_t>(r & 7) * 128u;
     const uint32_t sw = static_cast<uint32_t>(r & 7);
     // The weight slot of k block `it` was last used by k block it - GM_WS; that MMA's completion is the arrival on
@@ -194,6 +199,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x) {
       for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        if ((it & 1u) != grp) {  // the other group's k block: only advance the ring positions
+          if (it >= GM_WS && ++xs_old == GM_XS) { xs_old = 0; xph_old ^= 1u; }
+          if (++ps == GM_PS) { ps = 0; pph ^= 1u; }
+          if (++ws == GM_WS) ws = 0;
+          if (++xs == GM_XS) xs = 0;
+          continue;
+        }
         if (!ptx::mbar_wait(bar_p_full + 8 * ps, pph)) { report_timeout(GM_WAIT_P_FULL); ok = false; break; }
         const uint32_t paddr = base + GM_OFF_P + ps * GM_P_BYTES + r * TILE_ROW_BYTES;
         const uint4 p0 = ptx::lds128(paddr), p1 = ptx::lds128(paddr + 16);
