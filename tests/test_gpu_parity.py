@@ -405,3 +405,51 @@ def test_bounded_wait_reports_timeout_and_context_survives(oracle_mod, B):
     assert e.value.status == B.ERR_TIMEOUT and L.bitrl_last_timeout_stage() == 99
     B.poll_status()  # cleared
     check_layer(oracle_mod, B, 2, 256, 384, 7, 2999, 1)
+
+
+# ------------------------------------------------------------------------------------ less common code paths
+
+def test_gemv_k_beyond_prefetch_window(oracle_mod, B):
+    """K > 7168: the streaming kernel leaves its register prefetch window and streams the remaining k blocks."""
+    for M in (1, 5):
+        check_layer(oracle_mod, B, M, 7680, 128, 31, 3300 + M, 1)
+    check_layer(oracle_mod, B, 2, 13824, 256, 32, 3310, 0)
+
+
+def test_forward_multi_large_k_and_many_jobs(oracle_mod, B):
+    M = 4
+    specs = [(128, 7680, 31), (256, 13824, 32)] + [(128, 128, 6)] * 20
+    xs_cpu = {K: inputs.activations(M, K, 3400 + K) for K in {k for _, k, _ in specs}}
+    xs_gpu = {K: v.cuda() for K, v in xs_cpu.items()}
+    ws, xs, ys = [], [], []
+    for N, K, seed in specs:
+        _, Wq, g, _, _, lin = layer(oracle_mod, B, N, K, seed)
+        ws.append(lin)
+        xs.append(xs_gpu[K])
+        ys.append(torch.zeros((M, N), dtype=torch.bfloat16, device="cuda"))
+    B.MultiCall(ws, xs, ys, B.OUT_BF16).run()
+    B.poll_status()
+    for (N, K, seed), y in zip(specs, ys):
+        _, Wq, g, _, _, _ = layer(oracle_mod, B, N, K, seed)
+        ref = oracle_mod.bitlinear(inputs.bf16_bits(xs_cpu[K]), Wq, g)
+        assert np.array_equal(gpu_bf16_bits(y), ref["ybf16"])
+
+
+def test_row_producers_generic_path(oracle_mod, B):
+    """Rows longer than the register-resident producer handles (> 14336 values) take the shared-memory kernel."""
+    T, K = 3, 16384
+    h = inputs.activations(T, K, 3500)
+    xq, a, rs, u = B.rmsnorm_quant(h.cuda(), want_u=True)
+    B.poll_status()
+    check_producer(oracle_mod, xq, a, rs, u, oracle_mod.rmsnorm_bf16(inputs.bf16_bits(h)))
+    xq2, a2, rs2 = B.quant_act(h.cuda())
+    xq_o, a_o = oracle_mod.quant_act(inputs.bf16_bits(h))
+    assert np.array_equal(xq2.cpu().numpy(), xq_o) and np.array_equal(a2.cpu().numpy(), a_o)
+
+
+def test_gemm_token_tile_variants(oracle_mod, B):
+    """Shapes that make the launcher pick each token-tile width (64, 128, 192, 256) and both weight paths."""
+    check_layer(oracle_mod, B, 40, 640, 128, 8, 3600, 1)        # 64
+    check_layer(oracle_mod, B, 256, 2560, 6912, 1005, 3601, 1)  # 128
+    check_layer(oracle_mod, B, 300, 2560, 6912, 1005, 3602, 1)  # 192
+    check_layer(oracle_mod, B, 1100, 256, 384, 7, 3603, 0)      # fp32 output through the GEMM epilogue
