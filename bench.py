@@ -72,7 +72,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -307,6 +307,7 @@ def run_ours(args):
     e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3, world)
     e2e_gbs = world * bytes_step * args.steps / (e2e_ms * 1e-3) / 1e9
     clocks = sampler.stop() if sampler else None
+    sampler2 = ClockSampler(local).start() if rank == 0 else None  # clocks during the secondary sections
 
     extra, cpu = {}, None
     if rank == 0 and "decode8" in sections:
@@ -379,6 +380,7 @@ def run_ours(args):
             "frac_of_int8_peak_sustained": enc_ops / (mse * 1e-3) / 1e12 / i8_sus, "launches": le}
         del ge
     bitrl.poll_status()
+    clocks_sections = sampler2.stop() if sampler2 else None
     if rank == 0 and "cpu" in sections:
         cpu = oracle_decode_sample()
 
@@ -406,6 +408,7 @@ def run_ours(args):
                     "ms_per_step": e2e_ms / args.steps},
             "gpu_launches": launches1 * args.steps,
             "clocks": clocks,
+            "clocks_secondary_sections": clocks_sections,
             "extra": extra,
         }
         print(json.dumps(line))
@@ -416,7 +419,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=FULL_LAYERS, help="blocks in the backbone (30 = full model)")
