@@ -29,6 +29,17 @@ bool gemm_a_in_tmem() {
   return v == 1;
 }
 
+// BITRL_GEMM_TOK=<64|128|192|224|256> overrides the launcher's choice of token-tile width (for tuning runs).
+int gemm_forced_tok() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("BITRL_GEMM_TOK");
+    const int t = e ? atoi(e) : 0;
+    v = (t == 64 || t == 128 || t == 192 || t == 224 || t == 256) ? t : 0;
+  }
+  return v;
+}
+
 int sm_count() {
   static int cached[64] = {0};
   int dev = 0;

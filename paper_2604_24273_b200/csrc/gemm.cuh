@@ -72,12 +72,18 @@ template <int GM_TOK, bool A_TMEM>
 __global__ void __launch_bounds__(GM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   constexpr uint32_t GM_X_BYTES = GM_TOK * GM_BK;
-  constexpr uint32_t GM_XS = GM_X_RING_BYTES / GM_X_BYTES;  // 4 stages at 256 tokens, 5 at 192, 8 at 128, 16 at 64
+  // x_q ring: 128 KB, plus the 48 KB of the shared-memory weight ring when the weights go through tensor memory
+  // (4 stages at 256 tokens, 6 at 224, 7 at 192, 11 at 128, 16 at 64).
+  constexpr uint32_t GM_X_RING = A_TMEM ? GM_OFF_P - GM_OFF_X : GM_X_RING_BYTES;
+  constexpr uint32_t GM_XS = GM_X_RING / GM_X_BYTES < GM_XS_MAX ? GM_X_RING / GM_X_BYTES : GM_XS_MAX;
   static_assert(GM_TOK % 32 == 0 && GM_TOK >= 64 && GM_TOK <= GM_TOK_MAX && GM_XS <= GM_XS_MAX, "token tile");
-  // With the A operand in tensor memory the two accumulators sit at columns [0,TOK) and [256,256+TOK) and the ring
-  // of expanded weight slots (32 columns each) uses the columns they leave free: 192, 224, 448 (TOK <= 192).
-  static_assert(!A_TMEM || (GM_TOK <= 192 && GM_WS <= 3), "tensor-memory column budget");
-  static_assert(GM_WS < GM_XS, "the expanders watch the x_q ring GM_WS steps behind; a watched barrier must not flip twice");
+  // With the A operand in tensor memory the two accumulators sit at columns [0,TOK) and [256,256+TOK).
+  // Weight slots in tensor memory are the 32-column pieces between the end of each accumulator and the next multiple
+  // of 256: slot i sits behind accumulator (i & 1), piece i / 2.  TOK = 224 leaves two slots, TOK <= 192 four.
+  constexpr uint32_t WSK = !A_TMEM ? GM_WS : ((256 - GM_TOK) / 32 >= 2 ? 4 : 2 * ((256 - GM_TOK) / 32));
+  static_assert(!A_TMEM || (GM_TOK <= 224 && WSK >= 2), "tensor-memory column budget");
+  static_assert(WSK < GM_XS, "the expanders watch the x_q ring WSK steps behind; a watched barrier must not flip twice");
+  auto a_slot = [](uint32_t slot) { return (slot & 1u) * 256u + GM_TOK + 32u * (slot >> 1); };
   extern __shared__ unsigned char gm_smem_raw[];
   const uint32_t raw_addr = ptx::smem_u32(gm_smem_raw);
   const uint32_t base = (raw_addr + 1023u) & ~1023u;
@@ -157,12 +163,15 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
           report_timeout(GM_WAIT_TMEM_EMPTY); ok = false; break;
         }
         const uint32_t d_tmem = tmem_base + buf * GM_TOK_MAX;
+        ptx::tc_fence_after_sync();  // orders this tile's MMAs after the epilogue's reads of the accumulator
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!ptx::mbar_wait(bar_x_full + 8 * xs, xph)) { report_timeout(GM_WAIT_X_FULL); ok = false; break; }
-          ptx::tc_fence_after_sync();
+          // Weights written with tcgen05.st by other threads need the tcgen05 fence on this side of the barrier;
+          // TMA data and expander stores to shared memory (already fenced into the async proxy by their writers) do not.
+          if (A_TMEM) ptx::tc_fence_after_sync();
           const uint64_t bdesc = ptx::smem_desc_sw128(base + GM_OFF_X + xs * GM_X_BYTES);
           if (A_TMEM) {
-            const uint32_t a_tmem = tmem_base + (ws < 2 ? 192u + 32u * ws : 448u);
+            const uint32_t a_tmem = tmem_base + a_slot(ws);
 #pragma unroll
             for (int k4 = 0; k4 < GM_BK / 32; ++k4)
               ptx::mma_i8_ts(d_tmem, a_tmem + 8 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
@@ -174,7 +183,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
           }
           ptx::mma_commit(bar_x_empty + 8 * xs);  // frees the x_q slot and the weight slot of this k block
           if (++xs == GM_XS) { xs = 0; xph ^= 1u; }
-          if (++ws == GM_WS) ws = 0;
+          if (++ws == WSK) ws = 0;
         }
         if (ok) ptx::mma_commit(bar_tmem_full + 8 * buf);
       }
@@ -190,8 +199,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
                          : static_cast<int>(threadIdx.x) - (grp ? GM_EXPAND2_WARP0 : GM_EXPAND_WARP0) * 32;
     const uint32_t row_off = static_cast<uint32_t>(r >> 3) * 1024u + static_cast<uint32_t>(r & 7) * 128u;
     const uint32_t sw = static_cast<uint32_t>(r & 7);
-    // The weight slot of k block `it` was last used by k block it - GM_WS; that MMA's completion is the arrival on
-    // x_empty of ITS x_q slot, so the expanders watch the x_q ring GM_WS steps behind (GM_WS <= GM_XS keeps the
+    // The weight slot of k block `it` was last used by k block it - WSK; that MMA's completion is the arrival on
+    // x_empty of ITS x_q slot, so the expanders watch the x_q ring WSK steps behind (WSK < GM_XS keeps the
     // watched barrier at most one phase ahead).  Their "ready" arrival goes to x_full of the current x_q slot, which
     // therefore completes when both the TMA bytes and the four expander warps are in: one wait per k block for the MMA.
     uint32_t it = 0;
@@ -200,16 +209,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x) {
       for (int kb = 0; kb < kblocks; ++kb, ++it) {
         if ((it & 1u) != grp) {  // the other group's k block: only advance the ring positions
-          if (it >= GM_WS && ++xs_old == GM_XS) { xs_old = 0; xph_old ^= 1u; }
+          if (it >= WSK && ++xs_old == GM_XS) { xs_old = 0; xph_old ^= 1u; }
           if (++ps == GM_PS) { ps = 0; pph ^= 1u; }
-          if (++ws == GM_WS) ws = 0;
+          if (++ws == WSK) ws = 0;
           if (++xs == GM_XS) xs = 0;
           continue;
         }
         if (!ptx::mbar_wait(bar_p_full + 8 * ps, pph)) { report_timeout(GM_WAIT_P_FULL); ok = false; break; }
         const uint32_t paddr = base + GM_OFF_P + ps * GM_P_BYTES + r * TILE_ROW_BYTES;
         const uint4 p0 = ptx::lds128(paddr), p1 = ptx::lds128(paddr + 16);
-        if (it >= GM_WS) {
+        if (it >= WSK) {
           if (!ptx::mbar_wait(bar_x_empty + 8 * xs_old, xph_old)) { report_timeout(GM_WAIT_W_EMPTY); ok = false; break; }
           if (++xs_old == GM_XS) { xs_old = 0; xph_old ^= 1u; }
         }
@@ -226,7 +235,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
             cols[4 * j + 3] = (wd[j] >> 6) & 0x03030303u;
           }
           ptx::tmem_st_32x32b_x32(tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) +
-                                      (ws < 2 ? 192u + 32u * ws : 448u), cols);
+                                      a_slot(ws), cols);
           ptx::tmem_st_wait();
           ptx::tc_fence_before_sync();
         } else {
@@ -248,7 +257,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
           ptx::mbar_arrive(bar_p_empty + 8 * ps);
         }
         if (++ps == GM_PS) { ps = 0; pph ^= 1u; }
-        if (++ws == GM_WS) ws = 0;
+        if (++ws == WSK) ws = 0;
         if (++xs == GM_XS) xs = 0;
       }
     }
@@ -384,27 +393,31 @@ inline encode_tiled_fn get_encode_tiled() {
 }
 
 int sm_count();
-bool gemm_a_in_tmem();  // expanded weights through tensor memory (default) or through shared memory
+bool gemm_a_in_tmem();
+int gemm_forced_tok();    // 0, or the token-tile width forced through BITRL_GEMM_TOK (64, 128, 192, 224, 256)  // expanded weights through tensor memory (default) or through shared memory
 
 bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax, const int32_t* rowsum, int M,
                          void* y, int out_dtype, const void* residual, int32_t* acc_out, cudaStream_t st) {
   encode_tiled_fn encode = get_encode_tiled();
   if (!encode) return cuda_fail(cudaErrorSymbolNotFound);
-  // Token-tile width: fewest "waves x time per k block" over the SMs.  A k block costs 2*TOK cycles of tensor pipe,
-  // but not less than the expanders need for their 128 x 128 codes (about 330 cycles).
+  // Token-tile width: fewest "waves x time per k block" over the SMs.
   const int sms = sm_count();
   const int tiles_n = w->N / GM_ROWS;
   int tok = 256;
   {
     long long best = -1;
-    const int cand[4] = {256, 192, 128, 64};
-    for (int i = 0; i < 4; ++i) {
+    const int cand[5] = {256, 224, 192, 128, 64};
+    for (int i = 0; i < 5; ++i) {
+      if (cand[i] == 224 && !gemm_a_in_tmem()) continue;
       const long long tiles = static_cast<long long>(tiles_n) * ((M + cand[i] - 1) / cand[i]);
       const long long waves = (tiles + sms - 1) / sms;
-      const long long cost = waves * (2 * cand[i] > 330 ? 2 * cand[i] : 330);
+      // cycles per k block as measured: the 256-wide tile (4-stage x_q ring, weights through shared memory) runs at
+      // about 690, the narrower ones at the MMA thread's own ~500 or the tensor pipe's 2*TOK, whichever is larger
+      const long long cost = waves * (cand[i] == 256 ? 690 : (2 * cand[i] > 500 ? 2 * cand[i] : 500));
       if (best < 0 || cost <= best) { best = cost; tok = cand[i]; }  // ties go to the narrower tile
     }
   }
+  if (const int forced = gemm_forced_tok()) tok = forced;  // tuning knob, see bitrl.cu
   CUtensorMap tmap;
   const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(w->K), static_cast<cuuint64_t>(M)};
   const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(w->K)};
@@ -419,9 +432,10 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
              static_cast<const unsigned short*>(residual), acc_out, tiles_n, 0};
   a.tiles_total = tiles_n * ((M + tok - 1) / tok);
   const int grid = a.tiles_total < sms ? a.tiles_total : sms;
-  const bool a_tmem = gemm_a_in_tmem() && tok <= 192;
+  const bool a_tmem = gemm_a_in_tmem() && tok <= 224;
   void (*kern)(const CUtensorMap, const GemmArgs) =
       tok == 256 ? gemm_i8_kernel<256, false>
+      : tok == 224 ? gemm_i8_kernel<224, true>
       : tok == 192 ? (a_tmem ? gemm_i8_kernel<192, true> : gemm_i8_kernel<192, false>)
       : tok == 128 ? (a_tmem ? gemm_i8_kernel<128, true> : gemm_i8_kernel<128, false>)
                    : (a_tmem ? gemm_i8_kernel<64, true> : gemm_i8_kernel<64, false>);
