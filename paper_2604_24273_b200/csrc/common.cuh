@@ -27,6 +27,13 @@ __device__ __forceinline__ void report_timeout(int stage) {
   if (atomicCAS(&g_status[0], 0, BITRL_ERR_TIMEOUT) == 0) g_status[1] = stage;
 }
 
+// Lets the next kernel in the stream start its set-up, then waits until everything before this kernel has completed
+// and its memory is visible.
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ float bf16_bits_to_float(unsigned short h) {
   return __uint_as_float(static_cast<unsigned>(h) << 16);
 }
@@ -86,6 +93,24 @@ bitrl_status cuda_fail(cudaError_t e);  // records the code, returns BITRL_ERR_C
     cudaError_t e__ = (call);                              \
     if (e__ != cudaSuccess) return ::bitrl::cuda_fail(e__); \
   } while (0)
+
+// Launch with programmatic stream serialization: the kernel may be scheduled while its predecessor in the stream is
+// still draining, so launch latency and the kernel's own set-up overlap the predecessor's tail.  Such kernels call
+// pdl_enter() before they touch any global memory other than constant weights.
+template <class... KArgs, class... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -117,6 +117,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   __syncthreads();
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_enter();  // barriers and tensor memory are set up; inputs of the preceding kernel are read only from here on
 
   if (warp == 0) {
     // ------------------------------------------------------------------ X producer
@@ -289,6 +290,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
       const int tok_hi = min(GM_TOK, a.M - tok0);
       for (int c = 0; c < GM_TOK / 32; ++c) {
         if (c * 32 >= tok_hi) break;  // warp-uniform
+        // Residual rows of this chunk are requested first, so their latency hides behind the accumulator load, the
+        // rescale and the transpose (in-place updates make every later store a possible alias for the compiler).
+        uint4 rres[4];
+        if (a.residual && !f32) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int t = i * 8 + (lane >> 2);
+            if (c * 32 + t < tok_hi)
+              rres[i] = ptx::ldg128(a.residual + static_cast<size_t>(tok0 + c * 32 + t) * a.N + nbase + (lane & 3) * 8);
+          }
+        }
         uint32_t v[32];
         ptx::tmem_ld_32x32b_x32(tmem_base + buf * GM_TOK_MAX + c * 32 + (static_cast<uint32_t>(q * 32) << 16), v);
         ptx::tmem_ld_wait();
@@ -325,7 +337,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
             if (c * 32 + t < tok_hi) {
               const size_t off = static_cast<size_t>(tok0 + c * 32 + t) * a.N + nbase + part * 8;
               if (a.residual) {
-                const uint4 rr = *reinterpret_cast<const uint4*>(a.residual + off);
+                const uint4 rr = rres[i];
                 const uint32_t ov[4] = {o.x, o.y, o.z, o.w}, rv[4] = {rr.x, rr.y, rr.z, rr.w};
                 uint32_t res[4];
 #pragma unroll
@@ -440,9 +452,8 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
       : tok == 128 ? (a_tmem ? gemm_i8_kernel<128, true> : gemm_i8_kernel<128, false>)
                    : (a_tmem ? gemm_i8_kernel<64, true> : gemm_i8_kernel<64, false>);
   BITRL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM_BYTES));
-  kern<<<grid, GM_THREADS, GM_SMEM_BYTES, st>>>(tmap, a);
+  BITRL_CUDA(launch_pdl(kern, dim3(grid), dim3(GM_THREADS), GM_SMEM_BYTES, st, tmap, a));
   count_launch(1);
-  BITRL_CUDA(cudaGetLastError());
   return BITRL_OK;
 }
 

@@ -155,6 +155,7 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, i
   __shared__ float red_ss[ROW_THREADS / 32];
   __shared__ float red_mx[ROW_THREADS / 32];
   __shared__ int red_rs[ROW_THREADS / 32];
+  pdl_enter();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int sub = warp % WPR, grp = warp / WPR;
   const long long row = static_cast<long long>(blockIdx.x) * (ROW_THREADS / 32 / WPR) + grp;
@@ -280,9 +281,9 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, i
 template <int MODE, int WPR>
 bitrl_status launch_row_reg(const RowArgs& a, int T, cudaStream_t st) {
   const int rows_per_cta = ROW_THREADS / 32 / WPR;
-  row_quant_reg_kernel<MODE, WPR><<<(T + rows_per_cta - 1) / rows_per_cta, ROW_THREADS, 0, st>>>(a, T);
+  BITRL_CUDA(launch_pdl(row_quant_reg_kernel<MODE, WPR>, dim3((T + rows_per_cta - 1) / rows_per_cta), dim3(ROW_THREADS),
+                        0, st, a, T));
   count_launch(1);
-  BITRL_CUDA(cudaGetLastError());
   return BITRL_OK;
 }
 
