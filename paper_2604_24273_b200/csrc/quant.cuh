@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_kernel(RowArgs a) {
 // shared memory; only the three scalar reductions cross warps.  8 / WPR rows per CTA.
 constexpr int ROWQ_MAXG = 7;
 
-template <int MODE, int WPR>
+template <int MODE, int WPR, int NG>
 __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, int T) {
   __shared__ float red_ss[ROW_THREADS / 32];
   __shared__ float red_mx[ROW_THREADS / 32];
@@ -163,10 +163,10 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, i
   const int nvec8 = a.Kv >> 3;
   const unsigned short* src = a.in + (live ? row : 0) * a.in_stride + a.in_offset;
 
-  float v[ROWQ_MAXG][8];
+  float v[NG][8];
   float ss = 0.0f;
 #pragma unroll
-  for (int gi = 0; gi < ROWQ_MAXG; ++gi) {
+  for (int gi = 0; gi < NG; ++gi) {
     const int i = (gi * WPR + sub) * 32 + lane;
     if (live && i < nvec8) {
       const uint4 raw = *reinterpret_cast<const uint4*>(src + 8 * i);
@@ -208,7 +208,7 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, i
     }
     const float rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(ss, static_cast<float>(a.Kv)), 1e-5f)));
 #pragma unroll
-    for (int gi = 0; gi < ROWQ_MAXG; ++gi)
+    for (int gi = 0; gi < NG; ++gi)
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         v[gi][e] = bf16_bits_to_float(float_to_bf16_bits(__fmul_rn(v[gi][e], rstd)));
@@ -216,7 +216,7 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, i
       }
   } else {
 #pragma unroll
-    for (int gi = 0; gi < ROWQ_MAXG; ++gi)
+    for (int gi = 0; gi < NG; ++gi)
 #pragma unroll
       for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(v[gi][e]));
   }
@@ -234,7 +234,7 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, i
   int8_t* xq = a.xq + (live ? row : 0) * a.Kout;
   unsigned short* uo = a.u_out ? a.u_out + (live ? row : 0) * a.Kout : nullptr;
 #pragma unroll
-  for (int gi = 0; gi < ROWQ_MAXG; ++gi) {
+  for (int gi = 0; gi < NG; ++gi) {
     const int i = (gi * WPR + sub) * 32 + lane;
     if (live && i < nvec8) {
       int q[8];
@@ -278,10 +278,10 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, i
   }
 }
 
-template <int MODE, int WPR>
+template <int MODE, int WPR, int NG>
 bitrl_status launch_row_reg(const RowArgs& a, int T, cudaStream_t st) {
   const int rows_per_cta = ROW_THREADS / 32 / WPR;
-  BITRL_CUDA(launch_pdl(row_quant_reg_kernel<MODE, WPR>, dim3((T + rows_per_cta - 1) / rows_per_cta), dim3(ROW_THREADS),
+  BITRL_CUDA(launch_pdl(row_quant_reg_kernel<MODE, WPR, NG>, dim3((T + rows_per_cta - 1) / rows_per_cta), dim3(ROW_THREADS),
                         0, st, a, T));
   count_launch(1);
   return BITRL_OK;
@@ -290,13 +290,16 @@ bitrl_status launch_row_reg(const RowArgs& a, int T, cudaStream_t st) {
 template <int MODE>
 bitrl_status launch_row(const RowArgs& a, int T, cudaStream_t st) {
   // Rows of up to 8 * 32 * 7 * 8 = 14336 values fit the register-resident kernel (head_dim a multiple of 8 keeps
-  // the 8-value groups of the V-repeat producer inside one head).
+  // the 8-value groups of the V-repeat producer inside one head).  Few values per lane (NG <= 3 or 4) keep the
+  // register count low, so that several CTAs per SM overlap their load, compute and store phases.
   const int nvec8 = a.Kv >> 3;
   if (a.Kv % 8 == 0 && a.head_dim % 8 == 0) {
-    if (nvec8 <= 32 * ROWQ_MAXG) return launch_row_reg<MODE, 1>(a, T, st);
-    if (nvec8 <= 64 * ROWQ_MAXG) return launch_row_reg<MODE, 2>(a, T, st);
-    if (nvec8 <= 128 * ROWQ_MAXG) return launch_row_reg<MODE, 4>(a, T, st);
-    if (nvec8 <= 256 * ROWQ_MAXG) return launch_row_reg<MODE, 8>(a, T, st);
+    if (nvec8 <= 32 * 3) return launch_row_reg<MODE, 1, 3>(a, T, st);
+    if (nvec8 <= 64 * 3) return launch_row_reg<MODE, 2, 3>(a, T, st);
+    if (nvec8 <= 128 * 3) return launch_row_reg<MODE, 4, 3>(a, T, st);
+    if (nvec8 <= 256 * 3) return launch_row_reg<MODE, 8, 3>(a, T, st);
+    if (nvec8 <= 256 * 4) return launch_row_reg<MODE, 8, 4>(a, T, st);
+    if (nvec8 <= 256 * ROWQ_MAXG) return launch_row_reg<MODE, 8, ROWQ_MAXG>(a, T, st);
   }
   const size_t smem = static_cast<size_t>(a.Kv) * sizeof(float);
   if (smem > 40 * 1024) {
