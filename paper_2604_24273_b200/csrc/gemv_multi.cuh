@@ -183,6 +183,7 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
       }
 
       // ---- one row tile: this warp's 16 rows over the whole K ----
+      const float gamma = *job.gamma;  // requested now, needed after the k loop: its latency hides behind the loop
       // The GVM_UNROLL pieces of a slot are fetched from shared memory together and feed independent accumulator
       // chains, so that neither the loads nor the MMAs of one piece wait for those of another.
       constexpr int CH = NT == 8 ? 16 : 8;  // independent accumulator chains (the warp MMA has a long latency)
@@ -243,7 +244,6 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
           for (int e = 0; e < 4; ++e) acc[0][h][e] += acc[c][h][e];
       if (ok) {
         // C fragment: acc[h][0..1] = (row g, tokens 8h+2t, +1), acc[h][2..3] = (row g+8, same tokens)
-        const float gamma = *job.gamma;
         const int n0 = (u - job.unit_begin) * TILE_ROWS + warp * 16 + g;
 #pragma unroll
         for (int h = 0; h < NT / 8; ++h)
@@ -264,26 +264,30 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// M <= 2 variant: dp4a instead of the warp MMA (cheaper when only one or two tokens use the weights), and 16
-// consumer warps in two groups: group 0 takes the even pieces of every slot, group 1 the odd ones; their partial
-// sums meet in shared memory once per row tile.  Lane = 2*row + k half, as in the single-matrix kernel.
-constexpr int GVD_CONSUMERS = 16;
+// M <= 2 variant: dp4a instead of the warp MMA (cheaper when only one or two tokens use the weights), and
+// 8 * GVD_GROUPS consumer warps: group g takes pieces g, g + GROUPS of every ring slot (a slot holds 2 * GROUPS
+// pieces); the groups' partial sums meet in shared memory once per row tile.  Lane = 2*row + k half, as in the
+// single-matrix kernel.
+constexpr int GVD_GROUPS = 2;
+constexpr int GVD_CONSUMERS = 8 * GVD_GROUPS;
 constexpr int GVD_THREADS = (GVD_CONSUMERS + 1) * 32;
+constexpr int GVD_PIECES = 2 * GVD_GROUPS;                 // 4 KB pieces per ring slot
+constexpr int GVD_SLOT_BYTES = GVD_PIECES * TILE_BYTES;
 
 template <int MT>
 __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const __grid_constant__ GvmArgs a) {
   extern __shared__ __align__(128) unsigned char gvm_smem[];
-  const int depth = 1 << a.depth_log2;
+  const int depth = a.depth_log2;  // for this kernel the field holds the number of ring slots itself
   const uint32_t ring = ptx::smem_u32(gvm_smem);
-  int8_t* xq_s = reinterpret_cast<int8_t*>(gvm_smem + depth * GVM_SLOT_BYTES);  // [MT][K]
-  unsigned char* tail = gvm_smem + depth * GVM_SLOT_BYTES + static_cast<size_t>(MT) * a.kmax;
+  int8_t* xq_s = reinterpret_cast<int8_t*>(gvm_smem + depth * GVD_SLOT_BYTES);  // [MT][K]
+  unsigned char* tail = gvm_smem + depth * GVD_SLOT_BYTES + static_cast<size_t>(MT) * a.kmax;
   const uint32_t bar_full = ptx::smem_u32(tail);    // [depth]
   const uint32_t bar_empty = bar_full + 8 * depth;  // [depth]
   float* absmax_s = reinterpret_cast<float*>(tail + 16 * depth);  // [MT]
   int* rowsum_s = reinterpret_cast<int*>(absmax_s + MT);          // [MT]
-  float* redf = reinterpret_cast<float*>(rowsum_s + MT);          // [16]
-  int* redi = reinterpret_cast<int*>(redf + GVD_CONSUMERS);       // [16]
-  int* comb = redi + GVD_CONSUMERS;                               // [2][8 warps][16 rows][MT]
+  float* redf = reinterpret_cast<float*>(rowsum_s + MT);          // [GVD_CONSUMERS]
+  int* redi = reinterpret_cast<int*>(redf + GVD_CONSUMERS);       // [GVD_CONSUMERS]
+  int* comb = redi + GVD_CONSUMERS;                               // [2][GROUPS-1][8 warps][16 rows][MT]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int u_begin = a.unit_start[blockIdx.x], u_end = a.unit_start[blockIdx.x + 1];
@@ -301,19 +305,19 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
   if (warp == GVD_CONSUMERS) {
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
-      uint32_t pc = 0;
+      uint32_t s = 0, ph = 0;
       int j = 0;
       bool ok = true;
       for (int u = u_begin; ok && u < u_end; ++u) {
         while (j + 1 < a.njobs && a.jobs[j + 1].unit_begin <= u) ++j;
         const int kblocks = a.jobs[j].K / TILE_K;
         const uint8_t* src = a.jobs[j].tiles + static_cast<size_t>(u - a.jobs[j].unit_begin) * kblocks * TILE_BYTES;
-        for (int kb = 0; kb < kblocks; kb += GVM_UNROLL, ++pc) {
-          const uint32_t bytes = static_cast<uint32_t>(min(GVM_UNROLL, kblocks - kb)) * TILE_BYTES;
-          const uint32_t s = pc & (depth - 1), ph = (pc >> a.depth_log2) & 1u;
+        for (int kb = 0; kb < kblocks; kb += GVD_PIECES) {
+          const uint32_t bytes = static_cast<uint32_t>(min(GVD_PIECES, kblocks - kb)) * TILE_BYTES;
           if (!ptx::mbar_wait(bar_empty + 8 * s, ph ^ 1u)) { report_timeout(GVM_WAIT_EMPTY); ok = false; break; }
           ptx::mbar_arrive_expect_tx(bar_full + 8 * s, bytes);
-          ptx::bulk_g2s(ring + s * GVM_SLOT_BYTES, src + static_cast<size_t>(kb) * TILE_BYTES, bytes, bar_full + 8 * s);
+          ptx::bulk_g2s(ring + s * GVD_SLOT_BYTES, src + static_cast<size_t>(kb) * TILE_BYTES, bytes, bar_full + 8 * s);
+          if (++s == static_cast<uint32_t>(depth)) { s = 0; ph ^= 1u; }
         }
       }
     }
@@ -323,7 +327,7 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
     const int half = lane & 1, grp = warp >> 3, rw = warp & 7;
     const unsigned short* cached_x = nullptr;
     int cached_k = 0;
-    uint32_t pc = 0, tile_no = 0;
+    uint32_t s = 0, ph = 0, tile_no = 0;
     int j = 0;
     bool ok = true;
     for (int u = u_begin; u < u_end; ++u, ++tile_no) {
@@ -331,26 +335,26 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
       const GvmJob& job = a.jobs[j];
       const int K = job.K, kblocks = K / TILE_K;
       if (job.x != cached_x || K != cached_k) {
-        asm volatile("bar.sync 2, 512;" ::: "memory");  // everyone is done with the previous contents
+        asm volatile("bar.sync 2, %0;" ::"n"(GVD_CONSUMERS * 32) : "memory");  // done with the previous contents
         const int nvec8 = K >> 3;
         for (int m = 0; m < MT; ++m) {
           uint2* dst = reinterpret_cast<uint2*>(xq_s + m * K);
           if (m >= a.M) {
-            for (int i = threadIdx.x; i < nvec8; i += 512) dst[i] = make_uint2(0u, 0u);
+            for (int i = threadIdx.x; i < nvec8; i += GVD_CONSUMERS * 32) dst[i] = make_uint2(0u, 0u);
             continue;
           }
           const uint4* xr = reinterpret_cast<const uint4*>(job.x + static_cast<size_t>(m) * K);
           float mx = 0.0f;
-          for (int i = threadIdx.x; i < nvec8; i += 512) mx = fmaxf(mx, absmax8(xr[i]));
+          for (int i = threadIdx.x; i < nvec8; i += GVD_CONSUMERS * 32) mx = fmaxf(mx, absmax8(xr[i]));
           mx = warp_max(mx);
           if (lane == 0) redf[warp] = mx;
-          asm volatile("bar.sync 2, 512;" ::: "memory");
+          asm volatile("bar.sync 2, %0;" ::"n"(GVD_CONSUMERS * 32) : "memory");
 #pragma unroll
           for (int i = 0; i < GVD_CONSUMERS; ++i) mx = fmaxf(mx, redf[i]);
           const float amax = fmaxf(mx, 1e-5f);
           const float inv = __fdiv_rn(127.0f, amax);
           int rs = 0;
-          for (int i = threadIdx.x; i < nvec8; i += 512) {
+          for (int i = threadIdx.x; i < nvec8; i += GVD_CONSUMERS * 32) {
             const uint4 raw = xr[i];
             const uint32_t rwd[4] = {raw.x, raw.y, raw.z, raw.w};
             int q[8];
@@ -367,7 +371,7 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
           }
           rs = warp_sum_i(rs);
           if (lane == 0) redi[warp] = rs;
-          asm volatile("bar.sync 2, 512;" ::: "memory");
+          asm volatile("bar.sync 2, %0;" ::"n"(GVD_CONSUMERS * 32) : "memory");
           if (threadIdx.x == 0) {
             int tsum = 0;
 #pragma unroll
@@ -376,34 +380,35 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
             absmax_s[m] = amax;
           }
         }
-        asm volatile("bar.sync 2, 512;" ::: "memory");
+        asm volatile("bar.sync 2, %0;" ::"n"(GVD_CONSUMERS * 32) : "memory");
         cached_x = job.x;
         cached_k = K;
       }
 
-      // ---- one row tile: this warp's 16 rows, every second piece ----
+      // ---- one row tile: this warp's 16 rows, pieces grp and grp + GROUPS of every slot ----
+      const float gamma = *job.gamma;  // requested now, needed after the k loop: its latency hides behind the loop
       int acc[MT][4];
 #pragma unroll
       for (int m = 0; m < MT; ++m)
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[m][c] = 0;
-      for (int kb = 0; kb < kblocks; kb += GVM_UNROLL, ++pc) {
-        const int np = min(GVM_UNROLL, kblocks - kb);
-        const uint32_t s = pc & (depth - 1), ph = (pc >> a.depth_log2) & 1u;
+      // All addresses below are 32-bit shared-memory addresses with compile-time offsets, so that a piece costs its
+      // loads, masks and dp4a and little else.
+      const uint32_t w_lane = ring + rw * 512 + lane * 16 + grp * TILE_BYTES;   // this lane's 16 bytes in piece `grp`
+      uint32_t x_lane = ptx::smem_u32(xq_s) + half * 64 + grp * TILE_K;         // its 64 activations of that piece
+      for (int kb = 0; kb < kblocks; kb += GVD_PIECES, x_lane += GVD_PIECES * TILE_K) {
+        const int np = min(GVD_PIECES, kblocks - kb) - grp;  // pieces grp, grp + GROUPS exist if np > 0, GROUPS
         if (ok && !ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(GVM_WAIT_FULL); ok = false; }
         if (ok) {
-          uint4 wv[GVM_UNROLL / 2];
+          const uint32_t w_slot = w_lane + s * GVD_SLOT_BYTES;
+          uint4 wv[2];
 #pragma unroll
-          for (int pp = 0; pp < GVM_UNROLL / 2; ++pp) {
-            const int pidx = 2 * pp + grp;
-            if (pidx < np) wv[pp] = ptx::lds128(ring + s * GVM_SLOT_BYTES + pidx * TILE_BYTES + rw * 512 + lane * 16);
-          }
+          for (int pp = 0; pp < 2; ++pp)
+            if (GVD_GROUPS * pp < np) wv[pp] = ptx::lds128(w_slot + pp * GVD_GROUPS * TILE_BYTES);
 #pragma unroll
-          for (int pp = 0; pp < GVM_UNROLL / 2; ++pp) {
-            const int pidx = 2 * pp + grp;
-            if (pidx < np) {
+          for (int pp = 0; pp < 2; ++pp) {
+            if (GVD_GROUPS * pp < np) {
               const uint32_t wword[4] = {wv[pp].x, wv[pp].y, wv[pp].z, wv[pp].w};
-              const int k0 = (kb + pidx) * TILE_K + half * 64;
 #pragma unroll
               for (int jw = 0; jw < 4; ++jw) {
                 // The codes are left at their bit positions (c1 * 4, c2 * 16, c3 * 64 still fit an unsigned byte):
@@ -415,11 +420,11 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
                 const uint32_t c3 = wword[jw] & 0xc0c0c0c0u;
 #pragma unroll
                 for (int m = 0; m < MT; ++m) {
-                  const int4 xv = *reinterpret_cast<const int4*>(xq_s + m * K + k0 + 16 * jw);
-                  acc[m][0] = dp4a_u8s8(c0, xv.x, acc[m][0]);
-                  acc[m][1] = dp4a_u8s8(c1, xv.y, acc[m][1]);
-                  acc[m][2] = dp4a_u8s8(c2, xv.z, acc[m][2]);
-                  acc[m][3] = dp4a_u8s8(c3, xv.w, acc[m][3]);
+                  const uint4 xv = ptx::lds128(x_lane + m * K + pp * GVD_GROUPS * TILE_K + 16 * jw);
+                  acc[m][0] = dp4a_u8s8(c0, static_cast<int>(xv.x), acc[m][0]);
+                  acc[m][1] = dp4a_u8s8(c1, static_cast<int>(xv.y), acc[m][1]);
+                  acc[m][2] = dp4a_u8s8(c2, static_cast<int>(xv.z), acc[m][2]);
+                  acc[m][3] = dp4a_u8s8(c3, static_cast<int>(xv.w), acc[m][3]);
                 }
               }
             }
@@ -427,24 +432,26 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(bar_empty + 8 * s);
         }
+        if (++s == static_cast<uint32_t>(depth)) { s = 0; ph ^= 1u; }
       }
-      // ---- combine: k halves by shuffle, the two warp groups through shared memory ----
-      int* cb = comb + (tile_no & 1u) * (8 * 16 * MT) + (rw * 16 + (lane >> 1)) * MT;
+      // ---- combine: k halves by shuffle, the warp groups through shared memory ----
+      int* cb = comb + (tile_no & 1u) * ((GVD_GROUPS - 1) * 8 * 16 * MT) + (rw * 16 + (lane >> 1)) * MT;
       int tot[MT];
 #pragma unroll
       for (int m = 0; m < MT; ++m) {
         tot[m] = acc[m][0] + (acc[m][1] >> 2) + (acc[m][2] >> 4) + (acc[m][3] >> 6);  // exact: multiples of 4^i
         tot[m] += __shfl_xor_sync(0xffffffffu, tot[m], 1);
-        if (grp == 1 && half == 0) cb[m] = tot[m];
+        if (grp > 0 && half == 0) cb[(grp - 1) * (8 * 16 * MT) + m] = tot[m];
       }
-      asm volatile("bar.sync 3, 512;" ::: "memory");
+      asm volatile("bar.sync 3, %0;" ::"n"(GVD_CONSUMERS * 32) : "memory");
       if (grp == 0 && half == 0 && ok) {
-        const float gamma = *job.gamma;
         const int n = (u - job.unit_begin) * TILE_ROWS + rw * 16 + (lane >> 1);
 #pragma unroll
         for (int m = 0; m < MT; ++m) {
           if (m < a.M) {
-            const int tv = tot[m] + cb[m] - rowsum_s[m];
+            int tv = tot[m] - rowsum_s[m];
+#pragma unroll
+            for (int g2 = 0; g2 < GVD_GROUPS - 1; ++g2) tv += cb[g2 * (8 * 16 * MT) + m];
             const float yv = __fmul_rn(static_cast<float>(tv), out_scale(gamma, absmax_s[m]));
             const size_t o = static_cast<size_t>(m) * job.N + n;
             if (a.out_dtype == BITRL_OUT_F32) static_cast<float*>(job.y)[o] = yv;
@@ -498,7 +505,7 @@ bitrl_status launch_gemv_multi_dp4a_t(const GvmArgs& a, int grid, size_t smem, c
 inline int gvm_nt(int M) { return M <= 8 ? 8 : 16; }
 // Shared memory beside the ring: activations (+ barriers, reduction scratch, the group-combine buffer).
 inline size_t gvm_fixed_bytes(int M, int kmax) {
-  if (M <= 2) return static_cast<size_t>(M) * kmax + 1024 + 2 * 8 * 16 * 2 * sizeof(int);
+  if (M <= 2) return static_cast<size_t>(M) * kmax + 1024 + 2 * (GVD_GROUPS - 1) * 8 * 16 * 2 * sizeof(int);
   return static_cast<size_t>(gvm_nt(M)) * (kmax + GVM_XPAD) + 1024;
 }
 
@@ -521,7 +528,13 @@ bitrl_status launch_gemv_multi(int count, const Linear* const* w, const void* co
     pieces += static_cast<long long>(w[j]->N / TILE_ROWS) * (w[j]->K / TILE_K);
     if (w[j]->K > kmax) kmax = w[j]->K;
   }
-  const int dlog = gvm_depth_log2(M, kmax);
+  int dlog = gvm_depth_log2(M, kmax);
+  if (M <= 2) {  // the dp4a kernel takes the slot count itself (24 KB slots, any count from 2 to 8)
+    const long long room = static_cast<long long>(GVM_SMEM_BUDGET) - static_cast<long long>(gvm_fixed_bytes(M, kmax));
+    dlog = static_cast<int>(room / (GVD_SLOT_BYTES + 16));
+    if (dlog > 8) dlog = 8;
+    if (dlog < 2) dlog = -1;
+  }
   if (dlog < 0) return BITRL_ERR_SHAPE;
   int grid = sm_count();
   if (grid > GVM_MAX_CTAS) grid = GVM_MAX_CTAS;
@@ -547,7 +560,8 @@ bitrl_status launch_gemv_multi(int count, const Linear* const* w, const void* co
   a.out_dtype = out_dtype;
   a.depth_log2 = dlog;
   a.kmax = kmax;
-  const size_t smem = static_cast<size_t>(GVM_SLOT_BYTES + 16) * (1u << dlog) + gvm_fixed_bytes(M, kmax);
+  const size_t smem = (M <= 2 ? static_cast<size_t>(GVD_SLOT_BYTES + 16) * dlog
+                              : static_cast<size_t>(GVM_SLOT_BYTES + 16) * (1u << dlog)) + gvm_fixed_bytes(M, kmax);
   if (M == 1) return launch_gemv_multi_dp4a_t<1>(a, grid, smem, st);
   if (M == 2) return launch_gemv_multi_dp4a_t<2>(a, grid, smem, st);
   return gvm_nt(M) == 8 ? launch_gemv_multi_t<8>(a, grid, smem, st) : launch_gemv_multi_t<16>(a, grid, smem, st);
