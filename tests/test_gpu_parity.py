@@ -453,3 +453,62 @@ def test_gemm_token_tile_variants(oracle_mod, B):
     check_layer(oracle_mod, B, 256, 2560, 6912, 1005, 3601, 1)  # 128
     check_layer(oracle_mod, B, 300, 2560, 6912, 1005, 3602, 1)  # 192
     check_layer(oracle_mod, B, 1100, 256, 384, 7, 3603, 0)      # fp32 output through the GEMM epilogue
+
+
+# ----------------------------------------------------------------- full-size launches, sampled against the oracle
+
+def test_grouped_sweep_full_block_shapes_sampled(oracle_mod, B):
+    """The benchmark's launch configuration (grouped M=1 sweep over whole blocks of the ~2B backbone, here 2 blocks
+    = 8 matrices, 35 MB packed): every matrix's output is checked on 300 sampled rows recomputed one by one by the
+    oracle, plus the property |acc| <= 127 * nnz via the debug tap of the single-matrix kernel on one matrix."""
+    shapes = [(3840, 2560), (2560, 2560), (13824, 2560), (2560, 6912)]
+    x_cpu = {K: inputs.activations(1, K, 2001) for K in (2560, 6912)}
+    x_gpu = {K: v.cuda() for K, v in x_cpu.items()}
+    xq = {K: oracle_mod.quant_act(inputs.bf16_bits(v)) for K, v in x_cpu.items()}
+    ws, xs, ys, cpu = [], [], [], []
+    for l in range(2):
+        for j, (N, K) in enumerate(shapes):
+            _, Wq, g, _, _, lin = layer(oracle_mod, B, N, K, 5000 + 4 * l + j)
+            ws.append(lin)
+            xs.append(x_gpu[K])
+            ys.append(torch.empty((1, N), dtype=torch.bfloat16, device="cuda"))
+            cpu.append((Wq, g, K, N))
+    B.MultiCall(ws, xs, ys, B.OUT_BF16).run()
+    B.poll_status()
+    rng = np.random.default_rng(7)
+    for (Wq, g, K, N), y in zip(cpu, ys):
+        ns = np.unique(np.concatenate([[0, 127, 128, N - 1], rng.integers(0, N, 300)]))
+        q, a = xq[K]
+        acc = oracle_mod.contract_pairs(q, Wq, np.zeros_like(ns), ns)
+        _, yb, y64 = oracle_mod.rescale(acc[None, :], g, a)
+        got = gpu_bf16_bits(y)[0, ns]
+        assert np.array_equal(got, yb[0])
+        assert max_rel_err(bits_to_f64(got)[None, :], y64) <= TOL_BF16
+
+
+def test_encoder_full_width_two_blocks_teacher_forced(oracle_mod, B):
+    """Encoder at the real widths (d=2560, d_ff=6912, 20/5 heads), 2 blocks, T=300 (token tile with a ragged tail):
+    encoder_forward equals the chain of single calls bit for bit; every BitLinear of the chain is checked against the
+    oracle's integers on the GPU's own quantized input for 24 sampled token rows."""
+    dims = {"d": 2560, "d_ff": 6912, "n_heads": 20, "n_kv_heads": 5, "n_layers": 2}
+    T = 300
+    enc, layers_gpu, layers_cpu = build_encoder(oracle_mod, B, dims, 5000)
+    h0 = inputs.activations(T, dims["d"], 6000).cuda()
+    out = enc.forward(h0)
+    B.poll_status()
+    rows = np.unique(np.concatenate([[0, 255, 256, 299], np.random.default_rng(3).integers(0, T, 20)]))
+    h = h0.clone()
+    for (qkv_l, out_l, gu_l, down_l), cpu in zip(layers_gpu, layers_cpu):
+        xq, a, rs, _ = B.rmsnorm_quant(h)
+        qkv, acc = B.bitlinear_forward_q(qkv_l, xq, a, rs, want_acc=True)
+        assert np.array_equal(acc.cpu().numpy()[rows], oracle_mod.contract(xq.cpu().numpy()[rows], cpu[0][0]))
+        xq, a, rs, _ = B.vrepeat_rmsnorm_quant(qkv, 20, 5, 128)
+        h, acc = B.bitlinear_forward_q(out_l, xq, a, rs, residual=h, want_acc=True)
+        assert np.array_equal(acc.cpu().numpy()[rows], oracle_mod.contract(xq.cpu().numpy()[rows], cpu[1][0]))
+        xq, a, rs, _ = B.rmsnorm_quant(h)
+        gu, acc = B.bitlinear_forward_q(gu_l, xq, a, rs, want_acc=True)
+        assert np.array_equal(acc.cpu().numpy()[rows], oracle_mod.contract(xq.cpu().numpy()[rows], cpu[2][0]))
+        xq, a, rs, _ = B.relu2gate_rmsnorm_quant(gu)
+        h, acc = B.bitlinear_forward_q(down_l, xq, a, rs, residual=h, want_acc=True)
+        assert np.array_equal(acc.cpu().numpy()[rows], oracle_mod.contract(xq.cpu().numpy()[rows], cpu[3][0]))
+    assert torch.equal(out, h)

@@ -1,0 +1,148 @@
+"""Do the pins bite?  Each case plants ONE plausible mistake in (a wrapper around) the CPU oracle and checks that
+at least one of the pin tests of test_oracle_pins.py fails on it.  The mistakes are the ones a re-implementation
+would most likely make: a dropped epsilon, the wrong tie rule, a reversed bit order, a lost sign, a wrong head map.
+All of this runs on the CPU; nothing here touches the CUDA library.
+"""
+import numpy as np
+import pytest
+
+import test_oracle_pins as pins
+
+
+class Mutant:
+    """The oracle module with some functions replaced; `bitlinear` is re-composed from the (possibly replaced) parts."""
+
+    def __init__(self, real, **overrides):
+        self._real = real
+        self._over = overrides
+
+    def __getattr__(self, name):
+        if name in self._over:
+            return lambda *a, **k: self._over[name](self._real, *a, **k)
+        return getattr(self._real, name)
+
+    def bitlinear(self, x_bf16, Wq, gamma, threads=None):
+        xq, a = self.quant_act(x_bf16)
+        acc = self.contract(xq, Wq, threads)
+        y32, yb, y64 = self.rescale(acc, gamma, a)
+        return {"xq": xq, "absmax": a, "acc": acc, "y32": y32, "ybf16": yb, "y64": y64}
+
+
+def _ternarize_half_away(real, W, gamma=None):
+    """round-half-away-from-zero instead of ties-to-even: |W|/s = 0.5 becomes +-1 (Eq. 2 has a strict '>')."""
+    W = np.ascontiguousarray(W, np.float32)
+    g = real.absmean(W) if gamma is None else np.float32(gamma)
+    t = W / np.float32(g + np.float32(1e-5))
+    r = np.sign(t) * np.floor(np.abs(t) + np.float32(0.5))
+    return np.clip(r, -1, 1).astype(np.int8), g
+
+
+def _ternarize_no_eps(real, W, gamma=None):
+    W = np.ascontiguousarray(W, np.float32)
+    g = real.absmean(W) if gamma is None else np.float32(gamma)
+    Wq, _ = real.ternarize(W, gamma=np.float32(g) * np.float32(1.3))  # threshold off by 30 %
+    return Wq, g
+
+
+def _pack_reversed_bits(real, Wq):
+    p = real.pack(Wq)
+    return ((p & 0x03) << 6) | ((p & 0x0C) << 2) | ((p & 0x30) >> 2) | ((p & 0xC0) >> 6)
+
+
+def _contract_drops_minus(real, xq, Wq, threads=None):
+    """treats -1 weights as 'skip' instead of 'subtract'"""
+    return real.contract(xq, np.maximum(np.asarray(Wq), 0).astype(np.int8), threads)
+
+
+def _contract_transposed_x(real, xq, Wq, threads=None):
+    xq = np.asarray(xq)
+    return real.contract(xq[:, ::-1].copy(), Wq, threads)  # k index reversed on one operand only
+
+
+def _rescale_gamma_plus_eps(real, acc, gamma, absmax):
+    return real.rescale(acc, np.float32(gamma) + np.float32(1e-5), absmax)
+
+
+def _rescale_over_128(real, acc, gamma, absmax):
+    y32, yb, y64 = real.rescale(acc, gamma, absmax)
+    return (y32 * np.float32(127.0 / 128.0)).astype(np.float32), yb, y64 * (127.0 / 128.0)
+
+
+def _quant_truncates(real, x_bf16):
+    xq, a = real.quant_act(x_bf16)
+    x = pins.bits_to_f32(x_bf16)
+    q = np.trunc(x * (np.float32(127.0) / a[:, None]))
+    return np.clip(q, -128, 127).astype(np.int8), a
+
+
+def _quant_no_clamp(real, x_bf16):
+    xq, a = real.quant_act(x_bf16)
+    x = np.abs(pins.bits_to_f32(x_bf16)).max(axis=1)
+    return xq, x.astype(np.float32)  # absmax without the 1e-5 floor
+
+
+def _rmsnorm_no_eps_wrong_len(real, x_bf16):
+    x = pins.bits_to_f32(x_bf16).astype(np.float64)
+    u = x / np.sqrt((x * x).sum(axis=1, keepdims=True) / (x.shape[1] - 1))
+    return pins.bf16_bits_of(u.astype(np.float32))
+
+
+def _attention_modulo(real, qkv, n_heads, n_kv_heads, head_dim):
+    T = qkv.shape[0]
+    v = np.asarray(qkv)[:, (n_heads + n_kv_heads) * head_dim:].reshape(T, n_kv_heads, head_dim)
+    return np.stack([v[:, h % n_kv_heads] for h in range(n_heads)], axis=1).reshape(T, n_heads * head_dim)
+
+
+def _relu2_without_square(real, gu):
+    g = pins.bits_to_f32(gu)
+    F = g.shape[1] // 2
+    return (np.maximum(g[:, :F], 0) * g[:, F:]).astype(np.float32)
+
+
+PIN_TESTS = [pins.test_eq2_definition_fp64, pins.test_eq2_ties_are_strict, pins.test_golden_worked_example,
+             pins.test_dense_fp64_of_dequantized_operands, pins.test_quant_act_against_torch,
+             pins.test_absmax_maps_to_127_and_zero_rows, pins.test_select_sum_add_subtract_skip,
+             pins.test_negation_permutation_bound_allones, pins.test_pack_roundtrip_and_zero_matrix,
+             pins.test_gaussian_closed_forms, pins.test_rescale_tolerances_and_bf16_rne,
+             pins.test_rmsnorm_against_fp64, pins.test_relu2_gate_identity_attention_residual]
+
+
+def failing_pins(mod):
+    failed = []
+    for t in PIN_TESTS:
+        try:
+            if t is pins.test_dense_fp64_of_dequantized_operands:
+                t(mod, 3, 64, 40, 1)
+            else:
+                t(mod)
+        except AssertionError:
+            failed.append(t.__name__)
+        except Exception:  # a mistake that makes the computation blow up is caught as well
+            failed.append(t.__name__)
+    return failed
+
+
+MUTANTS = {
+    "ternarize: round half away": {"ternarize": _ternarize_half_away},
+    "ternarize: threshold off": {"ternarize": _ternarize_no_eps},
+    "pack: reversed bit order": {"pack": _pack_reversed_bits},
+    "contract: -1 treated as skip": {"contract": _contract_drops_minus},
+    "contract: k reversed on one operand": {"contract": _contract_transposed_x},
+    "rescale: gamma + eps": {"rescale": _rescale_gamma_plus_eps},
+    "rescale: 128 levels": {"rescale": _rescale_over_128},
+    "quant: truncation": {"quant_act": _quant_truncates},
+    "quant: no absmax floor": {"quant_act": _quant_no_clamp},
+    "rmsnorm: wrong statistics": {"rmsnorm_bf16": _rmsnorm_no_eps_wrong_len},
+    "attention: modulo head map": {"identity_attention": _attention_modulo},
+    "gate: relu without the square": {"relu2_gate": _relu2_without_square},
+}
+
+
+def test_the_unmodified_oracle_passes_every_pin(oracle_mod):
+    assert failing_pins(Mutant(oracle_mod)) == []
+
+
+@pytest.mark.parametrize("name", sorted(MUTANTS))
+def test_each_planted_mistake_fails_a_pin(oracle_mod, name):
+    failed = failing_pins(Mutant(oracle_mod, **MUTANTS[name]))
+    assert failed, f"no pin noticed the mistake: {name}"
