@@ -413,6 +413,7 @@ def run_ours(args):
         }
         print(json.dumps(line))
     if world > 1:
+        torch.distributed.barrier()  # the other ranks wait for rank 0's secondary sections before tearing down
         torch.distributed.destroy_process_group()
 
 

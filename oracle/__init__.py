@@ -60,8 +60,14 @@ def _L():
         _lib.oracle_relu2_gate.argtypes = [_vp, _i64, _i64, _vp]
         _lib.oracle_identity_attention.argtypes = [_vp, _i64, _i64, _i64, _i64, _vp]
         _lib.oracle_residual_add.argtypes = [_vp, _vp, _i64]
+        _lib.oracle_attention.argtypes = [_vp, _vp, _i64, _i64, _i64, _i64, ctypes.c_double, _vp]
+        _lib.oracle_attention.restype = None
         _lib.oracle_encoder_block.argtypes = [_vp, _i64, _i64, _i64, _i64, _i64,
                                               _vp, _f32, _vp, _f32, _vp, _f32, _vp, _f32, _int]
+        _lib.oracle_encoder_block_states.argtypes = [_vp, _i64, _i64, _i64, _i64, _i64,
+                                                     _vp, _f32, _vp, _f32, _vp, _f32, _vp, _f32,
+                                                     _vp, _i64, ctypes.c_double, _int]
+        _lib.oracle_encoder_block_states.restype = None
         for name in ("oracle_ternarize", "oracle_pack", "oracle_unpack", "oracle_quant_act",
                      "oracle_contract", "oracle_contract_pairs", "oracle_rescale", "oracle_rmsnorm_f32",
                      "oracle_rmsnorm_bf16", "oracle_relu2_gate", "oracle_identity_attention",
@@ -206,6 +212,18 @@ def identity_attention(qkv_bf16: np.ndarray, n_heads: int, n_kv_heads: int, head
     return att
 
 
+def attention(qkv_bf16: np.ndarray, states, n_heads: int, n_kv_heads: int, head_dim: int, theta: float) -> np.ndarray:
+    """Causal GQA attention with rotary embedding inside each state; returns bf16 bits [T, n_heads*hd].
+    `states` is either one length S shared by all states or the offsets [n_states+1] of ragged states."""
+    qkv = _c(qkv_bf16, np.uint16)
+    T = qkv.shape[0]
+    off = _state_offsets(states, T)
+    assert qkv.shape[1] == (n_heads + 2 * n_kv_heads) * head_dim and head_dim % 2 == 0
+    att = np.empty((T, n_heads * head_dim), np.uint16)
+    _L().oracle_attention(_p(qkv), _p(off), len(off) - 1, n_heads, n_kv_heads, head_dim, ctypes.c_double(theta), _p(att))
+    return att
+
+
 def residual_add(h_bf16: np.ndarray, y_bf16: np.ndarray) -> np.ndarray:
     h = np.array(h_bf16, dtype=np.uint16, order="C", copy=True)
     y = _c(y_bf16, np.uint16)
@@ -214,20 +232,34 @@ def residual_add(h_bf16: np.ndarray, y_bf16: np.ndarray) -> np.ndarray:
     return h
 
 
-def encoder_block(h_bf16: np.ndarray, d_ff: int, n_heads: int, n_kv_heads: int, layer, threads=None):
-    """layer = ((Wq_qkv, g), (Wq_out, g), (Wq_gateup, g), (Wq_down, g)).  Returns the new h (bf16 bits)."""
+def _state_offsets(states, T):
+    if np.ndim(states) == 0:
+        assert T % int(states) == 0
+        return np.arange(0, T + 1, int(states), dtype=np.int64)
+    off = _c(np.asarray(states), np.int64)
+    assert off[0] == 0 and off[-1] == T and np.all(np.diff(off) >= 1)
+    return off
+
+
+def encoder_block(h_bf16: np.ndarray, d_ff: int, n_heads: int, n_kv_heads: int, layer, threads=None,
+                  states=None, theta: float = 500000.0):
+    """layer = ((Wq_qkv, g), (Wq_out, g), (Wq_gateup, g), (Wq_down, g)).  Returns the new h (bf16 bits).
+    states=None: identity attention; else a common state length or the offsets of ragged states (real attention)."""
     h = np.array(h_bf16, dtype=np.uint16, order="C", copy=True)
     T, d = h.shape
     mats = [(_c(w, np.int8), float(g)) for (w, g) in layer]
-    _L().oracle_encoder_block(_p(h), T, d, d_ff, n_heads, n_kv_heads,
-                              _p(mats[0][0]), _f32(mats[0][1]), _p(mats[1][0]), _f32(mats[1][1]),
-                              _p(mats[2][0]), _f32(mats[2][1]), _p(mats[3][0]), _f32(mats[3][1]),
-                              threads or default_threads())
+    off = None if states is None else _state_offsets(states, T)
+    _L().oracle_encoder_block_states(_p(h), T, d, d_ff, n_heads, n_kv_heads,
+                                     _p(mats[0][0]), _f32(mats[0][1]), _p(mats[1][0]), _f32(mats[1][1]),
+                                     _p(mats[2][0]), _f32(mats[2][1]), _p(mats[3][0]), _f32(mats[3][1]),
+                                     None if off is None else _p(off), 0 if off is None else len(off) - 1,
+                                     ctypes.c_double(theta), threads or default_threads())
     return h
 
 
-def encoder_forward(h_bf16: np.ndarray, d_ff: int, n_heads: int, n_kv_heads: int, layers, threads=None):
+def encoder_forward(h_bf16: np.ndarray, d_ff: int, n_heads: int, n_kv_heads: int, layers, threads=None,
+                    states=None, theta: float = 500000.0):
     h = h_bf16
     for layer in layers:
-        h = encoder_block(h, d_ff, n_heads, n_kv_heads, layer, threads)
+        h = encoder_block(h, d_ff, n_heads, n_kv_heads, layer, threads, states, theta)
     return h

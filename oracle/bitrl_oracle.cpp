@@ -253,6 +253,62 @@ void oracle_identity_attention(const uint16_t* qkv, int64_t T, int64_t n_heads, 
         att[t * d + hd * head_dim + e] = qkv[t * W + d + dkv + (hd / rep) * head_dim + e];
 }
 
+// Real attention inside each state (the step after the hot path; the paper only says that a state serializes to
+// 15-40 tokens that the backbone processes in one forward pass, Sec. V, and that h_t = f(serialize(s_t)), Eq. 3; the
+// form below is the causal grouped-query attention with rotary embedding of the cited architecture).
+// qkv: bf16 [T, (n_heads + 2 n_kv_heads) * head_dim] = [q | k | v]; state s owns the contiguous tokens
+// state_off[s] .. state_off[s+1]-1 (lengths may differ from state to state); T = state_off[n_states].
+//   rotary (rotate-half form), position p = index of the token inside its state, for i < head_dim/2:
+//     angle = p * theta^(-2 i / head_dim);  (x_i, x_{i+hd/2}) -> (x_i cos - x_{i+hd/2} sin, x_{i+hd/2} cos + x_i sin)
+//   applied to q and k.  score(p, r) = q_p . k_r / sqrt(head_dim) for r <= p, softmax over r, out_p = sum_r w_r v_r.
+// Query head h reads kv head h / (n_heads / n_kv_heads).  Everything in fp64; output rounded once to fp32, then bf16.
+void oracle_attention(const uint16_t* qkv, const int64_t* state_off, int64_t n_states, int64_t n_heads,
+                      int64_t n_kv_heads, int64_t head_dim, double theta, uint16_t* att) {
+  const int64_t d = n_heads * head_dim, dkv = n_kv_heads * head_dim, W = d + 2 * dkv, half = head_dim / 2;
+  const int64_t rep = n_heads / n_kv_heads;
+  std::vector<double> q, k, w;
+  auto rope = [&](const uint16_t* src, int64_t pos, double* dst) {
+    for (int64_t i = 0; i < half; ++i) {
+      const double ang = static_cast<double>(pos) * std::pow(theta, -2.0 * static_cast<double>(i) / static_cast<double>(head_dim));
+      const double c = std::cos(ang), sn = std::sin(ang);
+      const double a = bf16_to_f32(src[i]), b = bf16_to_f32(src[i + half]);
+      dst[i] = a * c - b * sn;
+      dst[i + half] = b * c + a * sn;
+    }
+  };
+  for (int64_t st = 0; st < n_states; ++st) {
+    const int64_t t0 = state_off[st], S = state_off[st + 1] - state_off[st];
+    q.assign(static_cast<size_t>(S * head_dim), 0.0);
+    k.assign(static_cast<size_t>(S * head_dim), 0.0);
+    w.assign(static_cast<size_t>(S), 0.0);
+    for (int64_t h = 0; h < n_heads; ++h) {
+      const int64_t kvh = h / rep;
+      for (int64_t p = 0; p < S; ++p) {
+        const uint16_t* row = qkv + (t0 + p) * W;
+        rope(row + h * head_dim, p, q.data() + p * head_dim);
+        rope(row + d + kvh * head_dim, p, k.data() + p * head_dim);
+      }
+      for (int64_t p = 0; p < S; ++p) {
+        double mx = -1e300;
+        for (int64_t r = 0; r <= p; ++r) {
+          double sc = 0.0;
+          for (int64_t e = 0; e < head_dim; ++e) sc += q[p * head_dim + e] * k[r * head_dim + e];
+          w[r] = sc / std::sqrt(static_cast<double>(head_dim));
+          if (w[r] > mx) mx = w[r];
+        }
+        double den = 0.0;
+        for (int64_t r = 0; r <= p; ++r) { w[r] = std::exp(w[r] - mx); den += w[r]; }
+        for (int64_t e = 0; e < head_dim; ++e) {
+          double o = 0.0;
+          for (int64_t r = 0; r <= p; ++r)
+            o += w[r] * static_cast<double>(bf16_to_f32(qkv[(t0 + r) * W + d + dkv + kvh * head_dim + e]));
+          att[(t0 + p) * d + h * head_dim + e] = f32_to_bf16_rne(static_cast<float>(o / den));
+        }
+      }
+    }
+  }
+}
+
 // Residual: h <- bf16( fp32(h) + fp32(y) ), both bf16.
 void oracle_residual_add(uint16_t* h, const uint16_t* y, int64_t count) {
   for (int64_t i = 0; i < count; ++i) h[i] = f32_to_bf16_rne(bf16_to_f32(h[i]) + bf16_to_f32(y[i]));
@@ -261,11 +317,12 @@ void oracle_residual_add(uint16_t* h, const uint16_t* y, int64_t count) {
 // One encoder block on a bf16 residual stream h [T,d], in place:
 //   h += BitLinear_out( RMSNorm( identity_attention( BitLinear_qkv( RMSNorm(h) ) ) ) )
 //   h += BitLinear_down( RMSNorm( relu2_gate( BitLinear_gateup( RMSNorm(h) ) ) ) )
-// Wq_* are int8 ternary matrices [N,K] with scales g_*.
-void oracle_encoder_block(uint16_t* h, int64_t T, int64_t d, int64_t d_ff, int64_t n_heads,
-                          int64_t n_kv_heads, const int8_t* Wq_qkv, float g_qkv, const int8_t* Wq_out,
-                          float g_out, const int8_t* Wq_gu, float g_gu, const int8_t* Wq_down, float g_down,
-                          int threads) {
+// Wq_* are int8 ternary matrices [N,K] with scales g_*.  With state_off == nullptr the attention step is the
+// identity on V above; otherwise it is oracle_attention over the states state_off describes (rotary base theta).
+void oracle_encoder_block_states(uint16_t* h, int64_t T, int64_t d, int64_t d_ff, int64_t n_heads,
+                                 int64_t n_kv_heads, const int8_t* Wq_qkv, float g_qkv, const int8_t* Wq_out,
+                                 float g_out, const int8_t* Wq_gu, float g_gu, const int8_t* Wq_down, float g_down,
+                                 const int64_t* state_off, int64_t n_states, double theta, int threads) {
   const int64_t head_dim = d / n_heads;
   const int64_t n_qkv = d + 2 * n_kv_heads * head_dim;
   std::vector<uint16_t> u(static_cast<size_t>(T * std::max(d, d_ff)));
@@ -278,7 +335,10 @@ void oracle_encoder_block(uint16_t* h, int64_t T, int64_t d, int64_t d_ff, int64
   oracle_rmsnorm_bf16(h, T, d, u.data());
   oracle_bitlinear(u.data(), Wq_qkv, g_qkv, T, n_qkv, d, nullptr, nullptr, nullptr, nullptr, qkv.data(),
                    nullptr, threads);
-  oracle_identity_attention(qkv.data(), T, n_heads, n_kv_heads, head_dim, att.data());
+  if (state_off)
+    oracle_attention(qkv.data(), state_off, n_states, n_heads, n_kv_heads, head_dim, theta, att.data());
+  else
+    oracle_identity_attention(qkv.data(), T, n_heads, n_kv_heads, head_dim, att.data());
   oracle_rmsnorm_bf16(att.data(), T, d, u.data());
   oracle_bitlinear(u.data(), Wq_out, g_out, T, d, d, nullptr, nullptr, nullptr, nullptr, y.data(), nullptr,
                    threads);
@@ -292,6 +352,14 @@ void oracle_encoder_block(uint16_t* h, int64_t T, int64_t d, int64_t d_ff, int64
   oracle_bitlinear(u.data(), Wq_down, g_down, T, d, d_ff, nullptr, nullptr, nullptr, nullptr, y.data(),
                    nullptr, threads);
   oracle_residual_add(h, y.data(), T * d);
+}
+
+void oracle_encoder_block(uint16_t* h, int64_t T, int64_t d, int64_t d_ff, int64_t n_heads,
+                          int64_t n_kv_heads, const int8_t* Wq_qkv, float g_qkv, const int8_t* Wq_out,
+                          float g_out, const int8_t* Wq_gu, float g_gu, const int8_t* Wq_down, float g_down,
+                          int threads) {
+  oracle_encoder_block_states(h, T, d, d_ff, n_heads, n_kv_heads, Wq_qkv, g_qkv, Wq_out, g_out, Wq_gu, g_gu, Wq_down,
+                              g_down, nullptr, 0, 0.0, threads);
 }
 
 }  // extern "C"

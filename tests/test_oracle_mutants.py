@@ -93,6 +93,52 @@ def _attention_modulo(real, qkv, n_heads, n_kv_heads, head_dim):
     return np.stack([v[:, h % n_kv_heads] for h in range(n_heads)], axis=1).reshape(T, n_heads * head_dim)
 
 
+def _softmax_attention(real, qkv, states, n_heads, n_kv_heads, head_dim, theta, causal=True, scale=None,
+                       interleaved=False):
+    """A separate fp64 attention used only to plant mistakes (no mask / wrong scale / wrong rotary pairing)."""
+    x = pins.bits_to_f32(qkv).astype(np.float64)
+    T = x.shape[0]
+    S = int(states)
+    d, dkv, half = n_heads * head_dim, n_kv_heads * head_dim, head_dim // 2
+    scale = 1.0 / np.sqrt(head_dim) if scale is None else scale
+    out = np.zeros((T, d))
+
+    def rope(v, p):
+        ang = p * theta ** (-2.0 * np.arange(half) / head_dim)
+        if interleaved:
+            a, b = v[0::2], v[1::2]
+            r = np.empty_like(v)
+            r[0::2], r[1::2] = a * np.cos(ang) - b * np.sin(ang), b * np.cos(ang) + a * np.sin(ang)
+            return r
+        a, b = v[:half], v[half:]
+        return np.concatenate([a * np.cos(ang) - b * np.sin(ang), b * np.cos(ang) + a * np.sin(ang)])
+
+    for t0 in range(0, T, S):
+        for h in range(n_heads):
+            kv = h // (n_heads // n_kv_heads)
+            q = np.stack([rope(x[t0 + p, h * head_dim:(h + 1) * head_dim], p) for p in range(S)])
+            k = np.stack([rope(x[t0 + p, d + kv * head_dim:d + (kv + 1) * head_dim], p) for p in range(S)])
+            v = x[t0:t0 + S, d + dkv + kv * head_dim:d + dkv + (kv + 1) * head_dim]
+            sc = q @ k.T * scale
+            if causal:
+                sc = np.where(np.tril(np.ones((S, S), bool)), sc, -np.inf)
+            w = np.exp(sc - sc.max(axis=1, keepdims=True))
+            out[t0:t0 + S, h * head_dim:(h + 1) * head_dim] = (w / w.sum(axis=1, keepdims=True)) @ v
+    return pins.bf16_bits_of(out.astype(np.float32))
+
+
+def _attention_no_mask(real, *a):
+    return _softmax_attention(real, *a, causal=False)
+
+
+def _attention_no_scale(real, *a):
+    return _softmax_attention(real, *a, scale=1.0)
+
+
+def _attention_interleaved_rope(real, *a):
+    return _softmax_attention(real, *a, interleaved=True)
+
+
 def _relu2_without_square(real, gu):
     g = pins.bits_to_f32(gu)
     F = g.shape[1] // 2
@@ -104,7 +150,8 @@ PIN_TESTS = [pins.test_eq2_definition_fp64, pins.test_eq2_ties_are_strict, pins.
              pins.test_absmax_maps_to_127_and_zero_rows, pins.test_select_sum_add_subtract_skip,
              pins.test_negation_permutation_bound_allones, pins.test_pack_roundtrip_and_zero_matrix,
              pins.test_gaussian_closed_forms, pins.test_rescale_tolerances_and_bf16_rne,
-             pins.test_rmsnorm_against_fp64, pins.test_relu2_gate_identity_attention_residual]
+             pins.test_rmsnorm_against_fp64, pins.test_relu2_gate_identity_attention_residual,
+             pins.test_attention_against_library_sdpa, pins.test_attention_special_cases]
 
 
 def failing_pins(mod):
@@ -135,6 +182,9 @@ MUTANTS = {
     "rmsnorm: wrong statistics": {"rmsnorm_bf16": _rmsnorm_no_eps_wrong_len},
     "attention: modulo head map": {"identity_attention": _attention_modulo},
     "gate: relu without the square": {"relu2_gate": _relu2_without_square},
+    "attention: no causal mask": {"attention": _attention_no_mask},
+    "attention: missing 1/sqrt(head_dim)": {"attention": _attention_no_scale},
+    "attention: interleaved rotary pairs": {"attention": _attention_interleaved_rope},
 }
 
 

@@ -337,3 +337,91 @@ def test_encoder_block_is_the_composition(oracle_mod):
     h = o.residual_add(h, y)
     assert np.array_equal(got, h)
     assert got.shape == (T, 256) and np.isfinite(bits_to_f32(got)).all()
+
+
+# ------------------------------------------------------------------------- attention (survey's NEXT row f1)
+
+def _rope_complex(x, pos, theta):
+    """Independent formulation of the rotary embedding: the pair (x_i, x_{i+hd/2}) as a complex number times e^{i*angle}."""
+    hd = x.shape[-1]
+    half = hd // 2
+    ang = pos[:, None] * theta ** (-2.0 * np.arange(half) / hd)[None, :]
+    z = (x[..., :half] + 1j * x[..., half:]) * np.exp(1j * ang)
+    return np.concatenate([z.real, z.imag], axis=-1)
+
+
+def test_attention_against_library_sdpa(oracle_mod):
+    nh, nkv, hd, S, ns, theta = 4, 2, 16, 7, 3, 500000.0
+    qkv = inputs.activations(ns * S, (nh + 2 * nkv) * hd, 41, outliers=False)
+    got = bits_to_f32(oracle_mod.attention(inputs.bf16_bits(qkv), S, nh, nkv, hd, theta)).astype(np.float64)
+    x = qkv.double().numpy().reshape(ns, S, -1)
+    d, dkv = nh * hd, nkv * hd
+    pos = np.arange(S, dtype=np.float64)
+    q = np.stack([_rope_complex(x[:, :, h * hd:(h + 1) * hd].reshape(ns * S, hd), np.tile(pos, ns), theta)
+                  for h in range(nh)], 1).reshape(ns, S, nh, hd)
+    k = np.stack([_rope_complex(x[:, :, d + h * hd:d + (h + 1) * hd].reshape(ns * S, hd), np.tile(pos, ns), theta)
+                  for h in range(nkv)], 1).reshape(ns, S, nkv, hd)
+    v = x[:, :, d + dkv:].reshape(ns, S, nkv, hd)
+    rep = nh // nkv
+    qt = torch.from_numpy(q).permute(0, 2, 1, 3)
+    kt = torch.from_numpy(np.repeat(k, rep, axis=2)).permute(0, 2, 1, 3)
+    vt = torch.from_numpy(np.repeat(v, rep, axis=2)).permute(0, 2, 1, 3)
+    want = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, is_causal=True)
+    want = want.permute(0, 2, 1, 3).reshape(ns * S, nh * hd).numpy()
+    assert np.max(np.abs(got - want) / np.maximum(np.abs(want), 1e-2)) <= 2.0 ** -8
+
+
+def test_attention_special_cases(oracle_mod):
+    nh, nkv, hd, theta = 4, 2, 16, 10000.0
+    W = (nh + 2 * nkv) * hd
+    d, dkv = nh * hd, nkv * hd
+    # one token per state: the softmax is 1 and the output is V - exactly the "identity on V" block of the benchmark
+    qkv1 = inputs.bf16_bits(inputs.activations(9, W, 42, outliers=False))
+    assert np.array_equal(oracle_mod.attention(qkv1, 1, nh, nkv, hd, theta),
+                          oracle_mod.identity_attention(qkv1, nh, nkv, hd))
+    # q = 0: uniform causal weights, output = running mean of V
+    S = 6
+    x = inputs.activations(2 * S, W, 43, outliers=False).float().numpy()
+    x[:, :d] = 0.0
+    out = bits_to_f32(oracle_mod.attention(bf16_bits_of(x), S, nh, nkv, hd, theta)).astype(np.float64)
+    xv = bits_to_f32(bf16_bits_of(x)).astype(np.float64)[:, d + dkv:].reshape(2, S, nkv, hd)
+    run = np.cumsum(xv, axis=1) / np.arange(1, S + 1)[None, :, None, None]
+    want = np.repeat(run, nh // nkv, axis=2).reshape(2 * S, d)
+    assert np.max(np.abs(out - want)) <= 2.0 ** -8 * np.max(np.abs(want)) + 1e-6
+    # causality: changing later tokens does not change earlier outputs; states do not see each other
+    y = inputs.activations(2 * S, W, 44, outliers=False).float().numpy()
+    base = oracle_mod.attention(bf16_bits_of(y), S, nh, nkv, hd, theta)
+    y2 = y.copy()
+    y2[4:6] += 1.0          # tokens 4, 5 of state 0
+    pert = oracle_mod.attention(bf16_bits_of(y2), S, nh, nkv, hd, theta)
+    assert np.array_equal(pert[:4], base[:4]) and np.array_equal(pert[S:], base[S:])
+    assert not np.array_equal(pert[4:6], base[4:6])
+    # constant V: every output equals that constant (weights sum to one)
+    z = inputs.activations(S, W, 45, outliers=False).float().numpy()
+    z[:, d + dkv:] = 0.75
+    assert np.all(bits_to_f32(oracle_mod.attention(bf16_bits_of(z), S, nh, nkv, hd, theta)) == 0.75)
+
+
+def test_attention_ragged_states_equal_separate_calls(oracle_mod):
+    nh, nkv, hd, theta = 4, 2, 16, 500000.0
+    lens = [3, 1, 8, 5]
+    off = np.concatenate([[0], np.cumsum(lens)])
+    qkv = inputs.bf16_bits(inputs.activations(int(off[-1]), (nh + 2 * nkv) * hd, 46, outliers=False))
+    whole = oracle_mod.attention(qkv, off, nh, nkv, hd, theta)
+    for s, n in enumerate(lens):
+        part = oracle_mod.attention(qkv[off[s]:off[s + 1]], n, nh, nkv, hd, theta)
+        assert np.array_equal(whole[off[s]:off[s + 1]], part)
+
+
+def test_encoder_block_with_one_token_states_is_the_identity_attention_block(oracle_mod):
+    """A state of one token attends to itself only, so the block with real attention reduces to the benchmark block."""
+    d, d_ff, nh, nkv = 128, 256, 4, 2
+    layer = []
+    for j, (N, K) in enumerate([(d + 2 * nkv * (d // nh), d), (d, d), (2 * d_ff, d), (d, d_ff)]):
+        layer.append(oracle_mod.ternarize(inputs.master_weights(N, K, 900 + j).numpy()))
+    h = inputs.bf16_bits(inputs.activations(6, d, 47))
+    a = oracle_mod.encoder_block(h, d_ff, nh, nkv, layer, threads=1)
+    b = oracle_mod.encoder_block(h, d_ff, nh, nkv, layer, threads=1, states=1)
+    c = oracle_mod.encoder_block(h, d_ff, nh, nkv, layer, threads=1, states=3)
+    assert np.array_equal(a, b) and not np.array_equal(a, c)
+    assert np.array_equal(a[[0, 3]], c[[0, 3]])   # the first token of each state sees only itself
