@@ -379,6 +379,23 @@ def run_ours(args):
             "states_per_s": 128.0 / (mse * 1e-3), "ms": mse, "TOPS": enc_ops / (mse * 1e-3) / 1e12,
             "frac_of_int8_peak_sustained": enc_ops / (mse * 1e-3) / 1e12 / i8_sus, "launches": le}
         del ge
+        # the same stack with real attention inside each state: equal 32-token states, then ragged 15-40-token ones
+        pooled = torch.empty((128, 2560), dtype=torch.bfloat16, device=dev)
+        off = inputs.state_offsets(128, 7000)
+        Tr = int(off[-1])
+        cases = (("uniform32", T, 32, h0, h1),
+                 ("ragged15to40", Tr, (off.to(torch.int32).to(dev), inputs.STATE_TOKENS_MAX),
+                  inputs.activations(Tr, 2560, 6001).to(dev), torch.empty((Tr, 2560), dtype=torch.bfloat16, device=dev)))
+        for label, Tc, states, hin, hout in cases:
+            max_len = states if isinstance(states, int) else states[1]
+            aws = torch.empty((enc.states_workspace_bytes(Tc, max_len),), dtype=torch.uint8, device=dev)
+            ga, la = capture(lambda: enc.forward_states(hin, states, h_out=hout, pooled=pooled, workspace=aws))
+            msa = time_graph(ga, sub_steps, args.warmup, 1) / sub_steps
+            ops = 2.0 * Tc * sum(k * n for _, k, n in BLOCK) * n_layers
+            extra[f"encoder_{n_layers}_blocks_attention_{label}"] = {
+                "states_per_s": 128.0 / (msa * 1e-3), "ms": msa, "tokens": Tc, "bitlinear_TOPS": ops / (msa * 1e-3) / 1e12,
+                "frac_of_int8_peak_sustained": ops / (msa * 1e-3) / 1e12 / i8_sus, "launches": la}
+            del ga, aws
     bitrl.poll_status()
     clocks_sections = sampler2.stop() if sampler2 else None
     if rank == 0 and "cpu" in sections:

@@ -41,7 +41,7 @@ extern "C" {
 typedef int32_t bitrl_status;
 #define BITRL_OK 0
 #define BITRL_ERR_NULL (-1)      /* a required pointer is NULL */
-#define BITRL_ERR_SHAPE (-2)     /* M < 1, K or N not a multiple of 128, shape does not match the handle */
+#define BITRL_ERR_SHAPE (-2)     /* M < 1, K or N not a multiple of 128, shape does not match the handle, bad state offsets */
 #define BITRL_ERR_ALIGN (-3)     /* a device pointer is not 16-byte aligned */
 #define BITRL_ERR_ARCH (-4)      /* current device is not compute capability 10.0 */
 #define BITRL_ERR_CUDA (-5)      /* a CUDA call failed; code in bitrl_last_cuda_error() */
@@ -159,6 +159,41 @@ BITRL_API bitrl_status bitrl_encoder_destroy(bitrl_encoder_t* enc);
 BITRL_API size_t bitrl_encoder_workspace_bytes(const bitrl_encoder_t* enc, int32_t T);
 BITRL_API bitrl_status bitrl_encoder_forward(const bitrl_encoder_t* enc, const void* h_in, int32_t T, void* h_out,
                                    void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---- attention inside each state (the step of the encoder block that the contraction feeds; Eq. 3 encodes every
+ * state s_t on its own, Sec. V: 15-40 tokens per state, one forward pass) --------------------------------------
+ * Causal grouped-query attention with rotary position embedding (rotate-half form) over independent states:
+ *   angle(p, i) = p * theta^(-2i/head_dim), p = index of the token inside its state, i < head_dim/2
+ *   (x_i, x_{i+hd/2}) -> (x_i cos - x_{i+hd/2} sin, x_{i+hd/2} cos + x_i sin)          applied to q and k
+ *   att[p] = sum_{r<=p} softmax_r(q_p . k_r / sqrt(head_dim)) v_r ; query head h reads kv head h / (n_heads/n_kv_heads)
+ * fp32 arithmetic, cos/sin from an fp64 table, one rounding to bf16.
+ * qkv: dev bf16 [T, (n_heads + 2 n_kv_heads) * head_dim] = [q | k | v].  att: dev bf16 [T, n_heads * head_dim].
+ * States: state_off = dev int32 [n_states + 1], ascending token offsets with state_off[0] = 0 and
+ * state_off[n_states] = T, every length in 1..max_state_len; or NULL, then every state has max_state_len tokens and
+ * T = n_states * max_state_len.  max_state_len <= BITRL_ATTN_MAX_STATE_TOKENS; head_dim is 64 or 128.
+ * Offsets are read on the device: a state that breaks the rules above is skipped (its rows of att are not written)
+ * and the next bitrl_poll_status returns BITRL_ERR_SHAPE.
+ * workspace: dev, >= bitrl_attention_workspace_bytes(max_state_len, head_dim) (the rotary table). */
+#define BITRL_ATTN_MAX_STATE_TOKENS 128
+BITRL_API size_t bitrl_attention_workspace_bytes(int32_t max_state_len, int32_t head_dim);
+BITRL_API bitrl_status bitrl_attention(const void* qkv, int32_t T, const int32_t* state_off, int32_t n_states,
+                                       int32_t max_state_len, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim,
+                                       double theta, void* att, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Last-token pooling: out[s, :] = h[last token of state s, :], the latent h_t of Eq. 3 (one per state).
+ * h: dev bf16 [T, d]; out: dev bf16 [n_states, d]; d a multiple of 8; states as for bitrl_attention. */
+BITRL_API bitrl_status bitrl_pool_last_token(const void* h, int32_t T, const int32_t* state_off, int32_t n_states,
+                                             int32_t max_state_len, int32_t d, void* out, void* stream);
+
+/* The encoder with real attention in place of the identity on V:
+ *   h += out(RMSNorm(attention(qkv(RMSNorm(h)))));  h += down(RMSNorm(relu(g)^2 * up))      per block,
+ * states and theta as for bitrl_attention.  pooled: NULL, or dev bf16 [n_states, d] that receives the last token
+ * of every state after the last block.  workspace >= bitrl_encoder_states_workspace_bytes(enc, T, max_state_len). */
+BITRL_API size_t bitrl_encoder_states_workspace_bytes(const bitrl_encoder_t* enc, int32_t T, int32_t max_state_len);
+BITRL_API bitrl_status bitrl_encoder_forward_states(const bitrl_encoder_t* enc, const void* h_in, int32_t T,
+                                                    const int32_t* state_off, int32_t n_states, int32_t max_state_len,
+                                                    double theta, void* h_out, void* pooled, void* workspace,
+                                                    size_t workspace_bytes, void* stream);
 
 /* ---- status ----------------------------------------------------------------------------------------- */
 /* Synchronizes `stream`, then reads and clears the device status word.  BITRL_OK, BITRL_ERR_TIMEOUT (a kernel

@@ -6,8 +6,8 @@ exception is raised.
 
 The functions mirror the C names without the ``bitrl_`` prefix:
 ``pack_ternary``, ``Linear`` (create/destroy), ``quant_act``, ``bitlinear_forward``, ``bitlinear_forward_debug``,
-``bitlinear_forward_q``, ``rmsnorm_quant``, ``vrepeat_rmsnorm_quant``, ``relu2gate_rmsnorm_quant``, ``Encoder``,
-``poll_status``.
+``bitlinear_forward_q``, ``rmsnorm_quant``, ``vrepeat_rmsnorm_quant``, ``relu2gate_rmsnorm_quant``, ``attention``,
+``pool_last_token``, ``Encoder`` (``forward``, ``forward_states``), ``poll_status``.
 """
 from __future__ import annotations
 
@@ -49,6 +49,11 @@ EXPORTS = {
     "bitrl_encoder_destroy": (_i32, [_vp]),
     "bitrl_encoder_workspace_bytes": (_sz, [_vp, _i32]),
     "bitrl_encoder_forward": (_i32, [_vp, _vp, _i32, _vp, _vp, _sz, _vp]),
+    "bitrl_attention_workspace_bytes": (_sz, [_i32, _i32]),
+    "bitrl_attention": (_i32, [_vp, _i32, _vp, _i32, _i32, _i32, _i32, _i32, ctypes.c_double, _vp, _vp, _sz, _vp]),
+    "bitrl_pool_last_token": (_i32, [_vp, _i32, _vp, _i32, _i32, _i32, _vp, _vp]),
+    "bitrl_encoder_states_workspace_bytes": (_sz, [_vp, _i32, _i32]),
+    "bitrl_encoder_forward_states": (_i32, [_vp, _vp, _i32, _vp, _i32, _i32, ctypes.c_double, _vp, _vp, _vp, _sz, _vp]),
     "bitrl_selftest_wait_timeout": (_i32, [ctypes.c_int64, _vp]),
     "bitrl_poll_status": (_i32, [_vp]),
     "bitrl_last_timeout_stage": (_i32, []),
@@ -300,6 +305,48 @@ def relu2gate_rmsnorm_quant(gu: torch.Tensor, want_u: bool = False):
     return xq, a, rs, u
 
 
+ATTN_MAX_STATE_TOKENS = 128
+ROPE_THETA = 500000.0
+
+
+def _states(states, T: int, device):
+    """``states``: an int (every state has that many tokens) or a CUDA int32 tensor of offsets [n_states+1] together
+    with the largest length, as a tuple ``(offsets, max_len)``.  Returns (offsets or None, n_states, max_len)."""
+    if isinstance(states, int):
+        if T % states != 0:
+            raise ValueError("T is not a multiple of the common state length")
+        return None, T // states, states
+    off, max_len = states
+    _dev(off, torch.int32, "state offsets")
+    return off, off.numel() - 1, int(max_len)
+
+
+def attention(qkv: torch.Tensor, states, n_heads: int, n_kv_heads: int, head_dim: int,
+              theta: float = ROPE_THETA) -> torch.Tensor:
+    """Causal GQA attention with rotary embedding inside each state: qkv bf16 [T, (nh+2nkv)*hd] -> att bf16 [T, nh*hd]."""
+    _dev(qkv, torch.bfloat16, "qkv")
+    T = qkv.shape[0]
+    assert qkv.shape[1] == (n_heads + 2 * n_kv_heads) * head_dim
+    off, n_states, max_len = _states(states, T, qkv.device)
+    att = torch.empty((T, n_heads * head_dim), dtype=torch.bfloat16, device=qkv.device)
+    nbytes = max(int(lib().bitrl_attention_workspace_bytes(max_len, head_dim)), 16)
+    ws = torch.empty((nbytes,), dtype=torch.uint8, device=qkv.device)
+    _check(lib().bitrl_attention(_ptr(qkv), T, _ptr(off), n_states, max_len, n_heads, n_kv_heads, head_dim,
+                                 float(theta), _ptr(att), _ptr(ws), nbytes, _stream()), "bitrl_attention")
+    return att
+
+
+def pool_last_token(h: torch.Tensor, states) -> torch.Tensor:
+    """h bf16 [T,d] -> bf16 [n_states,d]: the last token of every state."""
+    _dev(h, torch.bfloat16, "h")
+    T, d = h.shape
+    off, n_states, max_len = _states(states, T, h.device)
+    out = torch.empty((n_states, d), dtype=torch.bfloat16, device=h.device)
+    _check(lib().bitrl_pool_last_token(_ptr(h), T, _ptr(off), n_states, max_len, d, _ptr(out), _stream()),
+           "bitrl_pool_last_token")
+    return out
+
+
 class Encoder:
     """Owns a ``bitrl_encoder_t`` over ``layers`` = list of (qkv, out, gateup, down) ``Linear`` tuples."""
 
@@ -327,6 +374,27 @@ class Encoder:
         _check(lib().bitrl_encoder_forward(self.handle, _ptr(h_in), T, _ptr(h_out), _ptr(workspace), workspace.numel(),
                                            _stream()), "bitrl_encoder_forward")
         return h_out
+
+    def states_workspace_bytes(self, T: int, max_state_len: int) -> int:
+        return int(lib().bitrl_encoder_states_workspace_bytes(self.handle, T, max_state_len))
+
+    def forward_states(self, h_in: torch.Tensor, states, theta: float = ROPE_THETA, h_out: torch.Tensor | None = None,
+                       pooled: torch.Tensor | None = None, want_pooled: bool = False,
+                       workspace: torch.Tensor | None = None):
+        """The encoder with real attention inside each state; returns h_out, or (h_out, pooled) when pooling."""
+        _dev(h_in, torch.bfloat16, "h_in")
+        T = h_in.shape[0]
+        off, n_states, max_len = _states(states, T, h_in.device)
+        if h_out is None:
+            h_out = torch.empty_like(h_in)
+        if pooled is None and want_pooled:
+            pooled = torch.empty((n_states, self.d), dtype=torch.bfloat16, device=h_in.device)
+        if workspace is None:
+            workspace = torch.empty((self.states_workspace_bytes(T, max_len),), dtype=torch.uint8, device=h_in.device)
+        _check(lib().bitrl_encoder_forward_states(self.handle, _ptr(h_in), T, _ptr(off), n_states, max_len,
+                                                  float(theta), _ptr(h_out), _ptr(pooled), _ptr(workspace),
+                                                  workspace.numel(), _stream()), "bitrl_encoder_forward_states")
+        return (h_out, pooled) if pooled is not None else h_out
 
     def close(self):
         if getattr(self, "handle", None):

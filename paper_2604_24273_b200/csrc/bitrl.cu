@@ -73,6 +73,7 @@ static bitrl_status check_arch() {
 #include "gemv.cuh"
 #include "gemv_multi.cuh"
 #include "gemm.cuh"
+#include "attention.cuh"
 
 using namespace bitrl;
 
@@ -369,9 +370,11 @@ struct EncWs {
   float* absmax;    // [T]
   int32_t* rowsum;  // [T]
   unsigned short* wide;  // [T, max(n_qkv, 2 d_ff)] bf16: qkv, then gate/up
+  unsigned short* att;   // [T, d] bf16 attention output (only with real attention)
+  float2* rope;          // [max_state_len, head_dim/2] rotary table (only with real attention)
   size_t bytes;
 };
-EncWs carve_enc(void* ws, const bitrl_encoder* e, int T) {
+EncWs carve_enc(void* ws, const bitrl_encoder* e, int T, int max_state_len) {
   EncWs w;
   size_t off = 0;
   unsigned char* b = static_cast<unsigned char*>(ws);
@@ -386,14 +389,64 @@ EncWs carve_enc(void* ws, const bitrl_encoder* e, int T) {
   off += align_up(static_cast<size_t>(T) * 4, 256);
   w.wide = reinterpret_cast<unsigned short*>(b + off);
   off += align_up(static_cast<size_t>(T) * wmax * 2, 256);
+  w.att = nullptr;
+  w.rope = nullptr;
+  if (max_state_len > 0) {
+    w.att = reinterpret_cast<unsigned short*>(b + off);
+    off += align_up(static_cast<size_t>(T) * e->d * 2, 256);
+    w.rope = reinterpret_cast<float2*>(b + off);
+    off += rope_table_bytes(max_state_len, e->head_dim);
+  }
   w.bytes = off;
   return w;
+}
+
+bool attention_shape_ok(int n_heads, int n_kv_heads, int head_dim, int max_state_len) {
+  return n_heads >= 1 && n_kv_heads >= 1 && n_heads % n_kv_heads == 0 && (head_dim == 64 || head_dim == 128) &&
+         max_state_len >= 1 && max_state_len <= BITRL_ATTN_MAX_STATE_TOKENS;
+}
+
+// One pass over the blocks.  max_state_len == 0: identity attention (V repeated); else real attention per state.
+bitrl_status encoder_run(const bitrl_encoder_t* enc, const void* h_in, int32_t T, const int32_t* state_off,
+                         int32_t n_states, int32_t max_state_len, double theta, void* h_out, void* pooled,
+                         void* workspace, cudaStream_t st) {
+  bitrl_status s;
+  EncWs w = carve_enc(workspace, enc, T, max_state_len);
+  const int d = enc->d, F = enc->d_ff;
+  if (h_out != h_in)
+    BITRL_CUDA(cudaMemcpyAsync(h_out, h_in, static_cast<size_t>(T) * d * 2, cudaMemcpyDeviceToDevice, st));
+  if (max_state_len > 0 && (s = launch_rope_table(w.rope, max_state_len, enc->head_dim, theta, st)) != BITRL_OK) return s;
+  auto linear = [&](const bitrl_linear* lin, void* y, const void* residual) -> bitrl_status {
+    if (gemv_fits(T, lin->l.K))
+      return launch_gemv(&lin->l, nullptr, w.xq, w.absmax, T, y, BITRL_OUT_BF16, residual, nullptr, nullptr, nullptr, st);
+    return launch_gemm(&lin->l, w.xq, w.absmax, w.rowsum, T, y, BITRL_OUT_BF16, residual, nullptr, st);
+  };
+  for (int l = 0; l < enc->L; ++l) {
+    const bitrl_linear* const* q = enc->layers.data() + 4 * l;
+    if ((s = launch_rmsnorm_quant(h_out, T, d, w.xq, w.absmax, w.rowsum, nullptr, st)) != BITRL_OK) return s;
+    if ((s = linear(q[0], w.wide, nullptr)) != BITRL_OK) return s;
+    if (max_state_len > 0) {
+      if ((s = launch_attention(w.wide, T, state_off, n_states, max_state_len, enc->n_heads, enc->n_kv_heads,
+                                enc->head_dim, w.rope, w.att, st)) != BITRL_OK) return s;
+      if ((s = launch_rmsnorm_quant(w.att, T, d, w.xq, w.absmax, w.rowsum, nullptr, st)) != BITRL_OK) return s;
+    } else {
+      if ((s = launch_vrepeat_rmsnorm_quant(w.wide, T, enc->n_heads, enc->n_kv_heads, enc->head_dim, w.xq, w.absmax,
+                                            w.rowsum, nullptr, st)) != BITRL_OK) return s;
+    }
+    if ((s = linear(q[1], h_out, h_out)) != BITRL_OK) return s;
+    if ((s = launch_rmsnorm_quant(h_out, T, d, w.xq, w.absmax, w.rowsum, nullptr, st)) != BITRL_OK) return s;
+    if ((s = linear(q[2], w.wide, nullptr)) != BITRL_OK) return s;
+    if ((s = launch_relu2gate_rmsnorm_quant(w.wide, T, F, w.xq, w.absmax, w.rowsum, nullptr, st)) != BITRL_OK) return s;
+    if ((s = linear(q[3], h_out, h_out)) != BITRL_OK) return s;
+  }
+  if (pooled) return launch_pool_last_token(h_out, T, state_off, n_states, max_state_len, d, pooled, st);
+  return BITRL_OK;
 }
 }  // namespace
 
 size_t bitrl_encoder_workspace_bytes(const bitrl_encoder_t* enc, int32_t T) {
   if (!enc || T < 1) return 0;
-  return carve_enc(nullptr, enc, T).bytes;
+  return carve_enc(nullptr, enc, T, 0).bytes;
 }
 
 bitrl_status bitrl_encoder_forward(const bitrl_encoder_t* enc, const void* h_in, int32_t T, void* h_out,
@@ -404,29 +457,64 @@ bitrl_status bitrl_encoder_forward(const bitrl_encoder_t* enc, const void* h_in,
   if (!aligned16(h_in) || !aligned16(h_out) || !aligned16(workspace)) return BITRL_ERR_ALIGN;
   bitrl_status s = check_arch();
   if (s != BITRL_OK) return s;
+  return encoder_run(enc, h_in, T, nullptr, 0, 0, 0.0, h_out, nullptr, workspace, static_cast<cudaStream_t>(stream));
+}
+
+size_t bitrl_encoder_states_workspace_bytes(const bitrl_encoder_t* enc, int32_t T, int32_t max_state_len) {
+  if (!enc || T < 1 || max_state_len < 1) return 0;
+  return carve_enc(nullptr, enc, T, max_state_len).bytes;
+}
+
+bitrl_status bitrl_encoder_forward_states(const bitrl_encoder_t* enc, const void* h_in, int32_t T,
+                                          const int32_t* state_off, int32_t n_states, int32_t max_state_len,
+                                          double theta, void* h_out, void* pooled, void* workspace,
+                                          size_t workspace_bytes, void* stream) {
+  if (!enc || !h_in || !h_out) return BITRL_ERR_NULL;
+  if (T < 1 || n_states < 1 || !(theta > 0.0)) return BITRL_ERR_SHAPE;
+  if (!attention_shape_ok(enc->n_heads, enc->n_kv_heads, enc->head_dim, max_state_len)) return BITRL_ERR_SHAPE;
+  if (!state_off && static_cast<long long>(n_states) * max_state_len != T) return BITRL_ERR_SHAPE;
+  if (!workspace || workspace_bytes < bitrl_encoder_states_workspace_bytes(enc, T, max_state_len))
+    return BITRL_ERR_WORKSPACE;
+  if (!aligned16(h_in) || !aligned16(h_out) || !aligned16(workspace) || !aligned16(pooled)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  return encoder_run(enc, h_in, T, state_off, n_states, max_state_len, theta, h_out, pooled, workspace,
+                     static_cast<cudaStream_t>(stream));
+}
+
+// ---- attention inside each state, last-token pooling ------------------------------------------------------
+
+size_t bitrl_attention_workspace_bytes(int32_t max_state_len, int32_t head_dim) {
+  if (max_state_len < 1 || head_dim < 2) return 0;
+  return rope_table_bytes(max_state_len, head_dim);
+}
+
+bitrl_status bitrl_attention(const void* qkv, int32_t T, const int32_t* state_off, int32_t n_states,
+                             int32_t max_state_len, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim,
+                             double theta, void* att, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!qkv || !att) return BITRL_ERR_NULL;
+  if (T < 1 || n_states < 1 || !(theta > 0.0)) return BITRL_ERR_SHAPE;
+  if (!attention_shape_ok(n_heads, n_kv_heads, head_dim, max_state_len)) return BITRL_ERR_SHAPE;
+  if (!state_off && static_cast<long long>(n_states) * max_state_len != T) return BITRL_ERR_SHAPE;
+  if (!workspace || workspace_bytes < bitrl_attention_workspace_bytes(max_state_len, head_dim)) return BITRL_ERR_WORKSPACE;
+  if (!aligned16(qkv) || !aligned16(att) || !aligned16(workspace)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  EncWs w = carve_enc(workspace, enc, T);
-  const int d = enc->d, F = enc->d_ff;
-  if (h_out != h_in)
-    BITRL_CUDA(cudaMemcpyAsync(h_out, h_in, static_cast<size_t>(T) * d * 2, cudaMemcpyDeviceToDevice, st));
-  auto linear = [&](const bitrl_linear* lin, void* y, const void* residual) -> bitrl_status {
-    if (gemv_fits(T, lin->l.K))
-      return launch_gemv(&lin->l, nullptr, w.xq, w.absmax, T, y, BITRL_OUT_BF16, residual, nullptr, nullptr, nullptr, st);
-    return launch_gemm(&lin->l, w.xq, w.absmax, w.rowsum, T, y, BITRL_OUT_BF16, residual, nullptr, st);
-  };
-  for (int l = 0; l < enc->L; ++l) {
-    const bitrl_linear* const* q = enc->layers.data() + 4 * l;
-    if ((s = launch_rmsnorm_quant(h_out, T, d, w.xq, w.absmax, w.rowsum, nullptr, st)) != BITRL_OK) return s;
-    if ((s = linear(q[0], w.wide, nullptr)) != BITRL_OK) return s;
-    if ((s = launch_vrepeat_rmsnorm_quant(w.wide, T, enc->n_heads, enc->n_kv_heads, enc->head_dim, w.xq, w.absmax,
-                                          w.rowsum, nullptr, st)) != BITRL_OK) return s;
-    if ((s = linear(q[1], h_out, h_out)) != BITRL_OK) return s;
-    if ((s = launch_rmsnorm_quant(h_out, T, d, w.xq, w.absmax, w.rowsum, nullptr, st)) != BITRL_OK) return s;
-    if ((s = linear(q[2], w.wide, nullptr)) != BITRL_OK) return s;
-    if ((s = launch_relu2gate_rmsnorm_quant(w.wide, T, F, w.xq, w.absmax, w.rowsum, nullptr, st)) != BITRL_OK) return s;
-    if ((s = linear(q[3], h_out, h_out)) != BITRL_OK) return s;
-  }
-  return BITRL_OK;
+  float2* rope = static_cast<float2*>(workspace);
+  if ((s = launch_rope_table(rope, max_state_len, head_dim, theta, st)) != BITRL_OK) return s;
+  return launch_attention(qkv, T, state_off, n_states, max_state_len, n_heads, n_kv_heads, head_dim, rope, att, st);
+}
+
+bitrl_status bitrl_pool_last_token(const void* h, int32_t T, const int32_t* state_off, int32_t n_states,
+                                   int32_t max_state_len, int32_t d, void* out, void* stream) {
+  if (!h || !out) return BITRL_ERR_NULL;
+  if (T < 1 || n_states < 1 || max_state_len < 1 || d < 8 || d % 8 != 0) return BITRL_ERR_SHAPE;
+  if (!state_off && static_cast<long long>(n_states) * max_state_len != T) return BITRL_ERR_SHAPE;
+  if (!aligned16(h) || !aligned16(out)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  return launch_pool_last_token(h, T, state_off, n_states, max_state_len, d, out, static_cast<cudaStream_t>(stream));
 }
 
 // ---- self-test of the bounded-wait / status-word path ----

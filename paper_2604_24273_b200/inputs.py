@@ -8,7 +8,8 @@ Recipe (stands in for the real BitNet b1.58 weights and real serialized-state ac
 available offline):
   * master weights: fp32, N(0, sigma=0.02), shape [N_out, K_in];
   * activations: N(0,1) fp32; a fixed 1 % of the K channels (chosen by a seeded permutation) is
-    multiplied by 20 to imitate outlier channels; the result is cast to bf16.
+    multiplied by 20 to imitate outlier channels; the result is cast to bf16;
+  * states: 15-40 tokens each (uniform), the range the paper reports for serialized states.
 """
 from __future__ import annotations
 
@@ -58,6 +59,15 @@ def encoder_layer_weights(layer: int, seed: int = 5000, dims: dict | None = None
     n_qkv = d + 2 * e["n_kv_heads"] * hd
     shapes = [(n_qkv, d), (d, d), (2 * d_ff, d), (d, d_ff)]
     return [master_weights(n, k, seed + 4 * layer + j) for j, (n, k) in enumerate(shapes)]
+
+
+STATE_TOKENS_MIN, STATE_TOKENS_MAX = 15, 40  # tokens per serialized state (the range the paper reports, Sec. V)
+
+
+def state_offsets(n_states: int, seed: int, lo: int = STATE_TOKENS_MIN, hi: int = STATE_TOKENS_MAX) -> torch.Tensor:
+    """Token offsets [n_states+1] (int64, CPU) of states whose lengths are uniform integers in [lo, hi]."""
+    lens = torch.randint(lo, hi + 1, (n_states,), generator=_gen(seed), dtype=torch.int64)
+    return torch.cat([torch.zeros(1, dtype=torch.int64), torch.cumsum(lens, 0)])
 
 
 def bf16_bits(t: torch.Tensor):

@@ -1,0 +1,240 @@
+"""GPU parity of the attention step, last-token pooling and the encoder with real attention, through the C ABI,
+against the CPU oracle on the same seeded inputs.
+
+The oracle computes attention in fp64 and rounds once to bf16; the kernel computes in fp32 and rounds once.  An
+output is a convex combination of the values v_r of its column, so the fp32 path carries an absolute error of a few
+fp32 ulps of max_r |v_r| (64-128 fused multiply-adds per dot product, up to 128 keys): tolerance 4e-6 * max|v| of
+the column.  Outputs that are not tiny therefore agree to the bf16 bit, or differ in the last bit when that error
+crosses a rounding boundary (required: at most 0.5 % of the elements); outputs near zero (cancellation) may differ
+by more bf16 ulps but still lie within the absolute bound.  The integer stages that follow are checked by teacher
+forcing on the GPU's own bf16 values, bit-exactly.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2604_24273_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+THETA = 500000.0
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_24273_b200 import bitrl
+
+    bitrl.lib()
+    torch.cuda.set_device(0)
+    return bitrl
+
+
+def bits(t):
+    return inputs.bf16_bits(t.detach().cpu())
+
+
+def ulp_diff_bf16(a_bits, b_bits):
+    def key(u):
+        u = u.astype(np.int32)
+        return np.where(u & 0x8000, 0x8000 - u, u)
+    return np.abs(key(a_bits) - key(b_bits))
+
+
+def to_f64(b):
+    return (np.asarray(b, np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+ATOL_REL_TO_VMAX = 4e-6
+MAX_MISMATCH_FRACTION = 5e-3
+
+
+def check_attention(got_bits, want_bits, qkv_bits, nh, nkv, hd):
+    d = ulp_diff_bf16(got_bits, want_bits)
+    vmax = np.abs(to_f64(qkv_bits)[:, (nh + nkv) * hd:]).max(0).reshape(nkv, hd)
+    atol = ATOL_REL_TO_VMAX * np.repeat(vmax, nh // nkv, axis=0).reshape(-1)  # column of query head h <- kv head h/rep
+    err = np.abs(to_f64(got_bits) - to_f64(want_bits))
+    ok = (d <= 1) | (err <= atol[None, :])
+    assert ok.all(), f"{(~ok).sum()} outputs beyond one bf16 ulp and beyond the absolute bound (max {d.max()} ulps)"
+    assert (d != 0).mean() <= MAX_MISMATCH_FRACTION, f"{(d != 0).mean():.4f} of the outputs differ from the oracle"
+
+
+def dev_states(off64):
+    off = off64.to(torch.int32).cuda()
+    return off, int((off64[1:] - off64[:-1]).max())
+
+
+@pytest.mark.parametrize("nh,nkv,hd", [(20, 5, 128), (2, 1, 128), (6, 3, 64), (3, 3, 128), (8, 1, 64)])
+@pytest.mark.parametrize("S,n_states", [(32, 3), (1, 4), (17, 2), (40, 2), (64, 1), (100, 1), (128, 1)])
+def test_attention_equal_states(oracle_mod, B, nh, nkv, hd, S, n_states):
+    T = S * n_states
+    qkv = inputs.activations(T, (nh + 2 * nkv) * hd, 7100 + S, outliers=False)
+    att = B.attention(qkv.cuda(), S, nh, nkv, hd, THETA)
+    B.poll_status()
+    want = oracle_mod.attention(bits(qkv), S, nh, nkv, hd, THETA)
+    check_attention(bits(att), want, bits(qkv), nh, nkv, hd)
+
+
+@pytest.mark.parametrize("n_states,seed", [(7, 1), (40, 2)])
+def test_attention_ragged_states(oracle_mod, B, n_states, seed):
+    """States of 15-40 tokens, the backbone's head geometry."""
+    nh, nkv, hd = 20, 5, 128
+    off = inputs.state_offsets(n_states, 7200 + seed)
+    T = int(off[-1])
+    qkv = inputs.activations(T, (nh + 2 * nkv) * hd, 7300 + seed)
+    o32, max_len = dev_states(off)
+    att = B.attention(qkv.cuda(), (o32, max_len), nh, nkv, hd, THETA)
+    B.poll_status()
+    want = oracle_mod.attention(bits(qkv), off.numpy(), nh, nkv, hd, THETA)
+    check_attention(bits(att), want, bits(qkv), nh, nkv, hd)
+    # a larger allowed maximum (other kernel variant) gives the same bits
+    att2 = B.attention(qkv.cuda(), (o32, 128), nh, nkv, hd, THETA)
+    att3 = B.attention(qkv.cuda(), (o32, 64), nh, nkv, hd, THETA)
+    B.poll_status()
+    assert torch.equal(att, att2) and torch.equal(att, att3)
+
+
+def test_attention_other_theta_and_determinism(oracle_mod, B):
+    nh, nkv, hd, S = 4, 2, 128, 24
+    qkv = inputs.activations(2 * S, (nh + 2 * nkv) * hd, 7400, outliers=False)
+    a1 = B.attention(qkv.cuda(), S, nh, nkv, hd, 10000.0)
+    a2 = B.attention(qkv.cuda(), S, nh, nkv, hd, 10000.0)
+    B.poll_status()
+    assert torch.equal(a1, a2)
+    check_attention(bits(a1), oracle_mod.attention(bits(qkv), S, nh, nkv, hd, 10000.0), bits(qkv), nh, nkv, hd)
+
+
+def test_attention_bad_states_reported_not_faulted(oracle_mod, B):
+    """Offsets are read on the device: a state longer than the stated maximum (or running past T) is skipped and
+    reported by the status word; the other states are still computed and the context stays usable."""
+    nh, nkv, hd = 2, 1, 128
+    off = torch.tensor([0, 10, 60, 70], dtype=torch.int64)  # middle state has 50 tokens
+    qkv = inputs.activations(70, (nh + 2 * nkv) * hd, 7500, outliers=False)
+    o32 = off.to(torch.int32).cuda()
+    lib = B.lib()
+    att = torch.zeros((70, nh * hd), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty((max(lib.bitrl_attention_workspace_bytes(32, hd), 16),), dtype=torch.uint8, device="cuda")
+    st = lib.bitrl_attention(qkv.cuda().data_ptr(), 70, o32.data_ptr(), 3, 32, nh, nkv, hd, THETA, att.data_ptr(),
+                             ws.data_ptr(), ws.numel(), None)
+    assert st == B.OK
+    with pytest.raises(B.BitrlError) as e:
+        B.poll_status()
+    assert e.value.status == B.ERR_SHAPE
+    want = oracle_mod.attention(bits(qkv), off.numpy(), nh, nkv, hd, THETA)
+    got = bits(att)
+    keep = np.r_[0:10, 60:70]
+    check_attention(got[keep], want[keep], bits(qkv), nh, nkv, hd)
+    assert not got[10:60].any()  # skipped state: untouched
+    B.poll_status()  # cleared; context alive
+    # argument errors are returned at once
+    bad = lib.bitrl_attention(qkv.cuda().data_ptr(), 70, None, 3, 32, nh, nkv, hd, THETA, att.data_ptr(),
+                              ws.data_ptr(), ws.numel(), None)
+    assert bad == B.ERR_SHAPE  # 3 * 32 != 70
+    bad = lib.bitrl_attention(qkv.cuda().data_ptr(), 70, o32.data_ptr(), 3, 129, nh, nkv, hd, THETA, att.data_ptr(),
+                              ws.data_ptr(), ws.numel(), None)
+    assert bad == B.ERR_SHAPE
+    bad = lib.bitrl_attention(qkv.cuda().data_ptr(), 70, o32.data_ptr(), 3, 32, nh, nkv, 96, THETA, att.data_ptr(),
+                              ws.data_ptr(), ws.numel(), None)
+    assert bad == B.ERR_SHAPE
+    bad = lib.bitrl_attention(qkv.cuda().data_ptr(), 70, o32.data_ptr(), 3, 32, nh, nkv, hd, THETA, att.data_ptr(),
+                              ws.data_ptr(), 8, None)
+    assert bad == B.ERR_WORKSPACE
+
+
+def test_pool_last_token(oracle_mod, B):
+    off = inputs.state_offsets(9, 7600)
+    T = int(off[-1])
+    h = inputs.activations(T, 256, 7601)
+    o32, max_len = dev_states(off)
+    got = B.pool_last_token(h.cuda(), (o32, max_len))
+    B.poll_status()
+    assert torch.equal(got.cpu(), h[(off[1:] - 1)])
+    got = B.pool_last_token(h[:64].cuda(), 16)
+    B.poll_status()
+    assert torch.equal(got.cpu(), h[:64][15::16])
+
+
+SMALL = {"d": 256, "d_ff": 384, "n_heads": 2, "n_kv_heads": 1, "n_layers": 3}
+
+
+def build_encoder(oracle_mod, B, dims, seed):
+    layers_gpu, layers_cpu = [], []
+    for l in range(dims["n_layers"]):
+        Ws = inputs.encoder_layer_weights(l, seed=seed, dims=dims)
+        layers_cpu.append([oracle_mod.ternarize(w.numpy()) for w in Ws])
+        layers_gpu.append(tuple(B.Linear.from_master(w.cuda()) for w in Ws))
+    enc = B.Encoder(layers_gpu, dims["d"], dims["d_ff"], dims["n_heads"], dims["n_kv_heads"])
+    return enc, layers_gpu, layers_cpu
+
+
+@pytest.mark.parametrize("ragged", [False, True])
+def test_encoder_forward_states_small(oracle_mod, B, ragged):
+    """encoder_forward_states == the chain of single C-ABI calls (bit for bit); every BitLinear of the chain matches
+    the oracle's integers on the GPU's own quantized input; the attention step matches the oracle on the GPU's own
+    qkv; the end-to-end distance to the oracle's encoder is bounded; pooling returns the last token of each state."""
+    dims = SMALL
+    nh, nkv, hd = dims["n_heads"], dims["n_kv_heads"], dims["d"] // dims["n_heads"]
+    enc, layers_gpu, layers_cpu = build_encoder(oracle_mod, B, dims, 5000)
+    if ragged:
+        off = inputs.state_offsets(4, 7700)
+        T = int(off[-1])
+        o32, max_len = dev_states(off)
+        states, states_cpu = (o32, max_len), off.numpy()
+    else:
+        T, states, states_cpu = 72, 24, 24
+        off = torch.arange(0, T + 1, 24)
+    h0 = inputs.activations(T, dims["d"], 6000)
+    out, pooled = enc.forward_states(h0.cuda(), states, THETA, want_pooled=True)
+    out2 = enc.forward_states(h0.cuda(), states, THETA)
+    B.poll_status()
+    assert torch.equal(out, out2)
+    assert torch.equal(pooled, out[(off[1:] - 1).cuda()])
+    h = h0.cuda().clone()
+    for (qkv_l, out_l, gu_l, down_l), cpu in zip(layers_gpu, layers_cpu):
+        xq, a, rs, _ = B.rmsnorm_quant(h)
+        qkv, acc = B.bitlinear_forward_q(qkv_l, xq, a, rs, want_acc=True)
+        assert np.array_equal(acc.cpu().numpy(), oracle_mod.contract(xq.cpu().numpy(), cpu[0][0]))
+        att = B.attention(qkv, states, nh, nkv, hd, THETA)
+        check_attention(bits(att), oracle_mod.attention(bits(qkv), states_cpu, nh, nkv, hd, THETA), bits(qkv), nh, nkv, hd)
+        xq, a, rs, _ = B.rmsnorm_quant(att)
+        h, acc = B.bitlinear_forward_q(out_l, xq, a, rs, residual=h, want_acc=True)
+        assert np.array_equal(acc.cpu().numpy(), oracle_mod.contract(xq.cpu().numpy(), cpu[1][0]))
+        xq, a, rs, _ = B.rmsnorm_quant(h)
+        gu = B.bitlinear_forward_q(gu_l, xq, a, rs)
+        xq, a, rs, _ = B.relu2gate_rmsnorm_quant(gu)
+        h = B.bitlinear_forward_q(down_l, xq, a, rs, residual=h)
+    assert torch.equal(out, h)
+    ref = oracle_mod.encoder_forward(inputs.bf16_bits(h0), dims["d_ff"], nh, nkv, layers_cpu, states=states_cpu,
+                                     theta=THETA)
+    got = (bits(out).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    want = (np.asarray(ref, np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    rel = np.linalg.norm(got - want) / np.linalg.norm(want)
+    print(f"encoder with attention, end-to-end relative Frobenius distance to the oracle: {rel:.3e}")
+    assert rel < 3e-2
+
+
+def test_encoder_states_full_width_one_block(oracle_mod, B):
+    """Backbone widths (d=2560, 20/5 heads of 128), one block, ragged 15-40-token states: the fused call equals the
+    chain of single calls, whose attention step is checked against the oracle on the GPU's own qkv."""
+    dims = {"d": 2560, "d_ff": 6912, "n_heads": 20, "n_kv_heads": 5, "n_layers": 1}
+    enc, layers_gpu, layers_cpu = build_encoder(oracle_mod, B, dims, 5000)
+    off = inputs.state_offsets(10, 7800)
+    T = int(off[-1])
+    o32, max_len = dev_states(off)
+    h0 = inputs.activations(T, dims["d"], 6000).cuda()
+    out = enc.forward_states(h0, (o32, max_len), THETA)
+    B.poll_status()
+    (qkv_l, out_l, gu_l, down_l) = layers_gpu[0]
+    xq, a, rs, _ = B.rmsnorm_quant(h0)
+    qkv = B.bitlinear_forward_q(qkv_l, xq, a, rs)
+    att = B.attention(qkv, (o32, max_len), 20, 5, 128, THETA)
+    check_attention(bits(att), oracle_mod.attention(bits(qkv), off.numpy(), 20, 5, 128, THETA), bits(qkv), 20, 5, 128)
+    xq, a, rs, _ = B.rmsnorm_quant(att)
+    h = B.bitlinear_forward_q(out_l, xq, a, rs, residual=h0.clone())
+    xq, a, rs, _ = B.rmsnorm_quant(h)
+    gu = B.bitlinear_forward_q(gu_l, xq, a, rs)
+    xq, a, rs, _ = B.relu2gate_rmsnorm_quant(gu)
+    h = B.bitlinear_forward_q(down_l, xq, a, rs, residual=h)
+    B.poll_status()
+    assert torch.equal(out, h)
