@@ -6,13 +6,15 @@
 //
 // One persistent CTA per SM.  The work list is the concatenation of all jobs' row tiles (128 rows x all K, one
 // contiguous K/4*128-byte region of the tile layout); every CTA owns a contiguous, byte-balanced range of it.
-//   warp 8      producer: bulk copies (cp.async.bulk) of four consecutive 4 KB (row tile, k block) pieces into a ring of
+//   warp 16     producer: bulk copies (cp.async.bulk) of four consecutive 4 KB (row tile, k block) pieces into a ring of
 //               up to 8 slots of 16 KB - up to 128 KB in flight per SM, independent of the activations, so it runs ahead across jobs
-//   warps 0-7   consumers: warp w owns rows 16w..16w+15 of the row tile for the whole K.  The 2-bit codes are
+//   warps 0-15  consumers in two groups of 8: warp w of a group owns rows 16w..16w+15 of the row tile, the group every
+//               other 4 KB piece of the K range (sixteen warps hide the shared-memory and MMA latencies that eight
+//               leave exposed); the two partial sums meet in shared memory once per row tile.  The 2-bit codes are
 //               decoded by shift+mask straight into the A fragments of a warp-level integer MMA
 //               (mma.sync m16n8k32, A = unsigned codes, B = signed int8 activations of 8 tokens, int32 accumulate):
 //               the same instruction count serves 1 to 8 tokens (two MMAs per k step for 9 to 16), so the kernel
-//               stays memory-bound where a dp4a loop would be ALU-bound from M = 4 on.  No cross-warp reduction.
+//               stays memory-bound where a dp4a loop would be ALU-bound from M = 4 on.
 // The activations of a job are quantized into shared memory by the consumer warps when the job's x differs from the
 // cached one.  All mbarrier waits are bounded; after an expiry a warp keeps walking its work list (skipping waits and
 // stores) so that the consumer-wide named barriers stay matched, and the CTA exits normally.
@@ -26,7 +28,8 @@ namespace bitrl {
 
 constexpr int GVM_MAX_JOBS = 128;
 constexpr int GVM_MAX_CTAS = 192;
-constexpr int GVM_CONSUMERS = 8;
+constexpr int GVM_GROUPS = 2;                   // warp groups; group i takes pieces i and i + 2 of every ring slot
+constexpr int GVM_CONSUMERS = 8 * GVM_GROUPS;
 constexpr int GVM_THREADS = (GVM_CONSUMERS + 1) * 32;
 constexpr int GVM_SMEM_BUDGET = 220 * 1024;
 constexpr int GVM_UNROLL = 4;  // 4 KB pieces per ring slot: one bulk copy, one barrier, one consumer loop iteration
@@ -61,24 +64,24 @@ __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, 
 }
 
 // Fragment mapping used below.  Lane (g = lane/4, t = lane%4) holds weight rows g and g+8 of its warp's 16 rows.
-// Word j of a row covers k = 16j..16j+15 and (word >> 2t) & 0x03030303 are its codes k = 16j+4t..16j+4t+3: exactly
-// the bytes the A fragment wants from this lane (a0/a2: row g, k = 4t.. and 16+4t..; a1/a3: row g+8).  Activations
-// are stored so that the eight words k = 16q+4t.. (q = 0..7) of one token and one 128-k block are contiguous:
-// two 128-bit loads give the B fragments (b0, b1) of the block's four k steps.
+// A row of a piece is 8 words of 16 codes; (word >> 2s) & 0x03030303 are its codes k = 16w+4s..16w+4s+3.  The order
+// in which a block's 128 k enter the MMAs is free as long as both operands agree, so lane t takes words 2t and 2t+1 of
+// its rows: the lanes of a warp read disjoint 8-byte pieces (every shared-memory byte is fetched once), the shifts are
+// compile-time constants, and MMA step s of a block multiplies codes k = 32t+4s.. and 32t+16+4s.. of the lane's rows
+// with the activations of the same k - which are simply the lane's 32 contiguous bytes of the plain int8 row.
 template <int NT>
 __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid_constant__ GvmArgs a) {
   extern __shared__ __align__(128) unsigned char gvm_smem[];
   const int depth = 1 << a.depth_log2;
   const uint32_t ring = ptx::smem_u32(gvm_smem);
-  unsigned char* xq_s = gvm_smem + depth * GVM_SLOT_BYTES;  // [NT][K + GVM_XPAD], word-permuted per 128-k block
+  unsigned char* xq_s = gvm_smem + depth * GVM_SLOT_BYTES;  // [NT][K + GVM_XPAD] int8 rows
   const uint32_t xq_addr = ptx::smem_u32(xq_s);
   unsigned char* tail = xq_s + static_cast<size_t>(NT) * (a.kmax + GVM_XPAD);
   const uint32_t bar_full = ptx::smem_u32(tail);    // [depth]
   const uint32_t bar_empty = bar_full + 8 * depth;  // [depth]
   float* absmax_s = reinterpret_cast<float*>(tail + 16 * depth);  // [NT]
   int* rowsum_s = reinterpret_cast<int*>(absmax_s + NT);          // [NT]
-  float* redf = reinterpret_cast<float*>(rowsum_s + NT);          // [8]
-  int* redi = reinterpret_cast<int*>(redf + GVM_CONSUMERS);       // [8]
+  int* comb = reinterpret_cast<int*>(rowsum_s + NT);              // [2][8 warps][NT/8 * 4][32 lanes]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int u_begin = a.unit_start[blockIdx.x], u_end = a.unit_start[blockIdx.x + 1];
@@ -116,39 +119,37 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
     // ------------------------------------------------------------------ consumers
     asm volatile("griddepcontrol.wait;" ::: "memory");  // x may be produced by the preceding kernel
     const int g = lane >> 2, t = lane & 3;
-    const int sh = 2 * t;
+    const int grp = warp >> 3, rw = warp & 7;
     const unsigned short* cached_x = nullptr;
     int cached_k = 0;
-    uint32_t pc = 0;
+    uint32_t pc = 0, tile_no = 0;
     int j = 0;
     bool ok = true;
-    for (int u = u_begin; u < u_end; ++u) {
+    for (int u = u_begin; u < u_end; ++u, ++tile_no) {
       while (j + 1 < a.njobs && a.jobs[j + 1].unit_begin <= u) ++j;
       const GvmJob& job = a.jobs[j];
       const int K = job.K, kblocks = K / TILE_K;
       const int xstride = K + GVM_XPAD;
       if (job.x != cached_x || K != cached_k) {
-        // ---- quantize this job's activations (all consumer warps; the ring keeps filling meanwhile) ----
-        asm volatile("bar.sync 2, 256;" ::: "memory");  // everyone is done with the previous contents
+        // ---- quantize this job's activations: one warp per token, so the tokens proceed side by side with warp-local
+        // reductions only (the ring keeps filling meanwhile) ----
+        asm volatile("bar.sync 2, %0;" ::"n"(GVM_CONSUMERS * 32) : "memory");  // done with the previous contents
         const int nvec8 = K >> 3;
-        for (int m = 0; m < NT; ++m) {
+        for (int m = warp; m < NT; m += GVM_CONSUMERS) {
           unsigned char* row = xq_s + static_cast<size_t>(m) * xstride;
           if (m >= a.M) {
-            for (int i = threadIdx.x; i < (xstride >> 2); i += 256) reinterpret_cast<uint32_t*>(row)[i] = 0u;
+            for (int i = lane; i < (xstride >> 2); i += 32) reinterpret_cast<uint32_t*>(row)[i] = 0u;
             continue;
           }
           const uint4* xr = reinterpret_cast<const uint4*>(job.x + static_cast<size_t>(m) * K);
           float mx = 0.0f;
-          for (int i = threadIdx.x; i < nvec8; i += 256) mx = fmaxf(mx, absmax8(xr[i]));
-          mx = warp_max(mx);
-          if (lane == 0) redf[warp] = mx;
-          asm volatile("bar.sync 2, 256;" ::: "memory");
-#pragma unroll
-          for (int i = 0; i < GVM_CONSUMERS; ++i) mx = fmaxf(mx, redf[i]);
-          const float amax = fmaxf(mx, 1e-5f);
+#pragma unroll 4
+          for (int i = lane; i < nvec8; i += 32) mx = fmaxf(mx, absmax8(xr[i]));
+          const float amax = fmaxf(warp_max(mx), 1e-5f);
           const float inv = __fdiv_rn(127.0f, amax);
           int rs = 0;
-          for (int i = threadIdx.x; i < nvec8; i += 256) {
+#pragma unroll 2
+          for (int i = lane; i < nvec8; i += 32) {
             const uint4 raw = xr[i];
             const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
             int q[8];
@@ -160,33 +161,25 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
             const uint32_t lo = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | (static_cast<uint32_t>(q[3]) << 24);
             const uint32_t hi = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | (static_cast<uint32_t>(q[7]) << 24);
             rs += q[0] + q[1] + q[2] + q[3] + q[4] + q[5] + q[6] + q[7];
-            // word w = 4q+t of a 128-k block is stored at word position t*8+q of that block
-            const int kb = i >> 4, w = (i & 15) * 2;
-            uint32_t* blk = reinterpret_cast<uint32_t*>(row + kb * TILE_K);
-            blk[(w & 3) * 8 + (w >> 2)] = lo;
-            blk[((w + 1) & 3) * 8 + ((w + 1) >> 2)] = hi;
+            reinterpret_cast<uint2*>(row)[i] = make_uint2(lo, hi);
           }
           rs = warp_sum_i(rs);
-          if (lane == 0) redi[warp] = rs;
-          asm volatile("bar.sync 2, 256;" ::: "memory");
-          if (threadIdx.x == 0) {
-            int tsum = 0;
-#pragma unroll
-            for (int i = 0; i < GVM_CONSUMERS; ++i) tsum += redi[i];
-            rowsum_s[m] = tsum;
+          if (lane == 0) {
+            rowsum_s[m] = rs;
             absmax_s[m] = amax;
           }
         }
-        asm volatile("bar.sync 2, 256;" ::: "memory");
+        asm volatile("bar.sync 2, %0;" ::"n"(GVM_CONSUMERS * 32) : "memory");
         cached_x = job.x;
         cached_k = K;
       }
 
       // ---- one row tile: this warp's 16 rows over the whole K ----
       const float gamma = *job.gamma;  // requested now, needed after the k loop: its latency hides behind the loop
-      // The GVM_UNROLL pieces of a slot are fetched from shared memory together and feed independent accumulator
-      // chains, so that neither the loads nor the MMAs of one piece wait for those of another.
-      constexpr int CH = NT == 8 ? 16 : 8;  // independent accumulator chains (the warp MMA has a long latency)
+      // A group's two pieces of a slot are fetched from shared memory together and feed independent accumulator
+      // chains, so that neither the loads nor the MMAs of one piece wait for those of the other.
+      constexpr int PP = GVM_UNROLL / GVM_GROUPS;  // pieces of a slot per group
+      constexpr int CH = NT == 8 ? 8 : 4;          // independent accumulator chains (the warp MMA has a long latency)
       int acc[CH][NT / 8][4];
 #pragma unroll
       for (int c = 0; c < CH; ++c)
@@ -194,40 +187,35 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
         for (int h = 0; h < NT / 8; ++h)
 #pragma unroll
           for (int e = 0; e < 4; ++e) acc[c][h][e] = 0;
-      const uint32_t xlane = xq_addr + g * xstride + t * 32;
+      const uint32_t xlane = xq_addr + g * xstride + t * 32 + grp * TILE_K;
+      const uint32_t wlane = ring + grp * TILE_BYTES + rw * 512 + g * 32 + t * 8;
       for (int kb = 0; kb < kblocks; kb += GVM_UNROLL) {
-        const int np = min(GVM_UNROLL, kblocks - kb);
-        uint4 wr[GVM_UNROLL][4];
+        const int np = min(GVM_UNROLL, kblocks - kb) - grp;  // pieces grp, grp + GROUPS exist if np > 0, GROUPS
+        uint2 wr[PP][2];
         const uint32_t s = pc & (depth - 1), ph = (pc >> a.depth_log2) & 1u;
         if (ok && !ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(GVM_WAIT_FULL); ok = false; }
         if (ok) {
 #pragma unroll
-          for (int p = 0; p < GVM_UNROLL; ++p) {
-            if (p < np) {
-              const uint32_t wslice = ring + s * GVM_SLOT_BYTES + p * TILE_BYTES + warp * 512;
-              wr[p][0] = ptx::lds128(wslice + g * 32);
-              wr[p][1] = ptx::lds128(wslice + g * 32 + 16);
-              wr[p][2] = ptx::lds128(wslice + (g + 8) * 32);
-              wr[p][3] = ptx::lds128(wslice + (g + 8) * 32 + 16);
+          for (int p = 0; p < PP; ++p) {
+            if (GVM_GROUPS * p < np) {
+              const uint32_t wslice = wlane + s * GVM_SLOT_BYTES + p * GVM_GROUPS * TILE_BYTES;
+              wr[p][0] = ptx::lds64(wslice);
+              wr[p][1] = ptx::lds64(wslice + 8 * 32);
             }
           }
-        }
-        if (ok) {
 #pragma unroll
-          for (int p = 0; p < GVM_UNROLL; ++p) {
-            if (p < np) {
-              const uint32_t w0[8] = {wr[p][0].x, wr[p][0].y, wr[p][0].z, wr[p][0].w, wr[p][1].x, wr[p][1].y, wr[p][1].z, wr[p][1].w};
-              const uint32_t w1[8] = {wr[p][2].x, wr[p][2].y, wr[p][2].z, wr[p][2].w, wr[p][3].x, wr[p][3].y, wr[p][3].z, wr[p][3].w};
+          for (int p = 0; p < PP; ++p) {
+            if (GVM_GROUPS * p < np) {
 #pragma unroll
               for (int h = 0; h < NT / 8; ++h) {
-                const uint32_t xa_addr = xlane + h * 8 * xstride + (kb + p) * TILE_K;
+                const uint32_t xa_addr = xlane + h * 8 * xstride + (kb + p * GVM_GROUPS) * TILE_K;
                 const uint4 xa = ptx::lds128(xa_addr), xb = ptx::lds128(xa_addr + 16);
                 const uint32_t xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
-                  mma_u8s8(acc[(p * 4 + ks) % CH][h], (w0[2 * ks] >> sh) & 0x03030303u, (w1[2 * ks] >> sh) & 0x03030303u,
-                           (w0[2 * ks + 1] >> sh) & 0x03030303u, (w1[2 * ks + 1] >> sh) & 0x03030303u, xv[2 * ks],
-                           xv[2 * ks + 1]);
+                  mma_u8s8(acc[(p * 4 + ks) % CH][h], (wr[p][0].x >> (2 * ks)) & 0x03030303u,
+                           (wr[p][1].x >> (2 * ks)) & 0x03030303u, (wr[p][0].y >> (2 * ks)) & 0x03030303u,
+                           (wr[p][1].y >> (2 * ks)) & 0x03030303u, xv[ks], xv[4 + ks]);
               }
             }
           }
@@ -242,16 +230,25 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
         for (int h = 0; h < NT / 8; ++h)
 #pragma unroll
           for (int e = 0; e < 4; ++e) acc[0][h][e] += acc[c][h][e];
-      if (ok) {
+      // ---- the two groups' partial sums meet in shared memory (double-buffered by tile parity) ----
+      int* cb = comb + (tile_no & 1u) * (8 * (NT / 8) * 4 * 32) + rw * ((NT / 8) * 4 * 32) + lane;
+      if (grp == 1) {
+#pragma unroll
+        for (int h = 0; h < NT / 8; ++h)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) cb[(h * 4 + e) * 32] = acc[0][h][e];
+      }
+      asm volatile("bar.sync 3, %0;" ::"n"(GVM_CONSUMERS * 32) : "memory");
+      if (grp == 0 && ok) {
         // C fragment: acc[h][0..1] = (row g, tokens 8h+2t, +1), acc[h][2..3] = (row g+8, same tokens)
-        const int n0 = (u - job.unit_begin) * TILE_ROWS + warp * 16 + g;
+        const int n0 = (u - job.unit_begin) * TILE_ROWS + rw * 16 + g;
 #pragma unroll
         for (int h = 0; h < NT / 8; ++h)
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int m = 8 * h + 2 * t + (e & 1);
             if (m < a.M) {
-              const int tv = acc[0][h][e] - rowsum_s[m];
+              const int tv = acc[0][h][e] + cb[(h * 4 + e) * 32] - rowsum_s[m];
               const float yv = __fmul_rn(static_cast<float>(tv), out_scale(gamma, absmax_s[m]));
               const size_t o = static_cast<size_t>(m) * job.N + n0 + (e >> 1) * 8;
               if (a.out_dtype == BITRL_OUT_F32) static_cast<float*>(job.y)[o] = yv;
@@ -343,9 +340,18 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
             for (int i = threadIdx.x; i < nvec8; i += GVD_CONSUMERS * 32) dst[i] = make_uint2(0u, 0u);
             continue;
           }
+          // The first two vectors of every thread (rows up to 8192 values) stay in registers between the absmax pass
+          // and the quantization pass: one trip to global memory instead of two.
           const uint4* xr = reinterpret_cast<const uint4*>(job.x + static_cast<size_t>(m) * K);
-          float mx = 0.0f;
-          for (int i = threadIdx.x; i < nvec8; i += GVD_CONSUMERS * 32) mx = fmaxf(mx, absmax8(xr[i]));
+          constexpr int NTH = GVD_CONSUMERS * 32;
+          uint4 held[2];
+#pragma unroll
+          for (int jv = 0; jv < 2; ++jv) {
+            const int i = threadIdx.x + jv * NTH;
+            held[jv] = i < nvec8 ? xr[i] : make_uint4(0u, 0u, 0u, 0u);
+          }
+          float mx = fmaxf(absmax8(held[0]), absmax8(held[1]));
+          for (int i = threadIdx.x + 2 * NTH; i < nvec8; i += NTH) mx = fmaxf(mx, absmax8(xr[i]));
           mx = warp_max(mx);
           if (lane == 0) redf[warp] = mx;
           asm volatile("bar.sync 2, %0;" ::"n"(GVD_CONSUMERS * 32) : "memory");
@@ -354,8 +360,7 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
           const float amax = fmaxf(mx, 1e-5f);
           const float inv = __fdiv_rn(127.0f, amax);
           int rs = 0;
-          for (int i = threadIdx.x; i < nvec8; i += GVD_CONSUMERS * 32) {
-            const uint4 raw = xr[i];
+          auto quant8 = [&](const uint4 raw, int i) {
             const uint32_t rwd[4] = {raw.x, raw.y, raw.z, raw.w};
             int q[8];
 #pragma unroll
@@ -368,7 +373,13 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
             wd.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | (static_cast<uint32_t>(q[7]) << 24);
             rs += q[0] + q[1] + q[2] + q[3] + q[4] + q[5] + q[6] + q[7];
             dst[i] = wd;
+          };
+#pragma unroll
+          for (int jv = 0; jv < 2; ++jv) {
+            const int i = threadIdx.x + jv * NTH;
+            if (i < nvec8) quant8(held[jv], i);
           }
+          for (int i = threadIdx.x + 2 * NTH; i < nvec8; i += NTH) quant8(xr[i], i);
           rs = warp_sum_i(rs);
           if (lane == 0) redi[warp] = rs;
           asm volatile("bar.sync 2, %0;" ::"n"(GVD_CONSUMERS * 32) : "memory");
@@ -506,7 +517,7 @@ inline int gvm_nt(int M) { return M <= 8 ? 8 : 16; }
 // Shared memory beside the ring: activations (+ barriers, reduction scratch, the group-combine buffer).
 inline size_t gvm_fixed_bytes(int M, int kmax) {
   if (M <= 2) return static_cast<size_t>(M) * kmax + 1024 + 2 * (GVD_GROUPS - 1) * 8 * 16 * 2 * sizeof(int);
-  return static_cast<size_t>(gvm_nt(M)) * (kmax + GVM_XPAD) + 1024;
+  return static_cast<size_t>(gvm_nt(M)) * (kmax + GVM_XPAD) + 1024 + 2 * 8 * (gvm_nt(M) / 8) * 4 * 32 * sizeof(int);
 }
 
 // Ring depth (log2) that fits beside the activations, or -1.
