@@ -32,7 +32,7 @@ constexpr int GVM_GROUPS = 2;                   // warp groups; group i takes pi
 constexpr int GVM_CONSUMERS = 8 * GVM_GROUPS;
 constexpr int GVM_THREADS = (GVM_CONSUMERS + 1) * 32;
 constexpr int GVM_SMEM_BUDGET = 220 * 1024;
-constexpr int GVM_UNROLL = 4;  // 4 KB pieces per ring slot: one bulk copy, one barrier, one consumer loop iteration
+constexpr int GVM_UNROLL = 8;  // 4 KB pieces per ring slot: one bulk copy, one barrier, one consumer loop iteration
 constexpr int GVM_SLOT_BYTES = GVM_UNROLL * TILE_BYTES;
 constexpr int GVM_XPAD = 16;  // bytes added to each activation row so that the 8 token rows hit different banks
 
@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
   unsigned char* tail = xq_s + static_cast<size_t>(NT) * (a.kmax + GVM_XPAD);
   const uint32_t bar_full = ptx::smem_u32(tail);    // [depth]
   const uint32_t bar_empty = bar_full + 8 * depth;  // [depth]
-  float* absmax_s = reinterpret_cast<float*>(tail + 16 * depth);  // [NT]
+  float* absmax_s = reinterpret_cast<float*>(tail + 16 * depth);  // [NT] a_m / 127
   int* rowsum_s = reinterpret_cast<int*>(absmax_s + NT);          // [NT]
   int* comb = reinterpret_cast<int*>(rowsum_s + NT);              // [2][8 warps][NT/8 * 4][32 lanes]
 
@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
           rs = warp_sum_i(rs);
           if (lane == 0) {
             rowsum_s[m] = rs;
-            absmax_s[m] = amax;
+            absmax_s[m] = __fdiv_rn(amax, 127.0f);  // the epilogue's scale is gamma * (a_m / 127)
           }
         }
         asm volatile("bar.sync 2, %0;" ::"n"(GVM_CONSUMERS * 32) : "memory");
@@ -238,7 +238,7 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
 #pragma unroll
           for (int e = 0; e < 4; ++e) cb[(h * 4 + e) * 32] = acc[0][h][e];
       }
-      asm volatile("bar.sync 3, %0;" ::"n"(GVM_CONSUMERS * 32) : "memory");
+      asm volatile("bar.sync %0, 64;" ::"r"(4 + rw) : "memory");  // only the two warps that share these rows meet
       if (grp == 0 && ok) {
         // C fragment: acc[h][0..1] = (row g, tokens 8h+2t, +1), acc[h][2..3] = (row g+8, same tokens)
         const int n0 = (u - job.unit_begin) * TILE_ROWS + rw * 16 + g;
@@ -249,7 +249,7 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
             const int m = 8 * h + 2 * t + (e & 1);
             if (m < a.M) {
               const int tv = acc[0][h][e] + cb[(h * 4 + e) * 32] - rowsum_s[m];
-              const float yv = __fmul_rn(static_cast<float>(tv), out_scale(gamma, absmax_s[m]));
+              const float yv = __fmul_rn(static_cast<float>(tv), __fmul_rn(gamma, absmax_s[m]));
               const size_t o = static_cast<size_t>(m) * job.N + n0 + (e >> 1) * 8;
               if (a.out_dtype == BITRL_OUT_F32) static_cast<float*>(job.y)[o] = yv;
               else static_cast<unsigned short*>(job.y)[o] = float_to_bf16_bits(yv);
@@ -388,7 +388,7 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
 #pragma unroll
             for (int i = 0; i < GVD_CONSUMERS; ++i) tsum += redi[i];
             rowsum_s[m] = tsum;
-            absmax_s[m] = amax;
+            absmax_s[m] = __fdiv_rn(amax, 127.0f);  // the epilogue's scale is gamma * (a_m / 127)
           }
         }
         asm volatile("bar.sync 2, %0;" ::"n"(GVD_CONSUMERS * 32) : "memory");
@@ -454,7 +454,7 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
         tot[m] += __shfl_xor_sync(0xffffffffu, tot[m], 1);
         if (grp > 0 && half == 0) cb[(grp - 1) * (8 * 16 * MT) + m] = tot[m];
       }
-      asm volatile("bar.sync 3, %0;" ::"n"(GVD_CONSUMERS * 32) : "memory");
+      asm volatile("bar.sync %0, %1;" ::"r"(4 + rw), "n"(GVD_GROUPS * 32) : "memory");  // the warps sharing these rows
       if (grp == 0 && half == 0 && ok) {
         const int n = (u - job.unit_begin) * TILE_ROWS + rw * 16 + (lane >> 1);
 #pragma unroll
@@ -463,7 +463,7 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
             int tv = tot[m] - rowsum_s[m];
 #pragma unroll
             for (int g2 = 0; g2 < GVD_GROUPS - 1; ++g2) tv += cb[g2 * (8 * 16 * MT) + m];
-            const float yv = __fmul_rn(static_cast<float>(tv), out_scale(gamma, absmax_s[m]));
+            const float yv = __fmul_rn(static_cast<float>(tv), __fmul_rn(gamma, absmax_s[m]));
             const size_t o = static_cast<size_t>(m) * job.N + n;
             if (a.out_dtype == BITRL_OUT_F32) static_cast<float*>(job.y)[o] = yv;
             else static_cast<unsigned short*>(job.y)[o] = float_to_bf16_bits(yv);
