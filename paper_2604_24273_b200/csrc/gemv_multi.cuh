@@ -212,10 +212,13 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
                 const uint4 xa = ptx::lds128(xa_addr), xb = ptx::lds128(xa_addr + 16);
                 const uint32_t xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                  mma_u8s8(acc[(p * 4 + ks) % CH][h], (wr[p][0].x >> (2 * ks)) & 0x03030303u,
-                           (wr[p][1].x >> (2 * ks)) & 0x03030303u, (wr[p][0].y >> (2 * ks)) & 0x03030303u,
-                           (wr[p][1].y >> (2 * ks)) & 0x03030303u, xv[ks], xv[4 + ks]);
+                for (int ks = 0; ks < 4; ++ks) {
+                  // The codes stay at their bit positions (c * 4^ks still fits an unsigned byte): one mask and no
+                  // shift per operand.  Chain ks then holds 4^ks times its share and is scaled back once per tile.
+                  const uint32_t msk = 0x03030303u << (2 * ks);
+                  mma_u8s8(acc[((p * 4) % CH) + ks][h], wr[p][0].x & msk, wr[p][1].x & msk, wr[p][0].y & msk,
+                           wr[p][1].y & msk, xv[ks], xv[4 + ks]);
+                }
               }
             }
           }
@@ -229,7 +232,7 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
 #pragma unroll
         for (int h = 0; h < NT / 8; ++h)
 #pragma unroll
-          for (int e = 0; e < 4; ++e) acc[0][h][e] += acc[c][h][e];
+          for (int e = 0; e < 4; ++e) acc[0][h][e] += acc[c][h][e] >> (2 * (c & 3));  // exact: multiples of 4^(c&3)
       // ---- the two groups' partial sums meet in shared memory (double-buffered by tile parity) ----
       int* cb = comb + (tile_no & 1u) * (8 * (NT / 8) * 4 * 32) + rw * ((NT / 8) * 4 * 32) + lane;
       if (grp == 1) {
