@@ -265,13 +265,14 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
 
 // ---------------------------------------------------------------------------------------------------------
 // M <= 2 variant: dp4a instead of the warp MMA (cheaper when only one or two tokens use the weights), and
-// 8 * GVD_GROUPS consumer warps: group g takes pieces g, g + GROUPS of every ring slot (a slot holds 2 * GROUPS
+// 8 * GVD_GROUPS consumer warps: group g takes pieces g, g + GROUPS of every ring slot (a slot holds GVD_PPG * GROUPS
 // pieces); the groups' partial sums meet in shared memory once per row tile.  Lane = 2*row + k half, as in the
 // single-matrix kernel.
 constexpr int GVD_GROUPS = 2;
 constexpr int GVD_CONSUMERS = 8 * GVD_GROUPS;
 constexpr int GVD_THREADS = (GVD_CONSUMERS + 1) * 32;
-constexpr int GVD_PIECES = 2 * GVD_GROUPS;                 // 4 KB pieces per ring slot
+constexpr int GVD_PPG = 4;                                 // pieces of a slot per group
+constexpr int GVD_PIECES = GVD_PPG * GVD_GROUPS;           // 4 KB pieces per ring slot
 constexpr int GVD_SLOT_BYTES = GVD_PIECES * TILE_BYTES;
 
 template <int MT>
@@ -415,12 +416,12 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
         if (ok && !ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(GVM_WAIT_FULL); ok = false; }
         if (ok) {
           const uint32_t w_slot = w_lane + s * GVD_SLOT_BYTES;
-          uint4 wv[2];
+          uint4 wv[GVD_PPG];
 #pragma unroll
-          for (int pp = 0; pp < 2; ++pp)
+          for (int pp = 0; pp < GVD_PPG; ++pp)
             if (GVD_GROUPS * pp < np) wv[pp] = ptx::lds128(w_slot + pp * GVD_GROUPS * TILE_BYTES);
 #pragma unroll
-          for (int pp = 0; pp < 2; ++pp) {
+          for (int pp = 0; pp < GVD_PPG; ++pp) {
             if (GVD_GROUPS * pp < np) {
               const uint32_t wword[4] = {wv[pp].x, wv[pp].y, wv[pp].z, wv[pp].w};
 #pragma unroll
@@ -543,7 +544,7 @@ bitrl_status launch_gemv_multi(int count, const Linear* const* w, const void* co
     if (w[j]->K > kmax) kmax = w[j]->K;
   }
   int dlog = gvm_depth_log2(M, kmax);
-  if (M <= 2) {  // the dp4a kernel takes the slot count itself (24 KB slots, any count from 2 to 8)
+  if (M <= 2) {  // the dp4a kernel takes the slot count itself (any count from 2 to 8)
     const long long room = static_cast<long long>(GVM_SMEM_BUDGET) - static_cast<long long>(gvm_fixed_bytes(M, kmax));
     dlog = static_cast<int>(room / (GVD_SLOT_BYTES + 16));
     if (dlog > 8) dlog = 8;
