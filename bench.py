@@ -365,6 +365,27 @@ def run_ours(args):
             extra[name] = res
             del xs, y, ws, q
 
+        # configs[2]: batched state encoding, M = 64 and 256 (one token per state), the whole layer per call
+        for M in (64, 256):
+            for K, N in ((2560, 6912), (6912, 2560)):
+                mats = up_only if N == 6912 else [layers[l][3] for l in range(n_layers)]
+                xs = [inputs.activations(M, K, 2500 + i).to(dev) for i in range(4)]
+                y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+                ws = torch.empty((bitrl.workspace_bytes(M, K, N),), dtype=torch.uint8, device=dev)
+                reps = 24
+
+                def small():
+                    for i in range(reps):
+                        bitrl.bitlinear_forward(mats[i % len(mats)], xs[i % 4], bitrl.OUT_BF16, y=y, workspace=ws)
+
+                g, lc = capture(small)
+                ms = time_graph(g, sub_steps, args.warmup, 1)
+                us = ms * 1e3 / (sub_steps * reps)
+                extra[f"layer_m{M}_k{K}_n{N}"] = {"us": us, "TOPS": 2.0 * M * N * K / (us * 1e-6) / 1e12,
+                                                  "packed_GBps": N * K / 4 / (us * 1e-6) / 1e9,
+                                                  "launches_per_layer": lc / reps}
+                del g, xs, y, ws
+
     if rank == 0 and "encoder" in sections:
         T = 4096  # 128 states x 32 tokens
         enc = bitrl.Encoder(layers, 2560, 6912, 20, 5)

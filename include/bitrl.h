@@ -100,7 +100,10 @@ BITRL_API bitrl_status bitrl_quant_act(const void* x, int32_t M, int32_t K, int8
  * x: dev bf16 [M,K]; y: dev [M,N] fp32 (BITRL_OUT_F32) or bf16 (BITRL_OUT_BF16).  K, N must equal the
  * handle's.  M <= BITRL_GEMV_MAX_M: one streaming kernel (quantization in its prologue, rescale in its
  * epilogue; no workspace needed).  Larger M: quantization kernel into the workspace, then the tcgen05 GEMM.
- * workspace: dev, >= bitrl_workspace_bytes(M,K,N) (0 for M <= 16, then NULL is accepted). */
+ * workspace: dev, >= bitrl_workspace_bytes(M,K,N) (0 for M <= 16, then NULL is accepted).  Up to M = 512 it also
+ * holds M*N int32 of scratch: when a launch has too few output tiles to occupy the SMs, K is split across them, the
+ * exact int32 partial sums meet in that scratch (integer atomics: order-free, deterministic) and a finishing kernel
+ * applies the rescale.  The results are the same bits either way. */
 BITRL_API size_t bitrl_workspace_bytes(int32_t M, int32_t K, int32_t N);
 BITRL_API bitrl_status bitrl_bitlinear_forward(const bitrl_linear_t* w, const void* x, int32_t M, int32_t K, int32_t N,
                                      void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes,

@@ -91,14 +91,16 @@ namespace {
 inline bool shape_ok(int N, int K) { return N >= 128 && K >= 128 && N % 128 == 0 && K % 128 == 0; }
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Workspace of the M > 16 path: x_q [M,K] int8, absmax [M] f32, rowsum [M] i32.
+// Workspace of the M > 16 path: x_q [M,K] int8, absmax [M] f32, rowsum [M] i32, and for small M the split-K scratch
+// [M,N] int32.
 struct FwdWs {
   int8_t* xq;
   float* absmax;
   int32_t* rowsum;
+  int32_t* splitk;
   size_t bytes;
 };
-inline FwdWs carve_fwd(void* ws, int M, int K) {
+inline FwdWs carve_fwd(void* ws, int M, int K, int N) {
   FwdWs f;
   size_t off = 0;
   unsigned char* b = static_cast<unsigned char*>(ws);
@@ -108,6 +110,11 @@ inline FwdWs carve_fwd(void* ws, int M, int K) {
   off += align_up(static_cast<size_t>(M) * 4, 256);
   f.rowsum = reinterpret_cast<int32_t*>(b + off);
   off += align_up(static_cast<size_t>(M) * 4, 256);
+  f.splitk = nullptr;
+  if (M <= GM_SPLITK_MAX_M) {
+    f.splitk = reinterpret_cast<int32_t*>(b + off);
+    off += align_up(static_cast<size_t>(M) * N * 4, 256);
+  }
   f.bytes = off;
   return f;
 }
@@ -218,10 +225,9 @@ bitrl_status bitrl_quant_act(const void* x, int32_t M, int32_t K, int8_t* xq, fl
 }
 
 size_t bitrl_workspace_bytes(int32_t M, int32_t K, int32_t N) {
-  (void)N;
-  if (M < 1 || K < 1) return 0;
+  if (M < 1 || K < 1 || N < 1) return 0;
   if (gemv_fits(M, K)) return 0;
-  return carve_fwd(nullptr, M, K).bytes;
+  return carve_fwd(nullptr, M, K, N).bytes;
 }
 
 static bitrl_status forward_impl(const bitrl_linear_t* w, const void* x, int32_t M, int32_t K, int32_t N, void* y,
@@ -236,13 +242,13 @@ static bitrl_status forward_impl(const bitrl_linear_t* w, const void* x, int32_t
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (gemv_fits(M, K))
     return launch_gemv(&w->l, x, nullptr, nullptr, M, y, out_dtype, nullptr, xq_out, absmax_out, acc_out, st);
-  const size_t need = carve_fwd(nullptr, M, K).bytes;
+  const size_t need = carve_fwd(nullptr, M, K, N).bytes;
   if (!workspace || workspace_bytes < need) return BITRL_ERR_WORKSPACE;
   if (!aligned16(workspace)) return BITRL_ERR_ALIGN;
-  FwdWs f = carve_fwd(workspace, M, K);
+  FwdWs f = carve_fwd(workspace, M, K, N);
   s = launch_quant_act(x, M, K, f.xq, f.absmax, f.rowsum, st);
   if (s != BITRL_OK) return s;
-  s = launch_gemm(&w->l, f.xq, f.absmax, f.rowsum, M, y, out_dtype, nullptr, acc_out, st);
+  s = launch_gemm(&w->l, f.xq, f.absmax, f.rowsum, M, y, out_dtype, nullptr, acc_out, st, f.splitk);
   if (s != BITRL_OK) return s;
   if (debug) {
     if (xq_out) BITRL_CUDA(cudaMemcpyAsync(xq_out, f.xq, static_cast<size_t>(M) * K, cudaMemcpyDeviceToDevice, st));
@@ -370,6 +376,7 @@ struct EncWs {
   float* absmax;    // [T]
   int32_t* rowsum;  // [T]
   unsigned short* wide;  // [T, max(n_qkv, 2 d_ff)] bf16: qkv, then gate/up
+  int32_t* splitk;       // [T, max N] int32 split-K scratch of the GEMM (only for small T)
   unsigned short* att;   // [T, d] bf16 attention output (only with real attention)
   float2* rope;          // [max_state_len, head_dim/2] rotary table (only with real attention)
   size_t bytes;
@@ -389,6 +396,11 @@ EncWs carve_enc(void* ws, const bitrl_encoder* e, int T, int max_state_len) {
   off += align_up(static_cast<size_t>(T) * 4, 256);
   w.wide = reinterpret_cast<unsigned short*>(b + off);
   off += align_up(static_cast<size_t>(T) * wmax * 2, 256);
+  w.splitk = nullptr;
+  if (T <= GM_SPLITK_MAX_M) {
+    w.splitk = reinterpret_cast<int32_t*>(b + off);
+    off += align_up(static_cast<size_t>(T) * wmax * 4, 256);
+  }
   w.att = nullptr;
   w.rope = nullptr;
   if (max_state_len > 0) {
@@ -419,7 +431,7 @@ bitrl_status encoder_run(const bitrl_encoder_t* enc, const void* h_in, int32_t T
   auto linear = [&](const bitrl_linear* lin, void* y, const void* residual) -> bitrl_status {
     if (gemv_fits(T, lin->l.K))
       return launch_gemv(&lin->l, nullptr, w.xq, w.absmax, T, y, BITRL_OUT_BF16, residual, nullptr, nullptr, nullptr, st);
-    return launch_gemm(&lin->l, w.xq, w.absmax, w.rowsum, T, y, BITRL_OUT_BF16, residual, nullptr, st);
+    return launch_gemm(&lin->l, w.xq, w.absmax, w.rowsum, T, y, BITRL_OUT_BF16, residual, nullptr, st, w.splitk);
   };
   for (int l = 0; l < enc->L; ++l) {
     const bitrl_linear* const* q = enc->layers.data() + 4 * l;

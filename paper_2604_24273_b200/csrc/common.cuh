@@ -129,8 +129,9 @@ bitrl_status launch_relu2gate_rmsnorm_quant(const void* gu, int T, int F, int8_t
 bitrl_status launch_gemv(const Linear* w, const void* x, const int8_t* xq, const float* absmax, int M, void* y,
                          int out_dtype, const void* residual, int8_t* xq_out, float* absmax_out,
                          int32_t* acc_out, cudaStream_t st);
-// Any M >= 1, tcgen05 path, already quantized input.
+// Any M >= 1, tcgen05 path, already quantized input.  splitk_ws: nullptr or M*N int32 of scratch (see gemm.cuh).
 bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax, const int32_t* rowsum, int M,
-                         void* y, int out_dtype, const void* residual, int32_t* acc_out, cudaStream_t st);
+                         void* y, int out_dtype, const void* residual, int32_t* acc_out, cudaStream_t st,
+                         int32_t* splitk_ws = nullptr);
 
 }  // namespace bitrl

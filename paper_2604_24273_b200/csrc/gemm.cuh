@@ -66,6 +66,11 @@ struct GemmArgs {
   const unsigned short* residual;
   int32_t* acc_out;
   int tiles_n, tiles_total;
+  // Split-K for launches with few tiles: work item = (tile, k range); the raw int32 partial sums of an item are added
+  // into `part` [M,N] (zeroed by the launcher) with integer atomics - exact and order-free - and a second kernel applies
+  // the epilogue.  splits == 1: one item per tile, epilogue in this kernel, `part` unused.
+  int splits, kb_per_split;
+  int32_t* part;
 };
 
 template <int GM_TOK, bool A_TMEM>
@@ -101,6 +106,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kblocks = a.K / GM_BK;
+  const int items = a.tiles_total * a.splits;
+  auto item_range = [&](int item, int& tile, int& kb0, int& kb1) {
+    tile = item / a.splits;
+    kb0 = (item - tile * a.splits) * a.kb_per_split;
+    kb1 = min(kblocks, kb0 + a.kb_per_split);
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < GM_XS; ++s) { ptx::mbar_init(bar_x_full + 8 * s, 1 + 4); ptx::mbar_init(bar_x_empty + 8 * s, 1); }
@@ -124,9 +135,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x) {
+      for (int item = blockIdx.x; ok && item < items; item += gridDim.x) {
+        int tile, kb0, kb1;
+        item_range(item, tile, kb0, kb1);
         const int tm = tile / a.tiles_n;
-        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const uint32_t s = it % GM_XS, ph = (it / GM_XS) & 1u;
           if (!ptx::mbar_wait(bar_x_empty + 8 * s, ph ^ 1u)) { report_timeout(GM_WAIT_X_EMPTY); ok = false; break; }
           ptx::mbar_arrive_expect_tx(bar_x_full + 8 * s, GM_X_BYTES);
@@ -139,10 +152,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x) {
+      for (int item = blockIdx.x; ok && item < items; item += gridDim.x) {
+        int tile, kb0, kb1;
+        item_range(item, tile, kb0, kb1);
         const int tn = tile % a.tiles_n;
         const uint8_t* wsrc = a.tiles + static_cast<size_t>(tn) * kblocks * TILE_BYTES;
-        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const uint32_t s = it % GM_PS, ph = (it / GM_PS) & 1u;
           if (!ptx::mbar_wait(bar_p_empty + 8 * s, ph ^ 1u)) { report_timeout(GM_WAIT_P_EMPTY); ok = false; break; }
           ptx::mbar_arrive_expect_tx(bar_p_full + 8 * s, GM_P_BYTES);
@@ -158,14 +173,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
       uint32_t lt = 0;
       uint32_t xs = 0, xph = 0, ws = 0;  // ring slots and phase, advanced without divisions
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x, ++lt) {
+      for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++lt) {
+        int tile, kb0, kb1;
+        item_range(item, tile, kb0, kb1);
         const uint32_t buf = lt & 1u;
         if (!ptx::mbar_wait(bar_tmem_empty + 8 * buf, ((lt >> 1) & 1u) ^ 1u)) {
           report_timeout(GM_WAIT_TMEM_EMPTY); ok = false; break;
         }
         const uint32_t d_tmem = tmem_base + buf * GM_TOK_MAX;
         ptx::tc_fence_after_sync();  // orders this tile's MMAs after the epilogue's reads of the accumulator
-        for (int kb = 0; kb < kblocks; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!ptx::mbar_wait(bar_x_full + 8 * xs, xph)) { report_timeout(GM_WAIT_X_FULL); ok = false; break; }
           // Weights written with tcgen05.st by other threads need the tcgen05 fence on this side of the barrier;
           // TMA data and expander stores to shared memory (already fenced into the async proxy by their writers) do not.
@@ -175,12 +192,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
             const uint32_t a_tmem = tmem_base + a_slot(ws);
 #pragma unroll
             for (int k4 = 0; k4 < GM_BK / 32; ++k4)
-              ptx::mma_i8_ts(d_tmem, a_tmem + 8 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+              ptx::mma_i8_ts(d_tmem, a_tmem + 8 * k4, bdesc + 2 * k4, idesc, (kb != kb0 || k4 != 0) ? 1u : 0u);
           } else {
             const uint64_t adesc = ptx::smem_desc_sw128(base + GM_OFF_W + ws * GM_W_BYTES);
 #pragma unroll
             for (int k4 = 0; k4 < GM_BK / 32; ++k4)
-              ptx::mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+              ptx::mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb != kb0 || k4 != 0) ? 1u : 0u);
           }
           ptx::mma_commit(bar_x_empty + 8 * xs);  // frees the x_q slot and the weight slot of this k block
           if (++xs == GM_XS) { xs = 0; xph ^= 1u; }
@@ -207,8 +224,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     uint32_t it = 0;
     uint32_t ps = 0, pph = 0, ws = 0, xs = 0, xs_old = 0, xph_old = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x) {
-      for (int kb = 0; kb < kblocks; ++kb, ++it) {
+    for (int item = blockIdx.x; ok && item < items; item += gridDim.x) {
+      int tile, kb0, kb1;
+      item_range(item, tile, kb0, kb1);
+      for (int kb = kb0; kb < kb1; ++kb, ++it) {
         if ((it & 1u) != grp) {  // the other group's k block: only advance the ring positions
           if (it >= WSK && ++xs_old == GM_XS) { xs_old = 0; xph_old ^= 1u; }
           if (++ps == GM_PS) { ps = 0; pph ^= 1u; }
@@ -272,7 +291,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     const bool f32 = a.out_dtype == BITRL_OUT_F32;
     uint32_t lt = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x, ++lt) {
+    for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++lt) {
+      const int tile = item / a.splits;
       const int tn = tile % a.tiles_n, tm = tile / a.tiles_n;
       const uint32_t buf = lt & 1u;
       const uint32_t sc_addr = base + GM_OFF_TOK + buf * GM_TOK_MAX * 4;
@@ -304,6 +324,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
         uint32_t v[32];
         ptx::tmem_ld_32x32b_x32(tmem_base + buf * GM_TOK_MAX + c * 32 + (static_cast<uint32_t>(q * 32) << 16), v);
         ptx::tmem_ld_wait();
+        if (a.part) {  // split-K item: hand the raw partial sums over, the finishing kernel does the rest
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (c * 32 + j < tok_hi)
+              atomicAdd(a.part + static_cast<size_t>(tok0 + c * 32 + j) * a.N + nbase + lane, static_cast<int>(v[j]));
+          continue;
+        }
         // acc = D - rowsum (exact int32), y = acc * scale
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
@@ -408,28 +435,86 @@ int sm_count();
 bool gemm_a_in_tmem();
 int gemm_forced_tok();    // 0, or the token-tile width forced through BITRL_GEMM_TOK (64, 128, 192, 224, 256)  // expanded weights through tensor memory (default) or through shared memory
 
+// Second kernel of a split-K launch: y = (part - rowsum) * gamma * a_m / 127 (+ residual), 8 outputs per thread.
+__global__ void __launch_bounds__(256) gemm_splitk_finish_kernel(const int32_t* part, const float* gamma, const float* absmax,
+                                                               const int32_t* rowsum, int M, int N, void* y, int out_dtype,
+                                                               const unsigned short* residual, int32_t* acc_out) {
+  pdl_enter();
+  const int n8 = N >> 3;
+  const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= static_cast<long long>(M) * n8) return;
+  const int m = static_cast<int>(idx / n8);
+  const size_t off = static_cast<size_t>(idx) * 8;
+  const uint4 p0 = *reinterpret_cast<const uint4*>(part + off), p1 = *reinterpret_cast<const uint4*>(part + off + 4);
+  const int rs = rowsum[m];
+  const float scale = out_scale(*gamma, absmax[m]);
+  const int acc[8] = {static_cast<int>(p0.x) - rs, static_cast<int>(p0.y) - rs, static_cast<int>(p0.z) - rs,
+                      static_cast<int>(p0.w) - rs, static_cast<int>(p1.x) - rs, static_cast<int>(p1.y) - rs,
+                      static_cast<int>(p1.z) - rs, static_cast<int>(p1.w) - rs};
+  if (acc_out) {
+    *reinterpret_cast<int4*>(acc_out + off) = make_int4(acc[0], acc[1], acc[2], acc[3]);
+    *reinterpret_cast<int4*>(acc_out + off + 4) = make_int4(acc[4], acc[5], acc[6], acc[7]);
+  }
+  float v[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) v[e] = __fmul_rn(static_cast<float>(acc[e]), scale);
+  if (out_dtype == BITRL_OUT_F32) {
+    float* yf = static_cast<float*>(y) + off;
+    *reinterpret_cast<float4*>(yf) = make_float4(v[0], v[1], v[2], v[3]);
+    *reinterpret_cast<float4*>(yf + 4) = make_float4(v[4], v[5], v[6], v[7]);
+    return;
+  }
+  uint32_t o[4];
+  uint4 rr = make_uint4(0u, 0u, 0u, 0u);
+  if (residual) rr = *reinterpret_cast<const uint4*>(residual + off);
+  const uint32_t rv[4] = {rr.x, rr.y, rr.z, rr.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    unsigned short lo = float_to_bf16_bits(v[2 * e]), hi = float_to_bf16_bits(v[2 * e + 1]);
+    if (residual) {
+      lo = float_to_bf16_bits(__fadd_rn(__uint_as_float(rv[e] << 16), bf16_bits_to_float(lo)));
+      hi = float_to_bf16_bits(__fadd_rn(__uint_as_float(rv[e] & 0xffff0000u), bf16_bits_to_float(hi)));
+    }
+    o[e] = static_cast<uint32_t>(lo) | (static_cast<uint32_t>(hi) << 16);
+  }
+  *reinterpret_cast<uint4*>(static_cast<unsigned short*>(y) + off) = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// Largest M for which a split-K workspace (M*N int32) is offered.
+constexpr int GM_SPLITK_MAX_M = 512;
+
+// splitk_ws: nullptr, or M*N int32 of scratch that allows split-K when the launch has too few tiles to fill the SMs.
 bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax, const int32_t* rowsum, int M,
-                         void* y, int out_dtype, const void* residual, int32_t* acc_out, cudaStream_t st) {
+                         void* y, int out_dtype, const void* residual, int32_t* acc_out, cudaStream_t st,
+                         int32_t* splitk_ws) {
   encode_tiled_fn encode = get_encode_tiled();
   if (!encode) return cuda_fail(cudaErrorSymbolNotFound);
-  // Token-tile width: fewest "waves x time per k block" over the SMs.
+  // Token-tile width and split count: fewest "waves x k blocks per item x time per k block" over the SMs.
   const int sms = sm_count();
   const int tiles_n = w->N / GM_ROWS;
-  int tok = 256;
+  const int kblocks = w->K / GM_BK;
+  int tok = 256, splits = 1;
   {
     long long best = -1;
     const int cand[5] = {256, 224, 192, 128, 64};
     for (int i = 0; i < 5; ++i) {
       if (cand[i] == 224 && !gemm_a_in_tmem()) continue;
       const long long tiles = static_cast<long long>(tiles_n) * ((M + cand[i] - 1) / cand[i]);
-      const long long waves = (tiles + sms - 1) / sms;
       // cycles per k block as measured: the 256-wide tile (4-stage x_q ring, weights through shared memory) runs at
       // about 690, the narrower ones at the MMA thread's own ~500 or the tensor pipe's 2*TOK, whichever is larger
-      const long long cost = waves * (cand[i] == 256 ? 690 : (2 * cand[i] > 500 ? 2 * cand[i] : 500));
-      if (best < 0 || cost <= best) { best = cost; tok = cand[i]; }  // ties go to the narrower tile
+      const long long per_kb = cand[i] == 256 ? 690 : (2 * cand[i] > 500 ? 2 * cand[i] : 500);
+      const int smax = (splitk_ws && M <= GM_SPLITK_MAX_M && tiles * 2 <= sms) ? static_cast<int>(sms / tiles) : 1;
+      for (int sp = 1; sp <= smax && sp <= kblocks; ++sp) {
+        const int kps = (kblocks + sp - 1) / sp;
+        if ((kblocks + kps - 1) / kps != sp) continue;  // this count would leave an empty split
+        const long long waves = (tiles * sp + sms - 1) / sms;
+        // a split launch pays for clearing the scratch and for the finishing kernel (about 3 us)
+        const long long cost = waves * kps * per_kb + (sp > 1 ? 6000 : 0);
+        if (best < 0 || cost <= best) { best = cost; tok = cand[i]; splits = sp; }  // ties go to the narrower tile
+      }
     }
   }
-  if (const int forced = gemm_forced_tok()) tok = forced;  // tuning knob, see bitrl.cu
+  if (const int forced = gemm_forced_tok()) { tok = forced; splits = 1; }  // tuning knob, see bitrl.cu
   CUtensorMap tmap;
   const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(w->K), static_cast<cuuint64_t>(M)};
   const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(w->K)};
@@ -440,10 +525,14 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
 
+  const bool split = splits > 1;
   GemmArgs a{w->tiles, w->gamma, absmax, rowsum, M, w->N, w->K, y, out_dtype,
-             static_cast<const unsigned short*>(residual), acc_out, tiles_n, 0};
+             split ? nullptr : static_cast<const unsigned short*>(residual), split ? nullptr : acc_out, tiles_n, 0,
+             splits, (kblocks + splits - 1) / splits, split ? splitk_ws : nullptr};
   a.tiles_total = tiles_n * ((M + tok - 1) / tok);
-  const int grid = a.tiles_total < sms ? a.tiles_total : sms;
+  const int items = a.tiles_total * splits;
+  const int grid = items < sms ? items : sms;
+  if (split) BITRL_CUDA(cudaMemsetAsync(splitk_ws, 0, static_cast<size_t>(M) * w->N * sizeof(int32_t), st));
   const bool a_tmem = gemm_a_in_tmem() && tok <= 224;
   void (*kern)(const CUtensorMap, const GemmArgs) =
       tok == 256 ? gemm_i8_kernel<256, false>
@@ -454,6 +543,13 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
   BITRL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM_BYTES));
   BITRL_CUDA(launch_pdl(kern, dim3(grid), dim3(GM_THREADS), GM_SMEM_BYTES, st, tmap, a));
   count_launch(1);
+  if (split) {
+    const long long n = static_cast<long long>(M) * (w->N / 8);
+    BITRL_CUDA(launch_pdl(gemm_splitk_finish_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, st,
+                          static_cast<const int32_t*>(splitk_ws), w->gamma, absmax, rowsum, M, w->N, y, out_dtype,
+                          static_cast<const unsigned short*>(residual), acc_out));
+    count_launch(1);
+  }
   return BITRL_OK;
 }
 

@@ -154,6 +154,14 @@ def test_gemm_batched_state_shapes_full(oracle_mod, B, M, K, N, wseed):
     check_layer(oracle_mod, B, M, K, N, wseed, 2200 + M, 1)
 
 
+@pytest.mark.parametrize("M", [17, 100, 300, 512])
+@pytest.mark.parametrize("K,N,wseed,out_dtype", [(6912, 256, 1010, 1), (6912, 128, 1011, 0), (2560, 384, 1012, 1)])
+def test_gemm_split_k_few_tiles(oracle_mod, B, M, K, N, wseed, out_dtype):
+    """Few output tiles and a long K: the launcher splits K over the idle SMs (int32 partial sums added with integer
+    atomics, a finishing kernel applies the epilogue).  Every stage must still equal the oracle's."""
+    check_layer(oracle_mod, B, M, K, N, wseed, 2300 + M, out_dtype)
+
+
 @pytest.mark.parametrize("K,N,wseed", [(2560, 6912, 1005), (6912, 2560, 1004)])
 def test_gemm_m4096_sampled(oracle_mod, B, K, N, wseed):
     """Full-size launch; the oracle recomputes 40 whole token rows plus 20000 random (m, n) outputs."""
