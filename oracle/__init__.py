@@ -17,6 +17,8 @@ from pathlib import Path
 
 import numpy as np
 
+from .rl_math import gae, log_softmax, mlp_head, ppo_loss  # noqa: F401  (heads, GAE and PPO objective, numpy fp64)
+
 _HERE = Path(__file__).resolve().parent
 _SRC = _HERE / "bitrl_oracle.cpp"
 _LIB = _HERE / "liboracle.so"
