@@ -198,6 +198,40 @@ BITRL_API bitrl_status bitrl_encoder_forward_states(const bitrl_encoder_t* enc, 
                                                     double theta, void* h_out, void* pooled, void* workspace,
                                                     size_t workspace_bytes, void* stream);
 
+/* ---- after the encoder: trainable heads, advantage estimation, PPO objective (all fp32, batched over the parallel
+ * environments; Eq. 3, Eq. 1, Sec. III-B, Table VI) -----------------------------------------------------------
+ * Heads: out = tanh(tanh(h W1t + b1) W2t + b2) W3t + b3.  The paper fixes two hidden layers of 256 and 128 units in
+ * fp32 and gives no activation; tanh is used.  h: dev bf16 [B,d] (the pooled latents), d a multiple of 16.
+ * Weights are dev fp32, stored input-major: W1t [d,H1], W2t [H1,H2], W3t [H2,n_out]; H1, H2, n_out <= 256.
+ * heads: HOST array of n_heads (<= 4) descriptors (policy head: n_out = number of actions; value head: n_out = 1);
+ * out: HOST array of n_heads dev fp32 pointers, out[i] is [B, heads[i].n_out]. */
+typedef struct bitrl_head {
+  const float* W1t; const float* b1;
+  const float* W2t; const float* b2;
+  const float* W3t; const float* b3;
+  int32_t n_out;
+} bitrl_head_t;
+BITRL_API bitrl_status bitrl_heads_forward(const void* h, int32_t B, int32_t d, int32_t H1, int32_t H2,
+                                           const bitrl_head_t* heads, int32_t n_heads, float* const* out, void* stream);
+
+/* Generalized advantage estimation over T steps of E environments (time-major dev fp32 arrays):
+ *   delta_t = r_t + gamma V_{t+1} (1 - done_t) - V_t ;  A_t = delta_t + gamma lambda (1 - done_t) A_{t+1}, A_T = 0
+ * rewards, dones: [T,E]; values: [T+1,E] (row T is the bootstrap value); adv: [T,E]; returns: NULL or [T,E] = adv + V. */
+BITRL_API bitrl_status bitrl_gae(const float* rewards, const float* values, const float* dones, int32_t T, int32_t E,
+                                 float gamma, float lambda, float* adv, float* returns, void* stream);
+
+/* Clipped surrogate of Eq. 1 with entropy bonus, and the value error, over a batch of B samples with A actions:
+ *   r = exp(log pi(a|s) - old_logp);  L_clip = mean min(r Ahat, clip(r, 1-eps, 1+eps) Ahat);  H = mean entropy(pi)
+ *   policy_loss = -(L_clip + beta H);  value_loss = mean 0.5 (V - R)^2
+ * logits: dev fp32 [B,A]; actions: dev int32 [B]; old_logp, adv, values, returns: dev fp32 [B].
+ * terms: dev fp32 [B,4] = per sample {r, min(...), entropy, 0.5 (V-R)^2} (required; also the reduction's input).
+ * dlogits: NULL or dev fp32 [B,A] = d policy_loss / d logits; dvalues: NULL or dev fp32 [B] = d value_loss / d values.
+ * summary: dev fp32 [4] = {L_clip, H, policy_loss, value_loss}, summed in a fixed order (deterministic). */
+BITRL_API bitrl_status bitrl_ppo_loss(const float* logits, const int32_t* actions, const float* old_logp,
+                                      const float* adv, const float* values, const float* returns, int32_t B, int32_t A,
+                                      float eps, float beta, float* terms, float* dlogits, float* dvalues,
+                                      float* summary, void* stream);
+
 /* ---- status ----------------------------------------------------------------------------------------- */
 /* Synchronizes `stream`, then reads and clears the device status word.  BITRL_OK, BITRL_ERR_TIMEOUT (a kernel
  * wait expired; results of that launch are invalid) or BITRL_ERR_CUDA. */

@@ -7,7 +7,8 @@ exception is raised.
 The functions mirror the C names without the ``bitrl_`` prefix:
 ``pack_ternary``, ``Linear`` (create/destroy), ``quant_act``, ``bitlinear_forward``, ``bitlinear_forward_debug``,
 ``bitlinear_forward_q``, ``rmsnorm_quant``, ``vrepeat_rmsnorm_quant``, ``relu2gate_rmsnorm_quant``, ``attention``,
-``pool_last_token``, ``Encoder`` (``forward``, ``forward_states``), ``poll_status``.
+``pool_last_token``, ``Encoder`` (``forward``, ``forward_states``), ``heads_forward``, ``gae``, ``ppo_loss``,
+``poll_status``.
 """
 from __future__ import annotations
 
@@ -28,6 +29,14 @@ GEMV_MAX_M = 16
 _vp = ctypes.c_void_p
 _i32 = ctypes.c_int32
 _sz = ctypes.c_size_t
+
+class HeadDesc(ctypes.Structure):
+    """Mirror of ``bitrl_head_t``."""
+    _fields_ = [("W1t", ctypes.c_void_p), ("b1", ctypes.c_void_p), ("W2t", ctypes.c_void_p), ("b2", ctypes.c_void_p),
+                ("W3t", ctypes.c_void_p), ("b3", ctypes.c_void_p), ("n_out", ctypes.c_int32)]
+
+
+_f32 = ctypes.c_float
 
 EXPORTS = {
     "bitrl_pack_workspace_bytes": (_sz, [_i32, _i32]),
@@ -54,6 +63,9 @@ EXPORTS = {
     "bitrl_pool_last_token": (_i32, [_vp, _i32, _vp, _i32, _i32, _i32, _vp, _vp]),
     "bitrl_encoder_states_workspace_bytes": (_sz, [_vp, _i32, _i32]),
     "bitrl_encoder_forward_states": (_i32, [_vp, _vp, _i32, _vp, _i32, _i32, ctypes.c_double, _vp, _vp, _vp, _sz, _vp]),
+    "bitrl_heads_forward": (_i32, [_vp, _i32, _i32, _i32, _i32, ctypes.POINTER(HeadDesc), _i32, ctypes.POINTER(_vp), _vp]),
+    "bitrl_gae": (_i32, [_vp, _vp, _vp, _i32, _i32, _f32, _f32, _vp, _vp, _vp]),
+    "bitrl_ppo_loss": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _f32, _f32, _vp, _vp, _vp, _vp, _vp]),
     "bitrl_selftest_wait_timeout": (_i32, [ctypes.c_int64, _vp]),
     "bitrl_poll_status": (_i32, [_vp]),
     "bitrl_last_timeout_stage": (_i32, []),
@@ -345,6 +357,55 @@ def pool_last_token(h: torch.Tensor, states) -> torch.Tensor:
     _check(lib().bitrl_pool_last_token(_ptr(h), T, _ptr(off), n_states, max_len, d, _ptr(out), _stream()),
            "bitrl_pool_last_token")
     return out
+
+
+def heads_forward(h: torch.Tensor, heads):
+    """h bf16 [B,d]; heads = list of (W1t [d,H1], b1, W2t [H1,H2], b2, W3t [H2,O], b3) CUDA fp32 tensors.
+    Returns one fp32 [B,O] tensor per head."""
+    _dev(h, torch.bfloat16, "h")
+    B, d = h.shape
+    H1, H2 = heads[0][0].shape[1], heads[0][2].shape[1]
+    descs = (HeadDesc * len(heads))()
+    outs = []
+    for i, (W1t, b1, W2t, b2, W3t, b3) in enumerate(heads):
+        for t in (W1t, b1, W2t, b2, W3t, b3):
+            _dev(t, torch.float32, "head weights")
+        assert W1t.shape == (d, H1) and W2t.shape == (H1, H2) and W3t.shape[0] == H2
+        descs[i] = HeadDesc(W1t.data_ptr(), b1.data_ptr(), W2t.data_ptr(), b2.data_ptr(), W3t.data_ptr(), b3.data_ptr(),
+                            W3t.shape[1])
+        outs.append(torch.empty((B, W3t.shape[1]), dtype=torch.float32, device=h.device))
+    optr = (_vp * len(heads))(*[o.data_ptr() for o in outs])
+    _check(lib().bitrl_heads_forward(_ptr(h), B, d, H1, H2, descs, len(heads), optr, _stream()), "bitrl_heads_forward")
+    return outs
+
+
+def gae(rewards: torch.Tensor, values: torch.Tensor, dones: torch.Tensor, gamma: float = 0.99, lam: float = 0.95):
+    """rewards, dones fp32 [T,E]; values fp32 [T+1,E].  Returns (advantages, returns), both [T,E]."""
+    for t in (rewards, values, dones):
+        _dev(t, torch.float32, "gae input")
+    T, E = rewards.shape
+    assert values.shape == (T + 1, E) and dones.shape == (T, E)
+    adv, ret = torch.empty_like(rewards), torch.empty_like(rewards)
+    _check(lib().bitrl_gae(_ptr(rewards), _ptr(values), _ptr(dones), T, E, gamma, lam, _ptr(adv), _ptr(ret), _stream()),
+           "bitrl_gae")
+    return adv, ret
+
+
+def ppo_loss(logits, actions, old_logp, adv, values, returns, eps: float = 0.1, beta: float = 0.05):
+    """Returns dict(summary fp32 [4] = {L_clip, entropy, policy_loss, value_loss}, terms [B,4], dlogits [B,A], dvalues [B])."""
+    _dev(logits, torch.float32, "logits")
+    _dev(actions, torch.int32, "actions")
+    for t in (old_logp, adv, values, returns):
+        _dev(t, torch.float32, "ppo input")
+    B, A = logits.shape
+    terms = torch.empty((B, 4), dtype=torch.float32, device=logits.device)
+    dlogits = torch.empty_like(logits)
+    dvalues = torch.empty((B,), dtype=torch.float32, device=logits.device)
+    summary = torch.empty((4,), dtype=torch.float32, device=logits.device)
+    _check(lib().bitrl_ppo_loss(_ptr(logits), _ptr(actions), _ptr(old_logp), _ptr(adv), _ptr(values), _ptr(returns), B, A,
+                                eps, beta, _ptr(terms), _ptr(dlogits), _ptr(dvalues), _ptr(summary), _stream()),
+           "bitrl_ppo_loss")
+    return {"summary": summary, "terms": terms, "dlogits": dlogits, "dvalues": dvalues}
 
 
 class Encoder:

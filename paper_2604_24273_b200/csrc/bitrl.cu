@@ -74,6 +74,7 @@ static bitrl_status check_arch() {
 #include "gemv_multi.cuh"
 #include "gemm.cuh"
 #include "attention.cuh"
+#include "heads.cuh"
 
 using namespace bitrl;
 
@@ -527,6 +528,59 @@ bitrl_status bitrl_pool_last_token(const void* h, int32_t T, const int32_t* stat
   bitrl_status s = check_arch();
   if (s != BITRL_OK) return s;
   return launch_pool_last_token(h, T, state_off, n_states, max_state_len, d, out, static_cast<cudaStream_t>(stream));
+}
+
+// ---- heads, GAE, PPO objective ----------------------------------------------------------------------------
+
+bitrl_status bitrl_heads_forward(const void* h, int32_t B, int32_t d, int32_t H1, int32_t H2, const bitrl_head_t* heads,
+                                 int32_t n_heads, float* const* out, void* stream) {
+  if (!h || !heads || !out) return BITRL_ERR_NULL;
+  if (B < 1 || d < 16 || d % 16 != 0 || H1 < 1 || H1 > HEAD_MAX_WIDTH || H2 < 1 || H2 > HEAD_MAX_WIDTH || n_heads < 1 ||
+      n_heads > HEAD_MAX_HEADS)
+    return BITRL_ERR_SHAPE;
+  HeadsArgs a;
+  for (int i = 0; i < n_heads; ++i) {
+    const bitrl_head_t& p = heads[i];
+    if (!p.W1t || !p.b1 || !p.W2t || !p.b2 || !p.W3t || !p.b3 || !out[i]) return BITRL_ERR_NULL;
+    if (p.n_out < 1 || p.n_out > HEAD_MAX_WIDTH) return BITRL_ERR_SHAPE;
+    a.head[i] = p;
+    a.out[i] = out[i];
+  }
+  for (int i = n_heads; i < HEAD_MAX_HEADS; ++i) { a.head[i] = heads[0]; a.out[i] = nullptr; }
+  if (!aligned16(h)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  a.h = static_cast<const unsigned short*>(h);
+  a.B = B; a.d = d; a.H1 = H1; a.H2 = H2;
+  return launch_heads(a, n_heads, static_cast<cudaStream_t>(stream));
+}
+
+bitrl_status bitrl_gae(const float* rewards, const float* values, const float* dones, int32_t T, int32_t E, float gamma,
+                       float lambda, float* adv, float* returns, void* stream) {
+  if (!rewards || !values || !dones || !adv) return BITRL_ERR_NULL;
+  if (T < 1 || E < 1) return BITRL_ERR_SHAPE;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  BITRL_CUDA(launch_pdl(gae_kernel, dim3((E + 127) / 128), dim3(128), 0, static_cast<cudaStream_t>(stream), rewards, values,
+                        dones, T, E, gamma, lambda, adv, returns));
+  count_launch(1);
+  return BITRL_OK;
+}
+
+bitrl_status bitrl_ppo_loss(const float* logits, const int32_t* actions, const float* old_logp, const float* adv,
+                            const float* values, const float* returns, int32_t B, int32_t A, float eps, float beta,
+                            float* terms, float* dlogits, float* dvalues, float* summary, void* stream) {
+  if (!logits || !actions || !old_logp || !adv || !values || !returns || !terms || !summary) return BITRL_ERR_NULL;
+  if (B < 1 || A < 1) return BITRL_ERR_SHAPE;
+  if (!aligned16(terms)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  PpoArgs a{logits, actions, old_logp, adv, values, returns, B, A, eps, beta, terms, dlogits, dvalues};
+  BITRL_CUDA(launch_pdl(ppo_terms_kernel, dim3((B + 7) / 8), dim3(256), 0, st, a));
+  BITRL_CUDA(launch_pdl(ppo_summary_kernel, dim3(1), dim3(256), 0, st, static_cast<const float*>(terms), B, beta, summary));
+  count_launch(2);
+  return BITRL_OK;
 }
 
 // ---- self-test of the bounded-wait / status-word path ----

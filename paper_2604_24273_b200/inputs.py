@@ -70,6 +70,41 @@ def state_offsets(n_states: int, seed: int, lo: int = STATE_TOKENS_MIN, hi: int 
     return torch.cat([torch.zeros(1, dtype=torch.int64), torch.cumsum(lens, 0)])
 
 
+HEAD_HIDDEN = (256, 128)  # hidden widths of the policy and value heads (paper: Table VI)
+
+
+def head_weights(d: int, n_out: int, seed: int, hidden=HEAD_HIDDEN):
+    """fp32 (W1t [d,H1], b1, W2t [H1,H2], b2, W3t [H2,n_out], b3), N(0, 1/fan_in) weights and N(0, 0.1) biases."""
+    g = _gen(seed)
+    dims = [d, hidden[0], hidden[1], n_out]
+    out = []
+    for i in range(3):
+        out.append(torch.randn(dims[i], dims[i + 1], generator=g, dtype=torch.float32) / dims[i] ** 0.5)
+        out.append(torch.randn(dims[i + 1], generator=g, dtype=torch.float32) * 0.1)
+    return tuple(out)
+
+
+def rollout(T: int, E: int, seed: int, done_prob: float = 0.02):
+    """fp32 rewards [T,E] ~ N(0,1), values [T+1,E] ~ N(0,1), dones [T,E] in {0,1} with P(done) = done_prob."""
+    g = _gen(seed)
+    r = torch.randn(T, E, generator=g, dtype=torch.float32)
+    v = torch.randn(T + 1, E, generator=g, dtype=torch.float32)
+    d = (torch.rand(T, E, generator=g) < done_prob).to(torch.float32)
+    return r, v, d
+
+
+def ppo_batch(B: int, A: int, seed: int):
+    """logits fp32 [B,A] ~ 2 N(0,1); actions int32 [B]; old_logp = log-softmax of perturbed logits at the action;
+    advantages, values, returns fp32 [B] ~ N(0,1)."""
+    g = _gen(seed)
+    logits = torch.randn(B, A, generator=g, dtype=torch.float32) * 2.0
+    actions = torch.randint(0, A, (B,), generator=g, dtype=torch.int32)
+    old = torch.log_softmax(logits + 0.3 * torch.randn(B, A, generator=g, dtype=torch.float32), dim=1)
+    old_logp = old[torch.arange(B), actions.long()].contiguous()
+    adv, v, R = (torch.randn(B, generator=g, dtype=torch.float32) for _ in range(3))
+    return logits, actions, old_logp, adv, v, R
+
+
 def bf16_bits(t: torch.Tensor):
     """bf16 CPU tensor -> numpy uint16 bit patterns (same shape)."""
     assert t.dtype == torch.bfloat16
