@@ -38,9 +38,9 @@ FULL_LAYERS = 30
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 INT8_OVER_BF16 = 2.0  # nominal dense int8 : bf16 tensor throughput on B200 (4.5 : 2.25 PFLOP/s)
 # DRAM bytes (read + write) of one gemv_multi_dp4a_kernel<1> launch per backbone block, from an ncu capture of the
-# 8-block case (dram__bytes_read.sum 138.995 MB + dram__bytes_write.sum 4.238 MB); every weight byte is read exactly
+# 8-block case (dram__bytes_read.sum 138.990 MB + dram__bytes_write.sum 4.391 MB, means of two launches); every weight byte is read exactly
 # once, so traffic scales with the number of blocks.  Set to None whenever that kernel changes.
-HEADLINE_TRAFFIC_PER_BLOCK = (138.995456e6 + 4.237568e6) / 8
+HEADLINE_TRAFFIC_PER_BLOCK = (138.990336e6 + 4.391296e6) / 8
 
 
 def load_peaks():
@@ -259,8 +259,21 @@ def run_ours(args):
     # independent (same activations, distinct weights), so they go through the grouped entry point: one launch of
     # one persistent kernel per step.
     def decode_setup(M):
-        xs = {k: inputs.activations(M, k, 2000 + M).to(dev) for k in (2560, 6912)}
-        ys = [[torch.empty((M, n), dtype=torch.bfloat16, device=dev) for _, _, n in BLOCK] for _ in range(n_layers)]
+        # the two activation tensors share one device buffer, and so do the outputs of each block: a step's inputs and
+        # its result then cross PCIe as one copy each way in the end-to-end measurement
+        xflat = torch.empty((M * (2560 + 6912),), dtype=torch.bfloat16, device=dev)
+        xs = {2560: xflat[:M * 2560].view(M, 2560), 6912: xflat[M * 2560:].view(M, 6912)}
+        for k in xs:
+            xs[k].copy_(inputs.activations(M, k, 2000 + M))
+        ys = []
+        for _ in range(n_layers):
+            yflat = torch.empty((M * sum(n for _, _, n in BLOCK),), dtype=torch.bfloat16, device=dev)
+            off, row = 0, []
+            for _, _, n in BLOCK:
+                row.append(yflat[off:off + M * n].view(M, n))
+                off += M * n
+            row.append(yflat)
+            ys.append(row)
         ws = [layers[l][j] for l in range(n_layers) for j in range(len(BLOCK))]
         xl = [xs[k] for _ in range(n_layers) for _, k, _ in BLOCK]
         yl = [ys[l][j] for l in range(n_layers) for j in range(len(BLOCK))]
@@ -275,6 +288,7 @@ def run_ours(args):
             for l in range(n_layers):
                 for j, (_, k, n) in enumerate(BLOCK):
                     bitrl.bitlinear_forward(layers[l][j], xs[k], bitrl.OUT_BF16, y=ys[l][j])
+        xs["flat"] = xflat
         return xs, ys, sweep, chain
 
     xs1, ys1, step1, chain1 = decode_setup(1)
@@ -285,17 +299,15 @@ def run_ours(args):
     us_per_launch = ms1 * 1e3 / (args.steps * launches1)
 
     # end to end: pinned host x -> device, the same graph, last block's outputs back to pinned host memory
-    host_x = {k: inputs.activations(1, k, 2001).pin_memory() for k in (2560, 6912)}
-    host_y = [torch.empty((1, n), dtype=torch.bfloat16).pin_memory() for _, _, n in BLOCK]
-    h2d = sum(t.numel() * 2 for t in host_x.values())
-    d2h = sum(t.numel() * 2 for t in host_y)
+    host_x = torch.cat([inputs.activations(1, k, 2001).reshape(-1) for k in (2560, 6912)]).pin_memory()
+    host_y = torch.empty_like(ys1[n_layers - 1][-1], device="cpu").pin_memory()
+    h2d = host_x.numel() * 2
+    d2h = host_y.numel() * 2
 
     def e2e_step():
-        for k in (2560, 6912):
-            xs1[k].copy_(host_x[k], non_blocking=True)
+        xs1["flat"].copy_(host_x, non_blocking=True)
         g1.replay()
-        for j in range(len(BLOCK)):
-            host_y[j].copy_(ys1[n_layers - 1][j], non_blocking=True)
+        host_y.copy_(ys1[n_layers - 1][-1], non_blocking=True)
         torch.cuda.current_stream().synchronize()
 
     for _ in range(args.warmup):
@@ -417,6 +429,32 @@ def run_ours(args):
                 "states_per_s": 128.0 / (msa * 1e-3), "ms": msa, "tokens": Tc, "bitlinear_TOPS": ops / (msa * 1e-3) / 1e12,
                 "frac_of_int8_peak_sustained": ops / (msa * 1e-3) / 1e12 / i8_sus, "launches": la}
             del ga, aws
+        # one agent step for 128 parallel environments: encoder with attention -> last-token latents -> policy and value
+        # heads; then the update-side math on a 2048-step rollout of those environments (GAE) and a 64-sample mini-batch
+        n_act = 6
+        heads = [tuple(t.to(dev) for t in inputs.head_weights(2560, n_act, 8200)),
+                 tuple(t.to(dev) for t in inputs.head_weights(2560, 1, 8201))]
+        aws = torch.empty((enc.states_workspace_bytes(T, 32),), dtype=torch.uint8, device=dev)
+
+        def agent_step():
+            enc.forward_states(h0, 32, h_out=h1, pooled=pooled, workspace=aws)
+            return bitrl.heads_forward(pooled, heads)
+
+        gs, ls = capture(agent_step)
+        mss = time_graph(gs, sub_steps, args.warmup, 1) / sub_steps
+        extra["agent_step_128_states_x32_tokens"] = {"ms": mss, "states_per_s": 128.0 / (mss * 1e-3), "launches": ls}
+        del gs
+        r, v, dn = (t.to(dev) for t in inputs.rollout(2048, 128, 8300))
+        batch = [t.to(dev) for t in inputs.ppo_batch(64, n_act, 8400)]
+
+        def update_math():
+            bitrl.gae(r, v, dn)
+            bitrl.ppo_loss(*batch)
+
+        gu, lu = capture(update_math)
+        msu = time_graph(gu, sub_steps, args.warmup, 1) / sub_steps
+        extra["gae_2048x128_plus_ppo_loss_64"] = {"us": msu * 1e3, "launches": lu}
+        del gu
     bitrl.poll_status()
     clocks_sections = sampler2.stop() if sampler2 else None
     if rank == 0 and "cpu" in sections:

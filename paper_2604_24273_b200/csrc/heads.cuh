@@ -123,14 +123,30 @@ __global__ void gae_kernel(const float* __restrict__ r, const float* __restrict_
   if (e >= E) return;
   const float gl = __fmul_rn(gamma, lam);
   float next_adv = 0.0f, v_next = v[static_cast<size_t>(T) * E + e];
-  for (int t = T - 1; t >= 0; --t) {
-    const size_t i = static_cast<size_t>(t) * E + e;
-    const float nd = 1.0f - done[i], vt = v[i];
-    const float delta = r[i] + gamma * v_next * nd - vt;
-    next_adv = delta + gl * nd * next_adv;
-    adv[i] = next_adv;
-    if (ret) ret[i] = next_adv + vt;
-    v_next = vt;
+  // The recursion is serial in t, the loads are not: eight steps' inputs are requested together.
+  constexpr int CHUNK = 8;
+  for (int t1 = T; t1 > 0; t1 -= CHUNK) {
+    float rr[CHUNK], vv[CHUNK], nn[CHUNK];
+#pragma unroll
+    for (int c = 0; c < CHUNK; ++c) {
+      const int t = t1 - 1 - c;
+      if (t >= 0) {
+        const size_t i = static_cast<size_t>(t) * E + e;
+        rr[c] = r[i]; vv[c] = v[i]; nn[c] = 1.0f - done[i];
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < CHUNK; ++c) {
+      const int t = t1 - 1 - c;
+      if (t >= 0) {
+        const size_t i = static_cast<size_t>(t) * E + e;
+        const float delta = rr[c] + gamma * v_next * nn[c] - vv[c];
+        next_adv = delta + gl * nn[c] * next_adv;
+        adv[i] = next_adv;
+        if (ret) ret[i] = next_adv + vv[c];
+        v_next = vv[c];
+      }
+    }
   }
 }
 
