@@ -123,8 +123,8 @@ __global__ void gae_kernel(const float* __restrict__ r, const float* __restrict_
   if (e >= E) return;
   const float gl = __fmul_rn(gamma, lam);
   float next_adv = 0.0f, v_next = v[static_cast<size_t>(T) * E + e];
-  // The recursion is serial in t, the loads are not: eight steps' inputs are requested together.
-  constexpr int CHUNK = 8;
+  // The recursion is serial in t, the loads are not: 32 steps' inputs are requested together.
+  constexpr int CHUNK = 32;
   for (int t1 = T; t1 > 0; t1 -= CHUNK) {
     float rr[CHUNK], vv[CHUNK], nn[CHUNK];
 #pragma unroll

@@ -150,6 +150,20 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_kernel(RowArgs a) {
 // shared memory; only the three scalar reductions cross warps.  8 / WPR rows per CTA.
 constexpr int ROWQ_MAXG = 7;
 
+// Four int32 codes -> four saturated int8 in one word (q0 in the low byte): two pack-with-saturation conversions.
+__device__ __forceinline__ uint32_t pack_s8x4(int q0, int q1, int q2, int q3) {
+  uint32_t hi, d;
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0));
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(q1), "r"(q0), "r"(hi));
+  return d;
+}
+// Sum of the four signed bytes of a word, added to acc.
+__device__ __forceinline__ int dp4a_ones(uint32_t w, int acc) {
+  int d;
+  asm("dp4a.s32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(w), "r"(0x01010101), "r"(acc));
+  return d;
+}
+
 template <int MODE, int WPR, int NG>
 __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, int T) {
   __shared__ float red_ss[ROW_THREADS / 32];
@@ -163,8 +177,9 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, i
   const int nvec8 = a.Kv >> 3;
   const unsigned short* src = a.in + (live ? row : 0) * a.in_stride + a.in_offset;
 
+  // pass 1: the row vector v, its sum of squares and its largest magnitude in one sweep
   float v[NG][8];
-  float ss = 0.0f;
+  float ss = 0.0f, mx = 0.0f;
 #pragma unroll
   for (int gi = 0; gi < NG; ++gi) {
     const int i = (gi * WPR + sub) * 32 + lane;
@@ -186,50 +201,36 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, i
           v[gi][2 * e + 1] = __fmul_rn(__fmul_rn(g1, g1), __uint_as_float(ru[e] & 0xffff0000u));
         }
       }
-      if (MODE != ROW_PLAIN) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) ss += v[gi][e] * v[gi][e];
+      for (int e = 0; e < 8; ++e) {
+        if (MODE != ROW_PLAIN) ss += v[gi][e] * v[gi][e];
+        mx = fmaxf(mx, fabsf(v[gi][e]));
       }
     } else {
 #pragma unroll
       for (int e = 0; e < 8; ++e) v[gi][e] = 0.0f;
     }
   }
-
-  float amax = 0.0f;
-  if (MODE != ROW_PLAIN) {
-    ss = warp_sum(ss);
-    if (WPR > 1) {
-      if (lane == 0) red_ss[warp] = ss;
-      __syncthreads();
-      ss = 0.0f;
-#pragma unroll
-      for (int i = 0; i < WPR; ++i) ss += red_ss[grp * WPR + i];
-    }
-    const float rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(ss, static_cast<float>(a.Kv)), 1e-5f)));
-#pragma unroll
-    for (int gi = 0; gi < NG; ++gi)
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        v[gi][e] = bf16_bits_to_float(float_to_bf16_bits(__fmul_rn(v[gi][e], rstd)));
-        amax = fmaxf(amax, fabsf(v[gi][e]));
-      }
-  } else {
-#pragma unroll
-    for (int gi = 0; gi < NG; ++gi)
-#pragma unroll
-      for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(v[gi][e]));
-  }
-  amax = warp_max(amax);
+  if (MODE != ROW_PLAIN) ss = warp_sum(ss);
+  mx = warp_max(mx);
   if (WPR > 1) {
-    if (lane == 0) red_mx[warp] = amax;
+    if (lane == 0) { red_ss[warp] = ss; red_mx[warp] = mx; }
     __syncthreads();
+    ss = 0.0f;
 #pragma unroll
-    for (int i = 0; i < WPR; ++i) amax = fmaxf(amax, red_mx[grp * WPR + i]);
+    for (int i = 0; i < WPR; ++i) { ss += red_ss[grp * WPR + i]; mx = fmaxf(mx, red_mx[grp * WPR + i]); }
+  }
+  // u = bf16(v * rstd) is monotonic in |v| (one rounded multiply, one rounding to bf16), so the largest |u| of the row
+  // is the image of the largest |v|: no second reduction over the normalized values.
+  float rstd = 1.0f, amax = mx;
+  if (MODE != ROW_PLAIN) {
+    rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(ss, static_cast<float>(a.Kv)), 1e-5f)));
+    amax = bf16_bits_to_float(float_to_bf16_bits(__fmul_rn(mx, rstd)));
   }
   amax = fmaxf(amax, 1e-5f);
   const float inv = __fdiv_rn(127.0f, amax);
 
+  // pass 2: normalize, round to bf16, quantize (round-to-nearest-even conversion, saturating pack), row sum of the codes
   int rs = 0;
   int8_t* xq = a.xq + (live ? row : 0) * a.Kout;
   unsigned short* uo = a.u_out ? a.u_out + (live ? row : 0) * a.Kout : nullptr;
@@ -237,30 +238,38 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, i
   for (int gi = 0; gi < NG; ++gi) {
     const int i = (gi * WPR + sub) * 32 + lane;
     if (live && i < nvec8) {
+      uint32_t ub[4];
       int q[8];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) { q[e] = quant_code(v[gi][e], inv); rs += q[e]; }
-      uint2 wd;
-      wd.x = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | (static_cast<uint32_t>(q[3]) << 24);
-      wd.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | (static_cast<uint32_t>(q[7]) << 24);
-      uint4 ub;
-      if (uo) {
-        ub.x = static_cast<uint32_t>(float_to_bf16_bits(v[gi][0])) | (static_cast<uint32_t>(float_to_bf16_bits(v[gi][1])) << 16);
-        ub.y = static_cast<uint32_t>(float_to_bf16_bits(v[gi][2])) | (static_cast<uint32_t>(float_to_bf16_bits(v[gi][3])) << 16);
-        ub.z = static_cast<uint32_t>(float_to_bf16_bits(v[gi][4])) | (static_cast<uint32_t>(float_to_bf16_bits(v[gi][5])) << 16);
-        ub.w = static_cast<uint32_t>(float_to_bf16_bits(v[gi][6])) | (static_cast<uint32_t>(float_to_bf16_bits(v[gi][7])) << 16);
+      for (int e = 0; e < 4; ++e) {
+        float lo = v[gi][2 * e], hi = v[gi][2 * e + 1];
+        if (MODE != ROW_PLAIN) {
+          const __nv_bfloat162 pr = __floats2bfloat162_rn(__fmul_rn(lo, rstd), __fmul_rn(hi, rstd));
+          ub[e] = *reinterpret_cast<const uint32_t*>(&pr);
+          lo = __uint_as_float(ub[e] << 16);
+          hi = __uint_as_float(ub[e] & 0xffff0000u);
+        } else if (a.u_out) {
+          ub[e] = (__float_as_uint(lo) >> 16) | (__float_as_uint(hi) & 0xffff0000u);
+        }
+        q[2 * e] = __float2int_rn(__fmul_rn(lo, inv));
+        q[2 * e + 1] = __float2int_rn(__fmul_rn(hi, inv));
       }
+      uint2 wd;
+      wd.x = pack_s8x4(q[0], q[1], q[2], q[3]);
+      wd.y = pack_s8x4(q[4], q[5], q[6], q[7]);
+      rs = dp4a_ones(wd.y, dp4a_ones(wd.x, rs));
+      const uint4 ub4 = make_uint4(ub[0], ub[1], ub[2], ub[3]);
       if (MODE == ROW_VREPEAT) {
         const int k = 8 * i;
         const int kvh = k / a.head_dim, e0 = k - kvh * a.head_dim;
         for (int r = 0; r < a.rep; ++r) {
           const int ko = (kvh * a.rep + r) * a.head_dim + e0;
           *reinterpret_cast<uint2*>(xq + ko) = wd;
-          if (uo) *reinterpret_cast<uint4*>(uo + ko) = ub;
+          if (uo) *reinterpret_cast<uint4*>(uo + ko) = ub4;
         }
       } else {
         *reinterpret_cast<uint2*>(xq + 8 * i) = wd;
-        if (uo) *reinterpret_cast<uint4*>(uo + 8 * i) = ub;
+        if (uo) *reinterpret_cast<uint4*>(uo + 8 * i) = ub4;
       }
     }
   }
