@@ -12,6 +12,8 @@
 // is rounded once to bf16.  Also here: last-token pooling of the encoder output to one latent per state.
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace bitrl {
@@ -29,6 +31,10 @@ struct AttArgs {
   const float2* rope;         // [state_len][HD / 2]: (cos, sin) of position * theta^(-2i/HD)
   unsigned short* att;        // bf16 [T, n_heads * HD]
 };
+
+__device__ __forceinline__ uint32_t ptx_smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
 
 __device__ __forceinline__ void report_status(int status, int stage) {
   if (atomicCAS(&g_status[0], 0, status) == 0) g_status[1] = stage;
@@ -227,6 +233,258 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_kernel(AttArgs a) {
   }
 }
 
+// ---- tensor-core formulation ------------------------------------------------------------------------------
+// Same (state, kv head) decomposition, but scores and the weighted sum of values run on the warp-level tensor
+// instruction mma.sync.m16n8k16 (f16 operands, fp32 accumulators).  To keep the products as exact as the fp32 form,
+// every fp32 operand x is split into two halves x = hi + lo (hi = f16(x), lo = f16(x - hi): 22 significant bits) and
+// the product a*b is formed as hi*hi + hi*lo + lo*hi (the dropped lo*lo term is below 2^-22 relative).  Values are
+// bf16 numbers and convert to f16 exactly (down to 6e-5 in magnitude, 3e-8 absolute below); softmax weights are split.
+// A warp owns one (query head, 16-token tile): Q fragments are read straight from global memory (the rotary partner
+// of a dimension sits in the same lane four k-steps later), K/V fragments come from shared memory through ldmatrix.
+constexpr int ATC_PAD = 8;  // halves added to each shared-memory row: consecutive rows start in different bank groups
+
+__device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// (x0, x1) -> f16x2 high parts and f16x2 low parts; x0 goes to the low half of the word.
+__device__ __forceinline__ void split_f16x2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  const __half h0 = __float2half_rn(x0), h1 = __float2half_rn(x1);
+  const __half l0 = __float2half_rn(x0 - __half2float(h0)), l1 = __float2half_rn(x1 - __half2float(h1));
+  hi = static_cast<uint32_t>(__half_as_ushort(h0)) | (static_cast<uint32_t>(__half_as_ushort(h1)) << 16);
+  lo = static_cast<uint32_t>(__half_as_ushort(l0)) | (static_cast<uint32_t>(__half_as_ushort(l1)) << 16);
+}
+
+// NKT = 8-key tiles held per query tile (keys padded to 8 * NKT, a multiple of 16).
+template <int HD, int NKT>
+__global__ void __launch_bounds__(ATT_THREADS) attention_tc_kernel(AttArgs a) {
+  constexpr int KS = HD / 16;            // k-steps of the score product
+  constexpr int ND = HD / 8;             // 8-wide output tiles
+  constexpr int SP = NKT * 8;            // padded keys
+  constexpr int RS = HD + ATC_PAD;       // shared-memory row stride in halves
+  extern __shared__ __align__(16) unsigned char atc_smem[];
+  __half* Khi = reinterpret_cast<__half*>(atc_smem);  // [SP][RS]
+  __half* Klo = Khi + SP * RS;
+  __half* Vh = Klo + SP * RS;
+
+  pdl_enter();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int st = blockIdx.x / a.n_kv, kvh = blockIdx.x - st * a.n_kv;
+  int t0, S;
+  if (!state_range(a.state_off, a.state_len, a.T, st, t0, S)) return;
+  if (S > SP) S = SP;  // the launcher picks NKT from state_len, so this never cuts
+  const int rep = a.n_heads / a.n_kv;
+  const int d = a.n_heads * HD, dkv = a.n_kv * HD, W = d + 2 * dkv;
+
+  // ---- keys (rotated, split) and values of this state into shared memory; rows S..SP-1 are zero ----
+  for (int r = warp; r < SP; r += ATT_WARPS) {
+    __half* kh = Khi + r * RS;
+    __half* kl = Klo + r * RS;
+    __half* vh = Vh + r * RS;
+    if (r < S) {
+      const unsigned short* krow = a.qkv + static_cast<long long>(t0 + r) * W + d + kvh * HD;
+      const float2* tab = a.rope + r * (HD / 2);
+      for (int i = 2 * lane; i < HD / 2; i += 64) {  // dims i, i+1 and their partners i + HD/2, i + 1 + HD/2
+        const uint32_t r1 = *reinterpret_cast<const uint32_t*>(krow + i);
+        const uint32_t r2 = *reinterpret_cast<const uint32_t*>(krow + i + HD / 2);
+        const float4 cs = *reinterpret_cast<const float4*>(tab + i);  // (cos_i, sin_i, cos_i+1, sin_i+1)
+        const float x1a = __uint_as_float(r1 << 16), x1b = __uint_as_float(r1 & 0xffff0000u);
+        const float x2a = __uint_as_float(r2 << 16), x2b = __uint_as_float(r2 & 0xffff0000u);
+        uint32_t hi, lo;
+        split_f16x2(fmaf(-x2a, cs.y, __fmul_rn(x1a, cs.x)), fmaf(-x2b, cs.w, __fmul_rn(x1b, cs.z)), hi, lo);
+        *reinterpret_cast<uint32_t*>(kh + i) = hi;
+        *reinterpret_cast<uint32_t*>(kl + i) = lo;
+        split_f16x2(fmaf(x1a, cs.y, __fmul_rn(x2a, cs.x)), fmaf(x1b, cs.w, __fmul_rn(x2b, cs.z)), hi, lo);
+        *reinterpret_cast<uint32_t*>(kh + i + HD / 2) = hi;
+        *reinterpret_cast<uint32_t*>(kl + i + HD / 2) = lo;
+      }
+      for (int i = 2 * lane; i < HD; i += 64) {
+        const uint32_t rv = *reinterpret_cast<const uint32_t*>(krow + dkv + i);
+        const __half v0 = __float2half_rn(__uint_as_float(rv << 16)), v1 = __float2half_rn(__uint_as_float(rv & 0xffff0000u));
+        *reinterpret_cast<uint32_t*>(vh + i) =
+            static_cast<uint32_t>(__half_as_ushort(v0)) | (static_cast<uint32_t>(__half_as_ushort(v1)) << 16);
+      }
+    } else {
+      for (int i = 2 * lane; i < HD; i += 64) {
+        *reinterpret_cast<uint32_t*>(kh + i) = 0u;
+        *reinterpret_cast<uint32_t*>(kl + i) = 0u;
+        *reinterpret_cast<uint32_t*>(vh + i) = 0u;
+      }
+    }
+  }
+  __syncthreads();
+
+  const int g = lane >> 2, t = lane & 3;
+  const float inv_sqrt = __fdiv_rn(1.0f, __fsqrt_rn(static_cast<float>(HD)));
+  const uint32_t khi_s = ptx_smem_u32(Khi), klo_s = ptx_smem_u32(Klo), vh_s = ptx_smem_u32(Vh);
+  // ldmatrix row address of this lane: matrix lane/8, row lane%8
+  const int lm = lane >> 3, lr = lane & 7;
+  const int m_tiles = (S + 15) >> 4;
+  for (int task = warp; task < rep * m_tiles; task += ATT_WARPS) {
+    // larger query tiles first: they have more keys under the causal limit
+    const int mt = m_tiles - 1 - task / rep, j = task % rep;
+    const int head = kvh * rep + j;
+    const int p_lo = 16 * mt + g, p_hi = p_lo + 8;
+    const int nkt = min(NKT, 2 * mt + 2);  // key tiles under the causal limit of this query tile
+
+    // ---- Q fragments: rows g and g+8 of the tile, rotated and split ----
+    uint32_t qh[KS][4], ql[KS][4];
+#pragma unroll
+    for (int rr = 0; rr < 2; ++rr) {
+      const int p = rr ? p_hi : p_lo;
+      const bool live = p < S;
+      const unsigned short* qrow = a.qkv + static_cast<long long>(t0 + (live ? p : 0)) * W + head * HD;
+      const float2* tab = a.rope + (live ? p : 0) * (HD / 2);
+#pragma unroll
+      for (int ks = 0; ks < KS / 2; ++ks)
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          const int dim = 16 * ks + 8 * hf + 2 * t;  // dims dim, dim+1 (first half of the head) and their partners
+          uint32_t r1 = 0u, r2 = 0u;
+          if (live) {
+            r1 = *reinterpret_cast<const uint32_t*>(qrow + dim);
+            r2 = *reinterpret_cast<const uint32_t*>(qrow + dim + HD / 2);
+          }
+          const float4 cs = *reinterpret_cast<const float4*>(tab + dim);
+          const float x1a = __uint_as_float(r1 << 16), x1b = __uint_as_float(r1 & 0xffff0000u);
+          const float x2a = __uint_as_float(r2 << 16), x2b = __uint_as_float(r2 & 0xffff0000u);
+          split_f16x2(fmaf(-x2a, cs.y, __fmul_rn(x1a, cs.x)), fmaf(-x2b, cs.w, __fmul_rn(x1b, cs.z)),
+                      qh[ks][2 * hf + rr], ql[ks][2 * hf + rr]);
+          split_f16x2(fmaf(x1a, cs.y, __fmul_rn(x2a, cs.x)), fmaf(x1b, cs.w, __fmul_rn(x2b, cs.z)),
+                      qh[ks + KS / 2][2 * hf + rr], ql[ks + KS / 2][2 * hf + rr]);
+        }
+    }
+
+    // ---- scores: c[nt] = Q K^T for key tile nt (rows g / g+8, keys 8nt+2t, +1) ----
+    float c[NKT][4];
+#pragma unroll
+    for (int nt = 0; nt < NKT; ++nt) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) c[nt][e] = 0.0f;
+      if (nt < nkt) {
+#pragma unroll
+        for (int ks = 0; ks < KS; ks += 2) {
+          const uint32_t off = static_cast<uint32_t>(((8 * nt + lr) * RS + 16 * ks + 8 * lm) * 2);
+          uint32_t bh[4], bl[4];
+          ldmatrix_x4(khi_s + off, bh);
+          ldmatrix_x4(klo_s + off, bl);
+          mma_f16(c[nt], qh[ks], bh[0], bh[1]);
+          mma_f16(c[nt], qh[ks], bl[0], bl[1]);
+          mma_f16(c[nt], ql[ks], bh[0], bh[1]);
+          mma_f16(c[nt], qh[ks + 1], bh[2], bh[3]);
+          mma_f16(c[nt], qh[ks + 1], bl[2], bl[3]);
+          mma_f16(c[nt], ql[ks + 1], bh[2], bh[3]);
+        }
+      }
+    }
+
+    // ---- softmax over the keys r <= p of each row (unnormalized weights, row sums kept) ----
+    float m_lo = -INFINITY, m_hi = -INFINITY;
+#pragma unroll
+    for (int nt = 0; nt < NKT; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int key = 8 * nt + 2 * t + e;
+        c[nt][e] = (nt < nkt && key <= p_lo) ? __fmul_rn(c[nt][e], inv_sqrt) : -INFINITY;
+        c[nt][2 + e] = (nt < nkt && key <= p_hi) ? __fmul_rn(c[nt][2 + e], inv_sqrt) : -INFINITY;
+        m_lo = fmaxf(m_lo, c[nt][e]);
+        m_hi = fmaxf(m_hi, c[nt][2 + e]);
+      }
+    m_lo = fmaxf(m_lo, __shfl_xor_sync(0xffffffffu, m_lo, 1));
+    m_lo = fmaxf(m_lo, __shfl_xor_sync(0xffffffffu, m_lo, 2));
+    m_hi = fmaxf(m_hi, __shfl_xor_sync(0xffffffffu, m_hi, 1));
+    m_hi = fmaxf(m_hi, __shfl_xor_sync(0xffffffffu, m_hi, 2));
+    float s_lo = 0.0f, s_hi = 0.0f;
+#pragma unroll
+    for (int nt = 0; nt < NKT; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        c[nt][e] = expf(c[nt][e] - m_lo);  // key 0 is never masked, so the maxima are finite
+        c[nt][2 + e] = expf(c[nt][2 + e] - m_hi);
+        s_lo += c[nt][e];
+        s_hi += c[nt][2 + e];
+      }
+    s_lo += __shfl_xor_sync(0xffffffffu, s_lo, 1);
+    s_lo += __shfl_xor_sync(0xffffffffu, s_lo, 2);
+    s_hi += __shfl_xor_sync(0xffffffffu, s_hi, 1);
+    s_hi += __shfl_xor_sync(0xffffffffu, s_hi, 2);
+
+    // ---- out = P V: the score accumulators of two adjacent key tiles are the A fragment of one 16-key step ----
+    float o[ND][4];
+#pragma unroll
+    for (int nd = 0; nd < ND; ++nd)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) o[nd][e] = 0.0f;
+#pragma unroll
+    for (int kk = 0; kk < NKT / 2; ++kk) {
+      if (2 * kk < nkt) {
+        uint32_t ph[4], pl[4];
+        split_f16x2(c[2 * kk][0], c[2 * kk][1], ph[0], pl[0]);
+        split_f16x2(c[2 * kk][2], c[2 * kk][3], ph[1], pl[1]);
+        split_f16x2(c[2 * kk + 1][0], c[2 * kk + 1][1], ph[2], pl[2]);
+        split_f16x2(c[2 * kk + 1][2], c[2 * kk + 1][3], ph[3], pl[3]);
+#pragma unroll
+        for (int nd = 0; nd < ND; nd += 2) {
+          uint32_t bv[4];
+          ldmatrix_x4_trans(vh_s + static_cast<uint32_t>(((16 * kk + 8 * (lm & 1) + lr) * RS + 8 * (nd + (lm >> 1))) * 2), bv);
+          mma_f16(o[nd], ph, bv[0], bv[1]);
+          mma_f16(o[nd], pl, bv[0], bv[1]);
+          mma_f16(o[nd + 1], ph, bv[2], bv[3]);
+          mma_f16(o[nd + 1], pl, bv[2], bv[3]);
+        }
+      }
+    }
+
+    // ---- normalize, round to bf16, store rows g and g+8 ----
+#pragma unroll
+    for (int rr = 0; rr < 2; ++rr) {
+      const int p = rr ? p_hi : p_lo;
+      if (p < S) {
+        const float den = rr ? s_hi : s_lo;
+        unsigned short* orow = a.att + static_cast<long long>(t0 + p) * d + head * HD + 2 * t;
+#pragma unroll
+        for (int nd = 0; nd < ND; ++nd)
+          *reinterpret_cast<uint32_t*>(orow + 8 * nd) =
+              static_cast<uint32_t>(float_to_bf16_bits(__fdiv_rn(o[nd][2 * rr], den))) |
+              (static_cast<uint32_t>(float_to_bf16_bits(__fdiv_rn(o[nd][2 * rr + 1], den))) << 16);
+      }
+    }
+  }
+}
+
+template <int HD, int NKT>
+bitrl_status launch_attention_tc_t(const AttArgs& a, int n_states, cudaStream_t st) {
+  const size_t smem = static_cast<size_t>(3) * (NKT * 8) * (HD + ATC_PAD) * sizeof(__half);
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  BITRL_CUDA(cudaGetDevice(&dev));
+  if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+    BITRL_CUDA(cudaFuncSetAttribute(attention_tc_kernel<HD, NKT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    static_cast<int>(smem)));
+    attr_set[dev] = true;
+  }
+  BITRL_CUDA(launch_pdl(attention_tc_kernel<HD, NKT>, dim3(static_cast<unsigned>(n_states) * a.n_kv), dim3(ATT_THREADS),
+                        smem, st, a));
+  count_launch(1);
+  return BITRL_OK;
+}
+
+template <int HD>
+bitrl_status launch_attention_tc_hd(const AttArgs& a, int n_states, cudaStream_t st) {
+  if (a.state_len <= 32) return launch_attention_tc_t<HD, 4>(a, n_states, st);
+  if (a.state_len <= 64) return launch_attention_tc_t<HD, 8>(a, n_states, st);
+  return launch_attention_tc_t<HD, 16>(a, n_states, st);
+}
+
 template <int HD, int G, int NCH>
 bitrl_status launch_attention_t(const AttArgs& a, int n_states, cudaStream_t st) {
   constexpr int SMAX = NCH * 32;
@@ -278,8 +536,8 @@ bitrl_status launch_attention(const void* qkv, int T, const int* state_off, int 
                               int n_kv, int hd, const float2* rope, void* att, cudaStream_t st) {
   AttArgs a{static_cast<const unsigned short*>(qkv), state_off, state_len, T, n_heads, n_kv, rope,
             static_cast<unsigned short*>(att)};
-  if (hd == 128) return launch_attention_hd<128>(a, n_states, st);
-  if (hd == 64) return launch_attention_hd<64>(a, n_states, st);
+  if (hd == 128) return launch_attention_tc_hd<128>(a, n_states, st);
+  if (hd == 64) return launch_attention_tc_hd<64>(a, n_states, st);
   return BITRL_ERR_SHAPE;
 }
 
