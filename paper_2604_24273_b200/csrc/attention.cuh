@@ -2,14 +2,15 @@
 // to 15-40 tokens that go through the backbone in one forward pass).  Causal grouped-query attention with rotary
 // position embedding, the form of the architecture the backbone follows (Sec. III-B cites it, the paper does not
 // spell it out).  States are short and independent, so one CTA owns one (state, kv head): its rotated keys and its
-// values sit in shared memory as fp32 and every query of the heads that share the kv head streams over them.
+// values sit in shared memory and every query tile of the heads that share the kv head runs over them.
 //
 //   rotary (rotate-half), position p = index of the token inside its state, i < head_dim/2:
 //     angle = p * theta^(-2i/head_dim);  (x_i, x_{i+hd/2}) -> (x_i cos - x_{i+hd/2} sin, x_{i+hd/2} cos + x_i sin)
 //   score(p, r) = q_p . k_r / sqrt(head_dim), r <= p;  w = exp(score - max);  out_p = (sum_r w_r v_r) / sum_r w_r
 //
-// All arithmetic is fp32 (fused multiply-adds), the cos/sin table is computed in fp64 and rounded once; the output
-// is rounded once to bf16.  Also here: last-token pooling of the encoder output to one latent per state.
+// The rotation is fp32 with cos/sin from an fp64 table rounded once; the two contractions run on the warp-level
+// tensor instruction with split-precision operands (below); the output is rounded once to bf16.  Also here:
+// last-token pooling of the encoder output to one latent per state.
 #pragma once
 
 #include <cuda_fp16.h>
@@ -65,177 +66,11 @@ __global__ void rope_table_kernel(float2* tab, int max_len, int hd, double theta
   tab[idx] = make_float2(static_cast<float>(cos(ang)), static_cast<float>(sin(ang)));
 }
 
-// The HD/32 consecutive elements a lane holds of one head row, rotated.  The partner of element e is e +- HD/2,
-// which the lane 16 away holds at the same register index.
-template <int HD>
-__device__ __forceinline__ void rope_lane(const float (&x)[HD / 32], const float2* tab_row, int lane, float (&y)[HD / 32]) {
-  constexpr int EPL = HD / 32;
-#pragma unroll
-  for (int j = 0; j < EPL; ++j) {
-    const float partner = __shfl_xor_sync(0xffffffffu, x[j], 16);
-    const int i = (lane * EPL + j) & (HD / 2 - 1);
-    const float2 cs = tab_row[i];
-    y[j] = fmaf(partner, lane < 16 ? -cs.y : cs.y, __fmul_rn(x[j], cs.x));
-  }
-}
-
-template <int HD>
-__device__ __forceinline__ void load_lane(const unsigned short* row, int lane, float (&x)[HD / 32]) {
-  if constexpr (HD == 128) {
-    const uint2 raw = *reinterpret_cast<const uint2*>(row + lane * 4);
-    x[0] = __uint_as_float(raw.x << 16);
-    x[1] = __uint_as_float(raw.x & 0xffff0000u);
-    x[2] = __uint_as_float(raw.y << 16);
-    x[3] = __uint_as_float(raw.y & 0xffff0000u);
-  } else {
-    const uint32_t raw = *reinterpret_cast<const uint32_t*>(row + lane * 2);
-    x[0] = __uint_as_float(raw << 16);
-    x[1] = __uint_as_float(raw & 0xffff0000u);
-  }
-}
-
-// G = query heads of one kv head handled together (they share every key and value load); NCH = 32-key chunks.
-template <int HD, int G, int NCH>
-__global__ void __launch_bounds__(ATT_THREADS) attention_kernel(AttArgs a) {
-  constexpr int EPL = HD / 32;   // elements of a head row per lane
-  constexpr int KS = HD + 4;     // key row stride in floats: 16-byte rows, quarter-warps hit distinct banks
-  constexpr int SMAX = NCH * 32;
-  extern __shared__ __align__(16) float att_smem[];
-  float* Ks = att_smem;                     // [SMAX][KS]   rotated keys
-  float* Vs = Ks + SMAX * KS;               // [SMAX][HD]   values
-  float* Qs = Vs + SMAX * HD;               // [warps][G][HD] rotated queries of the token a warp works on
-  float* Ps = Qs + ATT_WARPS * G * HD;      // [warps][SMAX][G] unnormalized softmax weights
-
-  pdl_enter();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int st = blockIdx.x / a.n_kv, kvh = blockIdx.x - st * a.n_kv;
-  int t0, S;
-  if (!state_range(a.state_off, a.state_len, a.T, st, t0, S)) return;
-  if (S > SMAX) S = SMAX;  // the launcher picks NCH from state_len, so this never cuts
-  const int rep = a.n_heads / a.n_kv;
-  const int d = a.n_heads * HD, dkv = a.n_kv * HD, W = d + 2 * dkv;
-
-  for (int r = warp; r < S; r += ATT_WARPS) {
-    const unsigned short* krow = a.qkv + static_cast<long long>(t0 + r) * W + d + kvh * HD;
-    float kx[EPL], ky[EPL], vx[EPL];
-    load_lane<HD>(krow, lane, kx);
-    load_lane<HD>(krow + dkv, lane, vx);
-    rope_lane<HD>(kx, a.rope + r * (HD / 2), lane, ky);
-#pragma unroll
-    for (int j = 0; j < EPL; ++j) {
-      Ks[r * KS + lane * EPL + j] = ky[j];
-      Vs[r * HD + lane * EPL + j] = vx[j];
-    }
-  }
-  __syncthreads();
-
-  float* qw = Qs + warp * G * HD;
-  float* pw = Ps + warp * SMAX * G;
-  const float inv_sqrt = __fdiv_rn(1.0f, __fsqrt_rn(static_cast<float>(HD)));
-  const int n_groups = rep / G;
-  // Tokens are dealt to the warps in a zig-zag (w, 15-w, 16+w, 31-w, ...) so that every warp gets the same
-  // number of causal keys.
-  for (int k = 0; k * ATT_WARPS < S; ++k) {
-    const int p = (k & 1) ? k * ATT_WARPS + (ATT_WARPS - 1 - warp) : k * ATT_WARPS + warp;
-    if (p >= S) continue;
-    const unsigned short* qrow = a.qkv + static_cast<long long>(t0 + p) * W;
-    for (int grp = 0; grp < n_groups; ++grp) {
-      const int h0 = kvh * rep + grp * G;
-#pragma unroll
-      for (int j = 0; j < G; ++j) {
-        float qx[EPL], qy[EPL];
-        load_lane<HD>(qrow + (h0 + j) * HD, lane, qx);
-        rope_lane<HD>(qx, a.rope + p * (HD / 2), lane, qy);
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) qw[j * HD + lane * EPL + e] = qy[e];
-      }
-      __syncwarp();
-
-      // scores: lane = key r inside each 32-key chunk
-      float sc[G][NCH];
-#pragma unroll
-      for (int c = 0; c < NCH; ++c) {
-        const int r = c * 32 + lane;
-        float acc[G];
-#pragma unroll
-        for (int j = 0; j < G; ++j) acc[j] = 0.0f;
-        if (c * 32 <= p) {
-          const float4* kr = reinterpret_cast<const float4*>(Ks + r * KS);
-#pragma unroll 8
-          for (int e4 = 0; e4 < HD / 4; ++e4) {
-            const float4 kv = kr[e4];
-#pragma unroll
-            for (int j = 0; j < G; ++j) {
-              const float4 qv = *reinterpret_cast<const float4*>(qw + j * HD + 4 * e4);
-              acc[j] = fmaf(qv.x, kv.x, acc[j]);
-              acc[j] = fmaf(qv.y, kv.y, acc[j]);
-              acc[j] = fmaf(qv.z, kv.z, acc[j]);
-              acc[j] = fmaf(qv.w, kv.w, acc[j]);
-            }
-          }
-        }
-#pragma unroll
-        for (int j = 0; j < G; ++j) sc[j][c] = (r <= p) ? __fmul_rn(acc[j], inv_sqrt) : -INFINITY;
-      }
-
-      // softmax weights (unnormalized) and their sums
-      float den[G];
-#pragma unroll
-      for (int j = 0; j < G; ++j) {
-        float m = sc[j][0];
-#pragma unroll
-        for (int c = 1; c < NCH; ++c) m = fmaxf(m, sc[j][c]);
-        m = warp_max(m);
-        float s = 0.0f;
-#pragma unroll
-        for (int c = 0; c < NCH; ++c) {
-          const float w = (c * 32 + lane <= p) ? expf(sc[j][c] - m) : 0.0f;
-          s += w;
-          pw[(c * 32 + lane) * G + j] = w;
-        }
-        den[j] = warp_sum(s);
-      }
-      __syncwarp();
-
-      // out = sum_r w_r v_r: lane = EPL consecutive elements of the head row
-      float o[G][EPL];
-#pragma unroll
-      for (int j = 0; j < G; ++j)
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) o[j][e] = 0.0f;
-      for (int r = 0; r <= p; ++r) {
-        float v[EPL], w[G];
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) v[e] = Vs[r * HD + lane * EPL + e];
-#pragma unroll
-        for (int j = 0; j < G; ++j) w[j] = pw[r * G + j];
-#pragma unroll
-        for (int j = 0; j < G; ++j)
-#pragma unroll
-          for (int e = 0; e < EPL; ++e) o[j][e] = fmaf(w[j], v[e], o[j][e]);
-      }
-      unsigned short* orow = a.att + static_cast<long long>(t0 + p) * d;
-#pragma unroll
-      for (int j = 0; j < G; ++j) {
-        uint32_t wd[EPL / 2];
-#pragma unroll
-        for (int e = 0; e < EPL; e += 2)
-          wd[e / 2] = static_cast<uint32_t>(float_to_bf16_bits(__fdiv_rn(o[j][e], den[j]))) |
-                      (static_cast<uint32_t>(float_to_bf16_bits(__fdiv_rn(o[j][e + 1], den[j]))) << 16);
-        unsigned short* dst = orow + (h0 + j) * HD + lane * EPL;
-        if constexpr (EPL == 4)
-          *reinterpret_cast<uint2*>(dst) = make_uint2(wd[0], wd[1]);
-        else
-          *reinterpret_cast<uint32_t*>(dst) = wd[0];
-      }
-      __syncwarp();  // the next item overwrites this warp's query and weight rows
-    }
-  }
-}
-
-// ---- tensor-core formulation ------------------------------------------------------------------------------
-// Same (state, kv head) decomposition, but scores and the weighted sum of values run on the warp-level tensor
-// instruction mma.sync.m16n8k16 (f16 operands, fp32 accumulators).  To keep the products as exact as the fp32 form,
+// ---- the kernel ---------------------------------------------------------------------------------------------
+// Scores and the weighted sum of values run on the warp-level tensor instruction mma.sync.m16n8k16 (f16 operands,
+// fp32 accumulators; the contractions are 16..128 tokens wide, far below a tcgen05 tile).  To keep the products as
+// exact as an fp32 multiply-add chain (which a first version of this kernel used: 76 us per block, bound by
+// shared-memory wavefronts),
 // every fp32 operand x is split into two halves x = hi + lo (hi = f16(x), lo = f16(x - hi): 22 significant bits) and
 // the product a*b is formed as hi*hi + hi*lo + lo*hi (the dropped lo*lo term is below 2^-22 relative).  Values are
 // bf16 numbers and convert to f16 exactly (down to 6e-5 in magnitude, 3e-8 absolute below); softmax weights are split.
@@ -266,7 +101,7 @@ __device__ __forceinline__ void split_f16x2(float x0, float x1, uint32_t& hi, ui
 
 // NKT = 8-key tiles held per query tile (keys padded to 8 * NKT, a multiple of 16).
 template <int HD, int NKT>
-__global__ void __launch_bounds__(ATT_THREADS) attention_tc_kernel(AttArgs a) {
+__global__ void __launch_bounds__(ATT_THREADS, NKT <= 4 ? 2 : 1) attention_tc_kernel(AttArgs a) {
   constexpr int KS = HD / 16;            // k-steps of the score product
   constexpr int ND = HD / 8;             // 8-wide output tiles
   constexpr int SP = NKT * 8;            // padded keys
@@ -286,6 +121,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_tc_kernel(AttArgs a) {
   const int d = a.n_heads * HD, dkv = a.n_kv * HD, W = d + 2 * dkv;
 
   // ---- keys (rotated, split) and values of this state into shared memory; rows S..SP-1 are zero ----
+#pragma unroll 4
   for (int r = warp; r < SP; r += ATT_WARPS) {
     __half* kh = Khi + r * RS;
     __half* kl = Klo + r * RS;
@@ -365,27 +201,45 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_tc_kernel(AttArgs a) {
     }
 
     // ---- scores: c[nt] = Q K^T for key tile nt (rows g / g+8, keys 8nt+2t, +1) ----
-    float c[NKT][4];
+    // Consecutive tensor instructions go to different accumulators (four key tiles, and the terms that involve a low
+    // half are summed apart in c2), so that none waits for the one before it; the two sums are added at the end.
+    float c[NKT][4], c2[NKT][4];
 #pragma unroll
-    for (int nt = 0; nt < NKT; ++nt) {
+    for (int nt = 0; nt < NKT; ++nt)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) c[nt][e] = 0.0f;
-      if (nt < nkt) {
+      for (int e = 0; e < 4; ++e) c[nt][e] = c2[nt][e] = 0.0f;
+#pragma unroll
+    for (int n0 = 0; n0 < NKT; n0 += 4) {
+      if (n0 < nkt) {
 #pragma unroll
         for (int ks = 0; ks < KS; ks += 2) {
-          const uint32_t off = static_cast<uint32_t>(((8 * nt + lr) * RS + 16 * ks + 8 * lm) * 2);
-          uint32_t bh[4], bl[4];
-          ldmatrix_x4(khi_s + off, bh);
-          ldmatrix_x4(klo_s + off, bl);
-          mma_f16(c[nt], qh[ks], bh[0], bh[1]);
-          mma_f16(c[nt], qh[ks], bl[0], bl[1]);
-          mma_f16(c[nt], ql[ks], bh[0], bh[1]);
-          mma_f16(c[nt], qh[ks + 1], bh[2], bh[3]);
-          mma_f16(c[nt], qh[ks + 1], bl[2], bl[3]);
-          mma_f16(c[nt], ql[ks + 1], bh[2], bh[3]);
+          uint32_t bh[4][4], bl[4][4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            // key tiles beyond the causal limit hold finite numbers (keys of this state or zero rows) and are masked below
+            const uint32_t off = static_cast<uint32_t>(((8 * (n0 + i) + lr) * RS + 16 * ks + 8 * lm) * 2);
+            ldmatrix_x4(khi_s + off, bh[i]);
+            ldmatrix_x4(klo_s + off, bl[i]);
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) mma_f16(c[n0 + i], qh[ks], bh[i][0], bh[i][1]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) mma_f16(c2[n0 + i], qh[ks], bl[i][0], bl[i][1]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) mma_f16(c[n0 + i], qh[ks + 1], bh[i][2], bh[i][3]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) mma_f16(c2[n0 + i], ql[ks], bh[i][0], bh[i][1]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) mma_f16(c2[n0 + i], qh[ks + 1], bl[i][2], bl[i][3]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) mma_f16(c2[n0 + i], ql[ks + 1], bh[i][2], bh[i][3]);
         }
       }
     }
+#pragma unroll
+    for (int nt = 0; nt < NKT; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) c[nt][e] += c2[nt][e];
 
     // ---- softmax over the keys r <= p of each row (unnormalized weights, row sums kept) ----
     float m_lo = -INFINITY, m_hi = -INFINITY;
@@ -449,13 +303,13 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_tc_kernel(AttArgs a) {
     for (int rr = 0; rr < 2; ++rr) {
       const int p = rr ? p_hi : p_lo;
       if (p < S) {
-        const float den = rr ? s_hi : s_lo;
+        const float rden = __fdiv_rn(1.0f, rr ? s_hi : s_lo);  // one division per row, then multiplies
         unsigned short* orow = a.att + static_cast<long long>(t0 + p) * d + head * HD + 2 * t;
 #pragma unroll
-        for (int nd = 0; nd < ND; ++nd)
-          *reinterpret_cast<uint32_t*>(orow + 8 * nd) =
-              static_cast<uint32_t>(float_to_bf16_bits(__fdiv_rn(o[nd][2 * rr], den))) |
-              (static_cast<uint32_t>(float_to_bf16_bits(__fdiv_rn(o[nd][2 * rr + 1], den))) << 16);
+        for (int nd = 0; nd < ND; ++nd) {
+          const __nv_bfloat162 pr = __floats2bfloat162_rn(__fmul_rn(o[nd][2 * rr], rden), __fmul_rn(o[nd][2 * rr + 1], rden));
+          *reinterpret_cast<uint32_t*>(orow + 8 * nd) = *reinterpret_cast<const uint32_t*>(&pr);
+        }
       }
     }
   }
@@ -483,40 +337,6 @@ bitrl_status launch_attention_tc_hd(const AttArgs& a, int n_states, cudaStream_t
   if (a.state_len <= 32) return launch_attention_tc_t<HD, 4>(a, n_states, st);
   if (a.state_len <= 64) return launch_attention_tc_t<HD, 8>(a, n_states, st);
   return launch_attention_tc_t<HD, 16>(a, n_states, st);
-}
-
-template <int HD, int G, int NCH>
-bitrl_status launch_attention_t(const AttArgs& a, int n_states, cudaStream_t st) {
-  constexpr int SMAX = NCH * 32;
-  const size_t smem = sizeof(float) * (static_cast<size_t>(SMAX) * (HD + 4) + static_cast<size_t>(SMAX) * HD +
-                                       static_cast<size_t>(ATT_WARPS) * G * HD + static_cast<size_t>(ATT_WARPS) * SMAX * G);
-  static bool attr_set[64] = {false};
-  int dev = 0;
-  BITRL_CUDA(cudaGetDevice(&dev));
-  if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-    BITRL_CUDA(cudaFuncSetAttribute(attention_kernel<HD, G, NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    static_cast<int>(smem)));
-    attr_set[dev] = true;
-  }
-  BITRL_CUDA(launch_pdl(attention_kernel<HD, G, NCH>, dim3(static_cast<unsigned>(n_states) * a.n_kv), dim3(ATT_THREADS),
-                        smem, st, a));
-  count_launch(1);
-  return BITRL_OK;
-}
-
-template <int HD, int G>
-bitrl_status launch_attention_g(const AttArgs& a, int n_states, cudaStream_t st) {
-  if (a.state_len <= 32) return launch_attention_t<HD, G, 1>(a, n_states, st);
-  if (a.state_len <= 64) return launch_attention_t<HD, G, 2>(a, n_states, st);
-  return launch_attention_t<HD, G, 4>(a, n_states, st);
-}
-
-template <int HD>
-bitrl_status launch_attention_hd(const AttArgs& a, int n_states, cudaStream_t st) {
-  const int rep = a.n_heads / a.n_kv;
-  if (rep % 4 == 0) return launch_attention_g<HD, 4>(a, n_states, st);
-  if (rep % 2 == 0) return launch_attention_g<HD, 2>(a, n_states, st);
-  return launch_attention_g<HD, 1>(a, n_states, st);
 }
 
 inline size_t rope_table_bytes(int max_state_len, int hd) {
