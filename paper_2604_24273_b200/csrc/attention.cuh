@@ -74,8 +74,7 @@ __global__ void rope_table_kernel(float2* tab, int max_len, int hd, double theta
 // every fp32 operand x is split into two halves x = hi + lo (hi = f16(x), lo = f16(x - hi): 22 significant bits) and
 // the product a*b is formed as hi*hi + hi*lo + lo*hi (the dropped lo*lo term is below 2^-22 relative).  Values are
 // bf16 numbers and convert to f16 exactly (down to 6e-5 in magnitude, 3e-8 absolute below); softmax weights are split.
-// A warp owns one (query head, 16-token tile): Q fragments are read straight from global memory (the rotary partner
-// of a dimension sits in the same lane four k-steps later), K/V fragments come from shared memory through ldmatrix.
+// A warp owns one (query head, 16-token tile); all fragments come from shared memory through ldmatrix.
 constexpr int ATC_PAD = 8;  // halves added to each shared-memory row: consecutive rows start in different bank groups
 
 __device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
@@ -99,8 +98,42 @@ __device__ __forceinline__ void split_f16x2(float x0, float x1, uint32_t& hi, ui
   lo = static_cast<uint32_t>(__half_as_ushort(l0)) | (static_cast<uint32_t>(__half_as_ushort(l1)) << 16);
 }
 
+// Eight consecutive dimensions of the first half of a head row (x1) and their eight rotary partners (x2), rotated with
+// cs = (cos, sin) of those eight dimensions, split, and stored as f16 high/low rows at columns c0 and c1.
+__device__ __forceinline__ void rope_split_store8(const uint4& x1, const uint4& x2, const float4 (&cs)[4], __half* hi_row,
+                                                  __half* lo_row, int c0, int c1) {
+  const uint32_t w1[4] = {x1.x, x1.y, x1.z, x1.w}, w2[4] = {x2.x, x2.y, x2.z, x2.w};
+  uint32_t h1[4], l1[4], h2[4], l2[4];
+#pragma unroll
+  for (int w = 0; w < 4; ++w) {
+    const float x1a = __uint_as_float(w1[w] << 16), x1b = __uint_as_float(w1[w] & 0xffff0000u);
+    const float x2a = __uint_as_float(w2[w] << 16), x2b = __uint_as_float(w2[w] & 0xffff0000u);
+    split_f16x2(fmaf(-x2a, cs[w].y, __fmul_rn(x1a, cs[w].x)), fmaf(-x2b, cs[w].w, __fmul_rn(x1b, cs[w].z)), h1[w], l1[w]);
+    split_f16x2(fmaf(x1a, cs[w].y, __fmul_rn(x2a, cs[w].x)), fmaf(x1b, cs[w].w, __fmul_rn(x2b, cs[w].z)), h2[w], l2[w]);
+  }
+  *reinterpret_cast<uint4*>(hi_row + c0) = make_uint4(h1[0], h1[1], h1[2], h1[3]);
+  *reinterpret_cast<uint4*>(lo_row + c0) = make_uint4(l1[0], l1[1], l1[2], l1[3]);
+  *reinterpret_cast<uint4*>(hi_row + c1) = make_uint4(h2[0], h2[1], h2[2], h2[3]);
+  *reinterpret_cast<uint4*>(lo_row + c1) = make_uint4(l2[0], l2[1], l2[2], l2[3]);
+}
+// Eight bf16 values -> eight f16 values (exact for the magnitudes of activations).
+__device__ __forceinline__ uint4 bf16x8_to_f16x8(const uint4& x) {
+  const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+  uint32_t o[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const __half a = __float2half_rn(__uint_as_float(w[i] << 16)), b = __float2half_rn(__uint_as_float(w[i] & 0xffff0000u));
+    o[i] = static_cast<uint32_t>(__half_as_ushort(a)) | (static_cast<uint32_t>(__half_as_ushort(b)) << 16);
+  }
+  return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 // NKT = 8-key tiles held per query tile (keys padded to 8 * NKT, a multiple of 16).
-template <int HD, int NKT>
+// STAGED: the rotated, split queries of all heads of the kv group are staged in shared memory by the same cooperative
+// pass that stages keys and values (every global load of the CTA is a 16-byte load issued up front, one memory
+// latency for the whole CTA); otherwise (long states or many heads per kv head, which would not fit) each warp builds
+// the query fragments of its task from global memory.
+template <int HD, int NKT, bool STAGED>
 __global__ void __launch_bounds__(ATT_THREADS, NKT <= 4 ? 2 : 1) attention_tc_kernel(AttArgs a) {
   constexpr int KS = HD / 16;            // k-steps of the score product
   constexpr int ND = HD / 8;             // 8-wide output tiles
@@ -110,6 +143,7 @@ __global__ void __launch_bounds__(ATT_THREADS, NKT <= 4 ? 2 : 1) attention_tc_ke
   __half* Khi = reinterpret_cast<__half*>(atc_smem);  // [SP][RS]
   __half* Klo = Khi + SP * RS;
   __half* Vh = Klo + SP * RS;
+  __half* Qhi = Vh + SP * RS;  // STAGED: [rep * SP][RS], then Qlo the same
 
   pdl_enter();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -120,40 +154,54 @@ __global__ void __launch_bounds__(ATT_THREADS, NKT <= 4 ? 2 : 1) attention_tc_ke
   const int rep = a.n_heads / a.n_kv;
   const int d = a.n_heads * HD, dkv = a.n_kv * HD, W = d + 2 * dkv;
 
-  // ---- keys (rotated, split) and values of this state into shared memory; rows S..SP-1 are zero ----
-#pragma unroll 4
-  for (int r = warp; r < SP; r += ATT_WARPS) {
-    __half* kh = Khi + r * RS;
-    __half* kl = Klo + r * RS;
-    __half* vh = Vh + r * RS;
-    if (r < S) {
-      const unsigned short* krow = a.qkv + static_cast<long long>(t0 + r) * W + d + kvh * HD;
-      const float2* tab = a.rope + r * (HD / 2);
-      for (int i = 2 * lane; i < HD / 2; i += 64) {  // dims i, i+1 and their partners i + HD/2, i + 1 + HD/2
-        const uint32_t r1 = *reinterpret_cast<const uint32_t*>(krow + i);
-        const uint32_t r2 = *reinterpret_cast<const uint32_t*>(krow + i + HD / 2);
-        const float4 cs = *reinterpret_cast<const float4*>(tab + i);  // (cos_i, sin_i, cos_i+1, sin_i+1)
-        const float x1a = __uint_as_float(r1 << 16), x1b = __uint_as_float(r1 & 0xffff0000u);
-        const float x2a = __uint_as_float(r2 << 16), x2b = __uint_as_float(r2 & 0xffff0000u);
-        uint32_t hi, lo;
-        split_f16x2(fmaf(-x2a, cs.y, __fmul_rn(x1a, cs.x)), fmaf(-x2b, cs.w, __fmul_rn(x1b, cs.z)), hi, lo);
-        *reinterpret_cast<uint32_t*>(kh + i) = hi;
-        *reinterpret_cast<uint32_t*>(kl + i) = lo;
-        split_f16x2(fmaf(x1a, cs.y, __fmul_rn(x2a, cs.x)), fmaf(x1b, cs.w, __fmul_rn(x2b, cs.z)), hi, lo);
-        *reinterpret_cast<uint32_t*>(kh + i + HD / 2) = hi;
-        *reinterpret_cast<uint32_t*>(kl + i + HD / 2) = lo;
-      }
-      for (int i = 2 * lane; i < HD; i += 64) {
-        const uint32_t rv = *reinterpret_cast<const uint32_t*>(krow + dkv + i);
-        const __half v0 = __float2half_rn(__uint_as_float(rv << 16)), v1 = __float2half_rn(__uint_as_float(rv & 0xffff0000u));
-        *reinterpret_cast<uint32_t*>(vh + i) =
-            static_cast<uint32_t>(__half_as_ushort(v0)) | (static_cast<uint32_t>(__half_as_ushort(v1)) << 16);
-      }
-    } else {
-      for (int i = 2 * lane; i < HD; i += 64) {
-        *reinterpret_cast<uint32_t*>(kh + i) = 0u;
-        *reinterpret_cast<uint32_t*>(kl + i) = 0u;
-        *reinterpret_cast<uint32_t*>(vh + i) = 0u;
+  __half* Qlo = Qhi + rep * SP * RS;
+  // ---- keys (rotated, split), values and (STAGED) queries of this state into shared memory; rows S..SP-1 are zero.
+  // A thread owns eight dimensions of the first half of a row together with their eight rotary partners.
+  {
+    constexpr int CPR = HD / 16;  // such chunk pairs per row
+    const int frow = threadIdx.x / CPR, cp = threadIdx.x % CPR;
+    const int c0 = 8 * cp, c1 = HD / 2 + 8 * cp;
+    for (int r = frow; r < SP; r += ATT_THREADS / CPR) {
+      if (r < S) {
+        const unsigned short* row = a.qkv + static_cast<long long>(t0 + r) * W;
+        const unsigned short* krow = row + d + kvh * HD;
+        const float4* tab = reinterpret_cast<const float4*>(a.rope + r * (HD / 2) + c0);
+        const float4 cs[4] = {tab[0], tab[1], tab[2], tab[3]};
+        const uint4 k1 = *reinterpret_cast<const uint4*>(krow + c0), k2 = *reinterpret_cast<const uint4*>(krow + c1);
+        const uint4 v1 = *reinterpret_cast<const uint4*>(krow + dkv + c0), v2 = *reinterpret_cast<const uint4*>(krow + dkv + c1);
+        if constexpr (STAGED) {
+          for (int j0 = 0; j0 < rep; j0 += 4) {
+            uint4 q1[4], q2[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              if (j0 + i < rep) {
+                const unsigned short* qrow = row + (kvh * rep + j0 + i) * HD;
+                q1[i] = *reinterpret_cast<const uint4*>(qrow + c0);
+                q2[i] = *reinterpret_cast<const uint4*>(qrow + c1);
+              }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              if (j0 + i < rep)
+                rope_split_store8(q1[i], q2[i], cs, Qhi + ((j0 + i) * SP + r) * RS, Qlo + ((j0 + i) * SP + r) * RS, c0, c1);
+          }
+        }
+        rope_split_store8(k1, k2, cs, Khi + r * RS, Klo + r * RS, c0, c1);
+        *reinterpret_cast<uint4*>(Vh + r * RS + c0) = bf16x8_to_f16x8(v1);
+        *reinterpret_cast<uint4*>(Vh + r * RS + c1) = bf16x8_to_f16x8(v2);
+      } else {
+        const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int c = h ? c1 : c0;
+          *reinterpret_cast<uint4*>(Khi + r * RS + c) = z;
+          *reinterpret_cast<uint4*>(Klo + r * RS + c) = z;
+          *reinterpret_cast<uint4*>(Vh + r * RS + c) = z;
+          if constexpr (STAGED)
+            for (int j = 0; j < rep; ++j) {
+              *reinterpret_cast<uint4*>(Qhi + (j * SP + r) * RS + c) = z;
+              *reinterpret_cast<uint4*>(Qlo + (j * SP + r) * RS + c) = z;
+            }
+        }
       }
     }
   }
@@ -162,6 +210,7 @@ __global__ void __launch_bounds__(ATT_THREADS, NKT <= 4 ? 2 : 1) attention_tc_ke
   const int g = lane >> 2, t = lane & 3;
   const float inv_sqrt = __fdiv_rn(1.0f, __fsqrt_rn(static_cast<float>(HD)));
   const uint32_t khi_s = ptx_smem_u32(Khi), klo_s = ptx_smem_u32(Klo), vh_s = ptx_smem_u32(Vh);
+  const uint32_t qhi_s = ptx_smem_u32(Qhi), qlo_s = ptx_smem_u32(Qlo);
   // ldmatrix row address of this lane: matrix lane/8, row lane%8
   const int lm = lane >> 3, lr = lane & 7;
   const int m_tiles = (S + 15) >> 4;
@@ -172,33 +221,38 @@ __global__ void __launch_bounds__(ATT_THREADS, NKT <= 4 ? 2 : 1) attention_tc_ke
     const int p_lo = 16 * mt + g, p_hi = p_lo + 8;
     const int nkt = min(NKT, 2 * mt + 2);  // key tiles under the causal limit of this query tile
 
-    // ---- Q fragments: rows g and g+8 of the tile, rotated and split ----
-    uint32_t qh[KS][4], ql[KS][4];
+    // ---- Q fragments of the tile (rows g and g+8 per lane), rotated and split ----
+    uint32_t qh[STAGED ? 2 : KS][4], ql[STAGED ? 2 : KS][4];
+    if constexpr (!STAGED) {
+      // straight from global memory: the rotary partner of a dimension sits in the same lane KS/2 k-steps later
 #pragma unroll
-    for (int rr = 0; rr < 2; ++rr) {
-      const int p = rr ? p_hi : p_lo;
-      const bool live = p < S;
-      const unsigned short* qrow = a.qkv + static_cast<long long>(t0 + (live ? p : 0)) * W + head * HD;
-      const float2* tab = a.rope + (live ? p : 0) * (HD / 2);
+      for (int rr = 0; rr < 2; ++rr) {
+        const int p = rr ? p_hi : p_lo;
+        const bool live = p < S;
+        const unsigned short* qrow = a.qkv + static_cast<long long>(t0 + (live ? p : 0)) * W + head * HD;
+        const float2* tab = a.rope + (live ? p : 0) * (HD / 2);
 #pragma unroll
-      for (int ks = 0; ks < KS / 2; ++ks)
+        for (int ks = 0; ks < KS / 2; ++ks)
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          const int dim = 16 * ks + 8 * hf + 2 * t;  // dims dim, dim+1 (first half of the head) and their partners
-          uint32_t r1 = 0u, r2 = 0u;
-          if (live) {
-            r1 = *reinterpret_cast<const uint32_t*>(qrow + dim);
-            r2 = *reinterpret_cast<const uint32_t*>(qrow + dim + HD / 2);
+          for (int hf = 0; hf < 2; ++hf) {
+            const int dim = 16 * ks + 8 * hf + 2 * t;  // dims dim, dim+1 (first half of the head) and their partners
+            uint32_t r1 = 0u, r2 = 0u;
+            if (live) {
+              r1 = *reinterpret_cast<const uint32_t*>(qrow + dim);
+              r2 = *reinterpret_cast<const uint32_t*>(qrow + dim + HD / 2);
+            }
+            const float4 cs = *reinterpret_cast<const float4*>(tab + dim);
+            const float x1a = __uint_as_float(r1 << 16), x1b = __uint_as_float(r1 & 0xffff0000u);
+            const float x2a = __uint_as_float(r2 << 16), x2b = __uint_as_float(r2 & 0xffff0000u);
+            split_f16x2(fmaf(-x2a, cs.y, __fmul_rn(x1a, cs.x)), fmaf(-x2b, cs.w, __fmul_rn(x1b, cs.z)),
+                        qh[ks][2 * hf + rr], ql[ks][2 * hf + rr]);
+            split_f16x2(fmaf(x1a, cs.y, __fmul_rn(x2a, cs.x)), fmaf(x1b, cs.w, __fmul_rn(x2b, cs.z)),
+                        qh[ks + KS / 2][2 * hf + rr], ql[ks + KS / 2][2 * hf + rr]);
           }
-          const float4 cs = *reinterpret_cast<const float4*>(tab + dim);
-          const float x1a = __uint_as_float(r1 << 16), x1b = __uint_as_float(r1 & 0xffff0000u);
-          const float x2a = __uint_as_float(r2 << 16), x2b = __uint_as_float(r2 & 0xffff0000u);
-          split_f16x2(fmaf(-x2a, cs.y, __fmul_rn(x1a, cs.x)), fmaf(-x2b, cs.w, __fmul_rn(x1b, cs.z)),
-                      qh[ks][2 * hf + rr], ql[ks][2 * hf + rr]);
-          split_f16x2(fmaf(x1a, cs.y, __fmul_rn(x2a, cs.x)), fmaf(x1b, cs.w, __fmul_rn(x2b, cs.z)),
-                      qh[ks + KS / 2][2 * hf + rr], ql[ks + KS / 2][2 * hf + rr]);
-        }
+      }
     }
+    // STAGED: fragments come from shared memory, two k-steps at a time (matrix lm: rows 8 (lm & 1).., columns 8 (lm >> 1)..)
+    const uint32_t q_off = static_cast<uint32_t>(((j * SP + 16 * mt + 8 * (lm & 1) + lr) * RS + 8 * (lm >> 1)) * 2);
 
     // ---- scores: c[nt] = Q K^T for key tile nt (rows g / g+8, keys 8nt+2t, +1) ----
     // Consecutive tensor instructions go to different accumulators (four key tiles, and the terms that involve a low
@@ -213,6 +267,13 @@ __global__ void __launch_bounds__(ATT_THREADS, NKT <= 4 ? 2 : 1) attention_tc_ke
       if (n0 < nkt) {
 #pragma unroll
         for (int ks = 0; ks < KS; ks += 2) {
+          const int k0 = STAGED ? 0 : ks, k1 = STAGED ? 1 : ks + 1;  // where this pair of k-steps sits in qh / ql
+          if constexpr (STAGED) {
+            ldmatrix_x4(qhi_s + q_off + 32 * ks, qh[0]);
+            ldmatrix_x4(qlo_s + q_off + 32 * ks, ql[0]);
+            ldmatrix_x4(qhi_s + q_off + 32 * ks + 32, qh[1]);
+            ldmatrix_x4(qlo_s + q_off + 32 * ks + 32, ql[1]);
+          }
           uint32_t bh[4][4], bl[4][4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
@@ -222,17 +283,17 @@ __global__ void __launch_bounds__(ATT_THREADS, NKT <= 4 ? 2 : 1) attention_tc_ke
             ldmatrix_x4(klo_s + off, bl[i]);
           }
 #pragma unroll
-          for (int i = 0; i < 4; ++i) mma_f16(c[n0 + i], qh[ks], bh[i][0], bh[i][1]);
+          for (int i = 0; i < 4; ++i) mma_f16(c[n0 + i], qh[k0], bh[i][0], bh[i][1]);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) mma_f16(c2[n0 + i], qh[ks], bl[i][0], bl[i][1]);
+          for (int i = 0; i < 4; ++i) mma_f16(c2[n0 + i], qh[k0], bl[i][0], bl[i][1]);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) mma_f16(c[n0 + i], qh[ks + 1], bh[i][2], bh[i][3]);
+          for (int i = 0; i < 4; ++i) mma_f16(c[n0 + i], qh[k1], bh[i][2], bh[i][3]);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) mma_f16(c2[n0 + i], ql[ks], bh[i][0], bh[i][1]);
+          for (int i = 0; i < 4; ++i) mma_f16(c2[n0 + i], ql[k0], bh[i][0], bh[i][1]);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) mma_f16(c2[n0 + i], qh[ks + 1], bl[i][2], bl[i][3]);
+          for (int i = 0; i < 4; ++i) mma_f16(c2[n0 + i], qh[k1], bl[i][2], bl[i][3]);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) mma_f16(c2[n0 + i], ql[ks + 1], bh[i][2], bh[i][3]);
+          for (int i = 0; i < 4; ++i) mma_f16(c2[n0 + i], ql[k1], bh[i][2], bh[i][3]);
         }
       }
     }
@@ -315,28 +376,33 @@ __global__ void __launch_bounds__(ATT_THREADS, NKT <= 4 ? 2 : 1) attention_tc_ke
   }
 }
 
-template <int HD, int NKT>
+template <int HD, int NKT, bool STAGED>
 bitrl_status launch_attention_tc_t(const AttArgs& a, int n_states, cudaStream_t st) {
-  const size_t smem = static_cast<size_t>(3) * (NKT * 8) * (HD + ATC_PAD) * sizeof(__half);
-  static bool attr_set[64] = {false};
+  const int rep = a.n_heads / a.n_kv;
+  const size_t row_bytes = (HD + ATC_PAD) * sizeof(__half);
+  const size_t smem = static_cast<size_t>(3 + (STAGED ? 2 * rep : 0)) * (NKT * 8) * row_bytes;
+  static size_t attr_set[64] = {0};
   int dev = 0;
   BITRL_CUDA(cudaGetDevice(&dev));
-  if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-    BITRL_CUDA(cudaFuncSetAttribute(attention_tc_kernel<HD, NKT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if (dev >= 0 && dev < 64 && attr_set[dev] < smem) {
+    BITRL_CUDA(cudaFuncSetAttribute(attention_tc_kernel<HD, NKT, STAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     static_cast<int>(smem)));
-    attr_set[dev] = true;
+    attr_set[dev] = smem;
   }
-  BITRL_CUDA(launch_pdl(attention_tc_kernel<HD, NKT>, dim3(static_cast<unsigned>(n_states) * a.n_kv), dim3(ATT_THREADS),
-                        smem, st, a));
+  BITRL_CUDA(launch_pdl(attention_tc_kernel<HD, NKT, STAGED>, dim3(static_cast<unsigned>(n_states) * a.n_kv),
+                        dim3(ATT_THREADS), smem, st, a));
   count_launch(1);
   return BITRL_OK;
 }
 
 template <int HD>
 bitrl_status launch_attention_tc_hd(const AttArgs& a, int n_states, cudaStream_t st) {
-  if (a.state_len <= 32) return launch_attention_tc_t<HD, 4>(a, n_states, st);
-  if (a.state_len <= 64) return launch_attention_tc_t<HD, 8>(a, n_states, st);
-  return launch_attention_tc_t<HD, 16>(a, n_states, st);
+  // queries are staged in shared memory while (3 + 2 * heads per kv head) * padded keys rows fit beside the rest
+  const int rep = a.n_heads / a.n_kv;
+  const auto fits = [&](int sp) { return static_cast<size_t>(3 + 2 * rep) * sp * (HD + ATC_PAD) * sizeof(__half) <= 200 * 1024; };
+  if (a.state_len <= 32) return fits(32) ? launch_attention_tc_t<HD, 4, true>(a, n_states, st) : launch_attention_tc_t<HD, 4, false>(a, n_states, st);
+  if (a.state_len <= 64) return fits(64) ? launch_attention_tc_t<HD, 8, true>(a, n_states, st) : launch_attention_tc_t<HD, 8, false>(a, n_states, st);
+  return launch_attention_tc_t<HD, 16, false>(a, n_states, st);
 }
 
 inline size_t rope_table_bytes(int max_state_len, int hd) {
