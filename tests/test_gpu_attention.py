@@ -1,13 +1,14 @@
 """GPU parity of the attention step, last-token pooling and the encoder with real attention, through the C ABI,
 against the CPU oracle on the same seeded inputs.
 
-The oracle computes attention in fp64 and rounds once to bf16; the kernel computes in fp32 and rounds once.  An
-output is a convex combination of the values v_r of its column, so the fp32 path carries an absolute error of a few
-fp32 ulps of max_r |v_r| (64-128 fused multiply-adds per dot product, up to 128 keys): tolerance 4e-6 * max|v| of
-the column.  Outputs that are not tiny therefore agree to the bf16 bit, or differ in the last bit when that error
-crosses a rounding boundary (required: at most 0.5 % of the elements); outputs near zero (cancellation) may differ
-by more bf16 ulps but still lie within the absolute bound.  The integer stages that follow are checked by teacher
-forcing on the GPU's own bf16 values, bit-exactly.
+The oracle computes attention in fp64 and rounds once to bf16.  The kernel rotates in fp32, forms both contractions
+on tensor instructions whose operands are split into two f16 halves (22 significant bits, products exact, fp32
+accumulation) and rounds once.  An output is a convex combination of the values v_r of its column, so this path
+carries an absolute error of a few 2^-22 of max_r |v_r| (64-128 terms per dot product, up to 128 keys): tolerance
+4e-6 * max|v| of the column (measured: below 1e-6).  Outputs that are not tiny therefore agree to the bf16 bit, or
+differ in the last bit when that error crosses a rounding boundary (required: at most 0.5 % of the elements; measured:
+0.05 %); outputs near zero (cancellation) may differ by more bf16 ulps but still lie within the absolute bound.  The
+integer stages that follow are checked by teacher forcing on the GPU's own bf16 values, bit-exactly.
 """
 import numpy as np
 import pytest

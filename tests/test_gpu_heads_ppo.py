@@ -86,3 +86,26 @@ def test_ppo_loss(oracle_mod, B, nB, A):
     np.testing.assert_allclose(f64(out["dvalues"]), want["dvalues"], rtol=1e-6, atol=1e-9)
     # the gradient of a sample sitting exactly on the clip boundary is one-sided; none of the seeded samples does
     np.testing.assert_allclose(f64(out["dlogits"]), want["dlogits"], rtol=2e-5, atol=1e-6 / nB)
+
+
+def test_gae_and_ppo_argument_errors(oracle_mod, B):
+    L = B.lib()
+    r, v, d = (t.cuda() for t in inputs.rollout(4, 3, 1))
+    adv = torch.empty_like(r)
+    assert L.bitrl_gae(r.data_ptr(), v.data_ptr(), d.data_ptr(), 0, 3, 0.99, 0.95, adv.data_ptr(), None, None) == B.ERR_SHAPE
+    assert L.bitrl_gae(None, v.data_ptr(), d.data_ptr(), 4, 3, 0.99, 0.95, adv.data_ptr(), None, None) == B.ERR_NULL
+    assert L.bitrl_gae(r.data_ptr(), v.data_ptr(), d.data_ptr(), 4, 3, 0.99, 0.95, adv.data_ptr(), None, None) == B.OK
+    B.poll_status()
+    want, _ = oracle_mod.gae(f64(r), f64(v), f64(d), 0.99, 0.95)  # returns pointer omitted: advantages only
+    np.testing.assert_allclose(f64(adv), want, rtol=1e-5, atol=1e-5)
+    logits, actions, old_logp, a_hat, val, R = (t.cuda() for t in inputs.ppo_batch(5, 4, 2))
+    terms = torch.empty((5, 4), dtype=torch.float32, device="cuda")
+    summ = torch.empty((4,), dtype=torch.float32, device="cuda")
+    args = [logits.data_ptr(), actions.data_ptr(), old_logp.data_ptr(), a_hat.data_ptr(), val.data_ptr(), R.data_ptr()]
+    assert L.bitrl_ppo_loss(*args, 0, 4, 0.1, 0.05, terms.data_ptr(), None, None, summ.data_ptr(), None) == B.ERR_SHAPE
+    assert L.bitrl_ppo_loss(*args, 5, 4, 0.1, 0.05, None, None, None, summ.data_ptr(), None) == B.ERR_NULL
+    assert L.bitrl_ppo_loss(*args, 5, 4, 0.1, 0.05, terms.data_ptr(), None, None, summ.data_ptr(), None) == B.OK  # no gradients asked
+    B.poll_status()
+    want = oracle_mod.ppo_loss(f64(logits), actions.cpu().numpy(), f64(old_logp), f64(a_hat), f64(val), f64(R), 0.1, 0.05)
+    np.testing.assert_allclose(f64(summ), [want["l_clip"], want["entropy"], want["policy_loss"], want["value_loss"]],
+                               rtol=1e-5, atol=1e-6)
