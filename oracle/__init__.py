@@ -51,6 +51,8 @@ def _L():
         _lib.oracle_absmean.restype = _f32
         _lib.oracle_absmean.argtypes = [_vp, _i64]
         _lib.oracle_ternarize.argtypes = [_vp, _i64, _f32, _vp]
+        _lib.oracle_w8_quantize.argtypes = [_vp, _i64, _vp, _vp]
+        _lib.oracle_w8_quantize.restype = None
         _lib.oracle_pack.argtypes = [_vp, _i64, _i64, _vp]
         _lib.oracle_unpack.argtypes = [_vp, _i64, _i64, _vp]
         _lib.oracle_quant_act.argtypes = [_vp, _i64, _i64, _vp, _vp]
@@ -107,6 +109,16 @@ def ternarize(W: np.ndarray, gamma=None):
     Wq = np.empty(W.shape, np.int8)
     _L().oracle_ternarize(_p(W), W.size, _f32(float(g)), _p(Wq))
     return Wq, g
+
+
+def w8_quantize(W: np.ndarray):
+    """Symmetric absmax int8 quantization of a weight matrix (one scale per matrix).  Returns (W_q int8, scale fp32);
+    ``bitlinear(x, W_q, scale)`` is then the W8A8 layer of the higher-precision critic."""
+    W = _c(W, np.float32)
+    Wq = np.empty(W.shape, np.int8)
+    scale = np.zeros((1,), np.float32)
+    _L().oracle_w8_quantize(_p(W), W.size, _p(Wq), _p(scale))
+    return Wq, np.float32(scale[0])
 
 
 def pack(Wq: np.ndarray) -> np.ndarray:

@@ -139,7 +139,29 @@ void oracle_quant_act(const uint16_t* x, int64_t M, int64_t K, int8_t* xq, float
   }
 }
 
-// acc[m,n] = sum_k x_q[m,k] * W_q[n,k] in int32 (exact; |acc| <= 127*K).
+// Eight-bit weights for the higher-precision critic backbone (Sec. V ablations, Table IV: "INT8 critic + 1-bit
+// policy"; the paper names the precision only).  Reading: one symmetric absmax scale per matrix, the same rounding as
+// the activations:  a = max(max|W|, 1e-20),  W_q = clip(rint(W * (127 / a)), -128, 127),  scale = a / 127.
+// The layer then is the BitLinear formula with W_q in place of the ternary codes and `scale` in place of gamma:
+//   acc = sum_k x_q W_q (int32, |acc| <= 127*128*K),  y = (float)acc * (scale * (a_m / 127)).
+void oracle_w8_quantize(const float* W, int64_t count, int8_t* Wq, float* scale) {
+  float a = 0.0f;
+  for (int64_t i = 0; i < count; ++i) {
+    const float v = std::fabs(W[i]);
+    if (v > a) a = v;
+  }
+  if (a < 1e-20f) a = 1e-20f;
+  const float inv = 127.0f / a;
+  for (int64_t i = 0; i < count; ++i) {
+    float q = std::nearbyintf(W[i] * inv);
+    if (q > 127.0f) q = 127.0f;
+    if (q < -128.0f) q = -128.0f;
+    Wq[i] = static_cast<int8_t>(q);
+  }
+  *scale = a / 127.0f;
+}
+
+// acc[m,n] = sum_k x_q[m,k] * W_q[n,k] in int32 (exact; |acc| <= 127*K for ternary, 127*128*K for 8-bit weights).
 void oracle_contract(const int8_t* xq, const int8_t* Wq, int64_t M, int64_t N, int64_t K, int32_t* acc,
                      int threads) {
   parallel_rows(M, threads, [=](int64_t m) {
