@@ -232,6 +232,28 @@ BITRL_API bitrl_status bitrl_ppo_loss(const float* logits, const int32_t* action
                                       float eps, float beta, float* terms, float* dlogits, float* dvalues,
                                       float* summary, void* stream);
 
+/* ---- W8A8 layer: the higher-precision critic backbone (Sec. V ablations, Table IV: "INT8 critic + 1-bit policy";
+ * the paper names the precision only) -------------------------------------------------------------------------
+ * One symmetric absmax scale per matrix, rounding as for the activations:
+ *   a = max(max|W|, 1e-20),  W_q = clip(rint(W * (127 / a)), -128, 127),  scale = a / 127
+ *   acc[m,n] = sum_k x_q[m,k] * W_q[n,k] (int32),  y[m,n] = (float)acc[m,n] * (scale * (a_m / 127))
+ * with x_q, a_m exactly as in bitrl_quant_act.  |acc| can exceed 2^24, so (float)acc is the int32 -> fp32 conversion
+ * with round-to-nearest-even.
+ * bitrl_w8_quantize: W dev fp32 [N,K] -> wq dev int8 [N,K] (row-major, the format the forward call reads) and
+ * scale: dev fp32 [2] - scale[0] receives the scale, scale[1] is scratch of the call.
+ * bitrl_w8a8_forward: x dev bf16 [M,K], y dev [M,N] fp32 or bf16; any M >= 1 runs the tcgen05 GEMM (both operands
+ * straight from TMA tiles).  workspace: dev, >= bitrl_w8a8_workspace_bytes(M, K) (the quantized activations).
+ * The _debug variant also writes xq_out dev int8 [M,K], absmax_out dev fp32 [M], acc_out dev int32 [M,N] (any may be NULL). */
+BITRL_API bitrl_status bitrl_w8_quantize(const float* W, int32_t N, int32_t K, int8_t* wq, float* scale, void* stream);
+BITRL_API size_t bitrl_w8a8_workspace_bytes(int32_t M, int32_t K);
+BITRL_API bitrl_status bitrl_w8a8_forward(const int8_t* wq, const float* scale, const void* x, int32_t M, int32_t K,
+                                          int32_t N, void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes,
+                                          void* stream);
+BITRL_API bitrl_status bitrl_w8a8_forward_debug(const int8_t* wq, const float* scale, const void* x, int32_t M, int32_t K,
+                                                int32_t N, void* y, int32_t out_dtype, void* workspace,
+                                                size_t workspace_bytes, int8_t* xq_out, float* absmax_out,
+                                                int32_t* acc_out, void* stream);
+
 /* ---- status ----------------------------------------------------------------------------------------- */
 /* Synchronizes `stream`, then reads and clears the device status word.  BITRL_OK, BITRL_ERR_TIMEOUT (a kernel
  * wait expired; results of that launch are invalid) or BITRL_ERR_CUDA. */

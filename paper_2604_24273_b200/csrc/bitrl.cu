@@ -75,6 +75,7 @@ static bitrl_status check_arch() {
 #include "gemm.cuh"
 #include "attention.cuh"
 #include "heads.cuh"
+#include "gemm_w8.cuh"
 
 using namespace bitrl;
 
@@ -581,6 +582,53 @@ bitrl_status bitrl_ppo_loss(const float* logits, const int32_t* actions, const f
   BITRL_CUDA(launch_pdl(ppo_summary_kernel, dim3(1), dim3(256), 0, st, static_cast<const float*>(terms), B, beta, summary));
   count_launch(2);
   return BITRL_OK;
+}
+
+// ---- W8A8 layer of the higher-precision critic ----------------------------------------------------------------
+
+bitrl_status bitrl_w8_quantize(const float* W, int32_t N, int32_t K, int8_t* wq, float* scale, void* stream) {
+  if (!W || !wq || !scale) return BITRL_ERR_NULL;
+  if (!shape_ok(N, K)) return BITRL_ERR_SHAPE;
+  if (!aligned16(W) || !aligned16(wq)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  return launch_w8_quantize(W, N, K, wq, scale, static_cast<cudaStream_t>(stream));
+}
+
+size_t bitrl_w8a8_workspace_bytes(int32_t M, int32_t K) {
+  if (M < 1 || K < 1) return 0;
+  return align_up(static_cast<size_t>(M) * K, 256) + align_up(static_cast<size_t>(M) * 4, 256);
+}
+
+static bitrl_status w8a8_impl(const int8_t* wq, const float* scale, const void* x, int32_t M, int32_t K, int32_t N, void* y,
+                              int32_t out_dtype, void* workspace, size_t workspace_bytes, int8_t* xq_out,
+                              float* absmax_out, int32_t* acc_out, void* stream) {
+  if (!wq || !scale || !x || !y) return BITRL_ERR_NULL;
+  if (M < 1 || !shape_ok(N, K)) return BITRL_ERR_SHAPE;
+  if (out_dtype != BITRL_OUT_F32 && out_dtype != BITRL_OUT_BF16) return BITRL_ERR_DTYPE;
+  if (!workspace || workspace_bytes < bitrl_w8a8_workspace_bytes(M, K)) return BITRL_ERR_WORKSPACE;
+  if (!aligned16(wq) || !aligned16(x) || !aligned16(y) || !aligned16(workspace)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int8_t* xq = static_cast<int8_t*>(workspace);
+  float* absmax = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + align_up(static_cast<size_t>(M) * K, 256));
+  if ((s = launch_quant_act(x, M, K, xq, absmax, nullptr, st)) != BITRL_OK) return s;
+  if ((s = launch_gemm_w8(wq, scale, N, K, xq, absmax, M, y, out_dtype, nullptr, acc_out, st)) != BITRL_OK) return s;
+  if (xq_out) BITRL_CUDA(cudaMemcpyAsync(xq_out, xq, static_cast<size_t>(M) * K, cudaMemcpyDeviceToDevice, st));
+  if (absmax_out) BITRL_CUDA(cudaMemcpyAsync(absmax_out, absmax, static_cast<size_t>(M) * 4, cudaMemcpyDeviceToDevice, st));
+  return BITRL_OK;
+}
+
+bitrl_status bitrl_w8a8_forward(const int8_t* wq, const float* scale, const void* x, int32_t M, int32_t K, int32_t N,
+                                void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes, void* stream) {
+  return w8a8_impl(wq, scale, x, M, K, N, y, out_dtype, workspace, workspace_bytes, nullptr, nullptr, nullptr, stream);
+}
+
+bitrl_status bitrl_w8a8_forward_debug(const int8_t* wq, const float* scale, const void* x, int32_t M, int32_t K, int32_t N,
+                                      void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes, int8_t* xq_out,
+                                      float* absmax_out, int32_t* acc_out, void* stream) {
+  return w8a8_impl(wq, scale, x, M, K, N, y, out_dtype, workspace, workspace_bytes, xq_out, absmax_out, acc_out, stream);
 }
 
 // ---- self-test of the bounded-wait / status-word path ----

@@ -1,0 +1,329 @@
+// W8A8 layer for the higher-precision critic backbone (Sec. V ablations, Table IV: "INT8 critic + 1-bit policy"):
+// the same int8 activation quantization and int32 contraction as the ternary layer, with int8 weights (one symmetric
+// absmax scale per matrix).  There is nothing to decode, so both operands of tcgen05.mma kind::i8 come straight from
+// TMA tiles in shared memory: D[n, m] = sum_k W_q[n,k] * x_q[m,k], weights the 128-row A operand (signed), tokens the
+// TOK-wide B operand (signed).
+//
+// One persistent CTA per SM, 6 warps:
+//   warp 0      producer: per k block one TMA tile of W_q (128 rows x 128 k) and one of x_q (TOK tokens x 128 k),
+//               both 128-byte swizzled, on one barrier
+//   warp 1      MMA: one thread issues four K=32 instructions per k block into one of two TMEM accumulators
+//   warps 2-5   epilogue: TMEM -> registers -> (float)acc * scale_w * a_m / 127 -> bf16/fp32, transposed through a
+//               per-warp shared-memory tile for 16-byte stores; overlaps the next tile's main loop
+// Every mbarrier wait is bounded; on expiry the CTA records a status word and leaves through the normal exit.
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+#include "gemm.cuh"
+#include "ptx.cuh"
+
+namespace bitrl {
+
+constexpr int G8_THREADS = 192;
+constexpr int G8_EPI_WARP0 = 2;
+constexpr uint32_t G8_W_BYTES = 128 * 128;
+constexpr uint32_t G8_RING_BYTES = 196608;
+constexpr uint32_t G8_MAX_STAGES = 8;
+constexpr uint32_t G8_OFF_STAGE = G8_RING_BYTES;                      // 4 x 2 KB epilogue tiles
+constexpr uint32_t G8_OFF_TOK = G8_OFF_STAGE + 4 * 2048;              // scale[2][256] f32
+constexpr uint32_t G8_OFF_BAR = G8_OFF_TOK + 2 * 256 * 4;
+constexpr uint32_t G8_OFF_MISC = G8_OFF_BAR + (2 * G8_MAX_STAGES + 4) * 8;
+constexpr uint32_t G8_SMEM_BYTES = G8_OFF_MISC + 16 + 1024;           // + slack to align the base to 1024
+static_assert(G8_SMEM_BYTES <= 232448, "shared memory budget of one CTA");
+
+enum { G8_WAIT_EMPTY = 41, G8_WAIT_FULL = 42, G8_WAIT_TMEM_EMPTY = 43, G8_WAIT_TMEM_FULL = 44 };
+
+struct Gemm8Args {
+  const float* scale;   // [1] weight scale
+  const float* absmax;  // [M]
+  int M, N, K;
+  void* y;
+  int out_dtype;
+  const unsigned short* residual;
+  int32_t* acc_out;
+  int tiles_n, tiles_total;
+};
+
+template <int TOK>
+__global__ void __launch_bounds__(G8_THREADS, 1)
+gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const Gemm8Args a) {
+  constexpr uint32_t X_BYTES = TOK * 128;
+  constexpr uint32_t STAGE = X_BYTES + G8_W_BYTES;
+  constexpr uint32_t NS = G8_RING_BYTES / STAGE < G8_MAX_STAGES ? G8_RING_BYTES / STAGE : G8_MAX_STAGES;
+  static_assert(TOK % 32 == 0 && TOK >= 64 && TOK <= 256, "token tile");
+  extern __shared__ unsigned char g8_smem_raw[];
+  const uint32_t raw_addr = ptx::smem_u32(g8_smem_raw);
+  const uint32_t base = (raw_addr + 1023u) & ~1023u;
+  unsigned char* base_ptr = g8_smem_raw + (base - raw_addr);
+  const uint32_t bar_full = base + G8_OFF_BAR;
+  const uint32_t bar_empty = bar_full + 8 * G8_MAX_STAGES;
+  const uint32_t bar_tmem_full = bar_empty + 8 * G8_MAX_STAGES;  // [2]
+  const uint32_t bar_tmem_empty = bar_tmem_full + 16;            // [2]
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + G8_OFF_MISC);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kblocks = a.K / 128;
+
+  if (threadIdx.x == 0) {
+    for (uint32_t s = 0; s < NS; ++s) { ptx::mbar_init(bar_full + 8 * s, 1); ptx::mbar_init(bar_empty + 8 * s, 1); }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(bar_tmem_full + 8 * b, 1); ptx::mbar_init(bar_tmem_empty + 8 * b, 4); }
+    ptx::mbar_init_fence();
+    ptx::tma_prefetch_desc(&tmap_x);
+    ptx::tma_prefetch_desc(&tmap_w);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(base + G8_OFF_MISC, 512);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_enter();
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      uint32_t s = 0, ph = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x) {
+        const int tn = tile % a.tiles_n, tm = tile / a.tiles_n;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!ptx::mbar_wait(bar_empty + 8 * s, ph ^ 1u)) { report_timeout(G8_WAIT_EMPTY); ok = false; break; }
+          ptx::mbar_arrive_expect_tx(bar_full + 8 * s, STAGE);
+          ptx::tma_load_2d(base + s * STAGE, &tmap_w, kb * 128, tn * 128, bar_full + 8 * s);
+          ptx::tma_load_2d(base + s * STAGE + G8_W_BYTES, &tmap_x, kb * 128, tm * TOK, bar_full + 8 * s);
+          if (++s == NS) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = ptx::idesc_i8(128, TOK, /*a_signed=*/true, /*b_signed=*/true);
+      uint32_t s = 0, ph = 0, lt = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x, ++lt) {
+        const uint32_t buf = lt & 1u;
+        if (!ptx::mbar_wait(bar_tmem_empty + 8 * buf, ((lt >> 1) & 1u) ^ 1u)) {
+          report_timeout(G8_WAIT_TMEM_EMPTY); ok = false; break;
+        }
+        const uint32_t d_tmem = tmem_base + buf * 256;
+        ptx::tc_fence_after_sync();
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(G8_WAIT_FULL); ok = false; break; }
+          const uint64_t adesc = ptx::smem_desc_sw128(base + s * STAGE);
+          const uint64_t bdesc = ptx::smem_desc_sw128(base + s * STAGE + G8_W_BYTES);
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4)
+            ptx::mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+          ptx::mma_commit(bar_empty + 8 * s);
+          if (++s == NS) { s = 0; ph ^= 1u; }
+        }
+        if (ok) ptx::mma_commit(bar_tmem_full + 8 * buf);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int q = warp & 3;                          // TMEM lane quarter this warp may read
+    const int ep = threadIdx.x - G8_EPI_WARP0 * 32;  // 0..127
+    const int ew = warp - G8_EPI_WARP0;
+    const uint32_t stage = base + G8_OFF_STAGE + ew * 2048;
+    const float wscale = *a.scale;
+    const bool f32 = a.out_dtype == BITRL_OUT_F32;
+    uint32_t lt = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x, ++lt) {
+      const int tn = tile % a.tiles_n, tm = tile / a.tiles_n;
+      const uint32_t buf = lt & 1u;
+      const uint32_t sc_addr = base + G8_OFF_TOK + buf * 256 * 4;
+      for (int j = ep; j < TOK; j += 128) {
+        const int tok = tm * TOK + j;
+        ptx::sts32(sc_addr + 4 * j, __float_as_uint(tok < a.M ? out_scale(wscale, a.absmax[tok]) : 0.0f));
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (!ptx::mbar_wait(bar_tmem_full + 8 * buf, (lt >> 1) & 1u)) { report_timeout(G8_WAIT_TMEM_FULL); ok = false; break; }
+      ptx::tc_fence_after_sync();
+      const int nbase = tn * 128 + q * 32;
+      const int tok0 = tm * TOK;
+      const int tok_hi = min(TOK, a.M - tok0);
+      for (int c = 0; c < TOK / 32; ++c) {
+        if (c * 32 >= tok_hi) break;  // warp-uniform
+        uint4 rres[4];
+        if (a.residual && !f32) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int t = i * 8 + (lane >> 2);
+            if (c * 32 + t < tok_hi)
+              rres[i] = ptx::ldg128(a.residual + static_cast<size_t>(tok0 + c * 32 + t) * a.N + nbase + (lane & 3) * 8);
+          }
+        }
+        uint32_t v[32];
+        ptx::tmem_ld_32x32b_x32(tmem_base + buf * 256 + c * 32 + (static_cast<uint32_t>(q * 32) << 16), v);
+        ptx::tmem_ld_wait();
+        if (a.acc_out) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (c * 32 + j < tok_hi)
+              a.acc_out[static_cast<size_t>(tok0 + c * 32 + j) * a.N + nbase + lane] = static_cast<int>(v[j]);
+        }
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          const uint4 sc4 = ptx::lds128(sc_addr + (c * 32 + 4 * g) * 4);
+          v[4 * g + 0] = __float_as_uint(__fmul_rn(static_cast<float>(static_cast<int>(v[4 * g + 0])), __uint_as_float(sc4.x)));
+          v[4 * g + 1] = __float_as_uint(__fmul_rn(static_cast<float>(static_cast<int>(v[4 * g + 1])), __uint_as_float(sc4.y)));
+          v[4 * g + 2] = __float_as_uint(__fmul_rn(static_cast<float>(static_cast<int>(v[4 * g + 2])), __uint_as_float(sc4.z)));
+          v[4 * g + 3] = __float_as_uint(__fmul_rn(static_cast<float>(static_cast<int>(v[4 * g + 3])), __uint_as_float(sc4.w)));
+        }
+        if (!f32) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) ptx::sts16(stage + j * 64 + lane * 2, float_to_bf16_bits(__uint_as_float(v[j])));
+          __syncwarp();
+          unsigned short* yb = static_cast<unsigned short*>(a.y);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int t = i * 8 + (lane >> 2), part = lane & 3;
+            uint4 o = ptx::lds128(stage + i * 512 + lane * 16);
+            if (c * 32 + t < tok_hi) {
+              const size_t off = static_cast<size_t>(tok0 + c * 32 + t) * a.N + nbase + part * 8;
+              if (a.residual) {
+                const uint4 rr = rres[i];
+                const uint32_t ov[4] = {o.x, o.y, o.z, o.w}, rv[4] = {rr.x, rr.y, rr.z, rr.w};
+                uint32_t res[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const float lo = __fadd_rn(__uint_as_float(rv[e] << 16), __uint_as_float(ov[e] << 16));
+                  const float hi = __fadd_rn(__uint_as_float(rv[e] & 0xffff0000u), __uint_as_float(ov[e] & 0xffff0000u));
+                  res[e] = static_cast<uint32_t>(float_to_bf16_bits(lo)) | (static_cast<uint32_t>(float_to_bf16_bits(hi)) << 16);
+                }
+                o = make_uint4(res[0], res[1], res[2], res[3]);
+              }
+              *reinterpret_cast<uint4*>(yb + off) = o;
+            }
+          }
+          __syncwarp();
+        } else {
+          float* yf = static_cast<float*>(a.y);
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) ptx::sts32(stage + j * 128 + lane * 4, v[h * 16 + j]);
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int t = h * 16 + i * 4 + (lane >> 3), part = lane & 7;
+              const uint4 o = ptx::lds128(stage + i * 512 + lane * 16);
+              if (c * 32 + t < tok_hi)
+                *reinterpret_cast<uint4*>(yf + static_cast<size_t>(tok0 + c * 32 + t) * a.N + nbase + part * 4) = o;
+            }
+            __syncwarp();
+          }
+        }
+      }
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar_tmem_empty + 8 * buf);
+    }
+  }
+
+  // ---- teardown: every role leaves through here, also after a timeout ----
+  __syncwarp();
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// Symmetric absmax quantization of a weight matrix: pass 1 = largest magnitude (integer atomicMax on the bit pattern of a
+// non-negative float: order-free, deterministic), pass 2 = codes.
+__global__ void w8_absmax_kernel(const float4* W, long long n4, unsigned int* amax_bits) {
+  float m = 0.0f;
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n4;
+       i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const float4 v = W[i];
+    m = fmaxf(m, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+  }
+  m = warp_max(m);
+  if ((threadIdx.x & 31) == 0) atomicMax(amax_bits, __float_as_uint(m));
+}
+__global__ void w8_quantize_kernel(const float4* W, long long n4, const unsigned int* amax_bits, uint32_t* Wq, float* scale) {
+  const float a = fmaxf(__uint_as_float(*amax_bits), 1e-20f);
+  const float inv = __fdiv_rn(127.0f, a);
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n4;
+       i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const float4 v = W[i];
+    const int q0 = quant_code(v.x, inv), q1 = quant_code(v.y, inv), q2 = quant_code(v.z, inv), q3 = quant_code(v.w, inv);
+    Wq[i] = (q0 & 0xff) | ((q1 & 0xff) << 8) | ((q2 & 0xff) << 16) | (static_cast<uint32_t>(q3) << 24);
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) *scale = __fdiv_rn(a, 127.0f);
+}
+
+// amax_bits: 4 bytes of scratch inside the caller's `scale` buffer would alias the result, so the launcher uses the
+// second float of a two-float scale buffer: scale[0] = result, scale[1] = scratch.
+bitrl_status launch_w8_quantize(const float* W, int N, int K, int8_t* Wq, float* scale2, cudaStream_t st) {
+  const long long n4 = static_cast<long long>(N) * K / 4;
+  unsigned int* amax_bits = reinterpret_cast<unsigned int*>(scale2 + 1);
+  BITRL_CUDA(cudaMemsetAsync(amax_bits, 0, 4, st));
+  const int grid = sm_count() * 8;
+  w8_absmax_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, amax_bits);
+  w8_quantize_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const float4*>(W), n4, amax_bits,
+                                           reinterpret_cast<uint32_t*>(Wq), scale2);
+  count_launch(2);
+  BITRL_CUDA(cudaGetLastError());
+  return BITRL_OK;
+}
+
+// y = W8A8(x_q): wq dev int8 [N,K] row-major, scale dev [1], x_q dev int8 [M,K], absmax dev [M].
+bitrl_status launch_gemm_w8(const int8_t* wq, const float* scale, int N, int K, const int8_t* xq, const float* absmax, int M,
+                            void* y, int out_dtype, const void* residual, int32_t* acc_out, cudaStream_t st) {
+  encode_tiled_fn encode = get_encode_tiled();
+  if (!encode) return cuda_fail(cudaErrorSymbolNotFound);
+  const int sms = sm_count();
+  const int tiles_n = N / 128;
+  int tok = 256;
+  {
+    long long best = -1;
+    const int cand[3] = {256, 128, 64};
+    for (int i = 0; i < 3; ++i) {
+      const long long tiles = static_cast<long long>(tiles_n) * ((M + cand[i] - 1) / cand[i]);
+      const long long waves = (tiles + sms - 1) / sms;
+      const long long cost = waves * (2 * cand[i] > 300 ? 2 * cand[i] : 300);  // tensor time per k block, floor for small tiles
+      if (best < 0 || cost <= best) { best = cost; tok = cand[i]; }
+    }
+  }
+  CUtensorMap tmx, tmw;
+  const cuuint32_t estr[2] = {1, 1};
+  {
+    const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(M)};
+    const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(K)};
+    const cuuint32_t box[2] = {128, static_cast<cuuint32_t>(tok)};
+    if (encode(&tmx, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(xq), gdim, gstride, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cuda_fail(cudaErrorInvalidValue);
+  }
+  {
+    const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(N)};
+    const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(K)};
+    const cuuint32_t box[2] = {128, 128};
+    if (encode(&tmw, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(wq), gdim, gstride, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cuda_fail(cudaErrorInvalidValue);
+  }
+  Gemm8Args a{scale, absmax, M, N, K, y, out_dtype, static_cast<const unsigned short*>(residual), acc_out, tiles_n, 0};
+  a.tiles_total = tiles_n * ((M + tok - 1) / tok);
+  const int grid = a.tiles_total < sms ? a.tiles_total : sms;
+  void (*kern)(const CUtensorMap, const CUtensorMap, const Gemm8Args) =
+      tok == 256 ? gemm_w8_kernel<256> : tok == 128 ? gemm_w8_kernel<128> : gemm_w8_kernel<64>;
+  BITRL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G8_SMEM_BYTES));
+  BITRL_CUDA(launch_pdl(kern, dim3(grid), dim3(G8_THREADS), G8_SMEM_BYTES, st, tmx, tmw, a));
+  count_launch(1);
+  return BITRL_OK;
+}
+
+}  // namespace bitrl

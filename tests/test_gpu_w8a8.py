@@ -1,0 +1,100 @@
+"""GPU parity of the W8A8 layer (int8 weights with one absmax scale per matrix, the higher-precision critic of the
+paper's ablations) through the C ABI against the CPU oracle: codes, int8 activations and int32 sums bit-exact, rescaled
+outputs within 1e-3 (fp32) / 8e-3 (bf16) of the fp64 reference - and in fact equal bit for bit, both sides doing the
+same int32 -> fp32 conversion and the same three fp32 operations."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2604_24273_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_24273_b200 import bitrl
+
+    bitrl.lib()
+    torch.cuda.set_device(0)
+    return bitrl
+
+
+def bits_to_f64(bits):
+    return (np.asarray(bits, np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def rel_err(y, y64):
+    denom = np.where(y64 == 0, 1.0, np.abs(y64))
+    return float((np.abs(np.asarray(y, np.float64) - y64) / denom).max())
+
+
+_cache = {}
+
+
+def weights(oracle_mod, B, N, K, seed):
+    if (N, K, seed) not in _cache:
+        W = inputs.master_weights(N, K, seed)
+        Wq, scale = oracle_mod.w8_quantize(W.numpy())
+        wq_gpu, scale_gpu = B.w8_quantize(W.cuda())
+        B.poll_status()
+        assert np.array_equal(wq_gpu.cpu().numpy(), Wq), "int8 weight codes differ from the oracle"
+        assert np.float32(scale_gpu.cpu().numpy()[0]) == scale
+        _cache[(N, K, seed)] = (Wq, scale, wq_gpu, scale_gpu)
+    return _cache[(N, K, seed)]
+
+
+@pytest.mark.parametrize("M", [1, 17, 64, 300, 513])
+@pytest.mark.parametrize("K,N,seed,out_dtype", [(256, 384, 9200, 1), (640, 128, 9201, 0), (2560, 2560, 9202, 1)])
+def test_w8a8_full(oracle_mod, B, M, K, N, seed, out_dtype):
+    Wq, scale, wq_gpu, scale_gpu = weights(oracle_mod, B, N, K, seed)
+    x = inputs.activations(M, K, 9300 + M)
+    ref = oracle_mod.bitlinear(inputs.bf16_bits(x), Wq, scale)
+    y, xq, a, acc = B.w8a8_forward(wq_gpu, scale_gpu, x.cuda(), out_dtype, debug=True)
+    y2 = B.w8a8_forward(wq_gpu, scale_gpu, x.cuda(), out_dtype)
+    B.poll_status()
+    assert np.array_equal(xq.cpu().numpy(), ref["xq"])
+    assert np.array_equal(a.cpu().numpy(), ref["absmax"])
+    assert np.array_equal(acc.cpu().numpy(), ref["acc"])
+    if out_dtype == B.OUT_F32:
+        assert rel_err(y.cpu().numpy(), ref["y64"]) <= 1e-3
+        assert np.array_equal(y.cpu().numpy(), ref["y32"]) and torch.equal(y, y2)
+    else:
+        yb = inputs.bf16_bits(y.cpu())
+        assert rel_err(bits_to_f64(yb), ref["y64"]) <= 8e-3
+        assert np.array_equal(yb, ref["ybf16"]) and torch.equal(y, y2)
+
+
+def test_w8a8_m4096_sampled(oracle_mod, B):
+    """The batched-state shape at full size (M = 4096, 2560 -> 6912): sampled outputs one by one."""
+    K, N, M = 2560, 6912, 4096
+    Wq, scale, wq_gpu, scale_gpu = weights(oracle_mod, B, N, K, 9203)
+    x = inputs.activations(M, K, 9400)
+    y, xq, a, acc = B.w8a8_forward(wq_gpu, scale_gpu, x.cuda(), B.OUT_BF16, debug=True)
+    B.poll_status()
+    xq_o, a_o = oracle_mod.quant_act(inputs.bf16_bits(x))
+    assert np.array_equal(xq.cpu().numpy(), xq_o) and np.array_equal(a.cpu().numpy(), a_o)
+    rng = np.random.default_rng(5)
+    ms = np.concatenate([[0, 255, 256, 4095], rng.integers(0, M, 500)])
+    ns = np.concatenate([[0, 127, 128, 6911], rng.integers(0, N, 500)])
+    want = oracle_mod.contract_pairs(xq_o, Wq, ms, ns)
+    assert np.array_equal(acc.cpu().numpy()[ms, ns], want)
+    y64 = want.astype(np.float64) * float(scale) * a_o[ms].astype(np.float64) / 127.0
+    assert rel_err(bits_to_f64(inputs.bf16_bits(y.cpu())[ms, ns]), y64) <= 8e-3
+
+
+def test_w8a8_argument_errors(oracle_mod, B):
+    L = B.lib()
+    Wq, scale, wq_gpu, scale_gpu = weights(oracle_mod, B, 384, 256, 9200)
+    x = inputs.activations(4, 256, 1).cuda()
+    y = torch.empty((4, 384), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty((L.bitrl_w8a8_workspace_bytes(4, 256),), dtype=torch.uint8, device="cuda")
+    call = lambda M, K, N, wsb: L.bitrl_w8a8_forward(wq_gpu.data_ptr(), scale_gpu.data_ptr(), x.data_ptr(), M, K, N,
+                                                     y.data_ptr(), 1, ws.data_ptr(), wsb, None)
+    assert call(0, 256, 384, ws.numel()) == B.ERR_SHAPE
+    assert call(4, 200, 384, ws.numel()) == B.ERR_SHAPE
+    assert call(4, 256, 384, 16) == B.ERR_WORKSPACE
+    assert call(4, 256, 384, ws.numel()) == B.OK
+    B.poll_status()
