@@ -383,6 +383,49 @@ def run_ours(args):
             extra[name] = res
             del xs, y, ws, q
 
+        # the higher-precision critic's W8A8 layer at the same M = 4096 shapes (int8 weights, nothing to decode)
+        for name, K, N in (("w8a8_m4096_k2560_n6912", 2560, 6912), ("w8a8_m4096_k6912_n2560", 6912, 2560)):
+            w8 = []
+            for i in range(4):
+                gen.manual_seed(1400 + i)
+                w8.append(bitrl.w8_quantize(torch.randn(N, K, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W))
+            xs = [inputs.activations(M, K, 2400 + i).to(dev) for i in range(4)]
+            y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            ws = torch.empty((int(bitrl.lib().bitrl_w8a8_workspace_bytes(M, K)),), dtype=torch.uint8, device=dev)
+            reps = 12
+
+            def w8_layer():
+                for i in range(reps):
+                    bitrl.w8a8_forward(*w8[i % 4], xs[i % 4], bitrl.OUT_BF16, y=y, workspace=ws)
+
+            g, _ = capture(w8_layer)
+            ms = time_graph(g, sub_steps, args.warmup, 1)
+            tops = 2.0 * M * N * K * reps * sub_steps / (ms * 1e-3) / 1e12
+            extra[name] = {"layer": {"TOPS": tops, "us": ms * 1e3 / (sub_steps * reps), "frac_of_int8_peak": tops / i8_peak,
+                                     "frac_of_nominal_4500": tops / 4500.0}}
+            del g, xs, y, ws, w8
+
+        # ... and its streaming kernel at M = 1 and 8 over eight 2560 -> 13824 matrices (283 MB of int8 weights, > L2)
+        w8 = []
+        for i in range(8):
+            gen.manual_seed(1500 + i)
+            w8.append(bitrl.w8_quantize(torch.randn(13824, 2560, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W))
+        for Ms in (1, 8):
+            xd = inputs.activations(Ms, 2560, 2000 + Ms).to(dev)
+            yd = torch.empty((Ms, 13824), dtype=torch.bfloat16, device=dev)
+
+            def w8_sweep():
+                for wq8, sc8 in w8:
+                    bitrl.w8a8_forward(wq8, sc8, xd, bitrl.OUT_BF16, y=yd)
+
+            g, lc = capture(w8_sweep)
+            ms = time_graph(g, sub_steps, args.warmup, 1) / sub_steps
+            gbs = 8 * 13824 * 2560 / (ms * 1e-3) / 1e9
+            extra[f"w8a8_m{Ms}_sweep_8x_k2560_n13824"] = {"GBps_of_weight_bytes": gbs, "us_per_matrix": ms * 1e3 / 8,
+                                                         "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "launches": lc}
+            del g
+        del w8
+
         # configs[2]: batched state encoding, M = 64 and 256 (one token per state), the whole layer per call
         for M in (64, 256):
             for K, N in ((2560, 6912), (6912, 2560)):

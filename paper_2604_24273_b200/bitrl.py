@@ -385,7 +385,7 @@ def w8a8_forward(wq: torch.Tensor, scale: torch.Tensor, x: torch.Tensor, out_dty
     if y is None:
         y = _out(M, N, out_dtype, x.device)
     if workspace is None:
-        workspace = torch.empty((int(lib().bitrl_w8a8_workspace_bytes(M, K)),), dtype=torch.uint8, device=x.device)
+        workspace = torch.empty((max(int(lib().bitrl_w8a8_workspace_bytes(M, K)), 16),), dtype=torch.uint8, device=x.device)
     if not debug:
         _check(lib().bitrl_w8a8_forward(_ptr(wq), _ptr(scale), _ptr(x), M, K, N, _ptr(y), out_dtype, _ptr(workspace),
                                         workspace.numel(), _stream()), "bitrl_w8a8_forward")

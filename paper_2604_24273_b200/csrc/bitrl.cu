@@ -597,6 +597,7 @@ bitrl_status bitrl_w8_quantize(const float* W, int32_t N, int32_t K, int8_t* wq,
 
 size_t bitrl_w8a8_workspace_bytes(int32_t M, int32_t K) {
   if (M < 1 || K < 1) return 0;
+  if (gemv_w8_fits(M, K)) return 0;
   return align_up(static_cast<size_t>(M) * K, 256) + align_up(static_cast<size_t>(M) * 4, 256);
 }
 
@@ -606,11 +607,13 @@ static bitrl_status w8a8_impl(const int8_t* wq, const float* scale, const void* 
   if (!wq || !scale || !x || !y) return BITRL_ERR_NULL;
   if (M < 1 || !shape_ok(N, K)) return BITRL_ERR_SHAPE;
   if (out_dtype != BITRL_OUT_F32 && out_dtype != BITRL_OUT_BF16) return BITRL_ERR_DTYPE;
-  if (!workspace || workspace_bytes < bitrl_w8a8_workspace_bytes(M, K)) return BITRL_ERR_WORKSPACE;
   if (!aligned16(wq) || !aligned16(x) || !aligned16(y) || !aligned16(workspace)) return BITRL_ERR_ALIGN;
   bitrl_status s = check_arch();
   if (s != BITRL_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (gemv_w8_fits(M, K))
+    return launch_gemv_w8(wq, scale, N, K, x, M, y, out_dtype, xq_out, absmax_out, acc_out, st);
+  if (!workspace || workspace_bytes < bitrl_w8a8_workspace_bytes(M, K)) return BITRL_ERR_WORKSPACE;
   int8_t* xq = static_cast<int8_t*>(workspace);
   float* absmax = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + align_up(static_cast<size_t>(M) * K, 256));
   if ((s = launch_quant_act(x, M, K, xq, absmax, nullptr, st)) != BITRL_OK) return s;

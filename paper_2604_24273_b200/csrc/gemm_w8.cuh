@@ -17,6 +17,7 @@
 
 #include "common.cuh"
 #include "gemm.cuh"
+#include "gemv.cuh"
 #include "ptx.cuh"
 
 namespace bitrl {
@@ -238,6 +239,148 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   }
 }
 
+// ---- M <= 16: streaming kernel ----------------------------------------------------------------------------------
+// The weights (N*K bytes) are read once; the kernel is bound by HBM.  Persistent CTAs of 8 warps: the activations are
+// quantized once per CTA into shared memory (one warp per token), then a warp owns a few weight rows at a time, every
+// lane streams 16-byte pieces of them and feeds dp4a (signed x signed) for all tokens; one shuffle tree per row.
+constexpr int GV8_THREADS = 256;
+
+struct Gemv8Args {
+  const int8_t* wq;
+  const float* scale;
+  const unsigned short* x;  // bf16 [M,K]
+  int M, N, K;
+  void* y;
+  int out_dtype;
+  int8_t* xq_out;      // debug taps (may be null)
+  float* absmax_out;
+  int32_t* acc_out;
+};
+
+__device__ __forceinline__ int dp4a_s8s8(uint32_t a, uint32_t b, int acc) {
+  int d;
+  asm("dp4a.s32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(acc));
+  return d;
+}
+
+template <int MT>
+__global__ void __launch_bounds__(GV8_THREADS) gemv_w8_kernel(Gemv8Args a) {
+  extern __shared__ __align__(16) unsigned char gv8_smem[];
+  int8_t* xq_s = reinterpret_cast<int8_t*>(gv8_smem);               // [MT][K]
+  float* sc_s = reinterpret_cast<float*>(gv8_smem + MT * a.K);      // [MT] a_m / 127
+  pdl_enter();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int K = a.K, nvec8 = K >> 3;
+  for (int m = warp; m < MT; m += GV8_THREADS / 32) {
+    uint2* dst = reinterpret_cast<uint2*>(xq_s + m * K);
+    if (m >= a.M) {
+      for (int i = lane; i < nvec8; i += 32) dst[i] = make_uint2(0u, 0u);
+      if (lane == 0) sc_s[m] = 0.0f;
+      continue;
+    }
+    const uint4* xr = reinterpret_cast<const uint4*>(a.x + static_cast<size_t>(m) * K);
+    float mx = 0.0f;
+#pragma unroll 4
+    for (int i = lane; i < nvec8; i += 32) mx = fmaxf(mx, absmax8(xr[i]));
+    const float amax = fmaxf(warp_max(mx), 1e-5f);
+    const float inv = __fdiv_rn(127.0f, amax);
+    uint2* tap = (a.xq_out && blockIdx.x == 0) ? reinterpret_cast<uint2*>(a.xq_out + static_cast<size_t>(m) * K) : nullptr;
+    for (int i = lane; i < nvec8; i += 32) {
+      const uint4 raw = xr[i];
+      const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+      int q[8];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        q[2 * e] = quant_code(__uint_as_float(rw[e] << 16), inv);
+        q[2 * e + 1] = quant_code(__uint_as_float(rw[e] & 0xffff0000u), inv);
+      }
+      uint2 wd;
+      wd.x = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | (static_cast<uint32_t>(q[3]) << 24);
+      wd.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | (static_cast<uint32_t>(q[7]) << 24);
+      dst[i] = wd;
+      if (tap) tap[i] = wd;
+    }
+    if (lane == 0) {
+      sc_s[m] = __fdiv_rn(amax, 127.0f);
+      if (a.absmax_out && blockIdx.x == 0) a.absmax_out[m] = amax;
+    }
+  }
+  __syncthreads();
+
+  const float wscale = *a.scale;
+  const int nvec16 = K >> 4;
+  // A warp streams R rows at a time (N is a multiple of 128): R times as many loads in flight per lane, and every
+  // 16-byte piece of the activations read from shared memory serves R rows.
+  constexpr int R = MT <= 4 ? 4 : 2;
+  for (int n0 = (blockIdx.x * (GV8_THREADS / 32) + warp) * R; n0 < a.N; n0 += gridDim.x * (GV8_THREADS / 32) * R) {
+    const uint4* wr = reinterpret_cast<const uint4*>(a.wq + static_cast<size_t>(n0) * K);
+    int acc[R][MT];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int m = 0; m < MT; ++m) acc[r][m] = 0;
+#pragma unroll 2
+    for (int i = lane; i < nvec16; i += 32) {
+      uint4 wv[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) wv[r] = wr[static_cast<size_t>(r) * nvec16 + i];
+#pragma unroll
+      for (int m = 0; m < MT; ++m) {
+        const uint4 xv = *reinterpret_cast<const uint4*>(xq_s + m * K + 16 * i);
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          acc[r][m] = dp4a_s8s8(wv[r].x, xv.x, acc[r][m]);
+          acc[r][m] = dp4a_s8s8(wv[r].y, xv.y, acc[r][m]);
+          acc[r][m] = dp4a_s8s8(wv[r].z, xv.z, acc[r][m]);
+          acc[r][m] = dp4a_s8s8(wv[r].w, xv.w, acc[r][m]);
+        }
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int m = 0; m < MT; ++m) acc[r][m] = warp_sum_i(acc[r][m]);
+    if (lane == 0) {
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+          if (m < a.M) {
+            const float yv = __fmul_rn(static_cast<float>(acc[r][m]), __fmul_rn(wscale, sc_s[m]));
+            const size_t o = static_cast<size_t>(m) * a.N + n0 + r;
+            if (a.acc_out) a.acc_out[o] = acc[r][m];
+            if (a.out_dtype == BITRL_OUT_F32) static_cast<float*>(a.y)[o] = yv;
+            else static_cast<unsigned short*>(a.y)[o] = float_to_bf16_bits(yv);
+          }
+        }
+    }
+  }
+}
+
+template <int MT>
+bitrl_status launch_gemv_w8_t(const Gemv8Args& a, cudaStream_t st) {
+  const size_t smem = static_cast<size_t>(MT) * a.K + MT * sizeof(float) + 16;
+  BITRL_CUDA(cudaFuncSetAttribute(gemv_w8_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  int grid = sm_count() * (smem <= 100 * 1024 ? 2 : 1);
+  const int row_groups = (a.N + GV8_THREADS / 8 - 1) / (GV8_THREADS / 8);  // at most four rows per warp and step
+  if (grid > row_groups) grid = row_groups;
+  BITRL_CUDA(launch_pdl(gemv_w8_kernel<MT>, dim3(grid), dim3(GV8_THREADS), smem, st, a));
+  count_launch(1);
+  return BITRL_OK;
+}
+
+inline bool gemv_w8_fits(int M, int K) { return M <= BITRL_GEMV_MAX_M && static_cast<size_t>(16) * K <= 200 * 1024; }
+
+bitrl_status launch_gemv_w8(const int8_t* wq, const float* scale, int N, int K, const void* x, int M, void* y, int out_dtype,
+                            int8_t* xq_out, float* absmax_out, int32_t* acc_out, cudaStream_t st) {
+  Gemv8Args a{wq, scale, static_cast<const unsigned short*>(x), M, N, K, y, out_dtype, xq_out, absmax_out, acc_out};
+  if (M == 1) return launch_gemv_w8_t<1>(a, st);
+  if (M == 2) return launch_gemv_w8_t<2>(a, st);
+  if (M <= 4) return launch_gemv_w8_t<4>(a, st);
+  if (M <= 8) return launch_gemv_w8_t<8>(a, st);
+  return launch_gemv_w8_t<16>(a, st);
+}
+
 // Symmetric absmax quantization of a weight matrix: pass 1 = largest magnitude (integer atomicMax on the bit pattern of a
 // non-negative float: order-free, deterministic), pass 2 = codes.
 __global__ void w8_absmax_kernel(const float4* W, long long n4, unsigned int* amax_bits) {
@@ -287,8 +430,8 @@ bitrl_status launch_gemm_w8(const int8_t* wq, const float* scale, int N, int K, 
   int tok = 256;
   {
     long long best = -1;
-    const int cand[3] = {256, 128, 64};
-    for (int i = 0; i < 3; ++i) {
+    const int cand[5] = {256, 224, 192, 128, 64};
+    for (int i = 0; i < 5; ++i) {
       const long long tiles = static_cast<long long>(tiles_n) * ((M + cand[i] - 1) / cand[i]);
       const long long waves = (tiles + sms - 1) / sms;
       const long long cost = waves * (2 * cand[i] > 300 ? 2 * cand[i] : 300);  // tensor time per k block, floor for small tiles
@@ -319,7 +462,8 @@ bitrl_status launch_gemm_w8(const int8_t* wq, const float* scale, int N, int K, 
   a.tiles_total = tiles_n * ((M + tok - 1) / tok);
   const int grid = a.tiles_total < sms ? a.tiles_total : sms;
   void (*kern)(const CUtensorMap, const CUtensorMap, const Gemm8Args) =
-      tok == 256 ? gemm_w8_kernel<256> : tok == 128 ? gemm_w8_kernel<128> : gemm_w8_kernel<64>;
+      tok == 256 ? gemm_w8_kernel<256> : tok == 224 ? gemm_w8_kernel<224> : tok == 192 ? gemm_w8_kernel<192>
+      : tok == 128 ? gemm_w8_kernel<128> : gemm_w8_kernel<64>;
   BITRL_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, G8_SMEM_BYTES));
   BITRL_CUDA(launch_pdl(kern, dim3(grid), dim3(G8_THREADS), G8_SMEM_BYTES, st, tmx, tmw, a));
   count_launch(1);

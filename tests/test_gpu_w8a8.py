@@ -46,7 +46,7 @@ def weights(oracle_mod, B, N, K, seed):
     return _cache[(N, K, seed)]
 
 
-@pytest.mark.parametrize("M", [1, 17, 64, 300, 513])
+@pytest.mark.parametrize("M", [1, 2, 3, 8, 13, 16, 17, 64, 300, 513])
 @pytest.mark.parametrize("K,N,seed,out_dtype", [(256, 384, 9200, 1), (640, 128, 9201, 0), (2560, 2560, 9202, 1)])
 def test_w8a8_full(oracle_mod, B, M, K, N, seed, out_dtype):
     Wq, scale, wq_gpu, scale_gpu = weights(oracle_mod, B, N, K, seed)
@@ -88,13 +88,15 @@ def test_w8a8_m4096_sampled(oracle_mod, B):
 def test_w8a8_argument_errors(oracle_mod, B):
     L = B.lib()
     Wq, scale, wq_gpu, scale_gpu = weights(oracle_mod, B, 384, 256, 9200)
-    x = inputs.activations(4, 256, 1).cuda()
-    y = torch.empty((4, 384), dtype=torch.bfloat16, device="cuda")
-    ws = torch.empty((L.bitrl_w8a8_workspace_bytes(4, 256),), dtype=torch.uint8, device="cuda")
+    x = inputs.activations(20, 256, 1).cuda()
+    y = torch.empty((20, 384), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty((L.bitrl_w8a8_workspace_bytes(20, 256),), dtype=torch.uint8, device="cuda")
+    assert L.bitrl_w8a8_workspace_bytes(4, 256) == 0  # the streaming kernel needs none
     call = lambda M, K, N, wsb: L.bitrl_w8a8_forward(wq_gpu.data_ptr(), scale_gpu.data_ptr(), x.data_ptr(), M, K, N,
                                                      y.data_ptr(), 1, ws.data_ptr(), wsb, None)
     assert call(0, 256, 384, ws.numel()) == B.ERR_SHAPE
-    assert call(4, 200, 384, ws.numel()) == B.ERR_SHAPE
-    assert call(4, 256, 384, 16) == B.ERR_WORKSPACE
-    assert call(4, 256, 384, ws.numel()) == B.OK
+    assert call(20, 200, 384, ws.numel()) == B.ERR_SHAPE
+    assert call(20, 256, 384, 16) == B.ERR_WORKSPACE
+    assert call(20, 256, 384, ws.numel()) == B.OK
+    assert call(4, 256, 384, 0) == B.OK
     B.poll_status()
