@@ -20,6 +20,9 @@
 // stores) so that the consumer-wide named barriers stay matched, and the CTA exits normally.
 #pragma once
 
+#include <algorithm>
+#include <vector>
+
 #include "common.cuh"
 #include "gemv.cuh"
 #include "ptx.cuh"
@@ -50,7 +53,11 @@ struct GvmJob {
 
 struct GvmArgs {
   GvmJob jobs[GVM_MAX_JOBS];
-  int unit_start[GVM_MAX_CTAS + 1];  // work-list range of each CTA
+  // Work of each CTA: two ranges of the work list, [seg[c][0], seg[c][1]) then [seg[c][2], seg[c][3]).  The jobs are
+  // sorted by K, largest first, so the first range holds long row tiles and the second short ones: a CTA takes long
+  // tiles while they fit its share and tops up with short ones, which balances the bytes per CTA to within half a
+  // short tile (one range per CTA left the slowest CTA 5 % above the mean on the 30-block sweep).
+  int seg[GVM_MAX_CTAS][4];
   int njobs, M, out_dtype, depth_log2, kmax;
 };
 
@@ -84,7 +91,8 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
   int* comb = reinterpret_cast<int*>(rowsum_s + NT);              // [2][8 warps][NT/8 * 4][32 lanes]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int u_begin = a.unit_start[blockIdx.x], u_end = a.unit_start[blockIdx.x + 1];
+  const int u_begin = a.seg[blockIdx.x][0], u_mid = a.seg[blockIdx.x][1], u_resume = a.seg[blockIdx.x][2],
+            u_end = a.seg[blockIdx.x][3];  // units u_begin..u_mid-1, then u_resume..u_end-1
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < depth; ++s) {
@@ -102,7 +110,7 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
       uint32_t pc = 0;
       int j = 0;
       bool ok = true;
-      for (int u = u_begin; ok && u < u_end; ++u) {
+      for (int u = u_begin == u_mid ? u_resume : u_begin; ok && u < u_end; u = (u + 1 == u_mid) ? u_resume : u + 1) {
         while (j + 1 < a.njobs && a.jobs[j + 1].unit_begin <= u) ++j;
         const int kblocks = a.jobs[j].K / TILE_K;
         const uint8_t* src = a.jobs[j].tiles + static_cast<size_t>(u - a.jobs[j].unit_begin) * kblocks * TILE_BYTES;
@@ -125,7 +133,7 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
     uint32_t pc = 0, tile_no = 0;
     int j = 0;
     bool ok = true;
-    for (int u = u_begin; u < u_end; ++u, ++tile_no) {
+    for (int u = u_begin == u_mid ? u_resume : u_begin; u < u_end; u = (u + 1 == u_mid) ? u_resume : u + 1, ++tile_no) {
       while (j + 1 < a.njobs && a.jobs[j + 1].unit_begin <= u) ++j;
       const GvmJob& job = a.jobs[j];
       const int K = job.K, kblocks = K / TILE_K;
@@ -291,7 +299,8 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
   int* comb = redi + GVD_CONSUMERS;                               // [2][GROUPS-1][8 warps][16 rows][MT]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int u_begin = a.unit_start[blockIdx.x], u_end = a.unit_start[blockIdx.x + 1];
+  const int u_begin = a.seg[blockIdx.x][0], u_mid = a.seg[blockIdx.x][1], u_resume = a.seg[blockIdx.x][2],
+            u_end = a.seg[blockIdx.x][3];  // units u_begin..u_mid-1, then u_resume..u_end-1
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < depth; ++s) {
@@ -309,7 +318,7 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
       uint32_t s = 0, ph = 0;
       int j = 0;
       bool ok = true;
-      for (int u = u_begin; ok && u < u_end; ++u) {
+      for (int u = u_begin == u_mid ? u_resume : u_begin; ok && u < u_end; u = (u + 1 == u_mid) ? u_resume : u + 1) {
         while (j + 1 < a.njobs && a.jobs[j + 1].unit_begin <= u) ++j;
         const int kblocks = a.jobs[j].K / TILE_K;
         const uint8_t* src = a.jobs[j].tiles + static_cast<size_t>(u - a.jobs[j].unit_begin) * kblocks * TILE_BYTES;
@@ -331,7 +340,7 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
     uint32_t s = 0, ph = 0, tile_no = 0;
     int j = 0;
     bool ok = true;
-    for (int u = u_begin; u < u_end; ++u, ++tile_no) {
+    for (int u = u_begin == u_mid ? u_resume : u_begin; u < u_end; u = (u + 1 == u_mid) ? u_resume : u + 1, ++tile_no) {
       while (j + 1 < a.njobs && a.jobs[j + 1].unit_begin <= u) ++j;
       const GvmJob& job = a.jobs[j];
       const int K = job.K, kblocks = K / TILE_K;
@@ -536,8 +545,12 @@ bitrl_status launch_gemv_multi(int count, const Linear* const* w, const void* co
   static thread_local GvmArgs a;  // 7 KB, kept off the stack
   int kmax = 0, units = 0;
   long long pieces = 0;
-  for (int j = 0; j < count; ++j) {
-    a.jobs[j] = GvmJob{w[j]->tiles, w[j]->gamma, static_cast<const unsigned short*>(x[j]), y[j], w[j]->N, w[j]->K,
+  int order[GVM_MAX_JOBS];  // jobs by K, largest first (stable)
+  for (int j = 0; j < count; ++j) order[j] = j;
+  std::stable_sort(order, order + count, [&](int x, int y) { return w[x]->K > w[y]->K; });
+  for (int i = 0; i < count; ++i) {
+    const int j = order[i];
+    a.jobs[i] = GvmJob{w[j]->tiles, w[j]->gamma, static_cast<const unsigned short*>(x[j]), y[j], w[j]->N, w[j]->K,
                        units, 0};
     units += w[j]->N / TILE_ROWS;
     pieces += static_cast<long long>(w[j]->N / TILE_ROWS) * (w[j]->K / TILE_K);
@@ -554,21 +567,25 @@ bitrl_status launch_gemv_multi(int count, const Linear* const* w, const void* co
   int grid = sm_count();
   if (grid > GVM_MAX_CTAS) grid = GVM_MAX_CTAS;
   if (grid > units) grid = units;
-  // Contiguous ranges of row tiles with about pieces/grid 4 KB pieces each.
+  // Two ranges per CTA (see GvmArgs::seg): long tiles from the head of the list while they fit the CTA's share of
+  // the remaining pieces, then short tiles from the tail up to the nearest fit.
   {
-    int j = 0, u = 0;
-    long long done = 0;
-    a.unit_start[0] = 0;
+    static thread_local std::vector<int> sz;  // 4 KB pieces of every unit, in work-list order
+    sz.clear();
+    for (int j = 0; j < count; ++j) sz.insert(sz.end(), a.jobs[j].N / TILE_ROWS, a.jobs[j].K / TILE_K);
+    int head = 0, tail = units;
+    long long remaining = pieces;
     for (int c = 0; c < grid; ++c) {
-      const long long target = pieces * (c + 1) / grid;
-      while (u < units && done < target) {
-        while (j + 1 < count && a.jobs[j + 1].unit_begin <= u) ++j;
-        done += a.jobs[j].K / TILE_K;
-        ++u;
-      }
-      a.unit_start[c + 1] = u;
+      const double target = static_cast<double>(remaining) / (grid - c);
+      long long load = 0;
+      a.seg[c][0] = head;
+      while (head < tail && (c == grid - 1 || load + sz[head] <= target)) load += sz[head++];
+      a.seg[c][1] = head;
+      a.seg[c][3] = tail;
+      while (head < tail && load + sz[tail - 1] <= target + 0.5 * sz[tail - 1]) load += sz[--tail];
+      a.seg[c][2] = tail;
+      remaining -= load;
     }
-    a.unit_start[grid] = units;
   }
   a.njobs = count;
   a.M = M;
