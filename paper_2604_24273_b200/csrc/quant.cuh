@@ -170,128 +170,171 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, i
   __shared__ float red_mx[ROW_THREADS / 32];
   __shared__ int red_rs[ROW_THREADS / 32];
   pdl_enter();
+  constexpr int ROWS = ROW_THREADS / 32 / WPR;           // rows a CTA works on at a time
+  constexpr int NRAW = MODE == ROW_RELU2 ? 2 * NG : NG;  // 16-byte words a lane holds of one row
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int sub = warp % WPR, grp = warp / WPR;
-  const long long row = static_cast<long long>(blockIdx.x) * (ROW_THREADS / 32 / WPR) + grp;
-  const bool live = row < T;
   const int nvec8 = a.Kv >> 3;
-  const unsigned short* src = a.in + (live ? row : 0) * a.in_stride + a.in_offset;
 
-  // pass 1: the row vector v, its sum of squares and its largest magnitude in one sweep
-  float v[NG][8];
-  float ss = 0.0f, mx = 0.0f;
+  // Persistent CTAs: the raw words of the NEXT row are requested before the current row is processed, so that the
+  // memory system stays busy during the arithmetic (a one-row-per-CTA version showed no overlap of the two).
+  auto request = [&](long long row, uint4 (&raw)[NRAW]) {
+    const unsigned short* src = a.in + row * a.in_stride + a.in_offset;
 #pragma unroll
-  for (int gi = 0; gi < NG; ++gi) {
-    const int i = (gi * WPR + sub) * 32 + lane;
-    if (live && i < nvec8) {
-      const uint4 raw = *reinterpret_cast<const uint4*>(src + 8 * i);
-      const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        v[gi][2 * e] = __uint_as_float(rw[e] << 16);
-        v[gi][2 * e + 1] = __uint_as_float(rw[e] & 0xffff0000u);
+    for (int gi = 0; gi < NG; ++gi) {
+      const int i = (gi * WPR + sub) * 32 + lane;
+      if (row < T && i < nvec8) {
+        raw[gi] = *reinterpret_cast<const uint4*>(src + 8 * i);
+        if (MODE == ROW_RELU2) raw[NG + gi] = *reinterpret_cast<const uint4*>(src + a.gate_offset + 8 * i);
       }
-      if (MODE == ROW_RELU2) {
-        const uint4 rawu = *reinterpret_cast<const uint4*>(src + a.gate_offset + 8 * i);
-        const uint32_t ru[4] = {rawu.x, rawu.y, rawu.z, rawu.w};
+    }
+  };
+
+  constexpr bool PREFETCH = MODE == ROW_RELU2;  // see launch_row_reg
+  uint4 raw[NRAW], nxt[PREFETCH ? NRAW : 1];
+  long long row = static_cast<long long>(blockIdx.x) * ROWS + grp;
+  const long long stride = static_cast<long long>(gridDim.x) * ROWS;
+  if constexpr (PREFETCH) request(row, raw);
+  // every group of the CTA runs the same number of iterations (the CTA-wide barriers below need that)
+  for (long long base = static_cast<long long>(blockIdx.x) * ROWS; base < T; base += stride, row += stride) {
+    const bool live = row < T;
+    if constexpr (PREFETCH) request(row + stride, nxt);
+
+    // pass 1: the row vector v, its sum of squares and its largest magnitude in one sweep
+    float v[NG][8];
+    float ss = 0.0f, mx = 0.0f;
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi) {
+      const int i = (gi * WPR + sub) * 32 + lane;
+      if (live && i < nvec8) {
+        uint4 rg;
+        if constexpr (PREFETCH) rg = raw[gi];
+        else rg = *reinterpret_cast<const uint4*>(a.in + row * a.in_stride + a.in_offset + 8 * i);
+        const uint32_t rw[4] = {rg.x, rg.y, rg.z, rg.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const float g0 = fmaxf(v[gi][2 * e], 0.0f), g1 = fmaxf(v[gi][2 * e + 1], 0.0f);
-          v[gi][2 * e] = __fmul_rn(__fmul_rn(g0, g0), __uint_as_float(ru[e] << 16));
-          v[gi][2 * e + 1] = __fmul_rn(__fmul_rn(g1, g1), __uint_as_float(ru[e] & 0xffff0000u));
+          v[gi][2 * e] = __uint_as_float(rw[e] << 16);
+          v[gi][2 * e + 1] = __uint_as_float(rw[e] & 0xffff0000u);
         }
-      }
+        if (MODE == ROW_RELU2) {
+          const uint4 rawu = raw[MODE == ROW_RELU2 ? NG + gi : gi];  // ROW_RELU2 always prefetches
+          const uint32_t ru[4] = {rawu.x, rawu.y, rawu.z, rawu.w};
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        if (MODE != ROW_PLAIN) ss += v[gi][e] * v[gi][e];
-        mx = fmaxf(mx, fabsf(v[gi][e]));
-      }
-    } else {
-#pragma unroll
-      for (int e = 0; e < 8; ++e) v[gi][e] = 0.0f;
-    }
-  }
-  if (MODE != ROW_PLAIN) ss = warp_sum(ss);
-  mx = warp_max(mx);
-  if (WPR > 1) {
-    if (lane == 0) { red_ss[warp] = ss; red_mx[warp] = mx; }
-    __syncthreads();
-    ss = 0.0f;
-#pragma unroll
-    for (int i = 0; i < WPR; ++i) { ss += red_ss[grp * WPR + i]; mx = fmaxf(mx, red_mx[grp * WPR + i]); }
-  }
-  // u = bf16(v * rstd) is monotonic in |v| (one rounded multiply, one rounding to bf16), so the largest |u| of the row
-  // is the image of the largest |v|: no second reduction over the normalized values.
-  float rstd = 1.0f, amax = mx;
-  if (MODE != ROW_PLAIN) {
-    rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(ss, static_cast<float>(a.Kv)), 1e-5f)));
-    amax = bf16_bits_to_float(float_to_bf16_bits(__fmul_rn(mx, rstd)));
-  }
-  amax = fmaxf(amax, 1e-5f);
-  const float inv = __fdiv_rn(127.0f, amax);
-
-  // pass 2: normalize, round to bf16, quantize (round-to-nearest-even conversion, saturating pack), row sum of the codes
-  int rs = 0;
-  int8_t* xq = a.xq + (live ? row : 0) * a.Kout;
-  unsigned short* uo = a.u_out ? a.u_out + (live ? row : 0) * a.Kout : nullptr;
-#pragma unroll
-  for (int gi = 0; gi < NG; ++gi) {
-    const int i = (gi * WPR + sub) * 32 + lane;
-    if (live && i < nvec8) {
-      uint32_t ub[4];
-      int q[8];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        float lo = v[gi][2 * e], hi = v[gi][2 * e + 1];
-        if (MODE != ROW_PLAIN) {
-          const __nv_bfloat162 pr = __floats2bfloat162_rn(__fmul_rn(lo, rstd), __fmul_rn(hi, rstd));
-          ub[e] = *reinterpret_cast<const uint32_t*>(&pr);
-          lo = __uint_as_float(ub[e] << 16);
-          hi = __uint_as_float(ub[e] & 0xffff0000u);
-        } else if (a.u_out) {
-          ub[e] = (__float_as_uint(lo) >> 16) | (__float_as_uint(hi) & 0xffff0000u);
+          for (int e = 0; e < 4; ++e) {
+            const float g0 = fmaxf(v[gi][2 * e], 0.0f), g1 = fmaxf(v[gi][2 * e + 1], 0.0f);
+            v[gi][2 * e] = __fmul_rn(__fmul_rn(g0, g0), __uint_as_float(ru[e] << 16));
+            v[gi][2 * e + 1] = __fmul_rn(__fmul_rn(g1, g1), __uint_as_float(ru[e] & 0xffff0000u));
+          }
         }
-        q[2 * e] = __float2int_rn(__fmul_rn(lo, inv));
-        q[2 * e + 1] = __float2int_rn(__fmul_rn(hi, inv));
-      }
-      uint2 wd;
-      wd.x = pack_s8x4(q[0], q[1], q[2], q[3]);
-      wd.y = pack_s8x4(q[4], q[5], q[6], q[7]);
-      rs = dp4a_ones(wd.y, dp4a_ones(wd.x, rs));
-      const uint4 ub4 = make_uint4(ub[0], ub[1], ub[2], ub[3]);
-      if (MODE == ROW_VREPEAT) {
-        const int k = 8 * i;
-        const int kvh = k / a.head_dim, e0 = k - kvh * a.head_dim;
-        for (int r = 0; r < a.rep; ++r) {
-          const int ko = (kvh * a.rep + r) * a.head_dim + e0;
-          *reinterpret_cast<uint2*>(xq + ko) = wd;
-          if (uo) *reinterpret_cast<uint4*>(uo + ko) = ub4;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          if (MODE != ROW_PLAIN) ss = fmaf(v[gi][e], v[gi][e], ss);
+          mx = fmaxf(mx, fabsf(v[gi][e]));
         }
       } else {
-        *reinterpret_cast<uint2*>(xq + 8 * i) = wd;
-        if (uo) *reinterpret_cast<uint4*>(uo + 8 * i) = ub4;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[gi][e] = 0.0f;
       }
     }
-  }
-  rs = warp_sum_i(rs);
-  if (WPR > 1) {
-    if (lane == 0) red_rs[warp] = rs;
-    __syncthreads();
-    rs = 0;
+    if (MODE != ROW_PLAIN) ss = warp_sum(ss);
+    mx = warp_max(mx);
+    if (WPR > 1) {
+      if (lane == 0) { red_ss[warp] = ss; red_mx[warp] = mx; }
+      __syncthreads();
+      ss = 0.0f;
 #pragma unroll
-    for (int i = 0; i < WPR; ++i) rs += red_rs[grp * WPR + i];
-  }
-  if (live && sub == 0 && lane == 0) {
-    a.absmax[row] = amax;
-    if (a.rowsum) a.rowsum[row] = rs * a.rep;
+      for (int i = 0; i < WPR; ++i) { ss += red_ss[grp * WPR + i]; mx = fmaxf(mx, red_mx[grp * WPR + i]); }
+    }
+    // u = bf16(v * rstd) is monotonic in |v| (one rounded multiply, one rounding to bf16), so the largest |u| of the
+    // row is the image of the largest |v|: no second reduction over the normalized values.
+    float rstd = 1.0f, amax = mx;
+    if (MODE != ROW_PLAIN) {
+      rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(ss, static_cast<float>(a.Kv)), 1e-5f)));
+      amax = bf16_bits_to_float(float_to_bf16_bits(__fmul_rn(mx, rstd)));
+    }
+    amax = fmaxf(amax, 1e-5f);
+    const float inv = __fdiv_rn(127.0f, amax);
+
+    // pass 2: normalize, round to bf16, quantize (round-to-nearest-even conversion, saturating pack), row sum of codes
+    int rs = 0;
+    int8_t* xq = a.xq + (live ? row : 0) * a.Kout;
+    unsigned short* uo = a.u_out ? a.u_out + (live ? row : 0) * a.Kout : nullptr;
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi) {
+      const int i = (gi * WPR + sub) * 32 + lane;
+      if (live && i < nvec8) {
+        uint32_t ub[4];
+        int q[8];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float lo = v[gi][2 * e], hi = v[gi][2 * e + 1];
+          if (MODE != ROW_PLAIN) {
+            const __nv_bfloat162 pr = __floats2bfloat162_rn(__fmul_rn(lo, rstd), __fmul_rn(hi, rstd));
+            ub[e] = *reinterpret_cast<const uint32_t*>(&pr);
+            lo = __uint_as_float(ub[e] << 16);
+            hi = __uint_as_float(ub[e] & 0xffff0000u);
+          } else if (a.u_out) {
+            ub[e] = (__float_as_uint(lo) >> 16) | (__float_as_uint(hi) & 0xffff0000u);
+          }
+          q[2 * e] = __float2int_rn(__fmul_rn(lo, inv));
+          q[2 * e + 1] = __float2int_rn(__fmul_rn(hi, inv));
+        }
+        uint2 wd;
+        wd.x = pack_s8x4(q[0], q[1], q[2], q[3]);
+        wd.y = pack_s8x4(q[4], q[5], q[6], q[7]);
+        rs = dp4a_ones(wd.y, dp4a_ones(wd.x, rs));
+        const uint4 ub4 = make_uint4(ub[0], ub[1], ub[2], ub[3]);
+        if (MODE == ROW_VREPEAT) {
+          const int k = 8 * i;
+          const int kvh = k / a.head_dim, e0 = k - kvh * a.head_dim;
+          for (int r = 0; r < a.rep; ++r) {
+            const int ko = (kvh * a.rep + r) * a.head_dim + e0;
+            *reinterpret_cast<uint2*>(xq + ko) = wd;
+            if (uo) *reinterpret_cast<uint4*>(uo + ko) = ub4;
+          }
+        } else {
+          *reinterpret_cast<uint2*>(xq + 8 * i) = wd;
+          if (uo) *reinterpret_cast<uint4*>(uo + 8 * i) = ub4;
+        }
+      }
+    }
+    rs = warp_sum_i(rs);
+    if (WPR > 1) {
+      if (lane == 0) red_rs[warp] = rs;
+      __syncthreads();
+      rs = 0;
+#pragma unroll
+      for (int i = 0; i < WPR; ++i) rs += red_rs[grp * WPR + i];
+    }
+    if (live && sub == 0 && lane == 0) {
+      a.absmax[row] = amax;
+      if (a.rowsum) a.rowsum[row] = rs * a.rep;
+    }
+    if constexpr (PREFETCH) {
+#pragma unroll
+      for (int i = 0; i < NRAW; ++i) raw[i] = nxt[i];
+    }
   }
 }
+
+int sm_count();
 
 template <int MODE, int WPR, int NG>
 bitrl_status launch_row_reg(const RowArgs& a, int T, cudaStream_t st) {
   const int rows_per_cta = ROW_THREADS / 32 / WPR;
-  BITRL_CUDA(launch_pdl(row_quant_reg_kernel<MODE, WPR, NG>, dim3((T + rows_per_cta - 1) / rows_per_cta), dim3(ROW_THREADS),
-                        0, st, a, T));
+  const int row_groups = (T + rows_per_cta - 1) / rows_per_cta;
+  // persistent: as many CTAs as are resident at once, each walking its rows with the next row's loads in flight
+  static int per_sm = 0;
+  if (per_sm == 0) {
+    int n = 0;
+    BITRL_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, row_quant_reg_kernel<MODE, WPR, NG>, ROW_THREADS, 0));
+    per_sm = n > 0 ? n : 1;
+  }
+  // The gate producer reads 4 F bytes per row from a tensor larger than L2 and gains from the prefetch (37 -> 27 us at
+  // T = 4096); the others read a row that the preceding GEMM left in L2 and run best with one row group per CTA.
+  int grid = MODE == ROW_RELU2 ? sm_count() * per_sm : row_groups;
+  if (grid > row_groups) grid = row_groups;
+  BITRL_CUDA(launch_pdl(row_quant_reg_kernel<MODE, WPR, NG>, dim3(grid), dim3(ROW_THREADS), 0, st, a, T));
   count_launch(1);
   return BITRL_OK;
 }
