@@ -111,7 +111,8 @@ bitrl_status launch_heads_t(const HeadsArgs& a, int n_heads, cudaStream_t st) {
 
 bitrl_status launch_heads(const HeadsArgs& a, int n_heads, cudaStream_t st) {
   // few states: small tiles so that more SMs share the first layer's weights stream; many: larger tiles re-read it less
-  return a.B > 1024 ? launch_heads_t<8>(a, n_heads, st) : launch_heads_t<4>(a, n_heads, st);
+  if (a.B > 1024) return launch_heads_t<8>(a, n_heads, st);
+  return a.B > 256 ? launch_heads_t<4>(a, n_heads, st) : launch_heads_t<2>(a, n_heads, st);
 }
 
 // GAE: one thread per environment walks its trajectory backwards.

@@ -190,7 +190,7 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, i
     }
   };
 
-  constexpr bool PREFETCH = MODE == ROW_RELU2;  // see launch_row_reg
+  constexpr bool PREFETCH = MODE == ROW_RELU2 || MODE == ROW_PLAIN;  // see launch_row_reg
   uint4 raw[NRAW], nxt[PREFETCH ? NRAW : 1];
   long long row = static_cast<long long>(blockIdx.x) * ROWS + grp;
   const long long stride = static_cast<long long>(gridDim.x) * ROWS;
@@ -217,7 +217,7 @@ __global__ void __launch_bounds__(ROW_THREADS) row_quant_reg_kernel(RowArgs a, i
           v[gi][2 * e + 1] = __uint_as_float(rw[e] & 0xffff0000u);
         }
         if (MODE == ROW_RELU2) {
-          const uint4 rawu = raw[MODE == ROW_RELU2 ? NG + gi : gi];  // ROW_RELU2 always prefetches
+          const uint4 rawu = raw[MODE == ROW_RELU2 ? NG + gi : gi];  // the gate producer always prefetches
           const uint32_t ru[4] = {rawu.x, rawu.y, rawu.z, rawu.w};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
@@ -332,7 +332,8 @@ bitrl_status launch_row_reg(const RowArgs& a, int T, cudaStream_t st) {
   }
   // The gate producer reads 4 F bytes per row from a tensor larger than L2 and gains from the prefetch (37 -> 27 us at
   // T = 4096); the others read a row that the preceding GEMM left in L2 and run best with one row group per CTA.
-  int grid = MODE == ROW_RELU2 ? sm_count() * per_sm : row_groups;
+  // The plain quantizer reads activations that come from outside the layer (HBM) and prefetches as well.
+  int grid = (MODE == ROW_RELU2 || MODE == ROW_PLAIN) ? sm_count() * per_sm : row_groups;
   if (grid > row_groups) grid = row_groups;
   BITRL_CUDA(launch_pdl(row_quant_reg_kernel<MODE, WPR, NG>, dim3(grid), dim3(ROW_THREADS), 0, st, a, T));
   count_launch(1);
