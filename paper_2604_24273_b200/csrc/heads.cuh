@@ -55,17 +55,24 @@ __global__ void __launch_bounds__(HEAD_THREADS) heads_forward_kernel(const __gri
     for (int s = 0; s < SB; ++s) acc[s] = 0.0f;
     const float* w = hp.W1t + static_cast<size_t>(q) * kq * a.H1 + j;
     const float* x = hs + q * kq;
-#pragma unroll 2
-    for (int k = 0; k < kq; k += 4) {
-      const float w0 = w[static_cast<size_t>(k) * a.H1], w1 = w[static_cast<size_t>(k + 1) * a.H1],
-                  w2 = w[static_cast<size_t>(k + 2) * a.H1], w3 = w[static_cast<size_t>(k + 3) * a.H1];
+    // Every CTA reads the same weights: each starts at its own offset into the input range (and wraps), so that the
+    // CTAs do not all ask the same L2 lines at the same moment.
+    const int k_rot = static_cast<int>((blockIdx.x * 37u + blockIdx.y * 11u) % static_cast<unsigned>(kq / 4)) * 4;
+#pragma unroll 1
+    for (int pass = 0; pass < 2; ++pass) {
+      const int k_lo = pass == 0 ? k_rot : 0, k_hi = pass == 0 ? kq : k_rot;
+#pragma unroll(SB <= 4 ? 8 : 2)
+      for (int k = k_lo; k < k_hi; k += 4) {
+        const float w0 = w[static_cast<size_t>(k) * a.H1], w1 = w[static_cast<size_t>(k + 1) * a.H1],
+                    w2 = w[static_cast<size_t>(k + 2) * a.H1], w3 = w[static_cast<size_t>(k + 3) * a.H1];
 #pragma unroll
-      for (int s = 0; s < SB; ++s) {
-        const float4 xv = *reinterpret_cast<const float4*>(x + s * a.d + k);
-        acc[s] = fmaf(xv.x, w0, acc[s]);
-        acc[s] = fmaf(xv.y, w1, acc[s]);
-        acc[s] = fmaf(xv.z, w2, acc[s]);
-        acc[s] = fmaf(xv.w, w3, acc[s]);
+        for (int s = 0; s < SB; ++s) {
+          const float4 xv = *reinterpret_cast<const float4*>(x + s * a.d + k);
+          acc[s] = fmaf(xv.x, w0, acc[s]);
+          acc[s] = fmaf(xv.y, w1, acc[s]);
+          acc[s] = fmaf(xv.z, w2, acc[s]);
+          acc[s] = fmaf(xv.w, w3, acc[s]);
+        }
       }
     }
 #pragma unroll
