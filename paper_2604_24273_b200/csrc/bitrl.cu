@@ -562,7 +562,8 @@ bitrl_status bitrl_gae(const float* rewards, const float* values, const float* d
   if (T < 1 || E < 1) return BITRL_ERR_SHAPE;
   bitrl_status s = check_arch();
   if (s != BITRL_OK) return s;
-  BITRL_CUDA(launch_pdl(gae_kernel, dim3((E + 127) / 128), dim3(128), 0, static_cast<cudaStream_t>(stream), rewards, values,
+  BITRL_CUDA(launch_pdl(gae_kernel, dim3((E + GAE_ENVS - 1) / GAE_ENVS), dim3(GAE_CHUNKS * GAE_ENVS), 0,
+                        static_cast<cudaStream_t>(stream), rewards, values,
                         dones, T, E, gamma, lambda, adv, returns));
   count_launch(1);
   return BITRL_OK;

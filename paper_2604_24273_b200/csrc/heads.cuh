@@ -122,39 +122,57 @@ bitrl_status launch_heads(const HeadsArgs& a, int n_heads, cudaStream_t st) {
   return a.B > 256 ? launch_heads_t<4>(a, n_heads, st) : launch_heads_t<2>(a, n_heads, st);
 }
 
-// GAE: one thread per environment walks its trajectory backwards.
-//   delta_t = r_t + gamma V_{t+1} (1 - done_t) - V_t ;  A_t = delta_t + gamma lambda (1 - done_t) A_{t+1}
-__global__ void gae_kernel(const float* __restrict__ r, const float* __restrict__ v, const float* __restrict__ done, int T,
-                           int E, float gamma, float lam, float* __restrict__ adv, float* __restrict__ ret) {
+// GAE.  The recursion A_t = delta_t + c_t A_{t+1} (delta_t = r_t + gamma V_{t+1} (1 - done_t) - V_t, c_t = gamma lambda
+// (1 - done_t)) is a chain of affine maps, and affine maps compose: a trajectory is cut into GAE_CHUNKS pieces, a thread
+// folds its piece into A_first = Q + P * A_after (pass 1), one thread per environment chains the pieces from the end
+// (pass 2), and every thread replays its piece with the now known A_after and writes the outputs (pass 3).  2048 steps
+// become 3 x 64 dependent steps; the order of the fp32 operations differs from the plain backward loop only in how the
+// pieces are joined.
+constexpr int GAE_CHUNKS = 32;
+constexpr int GAE_ENVS = 8;  // environments per CTA
+
+__global__ void __launch_bounds__(GAE_CHUNKS * GAE_ENVS)
+gae_kernel(const float* __restrict__ r, const float* __restrict__ v, const float* __restrict__ done, int T, int E,
+           float gamma, float lam, float* __restrict__ adv, float* __restrict__ ret) {
+  __shared__ float Ps[GAE_CHUNKS][GAE_ENVS], Qs[GAE_CHUNKS][GAE_ENVS], Ain[GAE_CHUNKS][GAE_ENVS];
   pdl_enter();
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= E) return;
+  const int el = threadIdx.x % GAE_ENVS, c = threadIdx.x / GAE_ENVS;
+  const int e = blockIdx.x * GAE_ENVS + el;
+  const bool live = e < E;
+  const int len = (T + GAE_CHUNKS - 1) / GAE_CHUNKS;
+  const int t_lo = c * len, t_hi = min(T, t_lo + len);  // this thread's steps [t_lo, t_hi)
   const float gl = __fmul_rn(gamma, lam);
-  float next_adv = 0.0f, v_next = v[static_cast<size_t>(T) * E + e];
-  // The recursion is serial in t, the loads are not: 32 steps' inputs are requested together.
-  constexpr int CHUNK = 32;
-  for (int t1 = T; t1 > 0; t1 -= CHUNK) {
-    float rr[CHUNK], vv[CHUNK], nn[CHUNK];
-#pragma unroll
-    for (int c = 0; c < CHUNK; ++c) {
-      const int t = t1 - 1 - c;
-      if (t >= 0) {
-        const size_t i = static_cast<size_t>(t) * E + e;
-        rr[c] = r[i]; vv[c] = v[i]; nn[c] = 1.0f - done[i];
-      }
+  float P = 1.0f, Q = 0.0f;
+  if (live) {
+    for (int t = t_hi - 1; t >= t_lo; --t) {
+      const size_t i = static_cast<size_t>(t) * E + e;
+      const float nd = 1.0f - done[i];
+      const float delta = r[i] + gamma * v[i + E] * nd - v[i];
+      const float ct = gl * nd;
+      Q = delta + ct * Q;
+      P = ct * P;
     }
-#pragma unroll
-    for (int c = 0; c < CHUNK; ++c) {
-      const int t = t1 - 1 - c;
-      if (t >= 0) {
-        const size_t i = static_cast<size_t>(t) * E + e;
-        const float delta = rr[c] + gamma * v_next * nn[c] - vv[c];
-        next_adv = delta + gl * nn[c] * next_adv;
-        adv[i] = next_adv;
-        if (ret) ret[i] = next_adv + vv[c];
-        v_next = vv[c];
-      }
+  }
+  Ps[c][el] = P;
+  Qs[c][el] = Q;
+  __syncthreads();
+  if (c == 0) {
+    float a_after = 0.0f;  // A_T = 0
+    for (int cc = GAE_CHUNKS - 1; cc >= 0; --cc) {
+      Ain[cc][el] = a_after;
+      a_after = Qs[cc][el] + Ps[cc][el] * a_after;
     }
+  }
+  __syncthreads();
+  if (!live) return;
+  float next_adv = Ain[c][el];
+  for (int t = t_hi - 1; t >= t_lo; --t) {
+    const size_t i = static_cast<size_t>(t) * E + e;
+    const float nd = 1.0f - done[i], vt = v[i];
+    const float delta = r[i] + gamma * v[i + E] * nd - vt;
+    next_adv = delta + gl * nd * next_adv;
+    adv[i] = next_adv;
+    if (ret) ret[i] = next_adv + vt;
   }
 }
 
