@@ -5,13 +5,15 @@
 // kernel streams all of their packed weights back to back at HBM speed.
 //
 // One persistent CTA per SM.  The work list is the concatenation of all jobs' row tiles (128 rows x all K, one
-// contiguous K/4*128-byte region of the tile layout); every CTA owns a contiguous, byte-balanced range of it.
-//   warp 16     producer: bulk copies (cp.async.bulk) of four consecutive 4 KB (row tile, k block) pieces into a ring of
-//               up to 8 slots of 16 KB - up to 128 KB in flight per SM, independent of the activations, so it runs ahead across jobs
+// contiguous K/4*128-byte region of the tile layout), jobs sorted by K; every CTA owns two ranges of it, balanced in
+// bytes (see GvmArgs::seg).
+//   warp 16     producer: bulk copies (cp.async.bulk) of eight consecutive 4 KB (row tile, k block) pieces into a ring
+//               of 32 KB slots - 128 to 192 KB in flight per SM, independent of the activations, so it runs ahead across jobs
 //   warps 0-15  consumers in two groups of 8: warp w of a group owns rows 16w..16w+15 of the row tile, the group every
 //               other 4 KB piece of the K range (sixteen warps hide the shared-memory and MMA latencies that eight
-//               leave exposed); the two partial sums meet in shared memory once per row tile.  The 2-bit codes are
-//               decoded by shift+mask straight into the A fragments of a warp-level integer MMA
+//               leave exposed); the two partial sums meet in shared memory once per row tile, behind a barrier of the
+//               two warps that share the rows.  The 2-bit codes are masked (not shifted) straight into the A
+//               fragments of a warp-level integer MMA
 //               (mma.sync m16n8k32, A = unsigned codes, B = signed int8 activations of 8 tokens, int32 accumulate):
 //               the same instruction count serves 1 to 8 tokens (two MMAs per k step for 9 to 16), so the kernel
 //               stays memory-bound where a dp4a loop would be ALU-bound from M = 4 on.
