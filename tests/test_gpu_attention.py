@@ -96,6 +96,23 @@ def test_attention_ragged_states(oracle_mod, B, n_states, seed):
     assert torch.equal(att, att2) and torch.equal(att, att3)
 
 
+def test_attention_full_size_as_benchmarked(oracle_mod, B):
+    """The benchmark's shapes: 128 states x 32 tokens (T = 4096) and 128 ragged states of 15-40 tokens, 20/5 heads of
+    128, every output against the oracle."""
+    nh, nkv, hd = 20, 5, 128
+    qkv = inputs.activations(4096, (nh + 2 * nkv) * hd, 7900)
+    att = B.attention(qkv.cuda(), 32, nh, nkv, hd, THETA)
+    B.poll_status()
+    check_attention(bits(att), oracle_mod.attention(bits(qkv), 32, nh, nkv, hd, THETA), bits(qkv), nh, nkv, hd)
+    off = inputs.state_offsets(128, 7000)
+    T = int(off[-1])
+    qkv = inputs.activations(T, (nh + 2 * nkv) * hd, 7901)
+    o32, max_len = dev_states(off)
+    att = B.attention(qkv.cuda(), (o32, inputs.STATE_TOKENS_MAX), nh, nkv, hd, THETA)
+    B.poll_status()
+    check_attention(bits(att), oracle_mod.attention(bits(qkv), off.numpy(), nh, nkv, hd, THETA), bits(qkv), nh, nkv, hd)
+
+
 def test_attention_other_theta_and_determinism(oracle_mod, B):
     nh, nkv, hd, S = 4, 2, 128, 24
     qkv = inputs.activations(2 * S, (nh + 2 * nkv) * hd, 7400, outliers=False)
