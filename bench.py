@@ -493,6 +493,21 @@ def run_ours(args):
         mss = time_graph(gs, sub_steps, args.warmup, 1) / sub_steps
         extra["agent_step_128_states_x32_tokens"] = {"ms": mss, "states_per_s": 128.0 / (mss * 1e-3), "launches": ls}
         del gs
+        # the paper's own operating point: ONE environment, one state of 32 tokens per step (latency, not throughput)
+        h_one = inputs.activations(32, 2560, 6002).to(dev)
+        h_one_out = torch.empty_like(h_one)
+        pooled_one = torch.empty((1, 2560), dtype=torch.bfloat16, device=dev)
+        ws_one = torch.empty((enc.states_workspace_bytes(32, 32),), dtype=torch.uint8, device=dev)
+
+        def agent_step_one():
+            enc.forward_states(h_one, 32, h_out=h_one_out, pooled=pooled_one, workspace=ws_one)
+            return bitrl.heads_forward(pooled_one, heads)
+
+        g1s, l1s = capture(agent_step_one)
+        ms1s = time_graph(g1s, sub_steps, args.warmup, 1) / sub_steps
+        extra["agent_step_1_state_x32_tokens"] = {"ms": ms1s, "launches": l1s,
+                                                  "context": "the paper reports 24.8 ms median per step on a Raspberry Pi 4"}
+        del g1s
         r, v, dn = (t.to(dev) for t in inputs.rollout(2048, 128, 8300))
         batch = [t.to(dev) for t in inputs.ppo_batch(64, n_act, 8400)]
 

@@ -508,8 +508,8 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
         const int kps = (kblocks + sp - 1) / sp;
         if ((kblocks + kps - 1) / kps != sp) continue;  // this count would leave an empty split
         const long long waves = (tiles * sp + sms - 1) / sms;
-        // a split launch pays for clearing the scratch and for the finishing kernel (about 3 us)
-        const long long cost = waves * kps * per_kb + (sp > 1 ? 6000 : 0);
+        // a split launch pays for clearing the scratch and for the finishing kernel (about 5 us in a chain of dependent launches)
+        const long long cost = waves * kps * per_kb + (sp > 1 ? 10000 : 0);
         if (best < 0 || cost <= best) { best = cost; tok = cand[i]; splits = sp; }  // ties go to the narrower tile
       }
     }
