@@ -520,3 +520,30 @@ def test_encoder_full_width_two_blocks_teacher_forced(oracle_mod, B):
         h, acc = B.bitlinear_forward_q(down_l, xq, a, rs, residual=h, want_acc=True)
         assert np.array_equal(acc.cpu().numpy()[rows], oracle_mod.contract(xq.cpu().numpy()[rows], cpu[3][0]))
     assert torch.equal(out, h)
+
+
+@pytest.mark.parametrize("M", [1, 8, 40])
+def test_zero_and_tiny_token_rows(oracle_mod, B, M):
+    """Degenerate activations: an all-zero token (absmax clamps to 1e-5, every code and output is zero), a token of
+    tiny values below the clamp, and a token with a single non-zero element, through the streaming kernel (M <= 16) and
+    the GEMM (M = 40), and through the RMSNorm producer."""
+    K, N = 640, 384
+    W, Wq, g, _, _, lin = layer(oracle_mod, B, N, K, 11)
+    x = inputs.activations(M, K, 2950 + M).float()
+    x[0] = 0.0
+    if M > 2:
+        x[1] = 1e-7
+        x[2] = 0.0
+        x[2, 5] = -3.0
+    x = x.to(torch.bfloat16)
+    ref = oracle_mod.bitlinear(inputs.bf16_bits(x), Wq, g)
+    y, xq, a, acc = B.bitlinear_forward_debug(lin, x.cuda(), B.OUT_BF16)
+    B.poll_status()
+    assert np.array_equal(xq.cpu().numpy(), ref["xq"]) and not xq[0].any()
+    assert np.array_equal(a.cpu().numpy(), ref["absmax"]) and a[0].item() == np.float32(1e-5)
+    assert np.array_equal(acc.cpu().numpy(), ref["acc"])
+    assert np.array_equal(gpu_bf16_bits(y), ref["ybf16"]) and not gpu_bf16_bits(y)[0].any()
+    xq2, a2, rs2, u = B.rmsnorm_quant(x.cuda(), want_u=True)
+    B.poll_status()
+    check_producer(oracle_mod, xq2, a2, rs2, u, oracle_mod.rmsnorm_bf16(inputs.bf16_bits(x)))
+    assert not xq2[0].any() and rs2[0].item() == 0
