@@ -53,6 +53,10 @@ def _L():
         _lib.oracle_ternarize.argtypes = [_vp, _i64, _f32, _vp]
         _lib.oracle_w8_quantize.argtypes = [_vp, _i64, _vp, _vp]
         _lib.oracle_w8_quantize.restype = None
+        _lib.oracle_w4_quantize.argtypes = [_vp, _i64, _vp, _vp]
+        _lib.oracle_w4_quantize.restype = None
+        _lib.oracle_w4_pack.argtypes = [_vp, _i64, _i64, _vp]
+        _lib.oracle_w4_pack.restype = None
         _lib.oracle_pack.argtypes = [_vp, _i64, _i64, _vp]
         _lib.oracle_unpack.argtypes = [_vp, _i64, _i64, _vp]
         _lib.oracle_quant_act.argtypes = [_vp, _i64, _i64, _vp, _vp]
@@ -119,6 +123,25 @@ def w8_quantize(W: np.ndarray):
     scale = np.zeros((1,), np.float32)
     _L().oracle_w8_quantize(_p(W), W.size, _p(Wq), _p(scale))
     return Wq, np.float32(scale[0])
+
+
+def w4_quantize(W: np.ndarray):
+    """Symmetric absmax int4 quantization (one scale per matrix).  Returns (W_q int8 with values in [-8, 7], scale)."""
+    W = _c(W, np.float32)
+    Wq = np.empty(W.shape, np.int8)
+    scale = np.zeros((1,), np.float32)
+    _L().oracle_w4_quantize(_p(W), W.size, _p(Wq), _p(scale))
+    return Wq, np.float32(scale[0])
+
+
+def w4_pack(Wq: np.ndarray) -> np.ndarray:
+    """Two biased codes (q + 8) per byte, even k in the low nibble."""
+    Wq = _c(Wq, np.int8)
+    N, K = Wq.shape
+    assert K % 2 == 0
+    out = np.empty((N, K // 2), np.uint8)
+    _L().oracle_w4_pack(_p(Wq), N, K, _p(out))
+    return out
 
 
 def pack(Wq: np.ndarray) -> np.ndarray:

@@ -161,6 +161,36 @@ void oracle_w8_quantize(const float* W, int64_t count, int8_t* Wq, float* scale)
   *scale = a / 127.0f;
 }
 
+// Four-bit weights (the "INT4 critic" row of the same table), same reading with 7 in place of 127:
+//   a = max(max|W|, 1e-20),  W_q = clip(rint(W * (7 / a)), -8, 7),  scale = a / 7.
+// Codes are returned as int8 values in [-8, 7]; the layer is again the BitLinear formula with these codes and `scale`.
+void oracle_w4_quantize(const float* W, int64_t count, int8_t* Wq, float* scale) {
+  float a = 0.0f;
+  for (int64_t i = 0; i < count; ++i) {
+    const float v = std::fabs(W[i]);
+    if (v > a) a = v;
+  }
+  if (a < 1e-20f) a = 1e-20f;
+  const float inv = 7.0f / a;
+  for (int64_t i = 0; i < count; ++i) {
+    float q = std::nearbyintf(W[i] * inv);
+    if (q > 7.0f) q = 7.0f;
+    if (q < -8.0f) q = -8.0f;
+    Wq[i] = static_cast<int8_t>(q);
+  }
+  *scale = a / 7.0f;
+}
+
+// Packed form of the four-bit codes: byte j of row n holds k = 2j (low nibble) and k = 2j+1 (high nibble), each as the
+// biased code q + 8 in [0, 15].
+void oracle_w4_pack(const int8_t* Wq, int64_t N, int64_t K, uint8_t* packed) {
+  for (int64_t n = 0; n < N; ++n)
+    for (int64_t j = 0; j < K / 2; ++j) {
+      const unsigned lo = static_cast<unsigned>(Wq[n * K + 2 * j] + 8), hi = static_cast<unsigned>(Wq[n * K + 2 * j + 1] + 8);
+      packed[n * (K / 2) + j] = static_cast<uint8_t>(lo | (hi << 4));
+    }
+}
+
 // acc[m,n] = sum_k x_q[m,k] * W_q[n,k] in int32 (exact; |acc| <= 127*K for ternary, 127*128*K for 8-bit weights).
 void oracle_contract(const int8_t* xq, const int8_t* Wq, int64_t M, int64_t N, int64_t K, int32_t* acc,
                      int threads) {

@@ -56,3 +56,33 @@ def test_w8a8_layer_against_fp64_and_integer_library_matmuls():
     big = np.full((1, 256), 127, np.int8)
     accb = oracle.contract(big, np.full((3, 256), 127, np.int8))
     assert accb[0, 0] == 127 * 127 * 256
+
+
+def test_w4_codes_definition_error_bound_and_packing():
+    """absmax element -> +-7, codes in [-8, 7] and equal to rint(7 W / max|W|) in fp64 away from ties, error at most
+    half a step; the packed byte holds k even in the low nibble as q + 8 (checked against numpy bit operations)."""
+    W = inputs.master_weights(64, 96, 9110).numpy()
+    Wq, scale = oracle.w4_quantize(W)
+    a = np.abs(W).max()
+    assert Wq.min() >= -8 and Wq.max() <= 7 and np.abs(Wq.astype(np.int32)).max() == 7
+    assert scale == np.float32(a) / np.float32(7.0)
+    t = W.astype(np.float64) * 7.0 / float(a)
+    away = np.abs(t - np.floor(t) - 0.5) > 1e-4
+    assert away.mean() > 0.99 and np.array_equal(Wq[away], np.rint(t[away]).astype(np.int8))
+    assert np.all(np.abs(W.astype(np.float64) - Wq.astype(np.float64) * float(scale)) <= float(scale) * 0.5 * (1 + 1e-5))
+    packed = oracle.w4_pack(Wq)
+    assert packed.shape == (64, 48)
+    lo = (packed & 0x0F).astype(np.int32) - 8
+    hi = (packed >> 4).astype(np.int32) - 8
+    assert np.array_equal(lo, Wq[:, 0::2]) and np.array_equal(hi, Wq[:, 1::2])
+
+
+def test_w4a8_layer_against_library_matmuls():
+    W = inputs.master_weights(32, 128, 9111).numpy()
+    Wq, scale = oracle.w4_quantize(W)
+    x = inputs.activations(3, 128, 9112)
+    ref = oracle.bitlinear(inputs.bf16_bits(x), Wq, scale)
+    acc_t = torch.from_numpy(ref["xq"].astype(np.int32)) @ torch.from_numpy(Wq.astype(np.int32)).T
+    assert np.array_equal(ref["acc"], acc_t.numpy())
+    dense = (ref["xq"].astype(np.float64) * (ref["absmax"].astype(np.float64)[:, None] / 127.0)) @ (Wq.astype(np.float64) * float(scale)).T
+    np.testing.assert_allclose(ref["y64"], dense, rtol=1e-12, atol=1e-300)
