@@ -255,6 +255,22 @@ BITRL_API bitrl_status bitrl_w8a8_forward_debug(const int8_t* wq, const float* s
                                                 size_t workspace_bytes, int8_t* xq_out, float* absmax_out,
                                                 int32_t* acc_out, void* stream);
 
+/* ---- W4A8 layer: the "INT4 critic" of the same table (the paper names the precision only) -------------------------
+ * Same reading with 7 in place of 127:  a = max(max|W|, 1e-20),  W_q = clip(rint(W * (7 / a)), -8, 7),  scale = a / 7,
+ * acc and y as for W8A8.  packed: dev uint8 [N, K/2], byte j of row n = (W_q[n,2j] + 8) | (W_q[n,2j+1] + 8) << 4.
+ * bitrl_w4_quantize: W dev fp32 [N,K] -> packed and scale (dev fp32 [2]: scale[0] the result, scale[1] scratch).
+ * bitrl_w4a8_forward: M <= BITRL_GEMV_MAX_M streams the packed bytes once (dp4a; no workspace); larger M expands the
+ * codes to int8 in the workspace and runs the W8A8 GEMM on them.  workspace >= bitrl_w4a8_workspace_bytes(M, K, N). */
+BITRL_API bitrl_status bitrl_w4_quantize(const float* W, int32_t N, int32_t K, uint8_t* packed, float* scale, void* stream);
+BITRL_API size_t bitrl_w4a8_workspace_bytes(int32_t M, int32_t K, int32_t N);
+BITRL_API bitrl_status bitrl_w4a8_forward(const uint8_t* packed, const float* scale, const void* x, int32_t M, int32_t K,
+                                          int32_t N, void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes,
+                                          void* stream);
+BITRL_API bitrl_status bitrl_w4a8_forward_debug(const uint8_t* packed, const float* scale, const void* x, int32_t M,
+                                                int32_t K, int32_t N, void* y, int32_t out_dtype, void* workspace,
+                                                size_t workspace_bytes, int8_t* xq_out, float* absmax_out,
+                                                int32_t* acc_out, void* stream);
+
 /* ---- status ----------------------------------------------------------------------------------------- */
 /* Synchronizes `stream`, then reads and clears the device status word.  BITRL_OK, BITRL_ERR_TIMEOUT (a kernel
  * wait expired; results of that launch are invalid) or BITRL_ERR_CUDA. */

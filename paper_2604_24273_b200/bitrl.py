@@ -8,7 +8,7 @@ The functions mirror the C names without the ``bitrl_`` prefix:
 ``pack_ternary``, ``Linear`` (create/destroy), ``quant_act``, ``bitlinear_forward``, ``bitlinear_forward_debug``,
 ``bitlinear_forward_q``, ``rmsnorm_quant``, ``vrepeat_rmsnorm_quant``, ``relu2gate_rmsnorm_quant``, ``attention``,
 ``pool_last_token``, ``Encoder`` (``forward``, ``forward_states``), ``heads_forward``, ``gae``, ``ppo_loss``,
-``w8_quantize``, ``w8a8_forward``,
+``w8_quantize``, ``w8a8_forward``, ``w4_quantize``, ``w4a8_forward``,
 ``poll_status``.
 """
 from __future__ import annotations
@@ -71,6 +71,10 @@ EXPORTS = {
     "bitrl_w8a8_workspace_bytes": (_sz, [_i32, _i32]),
     "bitrl_w8a8_forward": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp]),
     "bitrl_w8a8_forward_debug": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp, _vp, _vp, _vp]),
+    "bitrl_w4_quantize": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp]),
+    "bitrl_w4a8_workspace_bytes": (_sz, [_i32, _i32, _i32]),
+    "bitrl_w4a8_forward": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp]),
+    "bitrl_w4a8_forward_debug": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp, _vp, _vp, _vp]),
     "bitrl_selftest_wait_timeout": (_i32, [ctypes.c_int64, _vp]),
     "bitrl_poll_status": (_i32, [_vp]),
     "bitrl_last_timeout_stage": (_i32, []),
@@ -396,6 +400,41 @@ def w8a8_forward(wq: torch.Tensor, scale: torch.Tensor, x: torch.Tensor, out_dty
     _check(lib().bitrl_w8a8_forward_debug(_ptr(wq), _ptr(scale), _ptr(x), M, K, N, _ptr(y), out_dtype, _ptr(workspace),
                                           workspace.numel(), _ptr(xq), _ptr(a), _ptr(acc), _stream()),
            "bitrl_w8a8_forward_debug")
+    return y, xq, a, acc
+
+
+def w4_quantize(W: torch.Tensor):
+    """W CUDA fp32 [N,K] -> (packed uint8 [N,K/2], scale fp32 [2]; scale[0] is the scale)."""
+    _dev(W, torch.float32, "W")
+    N, K = W.shape
+    packed = torch.empty((N, K // 2), dtype=torch.uint8, device=W.device)
+    scale = torch.empty((2,), dtype=torch.float32, device=W.device)
+    _check(lib().bitrl_w4_quantize(_ptr(W), N, K, _ptr(packed), _ptr(scale), _stream()), "bitrl_w4_quantize")
+    return packed, scale
+
+
+def w4a8_forward(packed: torch.Tensor, scale: torch.Tensor, x: torch.Tensor, out_dtype: int = OUT_BF16,
+                 debug: bool = False, y: torch.Tensor | None = None, workspace: torch.Tensor | None = None):
+    """y = W4A8(x).  With debug=True returns (y, x_q, absmax, acc)."""
+    _dev(packed, torch.uint8, "packed")
+    _dev(scale, torch.float32, "scale")
+    _dev(x, torch.bfloat16, "x")
+    M, K = x.shape
+    N = packed.shape[0]
+    if y is None:
+        y = _out(M, N, out_dtype, x.device)
+    if workspace is None:
+        workspace = torch.empty((max(int(lib().bitrl_w4a8_workspace_bytes(M, K, N)), 16),), dtype=torch.uint8, device=x.device)
+    if not debug:
+        _check(lib().bitrl_w4a8_forward(_ptr(packed), _ptr(scale), _ptr(x), M, K, N, _ptr(y), out_dtype, _ptr(workspace),
+                                        workspace.numel(), _stream()), "bitrl_w4a8_forward")
+        return y
+    xq = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    a = torch.empty((M,), dtype=torch.float32, device=x.device)
+    acc = torch.empty((M, N), dtype=torch.int32, device=x.device)
+    _check(lib().bitrl_w4a8_forward_debug(_ptr(packed), _ptr(scale), _ptr(x), M, K, N, _ptr(y), out_dtype, _ptr(workspace),
+                                          workspace.numel(), _ptr(xq), _ptr(a), _ptr(acc), _stream()),
+           "bitrl_w4a8_forward_debug")
     return y, xq, a, acc
 
 

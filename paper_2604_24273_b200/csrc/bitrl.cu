@@ -76,6 +76,7 @@ static bitrl_status check_arch() {
 #include "attention.cuh"
 #include "heads.cuh"
 #include "gemm_w8.cuh"
+#include "w4.cuh"
 
 using namespace bitrl;
 
@@ -633,6 +634,59 @@ bitrl_status bitrl_w8a8_forward_debug(const int8_t* wq, const float* scale, cons
                                       void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes, int8_t* xq_out,
                                       float* absmax_out, int32_t* acc_out, void* stream) {
   return w8a8_impl(wq, scale, x, M, K, N, y, out_dtype, workspace, workspace_bytes, xq_out, absmax_out, acc_out, stream);
+}
+
+// ---- W4A8 layer (INT4 critic) -----------------------------------------------------------------------------------
+
+bitrl_status bitrl_w4_quantize(const float* W, int32_t N, int32_t K, uint8_t* packed, float* scale, void* stream) {
+  if (!W || !packed || !scale) return BITRL_ERR_NULL;
+  if (!shape_ok(N, K)) return BITRL_ERR_SHAPE;
+  if (!aligned16(W) || !aligned16(packed)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  return launch_w4_quantize(W, N, K, packed, scale, static_cast<cudaStream_t>(stream));
+}
+
+size_t bitrl_w4a8_workspace_bytes(int32_t M, int32_t K, int32_t N) {
+  if (M < 1 || K < 1 || N < 1) return 0;
+  if (gemv_w8_fits(M, K)) return 0;
+  return bitrl_w8a8_workspace_bytes(M, K) + align_up(static_cast<size_t>(N) * K, 256);
+}
+
+static bitrl_status w4a8_impl(const uint8_t* packed, const float* scale, const void* x, int32_t M, int32_t K, int32_t N,
+                              void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes, int8_t* xq_out,
+                              float* absmax_out, int32_t* acc_out, void* stream) {
+  if (!packed || !scale || !x || !y) return BITRL_ERR_NULL;
+  if (M < 1 || !shape_ok(N, K)) return BITRL_ERR_SHAPE;
+  if (out_dtype != BITRL_OUT_F32 && out_dtype != BITRL_OUT_BF16) return BITRL_ERR_DTYPE;
+  if (!aligned16(packed) || !aligned16(x) || !aligned16(y) || !aligned16(workspace)) return BITRL_ERR_ALIGN;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (gemv_w8_fits(M, K))
+    return launch_gemv_w4(packed, scale, N, K, x, M, y, out_dtype, xq_out, absmax_out, acc_out, st);
+  if (!workspace || workspace_bytes < bitrl_w4a8_workspace_bytes(M, K, N)) return BITRL_ERR_WORKSPACE;
+  unsigned char* b = static_cast<unsigned char*>(workspace);
+  int8_t* xq = reinterpret_cast<int8_t*>(b);
+  float* absmax = reinterpret_cast<float*>(b + align_up(static_cast<size_t>(M) * K, 256));
+  int8_t* w8 = reinterpret_cast<int8_t*>(b + bitrl_w8a8_workspace_bytes(M, K));
+  if ((s = launch_quant_act(x, M, K, xq, absmax, nullptr, st)) != BITRL_OK) return s;
+  if ((s = launch_w4_expand(packed, N, K, w8, st)) != BITRL_OK) return s;
+  if ((s = launch_gemm_w8(w8, scale, N, K, xq, absmax, M, y, out_dtype, nullptr, acc_out, st)) != BITRL_OK) return s;
+  if (xq_out) BITRL_CUDA(cudaMemcpyAsync(xq_out, xq, static_cast<size_t>(M) * K, cudaMemcpyDeviceToDevice, st));
+  if (absmax_out) BITRL_CUDA(cudaMemcpyAsync(absmax_out, absmax, static_cast<size_t>(M) * 4, cudaMemcpyDeviceToDevice, st));
+  return BITRL_OK;
+}
+
+bitrl_status bitrl_w4a8_forward(const uint8_t* packed, const float* scale, const void* x, int32_t M, int32_t K, int32_t N,
+                                void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes, void* stream) {
+  return w4a8_impl(packed, scale, x, M, K, N, y, out_dtype, workspace, workspace_bytes, nullptr, nullptr, nullptr, stream);
+}
+
+bitrl_status bitrl_w4a8_forward_debug(const uint8_t* packed, const float* scale, const void* x, int32_t M, int32_t K,
+                                      int32_t N, void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes,
+                                      int8_t* xq_out, float* absmax_out, int32_t* acc_out, void* stream) {
+  return w4a8_impl(packed, scale, x, M, K, N, y, out_dtype, workspace, workspace_bytes, xq_out, absmax_out, acc_out, stream);
 }
 
 // ---- self-test of the bounded-wait / status-word path ----
