@@ -426,6 +426,42 @@ def run_ours(args):
             del g
         del w8
 
+        # the INT4 critic's W4A8 layer: streaming kernel at M = 1 over eight 2560 -> 13824 matrices (141 MB packed),
+        # and the whole layer at M = 4096 (int8 expansion into the workspace, then the W8A8 GEMM)
+        w4 = []
+        for i in range(8):
+            gen.manual_seed(1600 + i)
+            w4.append(bitrl.w4_quantize(torch.randn(13824, 2560, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W))
+        xd = inputs.activations(1, 2560, 2001).to(dev)
+        yd = torch.empty((1, 13824), dtype=torch.bfloat16, device=dev)
+
+        def w4_sweep():
+            for p4, sc4 in w4:
+                bitrl.w4a8_forward(p4, sc4, xd, bitrl.OUT_BF16, y=yd)
+
+        g, lc = capture(w4_sweep)
+        ms = time_graph(g, sub_steps, args.warmup, 1) / sub_steps
+        gbs = 8 * 13824 * 2560 / 2 / (ms * 1e-3) / 1e9
+        extra["w4a8_m1_sweep_8x_k2560_n13824"] = {"GBps_of_packed_bytes": gbs, "us_per_matrix": ms * 1e3 / 8,
+                                                   "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "launches": lc}
+        del g, w4
+        gen.manual_seed(1700)
+        p4, sc4 = bitrl.w4_quantize(torch.randn(6912, 2560, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W)
+        xs = [inputs.activations(M, 2560, 2400 + i).to(dev) for i in range(4)]
+        y = torch.empty((M, 6912), dtype=torch.bfloat16, device=dev)
+        ws = torch.empty((int(bitrl.lib().bitrl_w4a8_workspace_bytes(M, 2560, 6912)),), dtype=torch.uint8, device=dev)
+
+        def w4_layer():
+            for i in range(12):
+                bitrl.w4a8_forward(p4, sc4, xs[i % 4], bitrl.OUT_BF16, y=y, workspace=ws)
+
+        g, _ = capture(w4_layer)
+        ms = time_graph(g, sub_steps, args.warmup, 1)
+        tops = 2.0 * M * 6912 * 2560 * 12 * sub_steps / (ms * 1e-3) / 1e12
+        extra["w4a8_m4096_k2560_n6912"] = {"layer": {"TOPS": tops, "us": ms * 1e3 / (sub_steps * 12),
+                                                     "frac_of_int8_peak": tops / i8_peak}}
+        del g, xs, y, ws
+
         # configs[2]: batched state encoding, M = 64 and 256 (one token per state), the whole layer per call
         for M in (64, 256):
             for K, N in ((2560, 6912), (6912, 2560)):
