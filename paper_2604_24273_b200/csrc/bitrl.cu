@@ -29,6 +29,16 @@ bool gemm_a_in_tmem() {
   return v == 1;
 }
 
+// BITRL_GEMM_PAIR=1 forces the paired-CTA GEMM wherever the shape allows it, 0 forbids it (tuning and fallback knob).
+int gemm_pair_mode() {
+  static int v = -2;
+  if (v == -2) {
+    const char* e = getenv("BITRL_GEMM_PAIR");
+    v = !e ? -1 : (e[0] == '1' ? 1 : 0);
+  }
+  return v;
+}
+
 // BITRL_GEMM_TOK=<64|128|192|224|256> overrides the launcher's choice of token-tile width (for tuning runs).
 int gemm_forced_tok() {
   static int v = -1;

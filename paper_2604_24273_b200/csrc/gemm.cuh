@@ -73,10 +73,18 @@ struct GemmArgs {
   int32_t* part;
 };
 
-template <int GM_TOK, bool A_TMEM>
+// PAIR: two CTAs of a cluster work on one 256-row x TOK-token tile with tcgen05.mma.cta_group::2.  CTA rank r expands
+// weight rows [256 t + 128 r, +128) into its own tensor memory, fetches tokens [TOK/2 * r, +TOK/2) of the tile into its
+// own shared memory and drains its own 128 x TOK slice of the accumulator; rank 0 issues the MMAs.  Per SM this halves
+// the B-operand traffic through shared memory, the binding resource of the single-CTA kernel.  The barriers that gate
+// the MMA (x_full, tmem_empty) are rank 0's and collect the arrivals of both CTAs; the barriers that the MMA's
+// completion releases (x_empty, tmem_full) exist in both CTAs and are reached by one multicast commit.
+template <int GM_TOK, bool A_TMEM, bool PAIR = false>
 __global__ void __launch_bounds__(GM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
-  constexpr uint32_t GM_X_BYTES = GM_TOK * GM_BK;
+  static_assert(!PAIR || A_TMEM, "the paired kernel keeps its weights in tensor memory");
+  static_assert(!PAIR || GM_TOK % 16 == 0, "each CTA holds TOK/2 tokens in whole 8-row swizzle groups");
+  constexpr uint32_t GM_X_BYTES = (PAIR ? GM_TOK / 2 : GM_TOK) * GM_BK;  // this CTA's part of a token tile
   // x_q ring: 128 KB, plus the 48 KB of the shared-memory weight ring when the weights go through tensor memory
   // (4 stages at 256 tokens, 6 at 224, 7 at 192, 11 at 128, 16 at 64).
   constexpr uint32_t GM_X_RING = A_TMEM ? GM_OFF_P - GM_OFF_X : GM_X_RING_BYTES;
@@ -107,6 +115,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kblocks = a.K / GM_BK;
   const int items = a.tiles_total * a.splits;
+  // PAIR: both CTAs of a cluster walk the same items (tiles_n then counts 256-row tiles); rank selects the halves.
+  const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;
+  const int item0 = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+  const int item_step = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
+  const uint32_t x_full_lead = PAIR ? ptx::mapa_u32(bar_x_full, 0) : bar_x_full;        // as seen from either CTA
+  const uint32_t tmem_empty_lead = PAIR ? ptx::mapa_u32(bar_tmem_empty, 0) : bar_tmem_empty;
   auto item_range = [&](int item, int& tile, int& kb0, int& kb1) {
     tile = item / a.splits;
     kb0 = (item - tile * a.splits) * a.kb_per_split;
@@ -114,18 +128,31 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   };
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < GM_XS; ++s) { ptx::mbar_init(bar_x_full + 8 * s, 1 + 4); ptx::mbar_init(bar_x_empty + 8 * s, 1); }
+    // x_full: the producer's expect_tx arrival plus one arrival per expander warp (of both CTAs when paired)
+    for (int s = 0; s < GM_XS; ++s) {
+      ptx::mbar_init(bar_x_full + 8 * s, PAIR ? 1 + 8 : 1 + 4);
+      ptx::mbar_init(bar_x_empty + 8 * s, 1);
+    }
     for (int s = 0; s < GM_PS; ++s) { ptx::mbar_init(bar_p_full + 8 * s, 1); ptx::mbar_init(bar_p_empty + 8 * s, 4); }
-    for (int b = 0; b < 2; ++b) { ptx::mbar_init(bar_tmem_full + 8 * b, 1); ptx::mbar_init(bar_tmem_empty + 8 * b, 4); }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(bar_tmem_full + 8 * b, 1);
+      ptx::mbar_init(bar_tmem_empty + 8 * b, PAIR ? 8 : 4);
+    }
     ptx::mbar_init_fence();
     ptx::tma_prefetch_desc(&tmap_x);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(base + GM_OFF_MISC, 512);
-    ptx::tmem_relinquish();
+    if (PAIR) {
+      ptx::tmem_alloc_pair(base + GM_OFF_MISC, 512);
+      ptx::tmem_relinquish_pair();
+    } else {
+      ptx::tmem_alloc(base + GM_OFF_MISC, 512);
+      ptx::tmem_relinquish();
+    }
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
+  if (PAIR) ptx::cluster_sync_all();  // the peer's barriers are initialised before anything is sent to them
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   pdl_enter();  // barriers and tensor memory are set up; inputs of the preceding kernel are read only from here on
@@ -135,15 +162,22 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int item = blockIdx.x; ok && item < items; item += gridDim.x) {
+      for (int item = item0; ok && item < items; item += item_step) {
         int tile, kb0, kb1;
         item_range(item, tile, kb0, kb1);
         const int tm = tile / a.tiles_n;
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const uint32_t s = it % GM_XS, ph = (it / GM_XS) & 1u;
           if (!ptx::mbar_wait(bar_x_empty + 8 * s, ph ^ 1u)) { report_timeout(GM_WAIT_X_EMPTY); ok = false; break; }
-          ptx::mbar_arrive_expect_tx(bar_x_full + 8 * s, GM_X_BYTES);
-          ptx::tma_load_2d(base + GM_OFF_X + s * GM_X_BYTES, &tmap_x, kb * GM_BK, tm * GM_TOK, bar_x_full + 8 * s);
+          if (PAIR) {
+            // Rank 0 announces the bytes of both halves on its barrier; each CTA's copy reports there.
+            if (rank == 0) ptx::mbar_arrive_expect_tx(bar_x_full + 8 * s, 2 * GM_X_BYTES);
+            ptx::tma_load_2d_pair(base + GM_OFF_X + s * GM_X_BYTES, &tmap_x, kb * GM_BK,
+                                  tm * GM_TOK + static_cast<int>(rank) * (GM_TOK / 2), x_full_lead + 8 * s);
+          } else {
+            ptx::mbar_arrive_expect_tx(bar_x_full + 8 * s, GM_X_BYTES);
+            ptx::tma_load_2d(base + GM_OFF_X + s * GM_X_BYTES, &tmap_x, kb * GM_BK, tm * GM_TOK, bar_x_full + 8 * s);
+          }
         }
       }
     }
@@ -152,10 +186,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int item = blockIdx.x; ok && item < items; item += gridDim.x) {
+      for (int item = item0; ok && item < items; item += item_step) {
         int tile, kb0, kb1;
         item_range(item, tile, kb0, kb1);
-        const int tn = tile % a.tiles_n;
+        const int tn = PAIR ? 2 * (tile % a.tiles_n) + static_cast<int>(rank) : tile % a.tiles_n;
         const uint8_t* wsrc = a.tiles + static_cast<size_t>(tn) * kblocks * TILE_BYTES;
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const uint32_t s = it % GM_PS, ph = (it / GM_PS) & 1u;
@@ -168,27 +202,41 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = ptx::idesc_i8(GM_ROWS, GM_TOK, /*a_signed=*/false, /*b_signed=*/true);
+    // The whole warp walks the loop (waits included) and one elected lane issues: with uniform control flow the
+    // descriptors and addresses stay in uniform registers, which is what the MMA instruction takes its operands from.
+    if (rank == 0) {
+      const uint32_t idesc = ptx::idesc_i8(PAIR ? 2 * GM_ROWS : GM_ROWS, GM_TOK, /*a_signed=*/false, /*b_signed=*/true);
       uint32_t lt = 0;
       uint32_t xs = 0, xph = 0, ws = 0;  // ring slots and phase, advanced without divisions
       bool ok = true;
-      for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++lt) {
+      for (int item = item0; ok && item < items; item += item_step, ++lt) {
         int tile, kb0, kb1;
         item_range(item, tile, kb0, kb1);
         const uint32_t buf = lt & 1u;
-        if (!ptx::mbar_wait(bar_tmem_empty + 8 * buf, ((lt >> 1) & 1u) ^ 1u)) {
-          report_timeout(GM_WAIT_TMEM_EMPTY); ok = false; break;
+        if (!__any_sync(0xffffffffu, ptx::mbar_wait(bar_tmem_empty + 8 * buf, ((lt >> 1) & 1u) ^ 1u))) {
+          if (lane == 0) report_timeout(GM_WAIT_TMEM_EMPTY);
+          ok = false;
+          break;
         }
         const uint32_t d_tmem = tmem_base + buf * GM_TOK_MAX;
         ptx::tc_fence_after_sync();  // orders this tile's MMAs after the epilogue's reads of the accumulator
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!ptx::mbar_wait(bar_x_full + 8 * xs, xph)) { report_timeout(GM_WAIT_X_FULL); ok = false; break; }
+          if (!__any_sync(0xffffffffu, ptx::mbar_wait(bar_x_full + 8 * xs, xph))) {
+            if (lane == 0) report_timeout(GM_WAIT_X_FULL);
+            ok = false;
+            break;
+          }
           // Weights written with tcgen05.st by other threads need the tcgen05 fence on this side of the barrier;
           // TMA data and expander stores to shared memory (already fenced into the async proxy by their writers) do not.
           if (A_TMEM) ptx::tc_fence_after_sync();
           const uint64_t bdesc = ptx::smem_desc_sw128(base + GM_OFF_X + xs * GM_X_BYTES);
-          if (A_TMEM) {
+          if (ptx::elect_one()) {
+          if (PAIR) {
+            const uint32_t a_tmem = tmem_base + a_slot(ws);
+#pragma unroll
+            for (int k4 = 0; k4 < GM_BK / 32; ++k4)
+              ptx::mma_i8_ts_pair(d_tmem, a_tmem + 8 * k4, bdesc + 2 * k4, idesc, (kb != kb0 || k4 != 0) ? 1u : 0u);
+          } else if (A_TMEM) {
             const uint32_t a_tmem = tmem_base + a_slot(ws);
 #pragma unroll
             for (int k4 = 0; k4 < GM_BK / 32; ++k4)
@@ -199,11 +247,19 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
             for (int k4 = 0; k4 < GM_BK / 32; ++k4)
               ptx::mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb != kb0 || k4 != 0) ? 1u : 0u);
           }
-          ptx::mma_commit(bar_x_empty + 8 * xs);  // frees the x_q slot and the weight slot of this k block
+          // frees the x_q slot and the weight slot of this k block (in both CTAs of a pair)
+          if (PAIR) ptx::mma_commit_pair(bar_x_empty + 8 * xs, 3);
+          else ptx::mma_commit(bar_x_empty + 8 * xs);
+          }
+          __syncwarp();
           if (++xs == GM_XS) { xs = 0; xph ^= 1u; }
           if (++ws == WSK) ws = 0;
         }
-        if (ok) ptx::mma_commit(bar_tmem_full + 8 * buf);
+        if (ok && ptx::elect_one()) {
+          if (PAIR) ptx::mma_commit_pair(bar_tmem_full + 8 * buf, 3);
+          else ptx::mma_commit(bar_tmem_full + 8 * buf);
+        }
+        __syncwarp();
       }
     }
   } else if (warp < GM_EPI_WARP0 || warp >= GM_EXPAND2_WARP0) {
@@ -224,7 +280,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     uint32_t it = 0;
     uint32_t ps = 0, pph = 0, ws = 0, xs = 0, xs_old = 0, xph_old = 0;
     bool ok = true;
-    for (int item = blockIdx.x; ok && item < items; item += gridDim.x) {
+    for (int item = item0; ok && item < items; item += item_step) {
       int tile, kb0, kb1;
       item_range(item, tile, kb0, kb1);
       for (int kb = kb0; kb < kb1; ++kb, ++it) {
@@ -273,7 +329,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
         }
         __syncwarp();
         if (lane == 0) {
-          ptx::mbar_arrive(bar_x_full + 8 * xs);
+          if (PAIR) ptx::mbar_arrive_cluster(x_full_lead + 8 * xs);
+          else ptx::mbar_arrive(bar_x_full + 8 * xs);
           ptx::mbar_arrive(bar_p_empty + 8 * ps);
         }
         if (++ps == GM_PS) { ps = 0; pph ^= 1u; }
@@ -291,9 +348,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     const bool f32 = a.out_dtype == BITRL_OUT_F32;
     uint32_t lt = 0;
     bool ok = true;
-    for (int item = blockIdx.x; ok && item < items; item += gridDim.x, ++lt) {
+    for (int item = item0; ok && item < items; item += item_step, ++lt) {
       const int tile = item / a.splits;
-      const int tn = tile % a.tiles_n, tm = tile / a.tiles_n;
+      const int tn = PAIR ? 2 * (tile % a.tiles_n) + static_cast<int>(rank) : tile % a.tiles_n, tm = tile / a.tiles_n;
       const uint32_t buf = lt & 1u;
       const uint32_t sc_addr = base + GM_OFF_TOK + buf * GM_TOK_MAX * 4;
       const uint32_t rs_addr = base + GM_OFF_TOK + 2 * GM_TOK_MAX * 4 + buf * GM_TOK_MAX * 4;
@@ -400,7 +457,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
       }
       ptx::tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(bar_tmem_empty + 8 * buf);
+      if (lane == 0) {
+        if (PAIR) ptx::mbar_arrive_cluster(tmem_empty_lead + 8 * buf);
+        else ptx::mbar_arrive(bar_tmem_empty + 8 * buf);
+      }
     }
   }
 
@@ -408,9 +468,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   __syncwarp();
   ptx::tc_fence_before_sync();
   __syncthreads();
+  if (PAIR) ptx::cluster_sync_all();  // neither CTA leaves (or frees tensor memory) while the other may still reach it
   if (warp == 1) {
     ptx::tc_fence_after_sync();
-    ptx::tmem_dealloc(tmem_base, 512);
+    if (PAIR) ptx::tmem_dealloc_pair(tmem_base, 512);
+    else ptx::tmem_dealloc(tmem_base, 512);
   }
 }
 
@@ -433,6 +495,7 @@ inline encode_tiled_fn get_encode_tiled() {
 
 int sm_count();
 bool gemm_a_in_tmem();
+int gemm_pair_mode();     // BITRL_GEMM_PAIR: 1 = paired CTAs wherever the shape allows, 0 = never, unset = launcher's choice
 int gemm_forced_tok();    // 0, or the token-tile width forced through BITRL_GEMM_TOK (64, 128, 192, 224, 256)  // expanded weights through tensor memory (default) or through shared memory
 
 // Second kernel of a split-K launch: y = (part - rowsum) * gamma * a_m / 127 (+ residual), 8 outputs per thread.
@@ -480,6 +543,53 @@ __global__ void __launch_bounds__(256) gemm_splitk_finish_kernel(const int32_t* 
   *reinterpret_cast<uint4*>(static_cast<unsigned short*>(y) + off) = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
+// Paired-CTA launches are considered from this M on (many tiles, no split-K).
+constexpr int GM_PAIR_MIN_M = 1024;
+
+// Time per k block (ns) of one CTA (or CTA pair) by token-tile width, as measured at M = 4096 on the block shapes: the
+// 192-wide tile runs close to the tensor pipe's own time; at 224 only two weight slots fit beside the accumulators in
+// tensor memory and the expand -> MMA -> release chain shows; at 256 the weights go through shared memory, whose
+// bandwidth then binds; below 192 the fixed cost per k block (barrier round trips, issue) is the floor.
+inline long long gemm_kb_ns(int tok, bool pair) {
+  if (pair) return tok == 224 ? 350 : tok == 192 ? 283 : 284;
+  return tok == 256 ? 466 : tok == 224 ? 372 : tok == 192 ? 295 : tok == 128 ? 284 : 270;
+}
+
+inline void (*gemm_pair_kernel(int tok))(const CUtensorMap, const GemmArgs) {
+  return tok == 224 ? gemm_i8_kernel<224, true, true> : tok == 192 ? gemm_i8_kernel<192, true, true>
+                                                                   : gemm_i8_kernel<128, true, true>;
+}
+
+// Clusters of two CTAs that can be resident at once (the persistent grid must not exceed it), per device and width.
+inline int gemm_pair_max_clusters(int tok) {
+  static int cached[64][3] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  const int slot = tok == 224 ? 0 : tok == 192 ? 1 : 2;
+  if (cached[dev][slot] == 0) {
+    void (*pk)(const CUtensorMap, const GemmArgs) = gemm_pair_kernel(tok);
+    int n = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * 74);
+    cfg.blockDim = dim3(GM_THREADS);
+    cfg.dynamicSmemBytes = GM_SMEM_BYTES;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaFuncSetAttribute(pk, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM_BYTES) != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&n, pk, &cfg) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      n = -1;
+    }
+    cached[dev][slot] = n;
+  }
+  return cached[dev][slot] > 0 ? cached[dev][slot] : 0;
+}
+
 // Largest M for which a split-K workspace (M*N int32) is offered.
 constexpr int GM_SPLITK_MAX_M = 512;
 
@@ -494,31 +604,53 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
   const int tiles_n = w->N / GM_ROWS;
   const int kblocks = w->K / GM_BK;
   int tok = 256, splits = 1;
+  long long best = -1;
   {
-    long long best = -1;
     const int cand[5] = {256, 224, 192, 128, 64};
     for (int i = 0; i < 5; ++i) {
       if (cand[i] == 224 && !gemm_a_in_tmem()) continue;
       const long long tiles = static_cast<long long>(tiles_n) * ((M + cand[i] - 1) / cand[i]);
-      // cycles per k block as measured: the 256-wide tile (4-stage x_q ring, weights through shared memory) runs at
-      // about 690, the narrower ones at the MMA thread's own ~500 or the tensor pipe's 2*TOK, whichever is larger
-      const long long per_kb = cand[i] == 256 ? 690 : (2 * cand[i] > 500 ? 2 * cand[i] : 500);
+      const long long per_kb = gemm_kb_ns(cand[i], false);
       const int smax = (splitk_ws && M <= GM_SPLITK_MAX_M && tiles * 2 <= sms) ? static_cast<int>(sms / tiles) : 1;
       for (int sp = 1; sp <= smax && sp <= kblocks; ++sp) {
         const int kps = (kblocks + sp - 1) / sp;
         if ((kblocks + kps - 1) / kps != sp) continue;  // this count would leave an empty split
         const long long waves = (tiles * sp + sms - 1) / sms;
         // a split launch pays for clearing the scratch and for the finishing kernel (about 5 us in a chain of dependent launches)
-        const long long cost = waves * kps * per_kb + (sp > 1 ? 10000 : 0);
+        const long long cost = waves * kps * per_kb + (sp > 1 ? 5000 : 0);
         if (best < 0 || cost <= best) { best = cost; tok = cand[i]; splits = sp; }  // ties go to the narrower tile
       }
     }
   }
   if (const int forced = gemm_forced_tok()) { tok = forced; splits = 1; }  // tuning knob, see bitrl.cu
+  // CTA pairs (256-row tiles): for launches with many tiles, an even number of 128-row tiles and weights in tensor memory.
+  bool pair = false;
+  int pair_clusters = 0;
+  if (gemm_pair_mode() != 0 && gemm_a_in_tmem() && tiles_n % 2 == 0 && splits == 1 && M >= GM_PAIR_MIN_M) {
+    int ptok = 0;
+    if (const int forced = gemm_forced_tok()) {
+      if (forced == 224 || forced == 192 || forced == 128) ptok = forced;
+    } else {
+      long long pbest = -1;
+      const int cand[3] = {224, 192, 128};
+      for (int i = 0; i < 3; ++i) {
+        const int clusters = gemm_pair_max_clusters(cand[i]);
+        if (clusters <= 0) continue;
+        const long long tiles = static_cast<long long>(tiles_n / 2) * ((M + cand[i] - 1) / cand[i]);
+        const long long cost = ((tiles + clusters - 1) / clusters) * kblocks * gemm_kb_ns(cand[i], true);
+        if (pbest < 0 || cost < pbest) { pbest = cost; ptok = cand[i]; }
+      }
+      if (gemm_pair_mode() != 1 && pbest >= best) ptok = 0;  // the single-CTA kernel is expected to be no slower
+    }
+    if (ptok) {
+      pair_clusters = gemm_pair_max_clusters(ptok);
+      if (pair_clusters > 0) { pair = true; tok = ptok; }
+    }
+  }
   CUtensorMap tmap;
   const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(w->K), static_cast<cuuint64_t>(M)};
   const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(w->K)};
-  const cuuint32_t box[2] = {GM_BK, static_cast<cuuint32_t>(tok)};
+  const cuuint32_t box[2] = {GM_BK, static_cast<cuuint32_t>(pair ? tok / 2 : tok)};  // a paired CTA fetches half a tile
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(xq), gdim, gstride, box,
                             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -529,6 +661,29 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
   GemmArgs a{w->tiles, w->gamma, absmax, rowsum, M, w->N, w->K, y, out_dtype,
              split ? nullptr : static_cast<const unsigned short*>(residual), split ? nullptr : acc_out, tiles_n, 0,
              splits, (kblocks + splits - 1) / splits, split ? splitk_ws : nullptr};
+  if (pair) {
+    a.tiles_n = tiles_n / 2;
+    a.tiles_total = a.tiles_n * ((M + tok - 1) / tok);
+    const int clusters = a.tiles_total < pair_clusters ? a.tiles_total : pair_clusters;
+    void (*pk)(const CUtensorMap, const GemmArgs) = gemm_pair_kernel(tok);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * clusters);
+    cfg.blockDim = dim3(GM_THREADS);
+    cfg.dynamicSmemBytes = GM_SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    BITRL_CUDA(cudaLaunchKernelEx(&cfg, pk, tmap, a));
+    count_launch(1);
+    return BITRL_OK;
+  }
   a.tiles_total = tiles_n * ((M + tok - 1) / tok);
   const int items = a.tiles_total * splits;
   const int grid = items < sms ? items : sms;

@@ -102,28 +102,40 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp walks the loop and one elected lane issues: uniform control flow keeps the descriptors in
+    // uniform registers, from which the MMA instruction takes its operands.
+    {
       const uint32_t idesc = ptx::idesc_i8(128, TOK, /*a_signed=*/true, /*b_signed=*/true);
       uint32_t s = 0, ph = 0, lt = 0;
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x, ++lt) {
         const uint32_t buf = lt & 1u;
-        if (!ptx::mbar_wait(bar_tmem_empty + 8 * buf, ((lt >> 1) & 1u) ^ 1u)) {
-          report_timeout(G8_WAIT_TMEM_EMPTY); ok = false; break;
+        if (!__any_sync(0xffffffffu, ptx::mbar_wait(bar_tmem_empty + 8 * buf, ((lt >> 1) & 1u) ^ 1u))) {
+          if (lane == 0) report_timeout(G8_WAIT_TMEM_EMPTY);
+          ok = false;
+          break;
         }
         const uint32_t d_tmem = tmem_base + buf * 256;
         ptx::tc_fence_after_sync();
         for (int kb = 0; kb < kblocks; ++kb) {
-          if (!ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(G8_WAIT_FULL); ok = false; break; }
+          if (!__any_sync(0xffffffffu, ptx::mbar_wait(bar_full + 8 * s, ph))) {
+            if (lane == 0) report_timeout(G8_WAIT_FULL);
+            ok = false;
+            break;
+          }
           const uint64_t adesc = ptx::smem_desc_sw128(base + s * STAGE);
           const uint64_t bdesc = ptx::smem_desc_sw128(base + s * STAGE + G8_W_BYTES);
+          if (ptx::elect_one()) {
 #pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4)
-            ptx::mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
-          ptx::mma_commit(bar_empty + 8 * s);
+            for (int k4 = 0; k4 < 4; ++k4)
+              ptx::mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+            ptx::mma_commit(bar_empty + 8 * s);
+          }
+          __syncwarp();
           if (++s == NS) { s = 0; ph ^= 1u; }
         }
-        if (ok) ptx::mma_commit(bar_tmem_full + 8 * buf);
+        if (ok && ptx::elect_one()) ptx::mma_commit(bar_tmem_full + 8 * buf);
+        __syncwarp();
       }
     }
   } else {
