@@ -637,7 +637,8 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
         const int clusters = gemm_pair_max_clusters(cand[i]);
         if (clusters <= 0) continue;
         const long long tiles = static_cast<long long>(tiles_n / 2) * ((M + cand[i] - 1) / cand[i]);
-        const long long cost = ((tiles + clusters - 1) / clusters) * kblocks * gemm_kb_ns(cand[i], true);
+        // a cluster launch starts and ends about 4 us later than a plain one (measured on one-wave launches)
+        const long long cost = ((tiles + clusters - 1) / clusters) * kblocks * gemm_kb_ns(cand[i], true) + 4000;
         if (pbest < 0 || cost < pbest) { pbest = cost; ptok = cand[i]; }
       }
       if (gemm_pair_mode() != 1 && pbest >= best) ptok = 0;  // the single-CTA kernel is expected to be no slower
