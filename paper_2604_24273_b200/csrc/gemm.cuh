@@ -551,7 +551,7 @@ constexpr int GM_PAIR_MIN_M = 1024;
 // tensor memory and the expand -> MMA -> release chain shows; at 256 the weights go through shared memory, whose
 // bandwidth then binds; below 192 the fixed cost per k block (barrier round trips, issue) is the floor.
 inline long long gemm_kb_ns(int tok, bool pair) {
-  if (pair) return tok == 224 ? 350 : tok == 192 ? 283 : 284;
+  if (pair) return tok == 224 ? 340 : tok == 192 ? 283 : 284;
   return tok == 256 ? 466 : tok == 224 ? 372 : tok == 192 ? 295 : tok == 128 ? 284 : 270;
 }
 
@@ -637,8 +637,9 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
         const int clusters = gemm_pair_max_clusters(cand[i]);
         if (clusters <= 0) continue;
         const long long tiles = static_cast<long long>(tiles_n / 2) * ((M + cand[i] - 1) / cand[i]);
-        // a cluster launch starts and ends about 4 us later than a plain one (measured on one-wave launches)
-        const long long cost = ((tiles + clusters - 1) / clusters) * kblocks * gemm_kb_ns(cand[i], true) + 4000;
+        // a cluster launch starts and ends a few us later than a plain one (one-wave launches at M = 1024 lose 4 us,
+        // seven-wave launches at M = 4096 win 2 us)
+        const long long cost = ((tiles + clusters - 1) / clusters) * kblocks * gemm_kb_ns(cand[i], true) + 3000;
         if (pbest < 0 || cost < pbest) { pbest = cost; ptok = cand[i]; }
       }
       if (gemm_pair_mode() != 1 && pbest >= best) ptok = 0;  // the single-CTA kernel is expected to be no slower

@@ -190,6 +190,22 @@ def test_gemm_m4096_sampled(oracle_mod, B, K, N, wseed):
     assert np.isfinite(bits_to_f64(yb)).all()
 
 
+def test_gemm_paired_ctas_forced(B):
+    """The paired-CTA kernel on small ragged shapes the launcher would give to the single-CTA kernel: a child process
+    with BITRL_GEMM_PAIR=1 (the knob is read once per process) checks every stage against the oracle."""
+    import os
+    import subprocess
+    import sys
+    from pathlib import Path
+
+    root = Path(__file__).resolve().parent.parent
+    env = dict(os.environ, BITRL_GEMM_PAIR="1", PYTHONPATH=str(root))
+    r = subprocess.run([sys.executable, str(root / "tests" / "pair_gemm_child.py")], env=env, cwd=str(root),
+                       capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+    assert "paired-CTA GEMM parity ok" in r.stdout
+
+
 def test_forward_q_with_residual(oracle_mod, B):
     for M in (4, 130):
         K, N = 256, 384
