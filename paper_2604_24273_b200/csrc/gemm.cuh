@@ -10,11 +10,13 @@
 //   warp 0      X producer : TMA tile of x_q (TOK tokens x 128 k, 128-byte swizzle)        ring of 128 KB
 //   warp 2      P producer : bulk copy of the 4 KB packed weight piece (128 rows x 128 k)    ring of 8 x 4 KB
 //   warps 3-6, 11-14 expand: packed piece -> int8 codes in the swizzled K-major layout       ring of 3 x 16 KB
-//   warp 1      MMA        : one thread issues tcgen05.mma kind::i8 (4 per k block, K = 32 each) into TMEM
+//   warp 1      MMA        : the warp walks the loop, one elected lane issues tcgen05.mma kind::i8 (4 per k block,
+//                            K = 32 each) into TMEM
 //   warps 7-10  epilogue   : TMEM -> registers -> (acc - rowsum) * gamma*a_m/127 -> bf16/fp32, transposed through
 //                            a per-warp shared-memory tile so that global stores are 16 bytes per lane
 // The token-tile width TOK (64..256) is chosen per launch to fill the SMs with whole waves.
 // Two 256-column accumulators in TMEM let the epilogue of tile i overlap the main loop of tile i+1.
+// A variant for large launches pairs two CTAs of a cluster on a 256-row tile (tcgen05 cta_group::2, see PAIR below).
 // Every mbarrier wait is bounded; on expiry the CTA records a status word and leaves through the normal exit.
 #pragma once
 
