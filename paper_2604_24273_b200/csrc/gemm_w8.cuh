@@ -34,6 +34,7 @@ constexpr uint32_t G8_OFF_MISC = G8_OFF_BAR + (2 * G8_MAX_STAGES + 4) * 8;
 constexpr uint32_t G8_SMEM_BYTES = G8_OFF_MISC + 16 + 1024;           // + slack to align the base to 1024
 static_assert(G8_SMEM_BYTES <= 232448, "shared memory budget of one CTA");
 
+constexpr int G8_PAIR_MIN_M = 2048;  // paired CTAs from this M on
 enum { G8_WAIT_EMPTY = 41, G8_WAIT_FULL = 42, G8_WAIT_TMEM_EMPTY = 43, G8_WAIT_TMEM_FULL = 44 };
 
 struct Gemm8Args {
@@ -47,10 +48,15 @@ struct Gemm8Args {
   int tiles_n, tiles_total;
 };
 
-template <int TOK>
+// PAIR: two CTAs of a cluster work on one 256-row x TOK-token tile with tcgen05.mma.cta_group::2, as in the ternary
+// GEMM: rank r fetches weight rows [256 t + 128 r, +128) and tokens [TOK/2 * r, +TOK/2) of the tile into its own
+// shared memory (completion counted on rank 0's barrier) and drains its own 128 x TOK slice of the accumulator;
+// rank 0 issues the MMAs and releases the stage in both CTAs with one multicast commit.  Per SM the B tile is halved,
+// and shared-memory traffic is what binds this kernel.
+template <int TOK, bool PAIR = false>
 __global__ void __launch_bounds__(G8_THREADS, 1)
 gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const Gemm8Args a) {
-  constexpr uint32_t X_BYTES = TOK * 128;
+  constexpr uint32_t X_BYTES = (PAIR ? TOK / 2 : TOK) * 128;
   constexpr uint32_t STAGE = X_BYTES + G8_W_BYTES;
   constexpr uint32_t NS = G8_RING_BYTES / STAGE < G8_MAX_STAGES ? G8_RING_BYTES / STAGE : G8_MAX_STAGES;
   static_assert(TOK % 32 == 0 && TOK >= 64 && TOK <= 256, "token tile");
@@ -66,20 +72,34 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kblocks = a.K / 128;
+  const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;
+  const int tile0 = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+  const int tile_step = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
+  const uint32_t full_lead = PAIR ? ptx::mapa_u32(bar_full, 0) : bar_full;  // rank 0's barriers as seen from either CTA
+  const uint32_t tmem_empty_lead = PAIR ? ptx::mapa_u32(bar_tmem_empty, 0) : bar_tmem_empty;
 
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < NS; ++s) { ptx::mbar_init(bar_full + 8 * s, 1); ptx::mbar_init(bar_empty + 8 * s, 1); }
-    for (int b = 0; b < 2; ++b) { ptx::mbar_init(bar_tmem_full + 8 * b, 1); ptx::mbar_init(bar_tmem_empty + 8 * b, 4); }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(bar_tmem_full + 8 * b, 1);
+      ptx::mbar_init(bar_tmem_empty + 8 * b, PAIR ? 8 : 4);
+    }
     ptx::mbar_init_fence();
     ptx::tma_prefetch_desc(&tmap_x);
     ptx::tma_prefetch_desc(&tmap_w);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(base + G8_OFF_MISC, 512);
-    ptx::tmem_relinquish();
+    if (PAIR) {
+      ptx::tmem_alloc_pair(base + G8_OFF_MISC, 512);
+      ptx::tmem_relinquish_pair();
+    } else {
+      ptx::tmem_alloc(base + G8_OFF_MISC, 512);
+      ptx::tmem_relinquish();
+    }
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
+  if (PAIR) ptx::cluster_sync_all();  // the peer's barriers are initialised before anything is sent to them
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   pdl_enter();
@@ -89,10 +109,19 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     if (lane == 0) {
       uint32_t s = 0, ph = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x) {
-        const int tn = tile % a.tiles_n, tm = tile / a.tiles_n;
+      for (int tile = tile0; ok && tile < a.tiles_total; tile += tile_step) {
+        const int tn = PAIR ? 2 * (tile % a.tiles_n) + static_cast<int>(rank) : tile % a.tiles_n, tm = tile / a.tiles_n;
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!ptx::mbar_wait(bar_empty + 8 * s, ph ^ 1u)) { report_timeout(G8_WAIT_EMPTY); ok = false; break; }
+          if (PAIR) {
+            // Rank 0 announces the bytes of both CTAs' stages on its barrier; each CTA's copies report there.
+            if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * s, 2 * STAGE);
+            ptx::tma_load_2d_pair(base + s * STAGE, &tmap_w, kb * 128, tn * 128, full_lead + 8 * s);
+            ptx::tma_load_2d_pair(base + s * STAGE + G8_W_BYTES, &tmap_x, kb * 128,
+                                  tm * TOK + static_cast<int>(rank) * (TOK / 2), full_lead + 8 * s);
+            if (++s == NS) { s = 0; ph ^= 1u; }
+            continue;
+          }
           ptx::mbar_arrive_expect_tx(bar_full + 8 * s, STAGE);
           ptx::tma_load_2d(base + s * STAGE, &tmap_w, kb * 128, tn * 128, bar_full + 8 * s);
           ptx::tma_load_2d(base + s * STAGE + G8_W_BYTES, &tmap_x, kb * 128, tm * TOK, bar_full + 8 * s);
@@ -104,11 +133,11 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     // ------------------------------------------------------------------ MMA issuer
     // The whole warp walks the loop and one elected lane issues: uniform control flow keeps the descriptors in
     // uniform registers, from which the MMA instruction takes its operands.
-    {
-      const uint32_t idesc = ptx::idesc_i8(128, TOK, /*a_signed=*/true, /*b_signed=*/true);
+    if (rank == 0) {
+      const uint32_t idesc = ptx::idesc_i8(PAIR ? 256 : 128, TOK, /*a_signed=*/true, /*b_signed=*/true);
       uint32_t s = 0, ph = 0, lt = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x, ++lt) {
+      for (int tile = tile0; ok && tile < a.tiles_total; tile += tile_step, ++lt) {
         const uint32_t buf = lt & 1u;
         if (!__any_sync(0xffffffffu, ptx::mbar_wait(bar_tmem_empty + 8 * buf, ((lt >> 1) & 1u) ^ 1u))) {
           if (lane == 0) report_timeout(G8_WAIT_TMEM_EMPTY);
@@ -126,15 +155,25 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
           const uint64_t adesc = ptx::smem_desc_sw128(base + s * STAGE);
           const uint64_t bdesc = ptx::smem_desc_sw128(base + s * STAGE + G8_W_BYTES);
           if (ptx::elect_one()) {
+            if (PAIR) {
 #pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4)
-              ptx::mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
-            ptx::mma_commit(bar_empty + 8 * s);
+              for (int k4 = 0; k4 < 4; ++k4)
+                ptx::mma_i8_ss_pair(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+              ptx::mma_commit_pair(bar_empty + 8 * s, 3);  // frees the stage in both CTAs
+            } else {
+#pragma unroll
+              for (int k4 = 0; k4 < 4; ++k4)
+                ptx::mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+              ptx::mma_commit(bar_empty + 8 * s);
+            }
           }
           __syncwarp();
           if (++s == NS) { s = 0; ph ^= 1u; }
         }
-        if (ok && ptx::elect_one()) ptx::mma_commit(bar_tmem_full + 8 * buf);
+        if (ok && ptx::elect_one()) {
+          if (PAIR) ptx::mma_commit_pair(bar_tmem_full + 8 * buf, 3);
+          else ptx::mma_commit(bar_tmem_full + 8 * buf);
+        }
         __syncwarp();
       }
     }
@@ -148,8 +187,8 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     const bool f32 = a.out_dtype == BITRL_OUT_F32;
     uint32_t lt = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < a.tiles_total; tile += gridDim.x, ++lt) {
-      const int tn = tile % a.tiles_n, tm = tile / a.tiles_n;
+    for (int tile = tile0; ok && tile < a.tiles_total; tile += tile_step, ++lt) {
+      const int tn = PAIR ? 2 * (tile % a.tiles_n) + static_cast<int>(rank) : tile % a.tiles_n, tm = tile / a.tiles_n;
       const uint32_t buf = lt & 1u;
       const uint32_t sc_addr = base + G8_OFF_TOK + buf * 256 * 4;
       for (int j = ep; j < TOK; j += 128) {
@@ -237,7 +276,10 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       }
       ptx::tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(bar_tmem_empty + 8 * buf);
+      if (lane == 0) {
+        if (PAIR) ptx::mbar_arrive_cluster(tmem_empty_lead + 8 * buf);
+        else ptx::mbar_arrive(bar_tmem_empty + 8 * buf);
+      }
     }
   }
 
@@ -245,10 +287,46 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   __syncwarp();
   ptx::tc_fence_before_sync();
   __syncthreads();
+  if (PAIR) ptx::cluster_sync_all();  // neither CTA leaves (or frees tensor memory) while the other may still reach it
   if (warp == 1) {
     ptx::tc_fence_after_sync();
-    ptx::tmem_dealloc(tmem_base, 512);
+    if (PAIR) ptx::tmem_dealloc_pair(tmem_base, 512);
+    else ptx::tmem_dealloc(tmem_base, 512);
   }
+}
+
+inline void (*gemm_w8_pair_kernel(int tok))(const CUtensorMap, const CUtensorMap, const Gemm8Args) {
+  return tok == 256 ? gemm_w8_kernel<256, true> : tok == 192 ? gemm_w8_kernel<192, true> : gemm_w8_kernel<128, true>;
+}
+
+// Clusters of two CTAs that can be resident at once, per device and width (0 = paired launches unavailable).
+inline int gemm_w8_pair_max_clusters(int tok) {
+  static int cached[64][3] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  const int slot = tok == 256 ? 0 : tok == 192 ? 1 : 2;
+  if (cached[dev][slot] == 0) {
+    void (*pk)(const CUtensorMap, const CUtensorMap, const Gemm8Args) = gemm_w8_pair_kernel(tok);
+    int n = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * 74);
+    cfg.blockDim = dim3(G8_THREADS);
+    cfg.dynamicSmemBytes = G8_SMEM_BYTES;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaFuncSetAttribute(pk, cudaFuncAttributeMaxDynamicSharedMemorySize, G8_SMEM_BYTES) != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&n, pk, &cfg) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      n = -1;
+    }
+    cached[dev][slot] = n;
+  }
+  return cached[dev][slot] > 0 ? cached[dev][slot] : 0;
 }
 
 // ---- M <= 16: streaming kernel ----------------------------------------------------------------------------------
@@ -450,12 +528,33 @@ bitrl_status launch_gemm_w8(const int8_t* wq, const float* scale, int N, int K, 
       if (best < 0 || cost <= best) { best = cost; tok = cand[i]; }
     }
   }
+  // Paired CTAs for large launches (same knob as the ternary GEMM): widest tile that fills whole waves of clusters.
+  bool pair = false;
+  int pair_clusters = 0;
+  if (gemm_pair_mode() != 0 && tiles_n % 2 == 0 && M >= G8_PAIR_MIN_M) {
+    long long best = -1;
+    int ptok = 0;
+    const int cand[3] = {256, 192, 128};
+    for (int i = 0; i < 3; ++i) {
+      const int clusters = gemm_w8_pair_max_clusters(cand[i]);
+      if (clusters <= 0) continue;
+      const long long tiles = static_cast<long long>(tiles_n / 2) * ((M + cand[i] - 1) / cand[i]);
+      const long long cost = ((tiles + clusters - 1) / clusters) * (2 * cand[i] > 300 ? 2 * cand[i] : 300);
+      if (best < 0 || cost < best) { best = cost; ptok = cand[i]; }
+    }
+    if (const int forced = gemm_forced_tok())
+      if (forced == 256 || forced == 192 || forced == 128) ptok = forced;
+    if (ptok) {
+      pair_clusters = gemm_w8_pair_max_clusters(ptok);
+      if (pair_clusters > 0) { pair = true; tok = ptok; }
+    }
+  }
   CUtensorMap tmx, tmw;
   const cuuint32_t estr[2] = {1, 1};
   {
     const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(M)};
     const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(K)};
-    const cuuint32_t box[2] = {128, static_cast<cuuint32_t>(tok)};
+    const cuuint32_t box[2] = {128, static_cast<cuuint32_t>(pair ? tok / 2 : tok)};
     if (encode(&tmx, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(xq), gdim, gstride, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -471,6 +570,28 @@ bitrl_status launch_gemm_w8(const int8_t* wq, const float* scale, int N, int K, 
       return cuda_fail(cudaErrorInvalidValue);
   }
   Gemm8Args a{scale, absmax, M, N, K, y, out_dtype, static_cast<const unsigned short*>(residual), acc_out, tiles_n, 0};
+  if (pair) {
+    a.tiles_n = tiles_n / 2;
+    a.tiles_total = a.tiles_n * ((M + tok - 1) / tok);
+    const int clusters = a.tiles_total < pair_clusters ? a.tiles_total : pair_clusters;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * clusters);
+    cfg.blockDim = dim3(G8_THREADS);
+    cfg.dynamicSmemBytes = G8_SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    BITRL_CUDA(cudaLaunchKernelEx(&cfg, gemm_w8_pair_kernel(tok), tmx, tmw, a));
+    count_launch(1);
+    return BITRL_OK;
+  }
   a.tiles_total = tiles_n * ((M + tok - 1) / tok);
   const int grid = a.tiles_total < sms ? a.tiles_total : sms;
   void (*kern)(const CUtensorMap, const CUtensorMap, const Gemm8Args) =

@@ -67,6 +67,14 @@ def test_w8a8_full(oracle_mod, B, M, K, N, seed, out_dtype):
         assert np.array_equal(yb, ref["ybf16"]) and torch.equal(y, y2)
 
 
+@pytest.mark.parametrize("M,K,N,seed,out_dtype", [(2048, 128, 256, 9210, 1), (2085, 640, 512, 9211, 0),
+                                                   (2300, 2560, 768, 9212, 1)])
+def test_w8a8_paired_cta_shapes_full(oracle_mod, B, M, K, N, seed, out_dtype):
+    """M >= 2048 with an even number of 128-row tiles: the paired-CTA kernel (tcgen05 cta_group::2); ragged token counts,
+    one and several k blocks, every stage against the oracle."""
+    test_w8a8_full(oracle_mod, B, M, K, N, seed, out_dtype)
+
+
 def test_w8a8_m4096_sampled(oracle_mod, B):
     """The batched-state shape at full size (M = 4096, 2560 -> 6912): sampled outputs one by one."""
     K, N, M = 2560, 6912, 4096
