@@ -1,0 +1,198 @@
+"""GPU parity at the sizes and in the launch configurations the benchmark times: the M >= 1024 launches of the block
+shapes (where the launcher takes the paired-CTA kernel) with the residual epilogue, the encoder at T = 4096, and the
+INT4 critic layer at M = 4096.  The oracle recomputes sampled token rows and sampled (m, n) pairs one by one; integer
+stages must be bit-exact and the bf16 outputs bit-identical to the oracle's three fp32 operations + RNE.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2604_24273_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 8e-3
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_24273_b200 import bitrl
+
+    bitrl.lib()
+    torch.cuda.set_device(0)
+    return bitrl
+
+
+def bits_to_f64(bits):
+    return (np.asarray(bits, np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def gpu_bits(t):
+    return inputs.bf16_bits(t.detach().cpu())
+
+
+def rel_err(y, y64):
+    denom = np.where(y64 == 0, 1.0, np.abs(y64))
+    return float((np.abs(np.asarray(y, np.float64) - y64) / denom).max())
+
+
+_layers = {}
+
+
+def layer(oracle_mod, B, N, K, seed):
+    if (N, K, seed) not in _layers:
+        W = inputs.master_weights(N, K, seed)
+        Wq, g = oracle_mod.ternarize(W.numpy())
+        lin = B.Linear.from_master(W.cuda())
+        _layers[(N, K, seed)] = (Wq, g, lin)
+    return _layers[(N, K, seed)]
+
+
+def sample_rows(M, rng, extra=28):
+    """First and last rows, the edges of every token-tile width the launcher uses (64 ... 256) and the ragged tail."""
+    edges = [0, 63, 64, 127, 128, 191, 192, 223, 224, 255, 256, 383, 384, 447, 448, M - 225, M - 193, M - 129, M - 2, M - 1]
+    rows = np.concatenate([np.array(edges), rng.integers(0, M, extra)])
+    return np.unique(rows[(rows >= 0) & (rows < M)])
+
+
+@pytest.mark.parametrize("M", [1024, 1061, 4096])
+@pytest.mark.parametrize("K,N,wseed", [(2560, 2560, 5001), (2560, 3840, 5000), (2560, 13824, 5002), (6912, 2560, 5003)])
+def test_forward_q_residual_block_shapes_large_m(oracle_mod, B, M, K, N, wseed):
+    """a2 + a3 + residual add on a quantized input, as the encoder calls it: int32 sums bit-exact on >= 40 sampled token
+    rows and 20000 sampled pairs, bf16(residual + bf16(acc * scale)) bit-identical to the oracle on the sampled rows, and
+    the in-place form (y aliases the residual) equal to the out-of-place one everywhere."""
+    Wq, g, lin = layer(oracle_mod, B, N, K, wseed)
+    x = inputs.activations(M, K, 7000 + M)
+    res = inputs.activations(M, N, 7100 + M, outliers=False)
+    xq_o, a_o = oracle_mod.quant_act(inputs.bf16_bits(x))
+    xq, a, rs = B.quant_act(x.cuda())
+    res_gpu = res.cuda()
+    y, acc = B.bitlinear_forward_q(lin, xq, a, rs, B.OUT_BF16, residual=res_gpu, want_acc=True)
+    inplace = res_gpu.clone()
+    B.bitlinear_forward_q(lin, xq, a, rs, B.OUT_BF16, residual=inplace, y=inplace)
+    plain = B.bitlinear_forward_q(lin, xq, a, rs, B.OUT_BF16)
+    B.poll_status()
+    assert np.array_equal(xq.cpu().numpy(), xq_o) and np.array_equal(a.cpu().numpy(), a_o)
+    assert torch.equal(inplace, y)
+    acc = acc.cpu().numpy()
+    rng = np.random.default_rng(M + N)
+    rows = sample_rows(M, rng)
+    assert len(rows) >= 40
+    acc_rows = oracle_mod.contract(xq_o[rows], Wq)
+    assert np.array_equal(acc[rows], acc_rows)
+    _, yb_o, y64 = oracle_mod.rescale(acc_rows, g, a_o[rows])
+    assert np.array_equal(gpu_bits(plain)[rows], yb_o)
+    assert rel_err(bits_to_f64(yb_o), y64) <= TOL_BF16
+    want = oracle_mod.residual_add(inputs.bf16_bits(res)[rows], yb_o)
+    assert np.array_equal(gpu_bits(y)[rows], want)
+    ms, ns = rng.integers(0, M, 20000), rng.integers(0, N, 20000)
+    assert np.array_equal(acc[ms, ns], oracle_mod.contract_pairs(xq_o, Wq, ms, ns))
+    nnz = (Wq != 0).sum(1)
+    assert np.all(np.abs(acc) <= 127 * nnz[None, :])
+
+
+FULL = {"d": 2560, "d_ff": 6912, "n_heads": 20, "n_kv_heads": 5}
+
+
+def chain_block(B, h, lins, taps=None):
+    """One encoder block as single C-ABI calls; `taps` collects (x_q, acc) of the four BitLinear calls."""
+    qkv_l, out_l, gu_l, down_l = lins
+    want = taps is not None
+
+    def lin(l, xq, a, rs, residual=None):
+        r = B.bitlinear_forward_q(l, xq, a, rs, residual=residual, want_acc=want)
+        if want:
+            taps.append((xq, r[1]))
+            return r[0]
+        return r
+
+    xq, a, rs, _ = B.rmsnorm_quant(h)
+    qkv = lin(qkv_l, xq, a, rs)
+    xq, a, rs, _ = B.vrepeat_rmsnorm_quant(qkv, FULL["n_heads"], FULL["n_kv_heads"], FULL["d"] // FULL["n_heads"])
+    h = lin(out_l, xq, a, rs, residual=h)
+    xq, a, rs, _ = B.rmsnorm_quant(h)
+    gu = lin(gu_l, xq, a, rs)
+    xq, a, rs, _ = B.relu2gate_rmsnorm_quant(gu)
+    return lin(down_l, xq, a, rs, residual=h)
+
+
+def test_encoder_t4096_two_blocks_teacher_forced(oracle_mod, B):
+    """The benchmarked token count (128 states x 32 tokens) at the real widths, 2 blocks: bitrl_encoder_forward equals the
+    chain of single calls bit for bit, and each of the 8 BitLinear calls of the chain has the oracle's int32 sums on the
+    GPU's own quantized input for 40+ sampled token rows (teacher forcing)."""
+    T = 4096
+    dims = dict(FULL, n_layers=2)
+    layers_gpu, layers_cpu = [], []
+    for l in range(2):
+        Ws = inputs.encoder_layer_weights(l, seed=5000, dims=dims)
+        layers_cpu.append([oracle_mod.ternarize(w.numpy())[0] for w in Ws])
+        layers_gpu.append(tuple(B.Linear.from_master(w.cuda()) for w in Ws))
+    enc = B.Encoder(layers_gpu, dims["d"], dims["d_ff"], dims["n_heads"], dims["n_kv_heads"])
+    h0 = inputs.activations(T, dims["d"], 6000).cuda()
+    out = enc.forward(h0)
+    B.poll_status()
+    rows = sample_rows(T, np.random.default_rng(11))
+    h = h0.clone()
+    for lins, cpu in zip(layers_gpu, layers_cpu):
+        taps = []
+        h = chain_block(B, h, lins, taps)
+        B.poll_status()
+        for (xq, acc), Wq in zip(taps, cpu):
+            assert np.array_equal(acc.cpu().numpy()[rows], oracle_mod.contract(xq.cpu().numpy()[rows], Wq))
+    assert torch.equal(out, h)
+    assert torch.isfinite(out.float()).all()
+
+
+def test_encoder_t4096_thirty_blocks_equals_chain(B):
+    """The benchmarked call itself (30 blocks, T = 4096): bit-identical to the chain of 240 single calls, each of which is
+    compared with the oracle elsewhere.  Master weights are drawn on the GPU here (no oracle value is needed)."""
+    T, L = 4096, 30
+    d, F, nh, nkv = FULL["d"], FULL["d_ff"], FULL["n_heads"], FULL["n_kv_heads"]
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5000)
+    shapes = [(d + 2 * nkv * (d // nh), d), (d, d), (2 * F, d), (d, F)]
+    layers = []
+    for _ in range(L):
+        layers.append(tuple(B.Linear.from_master(torch.randn(n, k, generator=gen, device="cuda") * inputs.SIGMA_W)
+                            for n, k in shapes))
+    enc = B.Encoder(layers, d, F, nh, nkv)
+    h0 = inputs.activations(T, d, 6000).cuda()
+    out = enc.forward(h0)
+    out_again = enc.forward(h0)
+    B.poll_status()
+    h = h0.clone()
+    for lins in layers:
+        h = chain_block(B, h, lins)
+    B.poll_status()
+    assert torch.equal(out, h) and torch.equal(out, out_again)
+    assert torch.isfinite(out.float()).all()
+
+
+def test_w4a8_m4096_sampled(oracle_mod, B):
+    """INT4 critic layer at the benchmarked size (M = 4096, 2560 -> 6912): the expansion pass plus the paired-CTA
+    int8 GEMM against the oracle on sampled rows and pairs."""
+    K, N, M = 2560, 6912, 4096
+    W = inputs.master_weights(N, K, 9503)
+    Wq, scale = oracle_mod.w4_quantize(W.numpy())
+    packed, scale_gpu = B.w4_quantize(W.cuda())
+    assert np.array_equal(packed.cpu().numpy(), oracle_mod.w4_pack(Wq))
+    assert np.float32(scale_gpu.cpu().numpy()[0]) == scale
+    x = inputs.activations(M, K, 9700)
+    y, xq, a, acc = B.w4a8_forward(packed, scale_gpu, x.cuda(), B.OUT_BF16, debug=True)
+    y2 = B.w4a8_forward(packed, scale_gpu, x.cuda(), B.OUT_BF16)
+    B.poll_status()
+    xq_o, a_o = oracle_mod.quant_act(inputs.bf16_bits(x))
+    assert np.array_equal(xq.cpu().numpy(), xq_o) and np.array_equal(a.cpu().numpy(), a_o)
+    assert torch.equal(y, y2)
+    acc = acc.cpu().numpy()
+    rng = np.random.default_rng(9)
+    rows = sample_rows(M, rng, extra=10)
+    acc_rows = oracle_mod.contract(xq_o[rows], Wq)
+    assert np.array_equal(acc[rows], acc_rows)
+    _, yb_o, y64 = oracle_mod.rescale(acc_rows, scale, a_o[rows])
+    assert np.array_equal(gpu_bits(y)[rows], yb_o)
+    assert rel_err(bits_to_f64(yb_o), y64) <= TOL_BF16
+    ms, ns = rng.integers(0, M, 20000), rng.integers(0, N, 20000)
+    assert np.array_equal(acc[ms, ns], oracle_mod.contract_pairs(xq_o, Wq, ms, ns))
