@@ -59,6 +59,10 @@ def _L():
         _lib.oracle_w4_pack.restype = None
         _lib.oracle_pack.argtypes = [_vp, _i64, _i64, _vp]
         _lib.oracle_unpack.argtypes = [_vp, _i64, _i64, _vp]
+        _lib.oracle_pack5.argtypes = [_vp, _i64, _i64, _vp]
+        _lib.oracle_pack5.restype = None
+        _lib.oracle_unpack5.argtypes = [_vp, _i64, _i64, _vp]
+        _lib.oracle_unpack5.restype = None
         _lib.oracle_quant_act.argtypes = [_vp, _i64, _i64, _vp, _vp]
         _lib.oracle_contract.argtypes = [_vp, _vp, _i64, _i64, _i64, _vp, _int]
         _lib.oracle_contract_pairs.argtypes = [_vp, _vp, _i64, _vp, _vp, _i64, _vp]
@@ -160,6 +164,24 @@ def unpack(packed: np.ndarray, K: int) -> np.ndarray:
     out = np.empty((N, K), np.int8)
     _L().oracle_unpack(_p(packed), N, K, _p(out))
     return out
+
+
+def pack5(Wq: np.ndarray) -> np.ndarray:
+    """Five weights per byte, base 3: uint8 [N, ceil(K/5)]; missing positions of a row's last byte count as zero weights."""
+    Wq = _c(Wq, np.int8)
+    N, K = Wq.shape
+    out = np.empty((N, (K + 4) // 5), np.uint8)
+    _L().oracle_pack5(_p(Wq), N, K, _p(out))
+    return out
+
+
+def unpack5(packed: np.ndarray, K: int) -> np.ndarray:
+    packed = _c(packed, np.uint8)
+    N = packed.shape[0]
+    assert packed.shape[1] == (K + 4) // 5
+    Wq = np.empty((N, K), np.int8)
+    _L().oracle_unpack5(_p(packed), N, K, _p(Wq))
+    return Wq
 
 
 def quant_act(x_bf16: np.ndarray):

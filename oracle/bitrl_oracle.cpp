@@ -117,6 +117,37 @@ void oracle_unpack(const uint8_t* packed, int64_t N, int64_t K, int8_t* Wq) {
     }
 }
 
+// Denser packing, five ternary weights per byte (1.6 bits per weight; the paper's "1.58-bit" weights of the Abstract
+// and the lookup-table decoding of its inference stack, Sec. V edge-deployment paragraph).  The paper gives no format;
+// the one used here is the base-3 number of the five codes c = W_q + 1:
+//   byte j of row n = sum_{i=0..4} c[n, 5j+i] * 3^i      (0..242),   ceil(K/5) bytes per row,
+// where positions 5j+i >= K (only in a row's last byte, when 5 does not divide K) count as W_q = 0, i.e. c = 1.
+void oracle_pack5(const int8_t* Wq, int64_t N, int64_t K, uint8_t* packed) {
+  const int64_t KB = (K + 4) / 5;
+  for (int64_t n = 0; n < N; ++n) {
+    for (int64_t j = 0; j < KB; ++j) {
+      unsigned b = 0, p = 1;
+      for (int i = 0; i < 5; ++i) {
+        const int64_t k = 5 * j + i;
+        const unsigned c = k < K ? static_cast<unsigned>(Wq[n * K + k] + 1) : 1u;
+        b += c * p;
+        p *= 3;
+      }
+      packed[n * KB + j] = static_cast<uint8_t>(b);
+    }
+  }
+}
+
+void oracle_unpack5(const uint8_t* packed, int64_t N, int64_t K, int8_t* Wq) {
+  const int64_t KB = (K + 4) / 5;
+  for (int64_t n = 0; n < N; ++n)
+    for (int64_t k = 0; k < K; ++k) {
+      unsigned b = packed[n * KB + k / 5];
+      for (int i = 0; i < k % 5; ++i) b /= 3;
+      Wq[n * K + k] = static_cast<int8_t>(static_cast<int>(b % 3) - 1);
+    }
+}
+
 // Per-token absmax int8 quantization, Q = 127.  x is bf16 (raw 16-bit patterns), [M,K] row-major.
 //   a = max_k |x|, a' = max(a, 1e-5), inv = 127/a' (fp32 divide), q = rint(x*inv) (one fp32 multiply,
 //   ties-to-even), x_q = clip(q, -128, 127).

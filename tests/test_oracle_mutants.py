@@ -7,6 +7,7 @@ import numpy as np
 import pytest
 
 import test_oracle_pins as pins
+import test_oracle_pins_pack5 as pins5
 
 
 class Mutant:
@@ -47,6 +48,24 @@ def _ternarize_no_eps(real, W, gamma=None):
 def _pack_reversed_bits(real, Wq):
     p = real.pack(Wq)
     return ((p & 0x03) << 6) | ((p & 0x0C) << 2) | ((p & 0x30) >> 2) | ((p & 0xC0) >> 6)
+
+
+def _pack5_most_significant_first(real, Wq):
+    """digit i weighted 3^(4-i) instead of 3^i"""
+    Wq = np.asarray(Wq, np.int8)
+    K = Wq.shape[1]
+    ext = np.zeros((Wq.shape[0], 5 * (-(-K // 5))), np.int8)
+    ext[:, :K] = Wq
+    return real.pack5(ext.reshape(ext.shape[0], -1, 5)[:, :, ::-1].reshape(ext.shape[0], -1))
+
+
+def _pack5_pads_with_minus_one(real, Wq):
+    """missing positions of the last byte packed as code 0 (a -1 weight) instead of code 1 (a zero weight)"""
+    Wq = np.asarray(Wq, np.int8)
+    K = Wq.shape[1]
+    ext = np.full((Wq.shape[0], 5 * (-(-K // 5))), -1, np.int8)
+    ext[:, :K] = Wq
+    return real.pack5(ext)
 
 
 def _contract_drops_minus(real, xq, Wq, threads=None):
@@ -151,7 +170,9 @@ PIN_TESTS = [pins.test_eq2_definition_fp64, pins.test_eq2_ties_are_strict, pins.
              pins.test_negation_permutation_bound_allones, pins.test_pack_roundtrip_and_zero_matrix,
              pins.test_gaussian_closed_forms, pins.test_rescale_tolerances_and_bf16_rne,
              pins.test_rmsnorm_against_fp64, pins.test_relu2_gate_identity_attention_residual,
-             pins.test_attention_against_library_sdpa, pins.test_attention_special_cases]
+             pins.test_attention_against_library_sdpa, pins.test_attention_special_cases,
+             pins5.test_pack5_golden_bytes, pins5.test_pack5_is_the_base3_number_of_every_digit_string,
+             pins5.test_pack5_byte_count_padding_and_roundtrip, pins5.test_pack5_digit_positions]
 
 
 def failing_pins(mod):
@@ -173,6 +194,8 @@ MUTANTS = {
     "ternarize: round half away": {"ternarize": _ternarize_half_away},
     "ternarize: threshold off": {"ternarize": _ternarize_no_eps},
     "pack: reversed bit order": {"pack": _pack_reversed_bits},
+    "pack5: most significant digit first": {"pack5": _pack5_most_significant_first},
+    "pack5: padding packed as -1": {"pack5": _pack5_pads_with_minus_one},
     "contract: -1 treated as skip": {"contract": _contract_drops_minus},
     "contract: k reversed on one operand": {"contract": _contract_transposed_x},
     "rescale: gamma + eps": {"rescale": _rescale_gamma_plus_eps},
