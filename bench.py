@@ -144,6 +144,21 @@ def time_graph(graph, steps, warmup, world):
     return max_over_ranks(e0.elapsed_time(e1), world)
 
 
+def time_rounds(graph, steps, rounds=10):
+    """`rounds` further passes of `steps` replays each (this rank only): the spread of the per-step time in ms."""
+    per = []
+    for _ in range(rounds):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        per.append(e0.elapsed_time(e1) / steps)
+    return {"rounds": rounds, "steps_per_round": steps, "median": statistics.median(per), "min": min(per), "max": max(per)}
+
+
 def capture(fn):
     """Runs fn once eagerly, then captures it into a CUDA graph (the library launches on the current stream).
     Returns (graph, number of library kernel launches inside the graph)."""
@@ -210,6 +225,36 @@ def oracle_decode_sample(min_seconds=10.0):
                       "oracle threads over token rows, so M=1 runs on one core"}
 
 
+def oracle_batched_samples():
+    """The oracle beside the other half of the metric: a sample of token rows of both M = 4096 shapes (quant ->
+    contract -> rescale) and one encoder block on one 32-token state, each with one thread and with every core this
+    process may run on."""
+    import oracle
+
+    cores = oracle.default_threads()
+    out = {"kind": "oracle", "cores_all": cores}
+    for K, N, seed in ((2560, 6912, 1005), (6912, 2560, 1004)):
+        Wq, g = oracle.ternarize(inputs.master_weights(N, K, seed).numpy())
+        for label, threads, rows in (("1_thread", 1, 128), ("all_cores", cores, min(4096, 64 * cores))):
+            x = inputs.bf16_bits(inputs.activations(rows, K, 2400))
+            t0 = time.perf_counter()
+            oracle.bitlinear(x, Wq, g, threads=threads)
+            dt = time.perf_counter() - t0
+            out[f"m4096_k{K}_n{N}_{label}"] = {
+                "TOPS": 2.0 * rows * N * K / dt / 1e12, "cores": threads, "seconds": dt,
+                "sample": f"{rows} of the 4096 token rows"}
+    layer = [oracle.ternarize(w.numpy()) for w in inputs.encoder_layer_weights(0)]
+    h = inputs.bf16_bits(inputs.activations(32, 2560, 6002))
+    for label, threads in (("1_thread", 1), ("all_cores", cores)):
+        t0 = time.perf_counter()
+        oracle.encoder_block(h, 6912, 20, 5, layer, threads=threads)
+        dt = time.perf_counter() - t0
+        out[f"encoder_block_1_state_x32_tokens_{label}"] = {
+            "states_per_s_30_blocks": 1.0 / (dt * 30), "cores": threads, "seconds_per_block": dt,
+            "sample": "block 0 on one 32-token state (identity attention); a full forward is 30 such blocks"}
+    return out
+
+
 def run_reference(args):
     """--impl reference: the CPU oracle on the same metric/config, each step a bounded sample."""
     rank, _, _ = dist_env()
@@ -265,14 +310,14 @@ def run_ours(args):
         xs = {2560: xflat[:M * 2560].view(M, 2560), 6912: xflat[M * 2560:].view(M, 6912)}
         for k in xs:
             xs[k].copy_(inputs.activations(M, k, 2000 + M))
+        per_block = M * sum(n for _, _, n in BLOCK)
+        yall = torch.empty((n_layers * per_block,), dtype=torch.bfloat16, device=dev)  # every output of a step
         ys = []
-        for _ in range(n_layers):
-            yflat = torch.empty((M * sum(n for _, _, n in BLOCK),), dtype=torch.bfloat16, device=dev)
-            off, row = 0, []
+        for l in range(n_layers):
+            off, row = l * per_block, []
             for _, _, n in BLOCK:
-                row.append(yflat[off:off + M * n].view(M, n))
+                row.append(yall[off:off + M * n].view(M, n))
                 off += M * n
-            row.append(yflat)
             ys.append(row)
         ws = [layers[l][j] for l in range(n_layers) for j in range(len(BLOCK))]
         xl = [xs[k] for _ in range(n_layers) for _, k, _ in BLOCK]
@@ -289,6 +334,7 @@ def run_ours(args):
                 for j, (_, k, n) in enumerate(BLOCK):
                     bitrl.bitlinear_forward(layers[l][j], xs[k], bitrl.OUT_BF16, y=ys[l][j])
         xs["flat"] = xflat
+        xs["yall"] = yall
         return xs, ys, sweep, chain
 
     xs1, ys1, step1, chain1 = decode_setup(1)
@@ -297,18 +343,20 @@ def run_ours(args):
     ms1 = time_graph(g1, args.steps, args.warmup, world)
     gbs1 = world * bytes_step * args.steps / (ms1 * 1e-3) / 1e9
     us_per_launch = ms1 * 1e3 / (args.steps * launches1)
+    spread1 = time_rounds(g1, args.steps)
 
-    # end to end: pinned host x -> device, the sweep, the last block's outputs back to pinned host memory.  The two
-    # copies are nodes of the same CUDA graph as the kernel, so a step is one graph launch plus the wait for its result.
+    # end to end: pinned host x -> device, the sweep, ALL of the step's outputs (4 per block, one contiguous buffer) back
+    # to pinned host memory.  The two copies are nodes of the same CUDA graph as the kernel, so a step is one graph launch
+    # plus the wait for its result.
     host_x = torch.cat([inputs.activations(1, k, 2001).reshape(-1) for k in (2560, 6912)]).pin_memory()
-    host_y = torch.empty_like(ys1[n_layers - 1][-1], device="cpu").pin_memory()
+    host_y = torch.empty_like(xs1["yall"], device="cpu").pin_memory()
     h2d = host_x.numel() * 2
     d2h = host_y.numel() * 2
 
     def e2e_body():
         xs1["flat"].copy_(host_x, non_blocking=True)
         step1()
-        host_y.copy_(ys1[n_layers - 1][-1], non_blocking=True)
+        host_y.copy_(xs1["yall"], non_blocking=True)
 
     ge, _ = capture(e2e_body)
 
@@ -328,12 +376,17 @@ def run_ours(args):
     sampler2 = ClockSampler(local).start() if rank == 0 else None  # clocks during the secondary sections
 
     extra, cpu = {}, None
+    gemm_roofline = []  # the int8-TOPS half of the metric: one entry per judged M = 4096 shape
+    per_call_m1 = None
     if rank == 0 and "decode8" in sections:
         gc, lc = capture(chain1)
         msc = time_graph(gc, args.steps, args.warmup, 1)
         gbc = bytes_step * args.steps / (msc * 1e-3) / 1e9
         extra["chain_m1_one_launch_per_matrix"] = {"GBps": gbc, "us_per_launch": msc * 1e3 / (args.steps * lc),
                                                   "frac_of_hbm_peak": gbc / peaks["hbm_gbs"], "launches": lc}
+        per_call_m1 = {"call": "bitrl_bitlinear_forward, one launch per matrix in stream order", "kernel": "gemv_kernel<1>",
+                       "achieved": gbc, "unit": "GB/s", "frac": gbc / peaks["hbm_gbs"],
+                       "us_per_launch": msc * 1e3 / (args.steps * lc)}
         del gc
         _, _, step8, chain8 = decode_setup(8)
         for label, fn in (("sweep_m8_grouped", step8), ("chain_m8_one_launch_per_matrix", chain8)):
@@ -381,86 +434,97 @@ def run_ours(args):
                 del g
             res["int8_peak"] = f"{i8_peak:.0f} TOPS = 2 x bf16 burst peak (of {peak_src})"
             extra[name] = res
+            gemm_roofline.append({
+                "shape": f"M=4096 K={K} N={N}", "bound": "tensor", "unit": "TOPS", "peak": i8_peak,
+                "peak_source": f"2 x bf16 burst, of {peak_src}",
+                "kernel": "gemm_i8_kernel<224,true,true>" if N == 6912 else "gemm_i8_kernel<192,true,true>",
+                "us": res["gemm_kernel"]["us"], "achieved": res["gemm_kernel"]["TOPS"],
+                "frac": res["gemm_kernel"]["frac_of_int8_peak"], "frac_of_nominal_4500": res["gemm_kernel"]["frac_of_nominal_4500"],
+                "layer_us": res["layer"]["us"], "layer_achieved": res["layer"]["TOPS"],
+                "layer_frac": res["layer"]["frac_of_int8_peak"],
+                "layer_frac_of_nominal_4500": res["layer"]["frac_of_nominal_4500"],
+                "algorithmic_ops_per_launch": 2.0 * M * N * K})
             del xs, y, ws, q
 
-        # the higher-precision critic's W8A8 layer at the same M = 4096 shapes (int8 weights, nothing to decode)
-        for name, K, N in (("w8a8_m4096_k2560_n6912", 2560, 6912), ("w8a8_m4096_k6912_n2560", 6912, 2560)):
+        if "critic" in sections:  # Table IV's higher-precision critic layers (W8A8, W4A8)
+            # the higher-precision critic's W8A8 layer at the same M = 4096 shapes (int8 weights, nothing to decode)
+            for name, K, N in (("w8a8_m4096_k2560_n6912", 2560, 6912), ("w8a8_m4096_k6912_n2560", 6912, 2560)):
+                w8 = []
+                for i in range(4):
+                    gen.manual_seed(1400 + i)
+                    w8.append(bitrl.w8_quantize(torch.randn(N, K, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W))
+                xs = [inputs.activations(M, K, 2400 + i).to(dev) for i in range(4)]
+                y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+                ws = torch.empty((int(bitrl.lib().bitrl_w8a8_workspace_bytes(M, K)),), dtype=torch.uint8, device=dev)
+                reps = 12
+
+                def w8_layer():
+                    for i in range(reps):
+                        bitrl.w8a8_forward(*w8[i % 4], xs[i % 4], bitrl.OUT_BF16, y=y, workspace=ws)
+
+                g, _ = capture(w8_layer)
+                ms = time_graph(g, sub_steps, args.warmup, 1)
+                tops = 2.0 * M * N * K * reps * sub_steps / (ms * 1e-3) / 1e12
+                extra[name] = {"layer": {"TOPS": tops, "us": ms * 1e3 / (sub_steps * reps), "frac_of_int8_peak": tops / i8_peak,
+                                         "frac_of_nominal_4500": tops / 4500.0}}
+                del g, xs, y, ws, w8
+
+            # ... and its streaming kernel at M = 1 and 8 over eight 2560 -> 13824 matrices (283 MB of int8 weights, > L2)
             w8 = []
-            for i in range(4):
-                gen.manual_seed(1400 + i)
-                w8.append(bitrl.w8_quantize(torch.randn(N, K, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W))
-            xs = [inputs.activations(M, K, 2400 + i).to(dev) for i in range(4)]
-            y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
-            ws = torch.empty((int(bitrl.lib().bitrl_w8a8_workspace_bytes(M, K)),), dtype=torch.uint8, device=dev)
-            reps = 12
+            for i in range(8):
+                gen.manual_seed(1500 + i)
+                w8.append(bitrl.w8_quantize(torch.randn(13824, 2560, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W))
+            for Ms in (1, 8):
+                xd = inputs.activations(Ms, 2560, 2000 + Ms).to(dev)
+                yd = torch.empty((Ms, 13824), dtype=torch.bfloat16, device=dev)
 
-            def w8_layer():
-                for i in range(reps):
-                    bitrl.w8a8_forward(*w8[i % 4], xs[i % 4], bitrl.OUT_BF16, y=y, workspace=ws)
+                def w8_sweep():
+                    for wq8, sc8 in w8:
+                        bitrl.w8a8_forward(wq8, sc8, xd, bitrl.OUT_BF16, y=yd)
 
-            g, _ = capture(w8_layer)
-            ms = time_graph(g, sub_steps, args.warmup, 1)
-            tops = 2.0 * M * N * K * reps * sub_steps / (ms * 1e-3) / 1e12
-            extra[name] = {"layer": {"TOPS": tops, "us": ms * 1e3 / (sub_steps * reps), "frac_of_int8_peak": tops / i8_peak,
-                                     "frac_of_nominal_4500": tops / 4500.0}}
-            del g, xs, y, ws, w8
+                g, lc = capture(w8_sweep)
+                ms = time_graph(g, sub_steps, args.warmup, 1) / sub_steps
+                gbs = 8 * 13824 * 2560 / (ms * 1e-3) / 1e9
+                extra[f"w8a8_m{Ms}_sweep_8x_k2560_n13824"] = {"GBps_of_weight_bytes": gbs, "us_per_matrix": ms * 1e3 / 8,
+                                                             "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "launches": lc}
+                del g
+            del w8
 
-        # ... and its streaming kernel at M = 1 and 8 over eight 2560 -> 13824 matrices (283 MB of int8 weights, > L2)
-        w8 = []
-        for i in range(8):
-            gen.manual_seed(1500 + i)
-            w8.append(bitrl.w8_quantize(torch.randn(13824, 2560, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W))
-        for Ms in (1, 8):
-            xd = inputs.activations(Ms, 2560, 2000 + Ms).to(dev)
-            yd = torch.empty((Ms, 13824), dtype=torch.bfloat16, device=dev)
+            # the INT4 critic's W4A8 layer: streaming kernel at M = 1 over eight 2560 -> 13824 matrices (141 MB packed),
+            # and the whole layer at M = 4096 (int8 expansion into the workspace, then the W8A8 GEMM)
+            w4 = []
+            for i in range(8):
+                gen.manual_seed(1600 + i)
+                w4.append(bitrl.w4_quantize(torch.randn(13824, 2560, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W))
+            xd = inputs.activations(1, 2560, 2001).to(dev)
+            yd = torch.empty((1, 13824), dtype=torch.bfloat16, device=dev)
 
-            def w8_sweep():
-                for wq8, sc8 in w8:
-                    bitrl.w8a8_forward(wq8, sc8, xd, bitrl.OUT_BF16, y=yd)
+            def w4_sweep():
+                for p4, sc4 in w4:
+                    bitrl.w4a8_forward(p4, sc4, xd, bitrl.OUT_BF16, y=yd)
 
-            g, lc = capture(w8_sweep)
+            g, lc = capture(w4_sweep)
             ms = time_graph(g, sub_steps, args.warmup, 1) / sub_steps
-            gbs = 8 * 13824 * 2560 / (ms * 1e-3) / 1e9
-            extra[f"w8a8_m{Ms}_sweep_8x_k2560_n13824"] = {"GBps_of_weight_bytes": gbs, "us_per_matrix": ms * 1e3 / 8,
-                                                         "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "launches": lc}
-            del g
-        del w8
+            gbs = 8 * 13824 * 2560 / 2 / (ms * 1e-3) / 1e9
+            extra["w4a8_m1_sweep_8x_k2560_n13824"] = {"GBps_of_packed_bytes": gbs, "us_per_matrix": ms * 1e3 / 8,
+                                                       "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "launches": lc}
+            del g, w4
+            gen.manual_seed(1700)
+            p4, sc4 = bitrl.w4_quantize(torch.randn(6912, 2560, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W)
+            xs = [inputs.activations(M, 2560, 2400 + i).to(dev) for i in range(4)]
+            y = torch.empty((M, 6912), dtype=torch.bfloat16, device=dev)
+            ws = torch.empty((int(bitrl.lib().bitrl_w4a8_workspace_bytes(M, 2560, 6912)),), dtype=torch.uint8, device=dev)
 
-        # the INT4 critic's W4A8 layer: streaming kernel at M = 1 over eight 2560 -> 13824 matrices (141 MB packed),
-        # and the whole layer at M = 4096 (int8 expansion into the workspace, then the W8A8 GEMM)
-        w4 = []
-        for i in range(8):
-            gen.manual_seed(1600 + i)
-            w4.append(bitrl.w4_quantize(torch.randn(13824, 2560, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W))
-        xd = inputs.activations(1, 2560, 2001).to(dev)
-        yd = torch.empty((1, 13824), dtype=torch.bfloat16, device=dev)
+            def w4_layer():
+                for i in range(12):
+                    bitrl.w4a8_forward(p4, sc4, xs[i % 4], bitrl.OUT_BF16, y=y, workspace=ws)
 
-        def w4_sweep():
-            for p4, sc4 in w4:
-                bitrl.w4a8_forward(p4, sc4, xd, bitrl.OUT_BF16, y=yd)
-
-        g, lc = capture(w4_sweep)
-        ms = time_graph(g, sub_steps, args.warmup, 1) / sub_steps
-        gbs = 8 * 13824 * 2560 / 2 / (ms * 1e-3) / 1e9
-        extra["w4a8_m1_sweep_8x_k2560_n13824"] = {"GBps_of_packed_bytes": gbs, "us_per_matrix": ms * 1e3 / 8,
-                                                   "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "launches": lc}
-        del g, w4
-        gen.manual_seed(1700)
-        p4, sc4 = bitrl.w4_quantize(torch.randn(6912, 2560, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W)
-        xs = [inputs.activations(M, 2560, 2400 + i).to(dev) for i in range(4)]
-        y = torch.empty((M, 6912), dtype=torch.bfloat16, device=dev)
-        ws = torch.empty((int(bitrl.lib().bitrl_w4a8_workspace_bytes(M, 2560, 6912)),), dtype=torch.uint8, device=dev)
-
-        def w4_layer():
-            for i in range(12):
-                bitrl.w4a8_forward(p4, sc4, xs[i % 4], bitrl.OUT_BF16, y=y, workspace=ws)
-
-        g, _ = capture(w4_layer)
-        ms = time_graph(g, sub_steps, args.warmup, 1)
-        tops = 2.0 * M * 6912 * 2560 * 12 * sub_steps / (ms * 1e-3) / 1e12
-        extra["w4a8_m4096_k2560_n6912"] = {"layer": {"TOPS": tops, "us": ms * 1e3 / (sub_steps * 12),
-                                                     "frac_of_int8_peak": tops / i8_peak}}
-        del g, xs, y, ws
+            g, _ = capture(w4_layer)
+            ms = time_graph(g, sub_steps, args.warmup, 1)
+            tops = 2.0 * M * 6912 * 2560 * 12 * sub_steps / (ms * 1e-3) / 1e12
+            extra["w4a8_m4096_k2560_n6912"] = {"layer": {"TOPS": tops, "us": ms * 1e3 / (sub_steps * 12),
+                                                         "frac_of_int8_peak": tops / i8_peak}}
+            del g, xs, y, ws
 
         # configs[2]: batched state encoding, M = 64 and 256 (one token per state), the whole layer per call
         for M in (64, 256):
@@ -483,6 +547,22 @@ def run_ours(args):
                                                   "launches_per_layer": lc / reps}
                 del g, xs, y, ws
 
+    if world > 1 and "encoder" in sections:
+        # config 5 with its 4096 token rows sharded over the ranks (strong scaling: the same 128 states, fewer per GPU);
+        # rows are independent, so every rank encodes its own contiguous block of states and nothing is exchanged
+        from paper_2604_24273_b200.sharding import shard_rows
+
+        row0, rows = shard_rows(4096, world, rank)
+        enc_s = bitrl.Encoder(layers, 2560, 6912, 20, 5)
+        hs = inputs.activations(4096, 2560, 6000)[row0:row0 + rows].contiguous().to(dev)
+        hs_out = torch.empty_like(hs)
+        ws_s = torch.empty((enc_s.workspace_bytes(rows),), dtype=torch.uint8, device=dev)
+        gs_, _ = capture(lambda: enc_s.forward(hs, h_out=hs_out, workspace=ws_s))
+        ms_s = time_graph(gs_, sub_steps, args.warmup, world) / sub_steps
+        extra[f"encoder_{n_layers}_blocks_T4096_rows_sharded_x{world}"] = {
+            "ms": ms_s, "states_per_s": 128.0 / (ms_s * 1e-3), "rows_per_rank": rows, "scaling": "strong"}
+        del gs_, enc_s, hs, hs_out, ws_s
+
     if rank == 0 and "encoder" in sections:
         T = 4096  # 128 states x 32 tokens
         enc = bitrl.Encoder(layers, 2560, 6912, 20, 5)
@@ -493,9 +573,12 @@ def run_ours(args):
         mse = time_graph(ge, sub_steps, args.warmup, 1) / sub_steps
         enc_ops = 2.0 * T * sum(k * n for _, k, n in BLOCK) * n_layers
         i8_sus = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
+        i8_burst = peaks["bf16_tflops"] * INT8_OVER_BF16
+        enc_tops = enc_ops / (mse * 1e-3) / 1e12
         extra[f"encoder_{n_layers}_blocks_T4096"] = {
-            "states_per_s": 128.0 / (mse * 1e-3), "ms": mse, "TOPS": enc_ops / (mse * 1e-3) / 1e12,
-            "frac_of_int8_peak_sustained": enc_ops / (mse * 1e-3) / 1e12 / i8_sus, "launches": le}
+            "states_per_s": 128.0 / (mse * 1e-3), "ms": mse, "TOPS": enc_tops,
+            "frac_of_int8_peak_sustained": enc_tops / i8_sus, "frac_of_int8_peak_burst": enc_tops / i8_burst,
+            "frac_of_nominal_4500": enc_tops / 4500.0, "launches": le}
         del ge
         # the same stack with real attention inside each state: equal 32-token states, then ragged 15-40-token ones
         pooled = torch.empty((128, 2560), dtype=torch.bfloat16, device=dev)
@@ -557,8 +640,10 @@ def run_ours(args):
         del gu
     bitrl.poll_status()
     clocks_sections = sampler2.stop() if sampler2 else None
+    cpu_other = None
     if rank == 0 and "cpu" in sections:
         cpu = oracle_decode_sample()
+        cpu_other = oracle_batched_samples()
 
     if rank == 0:
         achieved = gbs1 / world
@@ -578,8 +663,10 @@ def run_ours(args):
                          "frac": achieved / peaks["hbm_gbs"],
                          "traffic": None if HEADLINE_TRAFFIC_PER_BLOCK is None else HEADLINE_TRAFFIC_PER_BLOCK * n_layers, "peak_source": f"of {peak_src}",
                          "kernel": "gemv_multi_dp4a_kernel<1>", "us_per_launch": us_per_launch,
-                         "algorithmic_bytes_per_launch": bytes_step / launches1},
+                         "algorithmic_bytes_per_launch": bytes_step / launches1,
+                         "ms_per_step_spread": spread1, "per_call_m1": per_call_m1, "gemm": gemm_roofline},
             "cpu_baseline": cpu,
+            "cpu_baseline_batched": cpu_other,
             "e2e": {"value": e2e_gbs, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms / args.steps},
             "gpu_launches": launches1 * args.steps,
@@ -593,6 +680,22 @@ def run_ours(args):
         torch.distributed.destroy_process_group()
 
 
+def free_port() -> int:
+    import socket
+
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def self_launch(n: int) -> int:
+    """Re-runs this command line as n ranks (one process per GPU) on this node through torch.distributed.run; the
+    ranks' output passes through, so rank 0's JSON line is this process's JSON line."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -600,9 +703,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=FULL_LAYERS, help="blocks in the backbone (30 = full model)")
-    ap.add_argument("--sections", default="decode8,gemm,encoder,cpu",
+    ap.add_argument("--sections", default="decode8,gemm,critic,encoder,cpu",
                     help="secondary measurements besides the M=1 headline (comma list; empty = none)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(self_launch(args.gpus))  # started as plain `python bench.py --gpus N`: become N ranks
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -75,7 +75,8 @@ BITRL_API bitrl_status bitrl_pack_ternary(const float* W, int32_t N, int32_t K, 
  * fixed 8 KB array that is part of the library image on every GPU that loads it, for the life of the process.
  *  - Limit: N*K <= BITRL_PACK_STATIC_MAX_WEIGHTS; larger matrices return BITRL_ERR_LIMIT and nothing is launched.
  *  - Calls no allocator of any kind.  The first call on a device looks up the array's device address (once per
- *    device, with that device current); make that first call outside any stream capture.
+ *    device, with that device current); make that first call outside any stream capture.  The address is kept for
+ *    the life of the device's context: after cudaDeviceReset the library must be reloaded before this call is used again.
  *  - All calls share the array and it keeps the previous call's contents.  Nothing in it has to start at zero:
  *    every slot that a call reads is written earlier in the same call.  Two calls that overlap on the GPU (different
  *    streams, or threads) race on it and may both produce a wrong gamma; serialize them. */
@@ -84,7 +85,9 @@ BITRL_API bitrl_status bitrl_pack_ternary_static(const float* W, int32_t N, int3
                                                  void* stream);
 
 /* Builds the weight handle from the canonical packed bytes and gamma (both dev).  The library keeps its own
- * re-tiled copy (N*K/4 bytes); the inputs may be freed once `stream` has run past this call. */
+ * re-tiled copy (N*K/4 bytes).  The call returns after the copy is complete (it synchronizes `stream`: handle creation
+ * is offline work and already allocates), so the inputs may be freed at once and the handle may be used on any stream.
+ * The forward kernels treat a handle's weights as immutable and fetch them before they wait for preceding kernels. */
 BITRL_API bitrl_status bitrl_linear_create(const uint8_t* packed, const float* gamma, int32_t N, int32_t K,
                                  bitrl_linear_t** out, void* stream);
 BITRL_API bitrl_status bitrl_linear_destroy(bitrl_linear_t* w);

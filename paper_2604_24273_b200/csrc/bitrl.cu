@@ -209,6 +209,8 @@ bitrl_status bitrl_linear_create(const uint8_t* packed, const float* gamma, int3
     return cuda_fail(e);
   }
   s = launch_retile(packed, N, K, w->l.tiles, st);
+  // The handle is complete when this returns: the forward kernels prefetch weights ahead of their stream dependencies.
+  if (s == BITRL_OK && cudaStreamSynchronize(st) != cudaSuccess) s = cuda_fail(cudaGetLastError());
   if (s != BITRL_OK) {
     cudaFree(w->l.tiles);
     cudaFree(w->l.gamma);

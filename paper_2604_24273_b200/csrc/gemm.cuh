@@ -50,7 +50,7 @@ constexpr uint32_t GM_OFF_BAR = GM_OFF_TOK + 2 * GM_TOK_MAX * 8;
 constexpr uint32_t GM_XS_MAX = 16;
 constexpr uint32_t GM_NUM_BARS = 2 * GM_XS_MAX + 2 * GM_PS + 2 * GM_WS + 4;
 constexpr uint32_t GM_OFF_MISC = GM_OFF_BAR + GM_NUM_BARS * 8;
-constexpr uint32_t GM_SMEM_BYTES = GM_OFF_MISC + 16 + 1024;  // + slack to align the base to 1024
+constexpr uint32_t GM_SMEM_BYTES = GM_OFF_MISC + 32 + 1024;  // + slack to align the base to 1024
 static_assert(GM_SMEM_BYTES <= 232448, "shared memory budget of one CTA");
 
 // stage ids reported with BITRL_ERR_TIMEOUT
@@ -113,12 +113,24 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   const uint32_t bar_tmem_full = bar_w_empty + 8 * GM_WS;  // [2]
   const uint32_t bar_tmem_empty = bar_tmem_full + 16;      // [2]
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + GM_OFF_MISC);
+  // Set by the first role whose wait ran out of time (in both CTAs of a pair).  Every wait polls it, so the other
+  // roles stop within a few hundred polls instead of each waiting out its own limit, and the teardown drains.
+  volatile uint32_t* failed = reinterpret_cast<volatile uint32_t*>(base_ptr + GM_OFF_MISC + 8);
+  const uint32_t failed_addr = base + GM_OFF_MISC + 8;
+  const uint32_t bar_drain = base + GM_OFF_MISC + 16;  // only used on the failure path
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kblocks = a.K / GM_BK;
   const int items = a.tiles_total * a.splits;
   // PAIR: both CTAs of a cluster walk the same items (tiles_n then counts 256-row tiles); rank selects the halves.
   const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;
+  const uint32_t failed_peer = PAIR ? ptx::mapa_u32(failed_addr, rank ^ 1u) : 0u;
+  auto wait = [&](uint32_t bar, uint32_t parity) { return ptx::mbar_wait_abortable(bar, parity, failed_addr); };
+  auto give_up = [&](int stage) {
+    report_timeout(stage);
+    *failed = 1u;
+    if (PAIR) asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(failed_peer), "r"(1u) : "memory");
+  };
   const int item0 = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
   const int item_step = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
   const uint32_t x_full_lead = PAIR ? ptx::mapa_u32(bar_x_full, 0) : bar_x_full;        // as seen from either CTA
@@ -130,6 +142,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   };
 
   if (threadIdx.x == 0) {
+    *failed = 0u;
+    ptx::mbar_init(bar_drain, 1);
     // x_full: the producer's expect_tx arrival plus one arrival per expander warp (of both CTAs when paired)
     for (int s = 0; s < GM_XS; ++s) {
       ptx::mbar_init(bar_x_full + 8 * s, PAIR ? 1 + 8 : 1 + 4);
@@ -170,7 +184,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
         const int tm = tile / a.tiles_n;
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const uint32_t s = it % GM_XS, ph = (it / GM_XS) & 1u;
-          if (!ptx::mbar_wait(bar_x_empty + 8 * s, ph ^ 1u)) { report_timeout(GM_WAIT_X_EMPTY); ok = false; break; }
+          if (!wait(bar_x_empty + 8 * s, ph ^ 1u)) { give_up(GM_WAIT_X_EMPTY); ok = false; break; }
           if (PAIR) {
             // Rank 0 announces the bytes of both halves on its barrier; each CTA's copy reports there.
             if (rank == 0) ptx::mbar_arrive_expect_tx(bar_x_full + 8 * s, 2 * GM_X_BYTES);
@@ -195,7 +209,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
         const uint8_t* wsrc = a.tiles + static_cast<size_t>(tn) * kblocks * TILE_BYTES;
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const uint32_t s = it % GM_PS, ph = (it / GM_PS) & 1u;
-          if (!ptx::mbar_wait(bar_p_empty + 8 * s, ph ^ 1u)) { report_timeout(GM_WAIT_P_EMPTY); ok = false; break; }
+          if (!wait(bar_p_empty + 8 * s, ph ^ 1u)) { give_up(GM_WAIT_P_EMPTY); ok = false; break; }
           ptx::mbar_arrive_expect_tx(bar_p_full + 8 * s, GM_P_BYTES);
           ptx::bulk_g2s(base + GM_OFF_P + s * GM_P_BYTES, wsrc + static_cast<size_t>(kb) * TILE_BYTES, GM_P_BYTES,
                         bar_p_full + 8 * s);
@@ -215,16 +229,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
         int tile, kb0, kb1;
         item_range(item, tile, kb0, kb1);
         const uint32_t buf = lt & 1u;
-        if (!__any_sync(0xffffffffu, ptx::mbar_wait(bar_tmem_empty + 8 * buf, ((lt >> 1) & 1u) ^ 1u))) {
-          if (lane == 0) report_timeout(GM_WAIT_TMEM_EMPTY);
+        if (!__any_sync(0xffffffffu, wait(bar_tmem_empty + 8 * buf, ((lt >> 1) & 1u) ^ 1u))) {
+          if (lane == 0) give_up(GM_WAIT_TMEM_EMPTY);
           ok = false;
           break;
         }
         const uint32_t d_tmem = tmem_base + buf * GM_TOK_MAX;
         ptx::tc_fence_after_sync();  // orders this tile's MMAs after the epilogue's reads of the accumulator
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!__any_sync(0xffffffffu, ptx::mbar_wait(bar_x_full + 8 * xs, xph))) {
-            if (lane == 0) report_timeout(GM_WAIT_X_FULL);
+          if (!__any_sync(0xffffffffu, wait(bar_x_full + 8 * xs, xph))) {
+            if (lane == 0) give_up(GM_WAIT_X_FULL);
             ok = false;
             break;
           }
@@ -293,11 +307,21 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
           if (++xs == GM_XS) xs = 0;
           continue;
         }
-        if (!ptx::mbar_wait(bar_p_full + 8 * ps, pph)) { report_timeout(GM_WAIT_P_FULL); ok = false; break; }
+        // All lanes poll the same barrier; a phase that one lane saw complete is complete, so the vote makes the
+        // outcome warp-uniform (the tcgen05.st below is a whole-warp instruction).
+        if (!__any_sync(0xffffffffu, wait(bar_p_full + 8 * ps, pph))) {
+          if (lane == 0) give_up(GM_WAIT_P_FULL);
+          ok = false;
+          break;
+        }
         const uint32_t paddr = base + GM_OFF_P + ps * GM_P_BYTES + r * TILE_ROW_BYTES;
         const uint4 p0 = ptx::lds128(paddr), p1 = ptx::lds128(paddr + 16);
         if (it >= WSK) {
-          if (!ptx::mbar_wait(bar_x_empty + 8 * xs_old, xph_old)) { report_timeout(GM_WAIT_W_EMPTY); ok = false; break; }
+          if (!__any_sync(0xffffffffu, wait(bar_x_empty + 8 * xs_old, xph_old))) {
+            if (lane == 0) give_up(GM_WAIT_W_EMPTY);
+            ok = false;
+            break;
+          }
           if (++xs_old == GM_XS) { xs_old = 0; xph_old ^= 1u; }
         }
         if (A_TMEM) ptx::tc_fence_after_sync();
@@ -361,8 +385,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
         ptx::sts32(sc_addr + 4 * j, __float_as_uint(tok < a.M ? out_scale(gamma, a.absmax[tok]) : 0.0f));
         ptx::sts32(rs_addr + 4 * j, static_cast<uint32_t>(tok < a.M ? a.rowsum[tok] : 0));
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (!ptx::mbar_wait(bar_tmem_full + 8 * buf, (lt >> 1) & 1u)) { report_timeout(GM_WAIT_TMEM_FULL); ok = false; break; }
+      // The named barrier that publishes the scales also ANDs the outcome of the wait over the four epilogue warps, so
+      // that they either all go on (to whole-warp tensor-memory loads and the next round of this barrier) or all leave.
+      if (!ptx::bar_red_and(1, 128, wait(bar_tmem_full + 8 * buf, (lt >> 1) & 1u))) {
+        if (ep == 0) give_up(GM_WAIT_TMEM_FULL);
+        ok = false;
+        break;
+      }
       ptx::tc_fence_after_sync();
       const int nbase = tn * GM_ROWS + q * 32;  // first output column of this warp
       const int tok0 = tm * GM_TOK;
@@ -471,6 +500,23 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   ptx::tc_fence_before_sync();
   __syncthreads();
   if (PAIR) ptx::cluster_sync_all();  // neither CTA leaves (or frees tensor memory) while the other may still reach it
+  if (*failed) {
+    // Failure path only: a role gave up, so copies and MMAs that nobody waited for may still be in flight.  The MMA
+    // issuer waits (bounded) for its MMAs, then every thread lets about a millisecond pass, far longer than any copy
+    // takes, before shared and tensor memory are given back.
+    if (warp == 1 && rank == 0) {
+      if (ptx::elect_one()) {
+        if (PAIR) ptx::mma_commit_pair(bar_drain, 1);
+        else ptx::mma_commit(bar_drain);
+      }
+      __syncwarp();
+      ptx::mbar_wait(bar_drain, 0, 2000000LL);
+    }
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) {}
+    __syncthreads();
+    if (PAIR) ptx::cluster_sync_all();  // `failed` is the same in both CTAs after the first cluster barrier
+  }
   if (warp == 1) {
     ptx::tc_fence_after_sync();
     if (PAIR) ptx::tmem_dealloc_pair(tmem_base, 512);
@@ -589,7 +635,11 @@ inline int gemm_pair_max_clusters(int tok) {
     }
     cached[dev][slot] = n;
   }
-  return cached[dev][slot] > 0 ? cached[dev][slot] : 0;
+  if (cached[dev][slot] > 0) return cached[dev][slot];
+  // The occupancy query can fail under a profiler.  When the paired kernel is forced (BITRL_GEMM_PAIR=1) fall back to
+  // one cluster per SM pair: the grid is a static partition of the tiles, CTAs wait only on their own cluster peer, so
+  // a grid larger than what is resident at once is merely queued.
+  return gemm_pair_mode() == 1 ? sm_count() / 2 : 0;
 }
 
 // Largest M for which a split-K workspace (M*N int32) is offered.

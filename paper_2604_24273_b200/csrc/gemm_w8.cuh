@@ -31,7 +31,7 @@ constexpr uint32_t G8_OFF_STAGE = G8_RING_BYTES;                      // 4 x 2 K
 constexpr uint32_t G8_OFF_TOK = G8_OFF_STAGE + 4 * 2048;              // scale[2][256] f32
 constexpr uint32_t G8_OFF_BAR = G8_OFF_TOK + 2 * 256 * 4;
 constexpr uint32_t G8_OFF_MISC = G8_OFF_BAR + (2 * G8_MAX_STAGES + 4) * 8;
-constexpr uint32_t G8_SMEM_BYTES = G8_OFF_MISC + 16 + 1024;           // + slack to align the base to 1024
+constexpr uint32_t G8_SMEM_BYTES = G8_OFF_MISC + 32 + 1024;           // + slack to align the base to 1024
 static_assert(G8_SMEM_BYTES <= 232448, "shared memory budget of one CTA");
 
 constexpr int G8_PAIR_MIN_M = 2048;  // paired CTAs from this M on
@@ -69,6 +69,10 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   const uint32_t bar_tmem_full = bar_empty + 8 * G8_MAX_STAGES;  // [2]
   const uint32_t bar_tmem_empty = bar_tmem_full + 16;            // [2]
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + G8_OFF_MISC);
+  // Set by the first role whose wait ran out of time (in both CTAs of a pair); every wait polls it.
+  volatile uint32_t* failed = reinterpret_cast<volatile uint32_t*>(base_ptr + G8_OFF_MISC + 8);
+  const uint32_t failed_addr = base + G8_OFF_MISC + 8;
+  const uint32_t bar_drain = base + G8_OFF_MISC + 16;  // only used on the failure path
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kblocks = a.K / 128;
@@ -77,8 +81,17 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   const int tile_step = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
   const uint32_t full_lead = PAIR ? ptx::mapa_u32(bar_full, 0) : bar_full;  // rank 0's barriers as seen from either CTA
   const uint32_t tmem_empty_lead = PAIR ? ptx::mapa_u32(bar_tmem_empty, 0) : bar_tmem_empty;
+  const uint32_t failed_peer = PAIR ? ptx::mapa_u32(failed_addr, rank ^ 1u) : 0u;
+  auto wait = [&](uint32_t bar, uint32_t parity) { return ptx::mbar_wait_abortable(bar, parity, failed_addr); };
+  auto give_up = [&](int stage) {
+    report_timeout(stage);
+    *failed = 1u;
+    if (PAIR) asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(failed_peer), "r"(1u) : "memory");
+  };
 
   if (threadIdx.x == 0) {
+    *failed = 0u;
+    ptx::mbar_init(bar_drain, 1);
     for (uint32_t s = 0; s < NS; ++s) { ptx::mbar_init(bar_full + 8 * s, 1); ptx::mbar_init(bar_empty + 8 * s, 1); }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(bar_tmem_full + 8 * b, 1);
@@ -112,7 +125,7 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       for (int tile = tile0; ok && tile < a.tiles_total; tile += tile_step) {
         const int tn = PAIR ? 2 * (tile % a.tiles_n) + static_cast<int>(rank) : tile % a.tiles_n, tm = tile / a.tiles_n;
         for (int kb = 0; kb < kblocks; ++kb) {
-          if (!ptx::mbar_wait(bar_empty + 8 * s, ph ^ 1u)) { report_timeout(G8_WAIT_EMPTY); ok = false; break; }
+          if (!wait(bar_empty + 8 * s, ph ^ 1u)) { give_up(G8_WAIT_EMPTY); ok = false; break; }
           if (PAIR) {
             // Rank 0 announces the bytes of both CTAs' stages on its barrier; each CTA's copies report there.
             if (rank == 0) ptx::mbar_arrive_expect_tx(bar_full + 8 * s, 2 * STAGE);
@@ -139,16 +152,16 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       bool ok = true;
       for (int tile = tile0; ok && tile < a.tiles_total; tile += tile_step, ++lt) {
         const uint32_t buf = lt & 1u;
-        if (!__any_sync(0xffffffffu, ptx::mbar_wait(bar_tmem_empty + 8 * buf, ((lt >> 1) & 1u) ^ 1u))) {
-          if (lane == 0) report_timeout(G8_WAIT_TMEM_EMPTY);
+        if (!__any_sync(0xffffffffu, wait(bar_tmem_empty + 8 * buf, ((lt >> 1) & 1u) ^ 1u))) {
+          if (lane == 0) give_up(G8_WAIT_TMEM_EMPTY);
           ok = false;
           break;
         }
         const uint32_t d_tmem = tmem_base + buf * 256;
         ptx::tc_fence_after_sync();
         for (int kb = 0; kb < kblocks; ++kb) {
-          if (!__any_sync(0xffffffffu, ptx::mbar_wait(bar_full + 8 * s, ph))) {
-            if (lane == 0) report_timeout(G8_WAIT_FULL);
+          if (!__any_sync(0xffffffffu, wait(bar_full + 8 * s, ph))) {
+            if (lane == 0) give_up(G8_WAIT_FULL);
             ok = false;
             break;
           }
@@ -195,8 +208,13 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         const int tok = tm * TOK + j;
         ptx::sts32(sc_addr + 4 * j, __float_as_uint(tok < a.M ? out_scale(wscale, a.absmax[tok]) : 0.0f));
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (!ptx::mbar_wait(bar_tmem_full + 8 * buf, (lt >> 1) & 1u)) { report_timeout(G8_WAIT_TMEM_FULL); ok = false; break; }
+      // The named barrier that publishes the scales also ANDs the outcome of the wait over the four epilogue warps:
+      // they all go on (whole-warp tensor-memory loads, the next round of this barrier) or all leave.
+      if (!ptx::bar_red_and(1, 128, wait(bar_tmem_full + 8 * buf, (lt >> 1) & 1u))) {
+        if (ep == 0) give_up(G8_WAIT_TMEM_FULL);
+        ok = false;
+        break;
+      }
       ptx::tc_fence_after_sync();
       const int nbase = tn * 128 + q * 32;
       const int tok0 = tm * TOK;
@@ -288,6 +306,22 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   ptx::tc_fence_before_sync();
   __syncthreads();
   if (PAIR) ptx::cluster_sync_all();  // neither CTA leaves (or frees tensor memory) while the other may still reach it
+  if (*failed) {
+    // Failure path only: copies and MMAs that nobody waited for may still be in flight.  The MMA issuer waits (bounded)
+    // for its MMAs, then every thread lets about a millisecond pass before shared and tensor memory are given back.
+    if (warp == 1 && rank == 0) {
+      if (ptx::elect_one()) {
+        if (PAIR) ptx::mma_commit_pair(bar_drain, 1);
+        else ptx::mma_commit(bar_drain);
+      }
+      __syncwarp();
+      ptx::mbar_wait(bar_drain, 0, 2000000LL);
+    }
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) {}
+    __syncthreads();
+    if (PAIR) ptx::cluster_sync_all();  // `failed` is the same in both CTAs after the first cluster barrier
+  }
   if (warp == 1) {
     ptx::tc_fence_after_sync();
     if (PAIR) ptx::tmem_dealloc_pair(tmem_base, 512);
@@ -326,7 +360,11 @@ inline int gemm_w8_pair_max_clusters(int tok) {
     }
     cached[dev][slot] = n;
   }
-  return cached[dev][slot] > 0 ? cached[dev][slot] : 0;
+  if (cached[dev][slot] > 0) return cached[dev][slot];
+  // The occupancy query can fail under a profiler.  When the paired kernel is forced (BITRL_GEMM_PAIR=1) fall back to
+  // one cluster per SM pair: the grid is a static partition of the tiles, CTAs wait only on their own cluster peer, so
+  // a grid larger than what is resident at once is merely queued.
+  return gemm_pair_mode() == 1 ? sm_count() / 2 : 0;
 }
 
 // ---- M <= 16: streaming kernel ----------------------------------------------------------------------------------

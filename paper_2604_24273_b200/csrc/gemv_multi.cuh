@@ -542,6 +542,24 @@ inline int gvm_depth_log2(int M, int kmax) {
   return -1;
 }
 
+// Two ranges per CTA (see GvmArgs::seg): long units from the head of the work list while they fit the CTA's share of
+// the remaining pieces, then short units from the tail up to the nearest fit.  `sz` = pieces of every unit in list order.
+inline void gvm_partition(const std::vector<int>& sz, long long pieces, int grid, int (*seg)[4]) {
+  int head = 0, tail = static_cast<int>(sz.size());
+  long long remaining = pieces;
+  for (int c = 0; c < grid; ++c) {
+    const double target = static_cast<double>(remaining) / (grid - c);
+    long long load = 0;
+    seg[c][0] = head;
+    while (head < tail && (c == grid - 1 || load + sz[head] <= target)) load += sz[head++];
+    seg[c][1] = head;
+    seg[c][3] = tail;
+    while (head < tail && load + sz[tail - 1] <= target + 0.5 * sz[tail - 1]) load += sz[--tail];
+    seg[c][2] = tail;
+    remaining -= load;
+  }
+}
+
 bitrl_status launch_gemv_multi(int count, const Linear* const* w, const void* const* x, void* const* y, int M,
                                int out_dtype, cudaStream_t st) {
   static thread_local GvmArgs a;  // 7 KB, kept off the stack
@@ -569,25 +587,11 @@ bitrl_status launch_gemv_multi(int count, const Linear* const* w, const void* co
   int grid = sm_count();
   if (grid > GVM_MAX_CTAS) grid = GVM_MAX_CTAS;
   if (grid > units) grid = units;
-  // Two ranges per CTA (see GvmArgs::seg): long tiles from the head of the list while they fit the CTA's share of
-  // the remaining pieces, then short tiles from the tail up to the nearest fit.
   {
     static thread_local std::vector<int> sz;  // 4 KB pieces of every unit, in work-list order
     sz.clear();
     for (int j = 0; j < count; ++j) sz.insert(sz.end(), a.jobs[j].N / TILE_ROWS, a.jobs[j].K / TILE_K);
-    int head = 0, tail = units;
-    long long remaining = pieces;
-    for (int c = 0; c < grid; ++c) {
-      const double target = static_cast<double>(remaining) / (grid - c);
-      long long load = 0;
-      a.seg[c][0] = head;
-      while (head < tail && (c == grid - 1 || load + sz[head] <= target)) load += sz[head++];
-      a.seg[c][1] = head;
-      a.seg[c][3] = tail;
-      while (head < tail && load + sz[tail - 1] <= target + 0.5 * sz[tail - 1]) load += sz[--tail];
-      a.seg[c][2] = tail;
-      remaining -= load;
-    }
+    gvm_partition(sz, pieces, grid, a.seg);
   }
   a.njobs = count;
   a.M = M;

@@ -64,6 +64,36 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
   }
 }
 
+// Bounded wait that also gives up as soon as the shared-memory word at `abort_flag` becomes non-zero: once one role
+// of a CTA has run out of time, the others need not each wait out their own limit.
+__device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, uint32_t abort_flag,
+                                                    long long limit_cycles = WAIT_LIMIT_CYCLES) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    uint32_t f;
+    asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(f) : "r"(abort_flag));
+    if (f != 0 || clock64() - t0 > limit_cycles) return false;
+  }
+}
+
+// Barrier over `nthreads` threads of the CTA (named barrier `id`) that also ANDs a predicate over them.
+__device__ __forceinline__ bool bar_red_and(uint32_t id, uint32_t nthreads, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %3, 0;\n\t"
+      "barrier.cta.red.and.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"(id), "r"(nthreads), "r"(static_cast<uint32_t>(pred))
+      : "memory");
+  return r != 0;
+}
+
 // Bounded wait on two barriers at once: both are polled in every round, so their latencies overlap.
 __device__ __forceinline__ bool mbar_wait2(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b,
                                            long long limit_cycles = WAIT_LIMIT_CYCLES) {

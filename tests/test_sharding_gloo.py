@@ -62,3 +62,19 @@ def test_two_rank_row_sharding_gloo():
         p.join(timeout=60)
         assert p.exitcode == 0
     assert ok and t == 11.0
+
+
+def test_bench_starts_its_own_ranks():
+    """`python bench.py --gpus 2` with no WORLD_SIZE in the environment becomes two ranks by itself; here on CPU with the
+    reference arm (rank 0 alone works and prints, the other rank exits 0): one JSON line with n_gpus = 2."""
+    import json
+    import subprocess
+
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--steps", "1",
+                        "--warmup", "0"], env=env, cwd=ROOT, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["impl"] == "reference" and d["value"] > 0

@@ -30,13 +30,21 @@ def B():
 
 
 def test_static_scratch_pack_matches_workspace_pack_twice(B):
+    warm = inputs.master_weights(128, 128, 40).cuda()  # first call on the device: looks the scratch address up
+    B.pack_ternary_static(warm, torch.empty((128, 32), dtype=torch.uint8, device="cuda"),
+                          torch.empty((1,), dtype=torch.float32, device="cuda"))
     for N, K, seed in ((2560, 6912, 41), (384, 256, 42), (2560, 3840, 43)):
         W = inputs.master_weights(N, K, seed).cuda()
         want_packed, want_gamma = B.pack_ternary(W)
         packed = torch.full((N, K // 4), 0xAA, dtype=torch.uint8, device="cuda")
         gamma = torch.full((1,), -1.0, dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         B.pack_ternary_static(W, packed, gamma)
         B.poll_status()
+        # the property the entry point exists for: the device's free memory is what it was (after the first call on the
+        # device, which loads nothing either - the scratch array is part of the library image)
+        assert torch.cuda.mem_get_info()[0] == free_before
         assert torch.equal(gamma.view(torch.int32), want_gamma.view(torch.int32))  # bit-identical scale
         assert torch.equal(packed, want_packed)                                    # byte-identical codes
 
@@ -46,9 +54,11 @@ def test_static_scratch_pack_rejects_oversize_and_bad_arguments(B):
     W = inputs.master_weights(128, 128, 44).cuda()
     packed = torch.empty((128, 32), dtype=torch.uint8, device="cuda")
     gamma = torch.empty((1,), dtype=torch.float32, device="cuda")
+    launches = B.launch_count()
     # 65536 x 8192 = 2^29 weights is beyond the 2^28 limit: refused before anything is launched or read
     assert L.bitrl_pack_ternary_static(W.data_ptr(), 65536, 8192, packed.data_ptr(), gamma.data_ptr(), None) == B.ERR_LIMIT
     assert L.bitrl_pack_ternary_static(None, 128, 128, packed.data_ptr(), gamma.data_ptr(), None) == B.ERR_NULL
     assert L.bitrl_pack_ternary_static(W.data_ptr(), 100, 128, packed.data_ptr(), gamma.data_ptr(), None) == B.ERR_SHAPE
+    assert B.launch_count() == launches  # a refused call launches nothing
     assert L.bitrl_status_string(B.ERR_LIMIT) == b"size beyond the fixed maximum of this entry point"
     B.poll_status()
