@@ -397,6 +397,31 @@ def run_ours(args):
                             "launches": l8}
             del g8
 
+    if rank == 0 and "pack5" in sections:
+        # the same M = 1 sweep on the five-weights-per-byte format (1.6 bits per weight, lookup-table decode): judged on
+        # microseconds per sweep against the 2-bit kernel's, and on GB/s of its own (smaller) packed bytes
+        gen5 = torch.Generator(device="cuda")
+        lin5 = []
+        for l in range(n_layers):
+            for j, (_, k, n) in enumerate(BLOCK):
+                gen5.manual_seed(5000 + 4 * l + j)
+                lin5.append(bitrl.Linear5.from_master(torch.randn(n, k, generator=gen5, device="cuda") * inputs.SIGMA_W))
+        x5 = [xs1[k] for _ in range(n_layers) for _, k, _ in BLOCK]
+        y5 = [torch.empty_like(ys1[l][j]) for l in range(n_layers) for j in range(len(BLOCK))]
+        call5 = bitrl.MultiCall5(lin5, x5, y5, bitrl.OUT_BF16)
+        g5, l5 = capture(call5.run)
+        ms5 = time_graph(g5, args.steps, args.warmup, 1) / args.steps
+        step1()
+        torch.cuda.synchronize()
+        same = all(torch.equal(a_, ys1[l][j]) for a_, (l, j) in zip(y5, [(l, j) for l in range(n_layers) for j in range(len(BLOCK))]))
+        bytes5 = sum(w.nbytes for w in lin5)
+        extra["sweep_m1_five_weights_per_byte"] = {
+            "us_per_sweep": ms5 * 1e3, "us_per_sweep_2bit": ms1 / args.steps * 1e3, "packed_bytes": bytes5,
+            "GBps_of_its_own_bytes": bytes5 / (ms5 * 1e-3) / 1e9, "frac_of_hbm_peak": bytes5 / (ms5 * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "bits_per_weight": 8.0 * bytes5 / (n_layers * sum(k * n for _, k, n in BLOCK)),
+            "outputs_equal_2bit_path": bool(same), "launches": l5}
+        del g5, lin5, y5
+
     if rank == 0 and "gemm" in sections:
         # M = 4096 GEMM, both judged shapes; weights rotate over several matrices, inputs over four buffers
         i8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
@@ -703,7 +728,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=FULL_LAYERS, help="blocks in the backbone (30 = full model)")
-    ap.add_argument("--sections", default="decode8,gemm,critic,encoder,cpu",
+    ap.add_argument("--sections", default="decode8,pack5,gemm,critic,encoder,cpu",
                     help="secondary measurements besides the M=1 headline (comma list; empty = none)")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:

@@ -274,6 +274,27 @@ BITRL_API bitrl_status bitrl_w4a8_forward_debug(const uint8_t* packed, const flo
                                                 size_t workspace_bytes, int8_t* xq_out, float* absmax_out,
                                                 int32_t* acc_out, void* stream);
 
+/* ---- five weights per byte: the denser, lookup-table-decoded format of the streaming path (Abstract: 1.58-bit
+ * weights; Sec. V, edge-deployment paragraph: ternary products as additions and subtractions "with lookup tables") ----
+ * Format (the paper gives none): byte j of row n = sum_{i=0..4} (W_q[n,5j+i] + 1) * 3^i, ceil(K/5) bytes per row,
+ * positions beyond K counted as zero weights; 1.6 bits per weight against 2.
+ * bitrl_pack5: packed dev [N,K/4] canonical 2-bit codes (the output of bitrl_pack_ternary) -> packed5 dev
+ * [N, ceil(K/5)] bytes.  bitrl_linear5_create re-tiles packed5 into the kernel's layout (library-owned copy; returns
+ * when it is complete) and bitrl_linear5_bytes reports the size of that copy, the bytes a forward call streams.
+ * bitrl_bitlinear5_forward_multi: `count` independent layers y[i] = BitLinear_{w[i]}(x[i]) in one launch, like
+ * bitrl_bitlinear_forward_multi, for M <= BITRL_LINEAR5_MAX_M tokens; every byte is decoded through a 243-entry table in
+ * shared memory.  Results are bit-identical to the 2-bit path.  w, x, y: HOST arrays of `count` entries. */
+#define BITRL_LINEAR5_MAX_M 2
+typedef struct bitrl_linear5 bitrl_linear5_t;
+BITRL_API bitrl_status bitrl_pack5(const uint8_t* packed, int32_t N, int32_t K, uint8_t* packed5, void* stream);
+BITRL_API bitrl_status bitrl_linear5_create(const uint8_t* packed5, const float* gamma, int32_t N, int32_t K,
+                                            bitrl_linear5_t** out, void* stream);
+BITRL_API bitrl_status bitrl_linear5_destroy(bitrl_linear5_t* w);
+BITRL_API size_t bitrl_linear5_bytes(const bitrl_linear5_t* w);
+BITRL_API bitrl_status bitrl_bitlinear5_forward_multi(int32_t count, const bitrl_linear5_t* const* w,
+                                                      const void* const* x, void* const* y, int32_t M,
+                                                      int32_t out_dtype, void* stream);
+
 /* ---- status ----------------------------------------------------------------------------------------- */
 /* Synchronizes `stream`, then reads and clears the device status word.  BITRL_OK, BITRL_ERR_TIMEOUT (a kernel
  * wait expired; results of that launch are invalid) or BITRL_ERR_CUDA. */

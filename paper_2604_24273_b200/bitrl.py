@@ -75,6 +75,12 @@ EXPORTS = {
     "bitrl_w4a8_workspace_bytes": (_sz, [_i32, _i32, _i32]),
     "bitrl_w4a8_forward": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp]),
     "bitrl_w4a8_forward_debug": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp, _vp, _vp, _vp]),
+    "bitrl_pack5": (_i32, [_vp, _i32, _i32, _vp, _vp]),
+    "bitrl_linear5_create": (_i32, [_vp, _vp, _i32, _i32, ctypes.POINTER(_vp), _vp]),
+    "bitrl_linear5_destroy": (_i32, [_vp]),
+    "bitrl_linear5_bytes": (_sz, [_vp]),
+    "bitrl_bitlinear5_forward_multi": (_i32, [_i32, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp), _i32,
+                                              _i32, _vp]),
     "bitrl_selftest_wait_timeout": (_i32, [ctypes.c_int64, _vp]),
     "bitrl_poll_status": (_i32, [_vp]),
     "bitrl_last_timeout_stage": (_i32, []),
@@ -254,6 +260,56 @@ class MultiCall:
     def run(self):
         _check(lib().bitrl_bitlinear_forward_multi(self.count, self.w, self.x, self.y, self.M, self.out_dtype,
                                                    _stream()), "bitrl_bitlinear_forward_multi")
+        return self.keep[2]
+
+
+LINEAR5_MAX_M = 2
+
+
+def pack5(packed: torch.Tensor, N: int, K: int) -> torch.Tensor:
+    """Canonical 2-bit codes [N,K/4] -> five weights per byte [N, ceil(K/5)] (base 3)."""
+    _dev(packed, torch.uint8, "packed")
+    out = torch.empty((N, (K + 4) // 5), dtype=torch.uint8, device=packed.device)
+    _check(lib().bitrl_pack5(_ptr(packed), N, K, _ptr(out), _stream()), "bitrl_pack5")
+    return out
+
+
+class Linear5:
+    """Owns a ``bitrl_linear5_t``: the weights in the five-per-byte kernel layout + gamma."""
+
+    def __init__(self, packed5: torch.Tensor, gamma: torch.Tensor, N: int, K: int):
+        _dev(packed5, torch.uint8, "packed5")
+        _dev(gamma, torch.float32, "gamma")
+        self.N, self.K = int(N), int(K)
+        h = _vp()
+        _check(lib().bitrl_linear5_create(_ptr(packed5), _ptr(gamma), self.N, self.K, ctypes.byref(h), _stream()),
+               "bitrl_linear5_create")
+        self.handle = h
+        self.nbytes = int(lib().bitrl_linear5_bytes(h))
+
+    @classmethod
+    def from_master(cls, W: torch.Tensor) -> "Linear5":
+        packed, gamma = pack_ternary(W)
+        return cls(pack5(packed, W.shape[0], W.shape[1]), gamma, W.shape[0], W.shape[1])
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().bitrl_linear5_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class MultiCall5(MultiCall):
+    """Argument block of ``bitrl_bitlinear5_forward_multi`` (M <= 2)."""
+
+    def run(self):
+        _check(lib().bitrl_bitlinear5_forward_multi(self.count, self.w, self.x, self.y, self.M, self.out_dtype,
+                                                    _stream()), "bitrl_bitlinear5_forward_multi")
         return self.keep[2]
 
 

@@ -87,11 +87,16 @@ static bitrl_status check_arch() {
 #include "heads.cuh"
 #include "gemm_w8.cuh"
 #include "w4.cuh"
+#include "gemv5.cuh"
 
 using namespace bitrl;
 
 struct bitrl_linear {
   Linear l;
+};
+
+struct bitrl_linear5 {
+  Linear5 l;
 };
 
 struct bitrl_encoder {
@@ -699,6 +704,78 @@ bitrl_status bitrl_w4a8_forward_debug(const uint8_t* packed, const float* scale,
                                       int32_t N, void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes,
                                       int8_t* xq_out, float* absmax_out, int32_t* acc_out, void* stream) {
   return w4a8_impl(packed, scale, x, M, K, N, y, out_dtype, workspace, workspace_bytes, xq_out, absmax_out, acc_out, stream);
+}
+
+// ---- five weights per byte: the denser format of the streaming path ---------------------------------------------
+
+bitrl_status bitrl_pack5(const uint8_t* packed, int32_t N, int32_t K, uint8_t* packed5, void* stream) {
+  if (!packed || !packed5) return BITRL_ERR_NULL;
+  if (!shape_ok(N, K)) return BITRL_ERR_SHAPE;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  const long long n = static_cast<long long>(N) * ((K + 4) / 5);
+  pack5_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(packed, N, K, packed5);
+  count_launch(1);
+  BITRL_CUDA(cudaGetLastError());
+  return BITRL_OK;
+}
+
+bitrl_status bitrl_linear5_create(const uint8_t* packed5, const float* gamma, int32_t N, int32_t K,
+                                  bitrl_linear5_t** out, void* stream) {
+  if (!packed5 || !gamma || !out) return BITRL_ERR_NULL;
+  if (!shape_ok(N, K)) return BITRL_ERR_SHAPE;
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  bitrl_linear5* w = new (std::nothrow) bitrl_linear5();
+  if (!w) return BITRL_ERR_CUDA;
+  w->l = Linear5{nullptr, nullptr, N, K, (K + T5_K - 1) / T5_K};
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = static_cast<size_t>(N / TILE_ROWS) * w->l.pieces * TILE_BYTES;
+  cudaError_t e = cudaMalloc(&w->l.tiles, bytes);
+  if (e == cudaSuccess) e = cudaMalloc(&w->l.gamma, 256);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(w->l.gamma, gamma, sizeof(float), cudaMemcpyDeviceToDevice, st);
+  if (e == cudaSuccess) {
+    retile5_kernel<<<static_cast<unsigned>((bytes + 255) / 256), 256, 0, st>>>(packed5, N, K, w->l.pieces, w->l.tiles);
+    count_launch(1);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);  // the handle is complete when this returns
+  if (e != cudaSuccess) {
+    cudaFree(w->l.tiles);
+    cudaFree(w->l.gamma);
+    delete w;
+    return cuda_fail(e);
+  }
+  *out = w;
+  return BITRL_OK;
+}
+
+bitrl_status bitrl_linear5_destroy(bitrl_linear5_t* w) {
+  if (!w) return BITRL_OK;
+  cudaFree(w->l.tiles);
+  cudaFree(w->l.gamma);
+  delete w;
+  return BITRL_OK;
+}
+
+size_t bitrl_linear5_bytes(const bitrl_linear5_t* w) {
+  return w ? static_cast<size_t>(w->l.N / TILE_ROWS) * w->l.pieces * TILE_BYTES : 0;
+}
+
+bitrl_status bitrl_bitlinear5_forward_multi(int32_t count, const bitrl_linear5_t* const* w, const void* const* x,
+                                            void* const* y, int32_t M, int32_t out_dtype, void* stream) {
+  if (!w || !x || !y) return BITRL_ERR_NULL;
+  if (count < 1 || count > BITRL_MULTI_MAX_JOBS || M < 1 || M > BITRL_LINEAR5_MAX_M) return BITRL_ERR_SHAPE;
+  if (out_dtype != BITRL_OUT_F32 && out_dtype != BITRL_OUT_BF16) return BITRL_ERR_DTYPE;
+  const Linear5* lins[BITRL_MULTI_MAX_JOBS];
+  for (int i = 0; i < count; ++i) {
+    if (!w[i] || !x[i] || !y[i]) return BITRL_ERR_NULL;
+    if (!aligned16(x[i]) || !aligned16(y[i])) return BITRL_ERR_ALIGN;
+    lins[i] = &w[i]->l;
+  }
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  return launch_gemv5_multi(count, lins, x, y, M, out_dtype, static_cast<cudaStream_t>(stream));
 }
 
 // ---- self-test of the bounded-wait / status-word path ----
