@@ -29,6 +29,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
            "-cudart", "static", "-Xlinker", "--exclude-libs,ALL", "-Xlinker", "-Bsymbolic"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("BITRL_NVCC_FLAGS", "").split()  # tuning builds, e.g. -DGM_MAXREG=128
     cmd += [str(s) for s in SOURCES] + ["-o", str(tmp)]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)

@@ -591,8 +591,10 @@ __global__ void __launch_bounds__(256) gemm_splitk_finish_kernel(const int32_t* 
   *reinterpret_cast<uint4*>(static_cast<unsigned short*>(y) + off) = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
-// Paired-CTA launches are considered from this M on (many tiles, no split-K).
-constexpr int GM_PAIR_MIN_M = 1024;
+// Paired-CTA launches are considered from this M on (many tiles, no split-K).  A sweep of the five block shapes showed
+// pairs never ahead at M = 1024 and 2048 (equal to 3 us behind) and ahead on four of five at M = 4096.
+constexpr int GM_PAIR_MIN_M = 3072;
+constexpr int GM_PAIR_FORCED_MIN_M = 1024;  // with BITRL_GEMM_PAIR=1 (tests of the paired kernel on small ragged shapes)
 
 // Time per k block (ns) of one CTA (or CTA pair) by token-tile width, as measured at M = 4096 on the block shapes: the
 // 192-wide tile runs close to the tensor pipe's own time; at 224 only two weight slots fit beside the accumulators in
@@ -678,7 +680,8 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
   // CTA pairs (256-row tiles): for launches with many tiles, an even number of 128-row tiles and weights in tensor memory.
   bool pair = false;
   int pair_clusters = 0;
-  if (gemm_pair_mode() != 0 && gemm_a_in_tmem() && tiles_n % 2 == 0 && splits == 1 && M >= GM_PAIR_MIN_M) {
+  if (gemm_pair_mode() != 0 && gemm_a_in_tmem() && tiles_n % 2 == 0 && splits == 1 &&
+      M >= (gemm_pair_mode() == 1 ? GM_PAIR_FORCED_MIN_M : GM_PAIR_MIN_M)) {
     int ptok = 0;
     if (const int forced = gemm_forced_tok()) {
       if (forced == 224 || forced == 192 || forced == 128) ptok = forced;
@@ -689,9 +692,9 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
         const int clusters = gemm_pair_max_clusters(cand[i]);
         if (clusters <= 0) continue;
         const long long tiles = static_cast<long long>(tiles_n / 2) * ((M + cand[i] - 1) / cand[i]);
-        // a cluster launch starts and ends a few us later than a plain one (one-wave launches at M = 1024 lose 4 us,
-        // seven-wave launches at M = 4096 win 2 us)
-        const long long cost = ((tiles + clusters - 1) / clusters) * kblocks * gemm_kb_ns(cand[i], true) + 3000;
+        // a cluster launch starts and ends a little later than a plain one; 1.5 us reproduces the measured choices at
+        // M = 4096 (pairs at 224 tokens for 2560 -> 3840 / 6912 / 13824, at 192 for 6912 -> 2560, single CTAs for 2560 -> 2560)
+        const long long cost = ((tiles + clusters - 1) / clusters) * kblocks * gemm_kb_ns(cand[i], true) + 1500;
         if (pbest < 0 || cost < pbest) { pbest = cost; ptok = cand[i]; }
       }
       if (gemm_pair_mode() != 1 && pbest >= best) ptok = 0;  // the single-CTA kernel is expected to be no slower

@@ -57,7 +57,7 @@ def sample_rows(M, rng, extra=28):
     return np.unique(rows[(rows >= 0) & (rows < M)])
 
 
-@pytest.mark.parametrize("M", [1024, 1061, 4096])
+@pytest.mark.parametrize("M", [1024, 1061, 3333, 4096])
 @pytest.mark.parametrize("K,N,wseed", [(2560, 2560, 5001), (2560, 3840, 5000), (2560, 13824, 5002), (6912, 2560, 5003)])
 def test_forward_q_residual_block_shapes_large_m(oracle_mod, B, M, K, N, wseed):
     """a2 + a3 + residual add on a quantized input, as the encoder calls it: int32 sums bit-exact on >= 40 sampled token
