@@ -4,16 +4,18 @@
 // not by HBM.  When several such calls are independent (a sweep over matrices, or the heads of one layer), this
 // kernel streams all of their packed weights back to back at HBM speed.
 //
-// One persistent CTA per SM.  The work list is the concatenation of all jobs' row tiles (128 rows x all K, one
-// contiguous K/4*128-byte region of the tile layout), jobs sorted by K; every CTA owns two ranges of it, balanced in
-// bytes (see GvmArgs::seg).
-//   warp 16     producer: bulk copies (cp.async.bulk) of eight consecutive 4 KB (row tile, k block) pieces into a ring
-//               of 32 KB slots - 128 to 192 KB in flight per SM, independent of the activations, so it runs ahead across jobs
-//   warps 0-15  consumers in two groups of 8: warp w of a group owns rows 16w..16w+15 of the row tile, the group every
-//               other 4 KB piece of the K range (sixteen warps hide the shared-memory and MMA latencies that eight
-//               leave exposed); the two partial sums meet in shared memory once per row tile, behind a barrier of the
-//               two warps that share the rows.  The 2-bit codes are masked (not shifted) straight into the A
-//               fragments of a warp-level integer MMA
+// One persistent CTA per SM.  The work list is the concatenation of all jobs' row-tile pairs (2 x 128 rows x all K, one
+// contiguous region of the tile layout), jobs sorted by K; every CTA owns two ranges of it, balanced in bytes (see
+// GvmArgs::seg).
+//   warp 16     producer: bulk copies (cp.async.bulk) of four consecutive 4 KB (row tile, k block) pieces of each of the
+//               unit's two row tiles into a ring of 32 KB slots - 128 to 192 KB in flight per SM, independent of the
+//               activations, so it runs ahead across jobs
+//   warps 0-15  consumers in two groups of 8: the work unit is a PAIR of row tiles of one job, group g owns row tile g
+//               of the pair and warp w of a group rows 16w..16w+15 of it over the whole K (a ring slot holds four
+//               consecutive pieces of either tile).  No two warps share an output row, so nothing is combined through
+//               shared memory and no barrier joins the warps: they drift apart freely, which hides the shared-memory
+//               and MMA latencies.  The 2-bit codes are masked (not shifted) straight into the A fragments of a
+//               warp-level integer MMA
 //               (mma.sync m16n8k32, A = unsigned codes, B = signed int8 activations of 8 tokens, int32 accumulate):
 //               the same instruction count serves 1 to 8 tokens (two MMAs per k step for 9 to 16), so the kernel
 //               stays memory-bound where a dp4a loop would be ALU-bound from M = 4 on.
@@ -37,7 +39,8 @@ constexpr int GVM_GROUPS = 2;                   // warp groups; group i takes pi
 constexpr int GVM_CONSUMERS = 8 * GVM_GROUPS;
 constexpr int GVM_THREADS = (GVM_CONSUMERS + 1) * 32;
 constexpr int GVM_SMEM_BUDGET = 220 * 1024;
-constexpr int GVM_UNROLL = 8;  // 4 KB pieces per ring slot: one bulk copy, one barrier, one consumer loop iteration
+constexpr int GVM_PPG = 4;     // 4 KB pieces of a ring slot per warp group (= per row tile of a unit)
+constexpr int GVM_UNROLL = GVM_PPG * GVM_GROUPS;  // pieces per ring slot: two bulk copies, one barrier
 constexpr int GVM_SLOT_BYTES = GVM_UNROLL * TILE_BYTES;
 constexpr int GVM_XPAD = 16;  // bytes added to each activation row so that the 8 token rows hit different banks
 
@@ -90,7 +93,6 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
   const uint32_t bar_empty = bar_full + 8 * depth;  // [depth]
   float* absmax_s = reinterpret_cast<float*>(tail + 16 * depth);  // [NT] a_m / 127
   int* rowsum_s = reinterpret_cast<int*>(absmax_s + NT);          // [NT]
-  int* comb = reinterpret_cast<int*>(rowsum_s + NT);              // [2][8 warps][NT/8 * 4][32 lanes]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int u_begin = a.seg[blockIdx.x][0], u_mid = a.seg[blockIdx.x][1], u_resume = a.seg[blockIdx.x][2],
@@ -115,13 +117,17 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
       for (int u = u_begin == u_mid ? u_resume : u_begin; ok && u < u_end; u = (u + 1 == u_mid) ? u_resume : u + 1) {
         while (j + 1 < a.njobs && a.jobs[j + 1].unit_begin <= u) ++j;
         const int kblocks = a.jobs[j].K / TILE_K;
-        const uint8_t* src = a.jobs[j].tiles + static_cast<size_t>(u - a.jobs[j].unit_begin) * kblocks * TILE_BYTES;
-        for (int kb = 0; kb < kblocks; kb += GVM_UNROLL, ++pc) {
-          const uint32_t bytes = static_cast<uint32_t>(min(GVM_UNROLL, kblocks - kb)) * TILE_BYTES;
+        const int tile0 = 2 * (u - a.jobs[j].unit_begin);
+        const int ntiles = min(2, a.jobs[j].N / TILE_ROWS - tile0);  // 1 for the half unit of an odd job
+        const uint8_t* src = a.jobs[j].tiles + static_cast<size_t>(tile0) * kblocks * TILE_BYTES;
+        for (int kb = 0; kb < kblocks; kb += GVM_PPG, ++pc) {
+          const uint32_t bytes = static_cast<uint32_t>(min(GVM_PPG, kblocks - kb)) * TILE_BYTES;
           const uint32_t s = pc & (depth - 1), ph = (pc >> a.depth_log2) & 1u;
           if (!ptx::mbar_wait(bar_empty + 8 * s, ph ^ 1u)) { report_timeout(GVM_WAIT_EMPTY); ok = false; break; }
-          ptx::mbar_arrive_expect_tx(bar_full + 8 * s, bytes);
-          ptx::bulk_g2s(ring + s * GVM_SLOT_BYTES, src + static_cast<size_t>(kb) * TILE_BYTES, bytes, bar_full + 8 * s);
+          ptx::mbar_arrive_expect_tx(bar_full + 8 * s, bytes * ntiles);
+          for (int t = 0; t < ntiles; ++t)
+            ptx::bulk_g2s(ring + s * GVM_SLOT_BYTES + t * GVM_PPG * TILE_BYTES,
+                          src + (static_cast<size_t>(t) * kblocks + kb) * TILE_BYTES, bytes, bar_full + 8 * s);
         }
       }
     }
@@ -132,10 +138,10 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
     const int grp = warp >> 3, rw = warp & 7;
     const unsigned short* cached_x = nullptr;
     int cached_k = 0;
-    uint32_t pc = 0, tile_no = 0;
+    uint32_t pc = 0;
     int j = 0;
     bool ok = true;
-    for (int u = u_begin == u_mid ? u_resume : u_begin; u < u_end; u = (u + 1 == u_mid) ? u_resume : u + 1, ++tile_no) {
+    for (int u = u_begin == u_mid ? u_resume : u_begin; u < u_end; u = (u + 1 == u_mid) ? u_resume : u + 1) {
       while (j + 1 < a.njobs && a.jobs[j + 1].unit_begin <= u) ++j;
       const GvmJob& job = a.jobs[j];
       const int K = job.K, kblocks = K / TILE_K;
@@ -184,12 +190,13 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
         cached_k = K;
       }
 
-      // ---- one row tile: this warp's 16 rows over the whole K ----
+      // ---- one unit: this warp's 16 rows of row tile `grp` of the pair, over the whole K ----
+      const int tile = 2 * (u - job.unit_begin) + grp;
+      const bool have_tile = tile < job.N / TILE_ROWS;  // false for group 1 in the half unit of an odd job
       const float gamma = *job.gamma;  // requested now, needed after the k loop: its latency hides behind the loop
-      // A group's two pieces of a slot are fetched from shared memory together and feed independent accumulator
-      // chains, so that neither the loads nor the MMAs of one piece wait for those of the other.
-      constexpr int PP = GVM_UNROLL / GVM_GROUPS;  // pieces of a slot per group
-      constexpr int CH = NT == 8 ? 8 : 4;          // independent accumulator chains (the warp MMA has a long latency)
+      // The pieces of a slot are fetched from shared memory together and feed independent accumulator chains, so that
+      // neither the loads nor the MMAs of one piece wait for those of another.
+      constexpr int CH = NT == 8 ? 8 : 4;  // independent accumulator chains (the warp MMA has a long latency)
       int acc[CH][NT / 8][4];
 #pragma unroll
       for (int c = 0; c < CH; ++c)
@@ -197,37 +204,39 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
         for (int h = 0; h < NT / 8; ++h)
 #pragma unroll
           for (int e = 0; e < 4; ++e) acc[c][h][e] = 0;
-      const uint32_t xlane = xq_addr + g * xstride + t * 32 + grp * TILE_K;
-      const uint32_t wlane = ring + grp * TILE_BYTES + rw * 512 + g * 32 + t * 8;
-      for (int kb = 0; kb < kblocks; kb += GVM_UNROLL) {
-        const int np = min(GVM_UNROLL, kblocks - kb) - grp;  // pieces grp, grp + GROUPS exist if np > 0, GROUPS
-        uint2 wr[PP][2];
+      const uint32_t xlane = xq_addr + g * xstride + t * 32;
+      const uint32_t wlane = ring + grp * GVM_PPG * TILE_BYTES + rw * 512 + g * 32 + t * 8;
+      for (int kb = 0; kb < kblocks; kb += GVM_PPG) {
+        const int np = min(GVM_PPG, kblocks - kb);
+        uint2 wr[GVM_PPG][2];
         const uint32_t s = pc & (depth - 1), ph = (pc >> a.depth_log2) & 1u;
         if (ok && !ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(GVM_WAIT_FULL); ok = false; }
         if (ok) {
+          if (have_tile) {
 #pragma unroll
-          for (int p = 0; p < PP; ++p) {
-            if (GVM_GROUPS * p < np) {
-              const uint32_t wslice = wlane + s * GVM_SLOT_BYTES + p * GVM_GROUPS * TILE_BYTES;
-              wr[p][0] = ptx::lds64(wslice);
-              wr[p][1] = ptx::lds64(wslice + 8 * 32);
+            for (int p = 0; p < GVM_PPG; ++p) {
+              if (p < np) {
+                const uint32_t wslice = wlane + s * GVM_SLOT_BYTES + p * TILE_BYTES;
+                wr[p][0] = ptx::lds64(wslice);
+                wr[p][1] = ptx::lds64(wslice + 8 * 32);
+              }
             }
-          }
 #pragma unroll
-          for (int p = 0; p < PP; ++p) {
-            if (GVM_GROUPS * p < np) {
+            for (int p = 0; p < GVM_PPG; ++p) {
+              if (p < np) {
 #pragma unroll
-              for (int h = 0; h < NT / 8; ++h) {
-                const uint32_t xa_addr = xlane + h * 8 * xstride + (kb + p * GVM_GROUPS) * TILE_K;
-                const uint4 xa = ptx::lds128(xa_addr), xb = ptx::lds128(xa_addr + 16);
-                const uint32_t xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+                for (int h = 0; h < NT / 8; ++h) {
+                  const uint32_t xa_addr = xlane + h * 8 * xstride + (kb + p) * TILE_K;
+                  const uint4 xa = ptx::lds128(xa_addr), xb = ptx::lds128(xa_addr + 16);
+                  const uint32_t xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                  // The codes stay at their bit positions (c * 4^ks still fits an unsigned byte): one mask and no
-                  // shift per operand.  Chain ks then holds 4^ks times its share and is scaled back once per tile.
-                  const uint32_t msk = 0x03030303u << (2 * ks);
-                  mma_u8s8(acc[((p * 4) % CH) + ks][h], wr[p][0].x & msk, wr[p][1].x & msk, wr[p][0].y & msk,
-                           wr[p][1].y & msk, xv[ks], xv[4 + ks]);
+                  for (int ks = 0; ks < 4; ++ks) {
+                    // The codes stay at their bit positions (c * 4^ks still fits an unsigned byte): one mask and no
+                    // shift per operand.  Chain ks then holds 4^ks times its share and is scaled back once per tile.
+                    const uint32_t msk = 0x03030303u << (2 * ks);
+                    mma_u8s8(acc[((p * 4) % CH) + ks][h], wr[p][0].x & msk, wr[p][1].x & msk, wr[p][0].y & msk,
+                             wr[p][1].y & msk, xv[ks], xv[4 + ks]);
+                  }
                 }
               }
             }
@@ -243,25 +252,16 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
         for (int h = 0; h < NT / 8; ++h)
 #pragma unroll
           for (int e = 0; e < 4; ++e) acc[0][h][e] += acc[c][h][e] >> (2 * (c & 3));  // exact: multiples of 4^(c&3)
-      // ---- the two groups' partial sums meet in shared memory (double-buffered by tile parity) ----
-      int* cb = comb + (tile_no & 1u) * (8 * (NT / 8) * 4 * 32) + rw * ((NT / 8) * 4 * 32) + lane;
-      if (grp == 1) {
-#pragma unroll
-        for (int h = 0; h < NT / 8; ++h)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) cb[(h * 4 + e) * 32] = acc[0][h][e];
-      }
-      asm volatile("bar.sync %0, 64;" ::"r"(4 + rw) : "memory");  // only the two warps that share these rows meet
-      if (grp == 0 && ok) {
+      if (have_tile && ok) {
         // C fragment: acc[h][0..1] = (row g, tokens 8h+2t, +1), acc[h][2..3] = (row g+8, same tokens)
-        const int n0 = (u - job.unit_begin) * TILE_ROWS + rw * 16 + g;
+        const int n0 = tile * TILE_ROWS + rw * 16 + g;
 #pragma unroll
         for (int h = 0; h < NT / 8; ++h)
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int m = 8 * h + 2 * t + (e & 1);
             if (m < a.M) {
-              const int tv = acc[0][h][e] + cb[(h * 4 + e) * 32] - rowsum_s[m];
+              const int tv = acc[0][h][e] - rowsum_s[m];
               const float yv = __fmul_rn(static_cast<float>(tv), __fmul_rn(gamma, absmax_s[m]));
               const size_t o = static_cast<size_t>(m) * job.N + n0 + (e >> 1) * 8;
               if (a.out_dtype == BITRL_OUT_F32) static_cast<float*>(job.y)[o] = yv;
@@ -274,14 +274,17 @@ __global__ void __launch_bounds__(GVM_THREADS, 1) gemv_multi_kernel(const __grid
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// M <= 2 variant: dp4a instead of the warp MMA (cheaper when only one or two tokens use the weights), and
-// 8 * GVD_GROUPS consumer warps: group g takes pieces g, g + GROUPS of every ring slot (a slot holds GVD_PPG * GROUPS
-// pieces); the groups' partial sums meet in shared memory once per row tile.  Lane = 2*row + k half, as in the
-// single-matrix kernel.
+// M <= 2 variant: dp4a instead of the warp MMA (cheaper when only one or two tokens use the weights).
+// The work unit is a PAIR of row tiles of one job (256 rows): warp group g (8 warps) owns row tile g of the pair, warp w
+// of a group rows 16w..16w+15 of that tile over the whole K, lane = 2*row + k half as in the single-matrix kernel.  A
+// ring slot holds four consecutive 4 KB pieces of either tile (two bulk copies, one barrier).  Since no two warps
+// share an output row, nothing is combined through shared memory and no barrier joins the warps: they drift apart
+// freely, which is what hides the shared-memory and dp4a latencies (two groups on the SAME rows with a pair barrier per
+// tile left every warp waiting for its partner's epilogue).  A job with an odd number of row tiles ends in a half unit.
 constexpr int GVD_GROUPS = 2;
 constexpr int GVD_CONSUMERS = 8 * GVD_GROUPS;
 constexpr int GVD_THREADS = (GVD_CONSUMERS + 1) * 32;
-constexpr int GVD_PPG = 4;                                 // pieces of a slot per group
+constexpr int GVD_PPG = 4;                                 // pieces of a slot per group (= per row tile of the pair)
 constexpr int GVD_PIECES = GVD_PPG * GVD_GROUPS;           // 4 KB pieces per ring slot
 constexpr int GVD_SLOT_BYTES = GVD_PIECES * TILE_BYTES;
 
@@ -298,7 +301,6 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
   int* rowsum_s = reinterpret_cast<int*>(absmax_s + MT);          // [MT]
   float* redf = reinterpret_cast<float*>(rowsum_s + MT);          // [GVD_CONSUMERS]
   int* redi = reinterpret_cast<int*>(redf + GVD_CONSUMERS);       // [GVD_CONSUMERS]
-  int* comb = redi + GVD_CONSUMERS;                               // [2][GROUPS-1][8 warps][16 rows][MT]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int u_begin = a.seg[blockIdx.x][0], u_mid = a.seg[blockIdx.x][1], u_resume = a.seg[blockIdx.x][2],
@@ -323,12 +325,16 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
       for (int u = u_begin == u_mid ? u_resume : u_begin; ok && u < u_end; u = (u + 1 == u_mid) ? u_resume : u + 1) {
         while (j + 1 < a.njobs && a.jobs[j + 1].unit_begin <= u) ++j;
         const int kblocks = a.jobs[j].K / TILE_K;
-        const uint8_t* src = a.jobs[j].tiles + static_cast<size_t>(u - a.jobs[j].unit_begin) * kblocks * TILE_BYTES;
-        for (int kb = 0; kb < kblocks; kb += GVD_PIECES) {
-          const uint32_t bytes = static_cast<uint32_t>(min(GVD_PIECES, kblocks - kb)) * TILE_BYTES;
+        const int tile0 = 2 * (u - a.jobs[j].unit_begin);
+        const int ntiles = min(2, a.jobs[j].N / TILE_ROWS - tile0);  // 1 for the half unit of an odd job
+        const uint8_t* src = a.jobs[j].tiles + static_cast<size_t>(tile0) * kblocks * TILE_BYTES;
+        for (int kb = 0; kb < kblocks; kb += GVD_PPG) {
+          const uint32_t bytes = static_cast<uint32_t>(min(GVD_PPG, kblocks - kb)) * TILE_BYTES;
           if (!ptx::mbar_wait(bar_empty + 8 * s, ph ^ 1u)) { report_timeout(GVM_WAIT_EMPTY); ok = false; break; }
-          ptx::mbar_arrive_expect_tx(bar_full + 8 * s, bytes);
-          ptx::bulk_g2s(ring + s * GVD_SLOT_BYTES, src + static_cast<size_t>(kb) * TILE_BYTES, bytes, bar_full + 8 * s);
+          ptx::mbar_arrive_expect_tx(bar_full + 8 * s, bytes * ntiles);
+          for (int t = 0; t < ntiles; ++t)
+            ptx::bulk_g2s(ring + s * GVD_SLOT_BYTES + t * GVD_PPG * TILE_BYTES,
+                          src + (static_cast<size_t>(t) * kblocks + kb) * TILE_BYTES, bytes, bar_full + 8 * s);
           if (++s == static_cast<uint32_t>(depth)) { s = 0; ph ^= 1u; }
         }
       }
@@ -339,10 +345,10 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
     const int half = lane & 1, grp = warp >> 3, rw = warp & 7;
     const unsigned short* cached_x = nullptr;
     int cached_k = 0;
-    uint32_t s = 0, ph = 0, tile_no = 0;
+    uint32_t s = 0, ph = 0;
     int j = 0;
     bool ok = true;
-    for (int u = u_begin == u_mid ? u_resume : u_begin; u < u_end; u = (u + 1 == u_mid) ? u_resume : u + 1, ++tile_no) {
+    for (int u = u_begin == u_mid ? u_resume : u_begin; u < u_end; u = (u + 1 == u_mid) ? u_resume : u + 1) {
       while (j + 1 < a.njobs && a.jobs[j + 1].unit_begin <= u) ++j;
       const GvmJob& job = a.jobs[j];
       const int K = job.K, kblocks = K / TILE_K;
@@ -411,7 +417,9 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
         cached_k = K;
       }
 
-      // ---- one row tile: this warp's 16 rows, pieces grp and grp + GROUPS of every slot ----
+      // ---- one unit: this warp's 16 rows of row tile `grp` of the pair, over the whole K ----
+      const int tile = 2 * (u - job.unit_begin) + grp;
+      const bool have_tile = tile < job.N / TILE_ROWS;  // false for group 1 in the half unit of an odd job
       const float gamma = *job.gamma;  // requested now, needed after the k loop: its latency hides behind the loop
       int acc[MT][4];
 #pragma unroll
@@ -420,37 +428,39 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
         for (int c = 0; c < 4; ++c) acc[m][c] = 0;
       // All addresses below are 32-bit shared-memory addresses with compile-time offsets, so that a piece costs its
       // loads, masks and dp4a and little else.
-      const uint32_t w_lane = ring + rw * 512 + lane * 16 + grp * TILE_BYTES;   // this lane's 16 bytes in piece `grp`
-      uint32_t x_lane = ptx::smem_u32(xq_s) + half * 64 + grp * TILE_K;         // its 64 activations of that piece
-      for (int kb = 0; kb < kblocks; kb += GVD_PIECES, x_lane += GVD_PIECES * TILE_K) {
-        const int np = min(GVD_PIECES, kblocks - kb) - grp;  // pieces grp, grp + GROUPS exist if np > 0, GROUPS
+      const uint32_t w_lane = ring + rw * 512 + lane * 16 + grp * GVD_PPG * TILE_BYTES;  // this lane's 16 bytes of a piece
+      uint32_t x_lane = ptx::smem_u32(xq_s) + half * 64;                                 // its 64 activations of that piece
+      for (int kb = 0; kb < kblocks; kb += GVD_PPG, x_lane += GVD_PPG * TILE_K) {
+        const int np = min(GVD_PPG, kblocks - kb);
         if (ok && !ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(GVM_WAIT_FULL); ok = false; }
         if (ok) {
-          const uint32_t w_slot = w_lane + s * GVD_SLOT_BYTES;
-          uint4 wv[GVD_PPG];
+          if (have_tile) {
+            const uint32_t w_slot = w_lane + s * GVD_SLOT_BYTES;
+            uint4 wv[GVD_PPG];
 #pragma unroll
-          for (int pp = 0; pp < GVD_PPG; ++pp)
-            if (GVD_GROUPS * pp < np) wv[pp] = ptx::lds128(w_slot + pp * GVD_GROUPS * TILE_BYTES);
+            for (int pp = 0; pp < GVD_PPG; ++pp)
+              if (pp < np) wv[pp] = ptx::lds128(w_slot + pp * TILE_BYTES);
 #pragma unroll
-          for (int pp = 0; pp < GVD_PPG; ++pp) {
-            if (GVD_GROUPS * pp < np) {
-              const uint32_t wword[4] = {wv[pp].x, wv[pp].y, wv[pp].z, wv[pp].w};
+            for (int pp = 0; pp < GVD_PPG; ++pp) {
+              if (pp < np) {
+                const uint32_t wword[4] = {wv[pp].x, wv[pp].y, wv[pp].z, wv[pp].w};
 #pragma unroll
-              for (int jw = 0; jw < 4; ++jw) {
-                // The codes are left at their bit positions (c1 * 4, c2 * 16, c3 * 64 still fit an unsigned byte):
-                // four masks and no shifts.  Accumulator i then holds 4^i times its share of the dot product and is
-                // scaled back by an exact shift once per row tile.
-                const uint32_t c0 = wword[jw] & 0x03030303u;
-                const uint32_t c1 = wword[jw] & 0x0c0c0c0cu;
-                const uint32_t c2 = wword[jw] & 0x30303030u;
-                const uint32_t c3 = wword[jw] & 0xc0c0c0c0u;
+                for (int jw = 0; jw < 4; ++jw) {
+                  // The codes are left at their bit positions (c1 * 4, c2 * 16, c3 * 64 still fit an unsigned byte):
+                  // four masks and no shifts.  Accumulator i then holds 4^i times its share of the dot product and is
+                  // scaled back by an exact shift once per row tile.
+                  const uint32_t c0 = wword[jw] & 0x03030303u;
+                  const uint32_t c1 = wword[jw] & 0x0c0c0c0cu;
+                  const uint32_t c2 = wword[jw] & 0x30303030u;
+                  const uint32_t c3 = wword[jw] & 0xc0c0c0c0u;
 #pragma unroll
-                for (int m = 0; m < MT; ++m) {
-                  const uint4 xv = ptx::lds128(x_lane + m * K + pp * GVD_GROUPS * TILE_K + 16 * jw);
-                  acc[m][0] = dp4a_u8s8(c0, static_cast<int>(xv.x), acc[m][0]);
-                  acc[m][1] = dp4a_u8s8(c1, static_cast<int>(xv.y), acc[m][1]);
-                  acc[m][2] = dp4a_u8s8(c2, static_cast<int>(xv.z), acc[m][2]);
-                  acc[m][3] = dp4a_u8s8(c3, static_cast<int>(xv.w), acc[m][3]);
+                  for (int m = 0; m < MT; ++m) {
+                    const uint4 xv = ptx::lds128(x_lane + m * K + pp * TILE_K + 16 * jw);
+                    acc[m][0] = dp4a_u8s8(c0, static_cast<int>(xv.x), acc[m][0]);
+                    acc[m][1] = dp4a_u8s8(c1, static_cast<int>(xv.y), acc[m][1]);
+                    acc[m][2] = dp4a_u8s8(c2, static_cast<int>(xv.z), acc[m][2]);
+                    acc[m][3] = dp4a_u8s8(c3, static_cast<int>(xv.w), acc[m][3]);
+                  }
                 }
               }
             }
@@ -460,29 +470,17 @@ __global__ void __launch_bounds__(GVD_THREADS, 1) gemv_multi_dp4a_kernel(const _
         }
         if (++s == static_cast<uint32_t>(depth)) { s = 0; ph ^= 1u; }
       }
-      // ---- combine: k halves by shuffle, the warp groups through shared memory ----
-      int* cb = comb + (tile_no & 1u) * ((GVD_GROUPS - 1) * 8 * 16 * MT) + (rw * 16 + (lane >> 1)) * MT;
-      int tot[MT];
+      // ---- epilogue of this warp's 16 rows: the k halves meet by one shuffle ----
 #pragma unroll
       for (int m = 0; m < MT; ++m) {
-        tot[m] = acc[m][0] + (acc[m][1] >> 2) + (acc[m][2] >> 4) + (acc[m][3] >> 6);  // exact: multiples of 4^i
-        tot[m] += __shfl_xor_sync(0xffffffffu, tot[m], 1);
-        if (grp > 0 && half == 0) cb[(grp - 1) * (8 * 16 * MT) + m] = tot[m];
-      }
-      asm volatile("bar.sync %0, %1;" ::"r"(4 + rw), "n"(GVD_GROUPS * 32) : "memory");  // the warps sharing these rows
-      if (grp == 0 && half == 0 && ok) {
-        const int n = (u - job.unit_begin) * TILE_ROWS + rw * 16 + (lane >> 1);
-#pragma unroll
-        for (int m = 0; m < MT; ++m) {
-          if (m < a.M) {
-            int tv = tot[m] - rowsum_s[m];
-#pragma unroll
-            for (int g2 = 0; g2 < GVD_GROUPS - 1; ++g2) tv += cb[g2 * (8 * 16 * MT) + m];
-            const float yv = __fmul_rn(static_cast<float>(tv), __fmul_rn(gamma, absmax_s[m]));
-            const size_t o = static_cast<size_t>(m) * job.N + n;
-            if (a.out_dtype == BITRL_OUT_F32) static_cast<float*>(job.y)[o] = yv;
-            else static_cast<unsigned short*>(job.y)[o] = float_to_bf16_bits(yv);
-          }
+        int tot = acc[m][0] + (acc[m][1] >> 2) + (acc[m][2] >> 4) + (acc[m][3] >> 6);  // exact: multiples of 4^i
+        tot += __shfl_xor_sync(0xffffffffu, tot, 1);
+        if (half == 0 && have_tile && ok && m < a.M) {
+          const int n = tile * TILE_ROWS + rw * 16 + (lane >> 1);
+          const float yv = __fmul_rn(static_cast<float>(tot - rowsum_s[m]), __fmul_rn(gamma, absmax_s[m]));
+          const size_t o = static_cast<size_t>(m) * job.N + n;
+          if (a.out_dtype == BITRL_OUT_F32) static_cast<float*>(job.y)[o] = yv;
+          else static_cast<unsigned short*>(job.y)[o] = float_to_bf16_bits(yv);
         }
       }
     }
@@ -568,12 +566,23 @@ bitrl_status launch_gemv_multi(int count, const Linear* const* w, const void* co
   int order[GVM_MAX_JOBS];  // jobs by K, largest first (stable)
   for (int j = 0; j < count; ++j) order[j] = j;
   std::stable_sort(order, order + count, [&](int x, int y) { return w[x]->K > w[y]->K; });
+  const bool pairs = true;  // the unit of both kernels is a pair of row tiles (one per warp group)
+  static thread_local std::vector<int> sz;  // 4 KB pieces of every unit, in work-list order
+  sz.clear();
   for (int i = 0; i < count; ++i) {
     const int j = order[i];
     a.jobs[i] = GvmJob{w[j]->tiles, w[j]->gamma, static_cast<const unsigned short*>(x[j]), y[j], w[j]->N, w[j]->K,
                        units, 0};
-    units += w[j]->N / TILE_ROWS;
-    pieces += static_cast<long long>(w[j]->N / TILE_ROWS) * (w[j]->K / TILE_K);
+    const int tiles = w[j]->N / TILE_ROWS, kb = w[j]->K / TILE_K;
+    if (pairs) {
+      sz.insert(sz.end(), tiles / 2, 2 * kb);
+      if (tiles & 1) sz.push_back(kb);
+      units += (tiles + 1) / 2;
+    } else {
+      sz.insert(sz.end(), tiles, kb);
+      units += tiles;
+    }
+    pieces += static_cast<long long>(tiles) * kb;
     if (w[j]->K > kmax) kmax = w[j]->K;
   }
   int dlog = gvm_depth_log2(M, kmax);
@@ -587,12 +596,7 @@ bitrl_status launch_gemv_multi(int count, const Linear* const* w, const void* co
   int grid = sm_count();
   if (grid > GVM_MAX_CTAS) grid = GVM_MAX_CTAS;
   if (grid > units) grid = units;
-  {
-    static thread_local std::vector<int> sz;  // 4 KB pieces of every unit, in work-list order
-    sz.clear();
-    for (int j = 0; j < count; ++j) sz.insert(sz.end(), a.jobs[j].N / TILE_ROWS, a.jobs[j].K / TILE_K);
-    gvm_partition(sz, pieces, grid, a.seg);
-  }
+  gvm_partition(sz, pieces, grid, a.seg);
   a.njobs = count;
   a.M = M;
   a.out_dtype = out_dtype;
