@@ -38,9 +38,10 @@ FULL_LAYERS = 30
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 INT8_OVER_BF16 = 2.0  # nominal dense int8 : bf16 tensor throughput on B200 (4.5 : 2.25 PFLOP/s)
 # DRAM bytes (read + write) of one gemv_multi_dp4a_kernel<1> launch per backbone block, from an ncu capture of the
-# 8-block case (dram__bytes_read.sum 138.989 MB + dram__bytes_write.sum 4.116 MB, means of two launches); every weight byte is read exactly
-# once, so traffic scales with the number of blocks.  Set to None whenever that kernel changes.
-HEADLINE_TRAFFIC_PER_BLOCK = (138.989056e6 + 4.116096e6) / 8
+# 8-block case (dram__bytes_read.sum 138.987 MB + dram__bytes_write.sum 3.904 MB, means of two launches of the kernel as
+# it is now); every weight byte is read exactly once, so traffic scales with the number of blocks.  Set to None whenever
+# that kernel changes.
+HEADLINE_TRAFFIC_PER_BLOCK = (138.987008e6 + 3.904e6) / 8
 
 
 def load_peaks():

@@ -5,7 +5,8 @@ written out term by term, imported only by tests, the smoke check and the benchm
 Paper anchors
   * Eq. 3: pi(a|s_t) = softmax(g_phi(h_t)), V(s_t) = v_psi(h_t); Table VI: both heads have two hidden layers of
     256 and 128 units and run in fp32.  The paper does not name the activation: tanh is taken (the usual choice
-    for PPO heads), see the readings table of the design notes.
+    for PPO heads); the first layer's width follows the latent (d -> 256 -> 128 -> outputs), so the "~50K parameters" the
+    paper quotes cannot hold for d = 2560 and the layer widths are followed, not the count.
   * Eq. 1: L_CLIP = E_t[min(r_t A_t, clip(r_t, 1-eps, 1+eps) A_t)], r_t = pi_new(a_t|s_t) / pi_old(a_t|s_t), eps = 0.1.
   * Sec. III-B: entropy regularization with coefficient beta = 0.05; advantages from GAE(lambda = 0.95, gamma = 0.99).
 """
