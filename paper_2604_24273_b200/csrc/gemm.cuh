@@ -95,7 +95,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   // With the A operand in tensor memory the two accumulators sit at columns [0,TOK) and [256,256+TOK).
   // Weight slots in tensor memory are the 32-column pieces between the end of each accumulator and the next multiple
   // of 256: slot i sits behind accumulator (i & 1), piece i / 2.  TOK = 224 leaves two slots, TOK <= 192 four.
-  constexpr uint32_t WSK = !A_TMEM ? GM_WS : ((256 - GM_TOK) / 32 >= 2 ? 4 : 2 * ((256 - GM_TOK) / 32));
+#ifndef GM_WSK_CAP
+#define GM_WSK_CAP 12
+#endif
+  constexpr uint32_t WSK_FREE = 2 * ((256 - GM_TOK) / 32);  // every free 32-column piece of tensor memory is a slot
+  constexpr uint32_t WSK = !A_TMEM ? GM_WS : (WSK_FREE < GM_WSK_CAP ? WSK_FREE : GM_WSK_CAP);
   static_assert(!A_TMEM || (GM_TOK <= 224 && WSK >= 2), "tensor-memory column budget");
   static_assert(WSK < GM_XS, "the expanders watch the x_q ring WSK steps behind; a watched barrier must not flip twice");
   auto a_slot = [](uint32_t slot) { return (slot & 1u) * 256u + GM_TOK + 32u * (slot >> 1); };
