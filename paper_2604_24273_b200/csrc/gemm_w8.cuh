@@ -396,62 +396,88 @@ __global__ void __launch_bounds__(GV8_THREADS) gemv_w8_kernel(Gemv8Args a) {
   extern __shared__ __align__(16) unsigned char gv8_smem[];
   int8_t* xq_s = reinterpret_cast<int8_t*>(gv8_smem);               // [MT][K]
   float* sc_s = reinterpret_cast<float*>(gv8_smem + MT * a.K);      // [MT] a_m / 127
-  pdl_enter();
+  __shared__ float redf[GV8_THREADS / 32];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int K = a.K, nvec8 = K >> 3;
-  for (int m = warp; m < MT; m += GV8_THREADS / 32) {
-    uint2* dst = reinterpret_cast<uint2*>(xq_s + m * K);
-    if (m >= a.M) {
-      for (int i = lane; i < nvec8; i += 32) dst[i] = make_uint2(0u, 0u);
-      if (lane == 0) sc_s[m] = 0.0f;
-      continue;
-    }
-    const uint4* xr = reinterpret_cast<const uint4*>(a.x + static_cast<size_t>(m) * K);
-    float mx = 0.0f;
-#pragma unroll 4
-    for (int i = lane; i < nvec8; i += 32) mx = fmaxf(mx, absmax8(xr[i]));
-    const float amax = fmaxf(warp_max(mx), 1e-5f);
-    const float inv = __fdiv_rn(127.0f, amax);
-    uint2* tap = (a.xq_out && blockIdx.x == 0) ? reinterpret_cast<uint2*>(a.xq_out + static_cast<size_t>(m) * K) : nullptr;
-    for (int i = lane; i < nvec8; i += 32) {
-      const uint4 raw = xr[i];
-      const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
-      int q[8];
+  const int K = a.K, nvec8 = K >> 3, nvec16 = K >> 4;
+  // A warp streams R rows at a time (N is a multiple of 128): R times as many loads in flight per lane, and every
+  // 16-byte piece of the activations read from shared memory serves R rows.
+  constexpr int R = MT <= 4 ? 4 : 2;
+  constexpr int PRE = 2;  // 16-byte steps of the first row group requested before anything else
+  const int n_first = (blockIdx.x * (GV8_THREADS / 32) + warp) * R;
+  // The weights depend neither on the activations nor on the preceding kernel: the first loads of this warp's first
+  // rows are in flight while the CTA waits for its predecessor and quantizes the activations.
+  uint4 pre[PRE][R];
+  if (n_first < a.N) {
+    const uint4* wr = reinterpret_cast<const uint4*>(a.wq + static_cast<size_t>(n_first) * K);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        q[2 * e] = quant_code(__uint_as_float(rw[e] << 16), inv);
-        q[2 * e + 1] = quant_code(__uint_as_float(rw[e] & 0xffff0000u), inv);
-      }
-      uint2 wd;
-      wd.x = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | (static_cast<uint32_t>(q[3]) << 24);
-      wd.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | (static_cast<uint32_t>(q[7]) << 24);
-      dst[i] = wd;
-      if (tap) tap[i] = wd;
+    for (int p = 0; p < PRE; ++p)
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+        if (lane + 32 * p < nvec16) pre[p][r] = __ldg(wr + static_cast<size_t>(r) * nvec16 + lane + 32 * p);
+  }
+  pdl_enter();
+  // Activations: WPR warps share a token (all eight for one token), largest magnitude through shared memory.
+  constexpr int NW = GV8_THREADS / 32;
+  constexpr int WPR = MT >= NW ? 1 : NW / MT;
+  constexpr int RPP = NW / WPR;
+  const int sub = warp % WPR;
+#pragma unroll 1
+  for (int pass = 0; pass < (MT + RPP - 1) / RPP; ++pass) {
+    const int m = pass * RPP + warp / WPR;
+    const bool live = m < a.M;
+    uint2* dst = reinterpret_cast<uint2*>(xq_s + (m < MT ? m : 0) * K);
+    const uint4* xr = reinterpret_cast<const uint4*>(a.x + static_cast<size_t>(live ? m : 0) * K);
+    float mx = 0.0f;
+    if (live) {
+#pragma unroll 4
+      for (int i = sub * 32 + lane; i < nvec8; i += WPR * 32) mx = fmaxf(mx, absmax8(xr[i]));
     }
-    if (lane == 0) {
-      sc_s[m] = __fdiv_rn(amax, 127.0f);
-      if (a.absmax_out && blockIdx.x == 0) a.absmax_out[m] = amax;
+    mx = warp_max(mx);
+    if (WPR > 1) {
+      if (lane == 0) redf[warp] = mx;
+      __syncthreads();
+#pragma unroll
+      for (int i = 0; i < WPR; ++i) mx = fmaxf(mx, redf[(warp / WPR) * WPR + i]);
+      __syncthreads();
+    }
+    const float amax = fmaxf(mx, 1e-5f);
+    const float inv = __fdiv_rn(127.0f, amax);
+    uint2* tap = (live && a.xq_out && blockIdx.x == 0) ? reinterpret_cast<uint2*>(a.xq_out + static_cast<size_t>(m) * K) : nullptr;
+    if (m < MT) {
+      for (int i = sub * 32 + lane; i < nvec8; i += WPR * 32) {
+        uint2 wd = make_uint2(0u, 0u);
+        if (live) {
+          const uint4 raw = xr[i];
+          const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+          int q[8];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            q[2 * e] = quant_code(__uint_as_float(rw[e] << 16), inv);
+            q[2 * e + 1] = quant_code(__uint_as_float(rw[e] & 0xffff0000u), inv);
+          }
+          wd.x = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | (static_cast<uint32_t>(q[3]) << 24);
+          wd.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | (static_cast<uint32_t>(q[7]) << 24);
+        }
+        dst[i] = wd;
+        if (tap) tap[i] = wd;
+      }
+      if (sub == 0 && lane == 0) {
+        sc_s[m] = live ? __fdiv_rn(amax, 127.0f) : 0.0f;
+        if (live && a.absmax_out && blockIdx.x == 0) a.absmax_out[m] = amax;
+      }
     }
   }
   __syncthreads();
 
   const float wscale = *a.scale;
-  const int nvec16 = K >> 4;
-  // A warp streams R rows at a time (N is a multiple of 128): R times as many loads in flight per lane, and every
-  // 16-byte piece of the activations read from shared memory serves R rows.
-  constexpr int R = MT <= 4 ? 4 : 2;
-  for (int n0 = (blockIdx.x * (GV8_THREADS / 32) + warp) * R; n0 < a.N; n0 += gridDim.x * (GV8_THREADS / 32) * R) {
+  for (int n0 = n_first; n0 < a.N; n0 += gridDim.x * (GV8_THREADS / 32) * R) {
     const uint4* wr = reinterpret_cast<const uint4*>(a.wq + static_cast<size_t>(n0) * K);
     int acc[R][MT];
 #pragma unroll
     for (int r = 0; r < R; ++r)
 #pragma unroll
       for (int m = 0; m < MT; ++m) acc[r][m] = 0;
-#pragma unroll 2
-    for (int i = lane; i < nvec16; i += 32) {
-      uint4 wv[R];
-#pragma unroll
-      for (int r = 0; r < R; ++r) wv[r] = wr[static_cast<size_t>(r) * nvec16 + i];
+    auto step = [&](const uint4 (&wv)[R], int i) {
 #pragma unroll
       for (int m = 0; m < MT; ++m) {
         const uint4 xv = *reinterpret_cast<const uint4*>(xq_s + m * K + 16 * i);
@@ -463,6 +489,19 @@ __global__ void __launch_bounds__(GV8_THREADS) gemv_w8_kernel(Gemv8Args a) {
           acc[r][m] = dp4a_s8s8(wv[r].w, xv.w, acc[r][m]);
         }
       }
+    };
+    int i = lane;
+    if (n0 == n_first) {  // the steps whose weights were requested up front
+#pragma unroll
+      for (int p = 0; p < PRE; ++p, i += 32)
+        if (i < nvec16) step(pre[p], i);
+    }
+#pragma unroll 2
+    for (; i < nvec16; i += 32) {
+      uint4 wv[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) wv[r] = wr[static_cast<size_t>(r) * nvec16 + i];
+      step(wv, i);
     }
 #pragma unroll
     for (int r = 0; r < R; ++r)
