@@ -547,6 +547,16 @@ def run_ours(args):
                 extra[f"w8a8_m{Ms}_sweep_8x_k2560_n13824"] = {"GBps_of_weight_bytes": gbs, "us_per_matrix": ms * 1e3 / 8,
                                                              "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "launches": lc}
                 del g
+            # ... and the M = 1 sweep over the same eight matrices as ONE grouped launch
+            xd = inputs.activations(1, 2560, 2001).to(dev)
+            yds = [torch.empty((1, 13824), dtype=torch.bfloat16, device=dev) for _ in w8]
+            call8 = bitrl.W8MultiCall(w8, [xd] * len(w8), yds, bitrl.OUT_BF16)
+            g, lc = capture(call8.run)
+            ms = time_graph(g, sub_steps, args.warmup, 1) / sub_steps
+            gbs = 8 * 13824 * 2560 / (ms * 1e-3) / 1e9
+            extra["w8a8_m1_sweep_8x_k2560_n13824_grouped"] = {"GBps_of_weight_bytes": gbs, "us_per_matrix": ms * 1e3 / 8,
+                                                             "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "launches": lc}
+            del g, call8, yds
             del w8
 
             # the INT4 critic's W4A8 layer: streaming kernel at M = 1 over eight 2560 -> 13824 matrices (141 MB packed),

@@ -258,6 +258,21 @@ BITRL_API bitrl_status bitrl_w8a8_forward_debug(const int8_t* wq, const float* s
                                                 size_t workspace_bytes, int8_t* xq_out, float* absmax_out,
                                                 int32_t* acc_out, void* stream);
 
+/* `count` independent W8A8 layers in one launch, for M <= BITRL_W8_MULTI_MAX_M tokens (one state per step through a critic
+ * backbone is a sweep over many decode-size matrices; a launch per matrix spends a third of its time ramping up):
+ * y[i] = W8A8_{mats[i]}(x[i]), bit-identical to `count` bitrl_w8a8_forward calls.  mats, x, y: HOST arrays of `count`
+ * entries (1 <= count <= BITRL_MULTI_MAX_JOBS); mats[i].wq dev int8 [N,K] row-major, mats[i].scale dev fp32 (the
+ * scale), M * K <= 27648 (six 32 KB slots and the quantized activations share the SM's shared memory; else BITRL_ERR_SHAPE);
+ * x[i] dev bf16 [M,K] (entries may repeat), y[i] dev [M,N], all distinct.  No workspace. */
+#define BITRL_W8_MULTI_MAX_M 2
+typedef struct bitrl_w8_matrix {
+  const int8_t* wq;
+  const float* scale;
+  int32_t N, K;
+} bitrl_w8_matrix_t;
+BITRL_API bitrl_status bitrl_w8a8_forward_multi(int32_t count, const bitrl_w8_matrix_t* mats, const void* const* x,
+                                                void* const* y, int32_t M, int32_t out_dtype, void* stream);
+
 /* ---- W4A8 layer: the "INT4 critic" of the same table (the paper names the precision only) -------------------------
  * Same reading with 7 in place of 127:  a = max(max|W|, 1e-20),  W_q = clip(rint(W * (7 / a)), -8, 7),  scale = a / 7,
  * acc and y as for W8A8.  packed: dev uint8 [N, K/2], byte j of row n = (W_q[n,2j] + 8) | (W_q[n,2j+1] + 8) << 4.

@@ -31,6 +31,11 @@ _vp = ctypes.c_void_p
 _i32 = ctypes.c_int32
 _sz = ctypes.c_size_t
 
+class W8Matrix(ctypes.Structure):
+    """Mirror of ``bitrl_w8_matrix_t``."""
+    _fields_ = [("wq", ctypes.c_void_p), ("scale", ctypes.c_void_p), ("N", ctypes.c_int32), ("K", ctypes.c_int32)]
+
+
 class HeadDesc(ctypes.Structure):
     """Mirror of ``bitrl_head_t``."""
     _fields_ = [("W1t", ctypes.c_void_p), ("b1", ctypes.c_void_p), ("W2t", ctypes.c_void_p), ("b2", ctypes.c_void_p),
@@ -71,6 +76,7 @@ EXPORTS = {
     "bitrl_w8a8_workspace_bytes": (_sz, [_i32, _i32]),
     "bitrl_w8a8_forward": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp]),
     "bitrl_w8a8_forward_debug": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp, _vp, _vp, _vp]),
+    "bitrl_w8a8_forward_multi": (_i32, [_i32, ctypes.POINTER(W8Matrix), ctypes.POINTER(_vp), ctypes.POINTER(_vp), _i32, _i32, _vp]),
     "bitrl_w4_quantize": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp]),
     "bitrl_w4a8_workspace_bytes": (_sz, [_i32, _i32, _i32]),
     "bitrl_w4a8_forward": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp]),
@@ -457,6 +463,35 @@ def w8a8_forward(wq: torch.Tensor, scale: torch.Tensor, x: torch.Tensor, out_dty
                                           workspace.numel(), _ptr(xq), _ptr(a), _ptr(acc), _stream()),
            "bitrl_w8a8_forward_debug")
     return y, xq, a, acc
+
+
+W8_MULTI_MAX_M = 2
+
+
+class W8MultiCall:
+    """Argument block of ``bitrl_w8a8_forward_multi``: ``count`` independent W8A8 layers (M <= 2), one launch.
+    ``mats`` = list of (W_q int8 [N,K], scale fp32) pairs as returned by ``w8_quantize``."""
+
+    def __init__(self, mats, xs, ys, out_dtype: int = OUT_BF16):
+        assert len(mats) == len(xs) == len(ys) >= 1
+        self.M = xs[0].shape[0]
+        for (wq, scale), x, y in zip(mats, xs, ys):
+            _dev(wq, torch.int8, "wq")
+            _dev(scale, torch.float32, "scale")
+            _dev(x, torch.bfloat16, "x")
+            assert x.shape == (self.M, wq.shape[1]) and tuple(y.shape) == (self.M, wq.shape[0]) and y.is_contiguous()
+            assert y.dtype == (torch.float32 if out_dtype == OUT_F32 else torch.bfloat16)
+        self.keep = (list(mats), list(xs), list(ys))
+        n = len(mats)
+        self.count, self.out_dtype = n, out_dtype
+        self.mats = (W8Matrix * n)(*[W8Matrix(wq.data_ptr(), sc.data_ptr(), wq.shape[0], wq.shape[1]) for wq, sc in mats])
+        self.x = (_vp * n)(*[x.data_ptr() for x in xs])
+        self.y = (_vp * n)(*[y.data_ptr() for y in ys])
+
+    def run(self):
+        _check(lib().bitrl_w8a8_forward_multi(self.count, self.mats, self.x, self.y, self.M, self.out_dtype, _stream()),
+               "bitrl_w8a8_forward_multi")
+        return self.keep[2]
 
 
 def w4_quantize(W: torch.Tensor):

@@ -88,6 +88,7 @@ static bitrl_status check_arch() {
 #include "gemm_w8.cuh"
 #include "w4.cuh"
 #include "gemv5.cuh"
+#include "gemv8_multi.cuh"
 
 using namespace bitrl;
 
@@ -651,6 +652,23 @@ bitrl_status bitrl_w8a8_forward_debug(const int8_t* wq, const float* scale, cons
                                       void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes, int8_t* xq_out,
                                       float* absmax_out, int32_t* acc_out, void* stream) {
   return w8a8_impl(wq, scale, x, M, K, N, y, out_dtype, workspace, workspace_bytes, xq_out, absmax_out, acc_out, stream);
+}
+
+bitrl_status bitrl_w8a8_forward_multi(int32_t count, const bitrl_w8_matrix_t* mats, const void* const* x, void* const* y,
+                                      int32_t M, int32_t out_dtype, void* stream) {
+  if (!mats || !x || !y) return BITRL_ERR_NULL;
+  if (count < 1 || count > BITRL_MULTI_MAX_JOBS || M < 1 || M > BITRL_W8_MULTI_MAX_M) return BITRL_ERR_SHAPE;
+  if (out_dtype != BITRL_OUT_F32 && out_dtype != BITRL_OUT_BF16) return BITRL_ERR_DTYPE;
+  W8Matrix w[BITRL_MULTI_MAX_JOBS];
+  for (int i = 0; i < count; ++i) {
+    if (!mats[i].wq || !mats[i].scale || !x[i] || !y[i]) return BITRL_ERR_NULL;
+    if (!shape_ok(mats[i].N, mats[i].K) || mats[i].K > 32768) return BITRL_ERR_SHAPE;
+    if (!aligned16(mats[i].wq) || !aligned16(x[i]) || !aligned16(y[i])) return BITRL_ERR_ALIGN;
+    w[i] = W8Matrix{mats[i].wq, mats[i].scale, mats[i].N, mats[i].K};
+  }
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  return launch_gemv8_multi(count, w, x, y, M, out_dtype, static_cast<cudaStream_t>(stream));
 }
 
 // ---- W4A8 layer (INT4 critic) -----------------------------------------------------------------------------------

@@ -93,6 +93,38 @@ def test_w8a8_m4096_sampled(oracle_mod, B):
     assert rel_err(bits_to_f64(inputs.bf16_bits(y.cpu())[ms, ns]), y64) <= 8e-3
 
 
+@pytest.mark.parametrize("M,out_dtype", [(1, 1), (2, 0), (2, 1)])
+def test_w8a8_forward_multi_matches_oracle_and_single_calls(oracle_mod, B, M, out_dtype):
+    """Several independent W8A8 layers in one launch (rows per ring slot: 12 at K = 2560, 4 at 6912, 25 at 1280, a ragged
+    last slot everywhere): bit-identical to the oracle and to separate calls."""
+    specs = [(384, 256, 9200), (2560, 2560, 9202), (2560, 6912, 9204), (128, 640, 9201), (6912, 2560, 9203), (640, 1280, 9205)]
+    xs_cpu = {K: inputs.activations(M, K, 9800 + K + M) for K in {k for _, k, _ in specs}}
+    xs_gpu = {K: v.cuda() for K, v in xs_cpu.items()}
+    mats, xs, ys, refs = [], [], [], []
+    dt = torch.float32 if out_dtype == 0 else torch.bfloat16
+    for N, K, seed in specs:
+        Wq, scale, wq_gpu, scale_gpu = weights(oracle_mod, B, N, K, seed)
+        mats.append((wq_gpu, scale_gpu))
+        xs.append(xs_gpu[K])
+        ys.append(torch.full((M, N), 7.0, dtype=dt, device="cuda"))
+        refs.append(oracle_mod.bitlinear(inputs.bf16_bits(xs_cpu[K]), Wq, scale))
+    call = B.W8MultiCall(mats, xs, ys, out_dtype)
+    call.run()
+    call.run()
+    B.poll_status()
+    for (wq_gpu, scale_gpu), x, y, ref in zip(mats, xs, ys, refs):
+        assert torch.equal(B.w8a8_forward(wq_gpu, scale_gpu, x, out_dtype), y)
+        if out_dtype == 0:
+            assert np.array_equal(y.cpu().numpy(), ref["y32"])
+        else:
+            yb = inputs.bf16_bits(y.cpu())
+            assert np.array_equal(yb, ref["ybf16"])
+            assert rel_err(bits_to_f64(yb), ref["y64"]) <= 8e-3
+    L = B.lib()
+    assert L.bitrl_w8a8_forward_multi(1, call.mats, call.x, call.y, 3, out_dtype, None) == B.ERR_SHAPE
+    assert L.bitrl_w8a8_forward_multi(0, call.mats, call.x, call.y, M, out_dtype, None) == B.ERR_SHAPE
+
+
 def test_w8a8_argument_errors(oracle_mod, B):
     L = B.lib()
     Wq, scale, wq_gpu, scale_gpu = weights(oracle_mod, B, 384, 256, 9200)
