@@ -577,7 +577,15 @@ def run_ours(args):
             gbs = 8 * 13824 * 2560 / 2 / (ms * 1e-3) / 1e9
             extra["w4a8_m1_sweep_8x_k2560_n13824"] = {"GBps_of_packed_bytes": gbs, "us_per_matrix": ms * 1e3 / 8,
                                                        "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "launches": lc}
-            del g, w4
+            del g
+            yds = [torch.empty((1, 13824), dtype=torch.bfloat16, device=dev) for _ in w4]
+            call4 = bitrl.W8MultiCall(w4, [xd] * len(w4), yds, bitrl.OUT_BF16, int4=True)
+            g, lc = capture(call4.run)
+            ms = time_graph(g, sub_steps, args.warmup, 1) / sub_steps
+            gbs = 8 * 13824 * 2560 / 2 / (ms * 1e-3) / 1e9
+            extra["w4a8_m1_sweep_8x_k2560_n13824_grouped"] = {"GBps_of_packed_bytes": gbs, "us_per_matrix": ms * 1e3 / 8,
+                                                               "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "launches": lc}
+            del g, call4, yds, w4
             gen.manual_seed(1700)
             p4, sc4 = bitrl.w4_quantize(torch.randn(6912, 2560, generator=gen, device="cuda", dtype=torch.float32) * inputs.SIGMA_W)
             xs = [inputs.activations(M, 2560, 2400 + i).to(dev) for i in range(4)]

@@ -289,6 +289,16 @@ BITRL_API bitrl_status bitrl_w4a8_forward_debug(const uint8_t* packed, const flo
                                                 size_t workspace_bytes, int8_t* xq_out, float* absmax_out,
                                                 int32_t* acc_out, void* stream);
 
+/* The grouped launch for W4A8 layers, as bitrl_w8a8_forward_multi (same limits; mats[i].packed dev uint8 [N,K/2]);
+ * bit-identical to `count` bitrl_w4a8_forward calls. */
+typedef struct bitrl_w4_matrix {
+  const uint8_t* packed;
+  const float* scale;
+  int32_t N, K;
+} bitrl_w4_matrix_t;
+BITRL_API bitrl_status bitrl_w4a8_forward_multi(int32_t count, const bitrl_w4_matrix_t* mats, const void* const* x,
+                                                void* const* y, int32_t M, int32_t out_dtype, void* stream);
+
 /* ---- five weights per byte: the denser, lookup-table-decoded format of the streaming path (Abstract: 1.58-bit
  * weights; Sec. V, edge-deployment paragraph: ternary products as additions and subtractions "with lookup tables") ----
  * Format (the paper gives none): byte j of row n = sum_{i=0..4} (W_q[n,5j+i] + 1) * 3^i, ceil(K/5) bytes per row,

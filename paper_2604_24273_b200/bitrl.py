@@ -77,6 +77,7 @@ EXPORTS = {
     "bitrl_w8a8_forward": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp]),
     "bitrl_w8a8_forward_debug": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp, _vp, _vp, _vp]),
     "bitrl_w8a8_forward_multi": (_i32, [_i32, ctypes.POINTER(W8Matrix), ctypes.POINTER(_vp), ctypes.POINTER(_vp), _i32, _i32, _vp]),
+    "bitrl_w4a8_forward_multi": (_i32, [_i32, ctypes.POINTER(W8Matrix), ctypes.POINTER(_vp), ctypes.POINTER(_vp), _i32, _i32, _vp]),
     "bitrl_w4_quantize": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp]),
     "bitrl_w4a8_workspace_bytes": (_sz, [_i32, _i32, _i32]),
     "bitrl_w4a8_forward": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _sz, _vp]),
@@ -470,27 +471,31 @@ W8_MULTI_MAX_M = 2
 
 class W8MultiCall:
     """Argument block of ``bitrl_w8a8_forward_multi``: ``count`` independent W8A8 layers (M <= 2), one launch.
-    ``mats`` = list of (W_q int8 [N,K], scale fp32) pairs as returned by ``w8_quantize``."""
+    ``mats`` = list of (W_q int8 [N,K], scale fp32) pairs as returned by ``w8_quantize``.
+    With ``int4=True``: ``bitrl_w4a8_forward_multi`` on (packed uint8 [N,K/2], scale) pairs from ``w4_quantize``."""
 
-    def __init__(self, mats, xs, ys, out_dtype: int = OUT_BF16):
+    def __init__(self, mats, xs, ys, out_dtype: int = OUT_BF16, int4: bool = False):
         assert len(mats) == len(xs) == len(ys) >= 1
         self.M = xs[0].shape[0]
+        self.int4 = int4
+        kmul = 2 if int4 else 1
         for (wq, scale), x, y in zip(mats, xs, ys):
-            _dev(wq, torch.int8, "wq")
+            _dev(wq, torch.uint8 if int4 else torch.int8, "wq")
             _dev(scale, torch.float32, "scale")
             _dev(x, torch.bfloat16, "x")
-            assert x.shape == (self.M, wq.shape[1]) and tuple(y.shape) == (self.M, wq.shape[0]) and y.is_contiguous()
+            assert x.shape == (self.M, wq.shape[1] * kmul) and tuple(y.shape) == (self.M, wq.shape[0]) and y.is_contiguous()
             assert y.dtype == (torch.float32 if out_dtype == OUT_F32 else torch.bfloat16)
         self.keep = (list(mats), list(xs), list(ys))
         n = len(mats)
         self.count, self.out_dtype = n, out_dtype
-        self.mats = (W8Matrix * n)(*[W8Matrix(wq.data_ptr(), sc.data_ptr(), wq.shape[0], wq.shape[1]) for wq, sc in mats])
+        self.mats = (W8Matrix * n)(*[W8Matrix(wq.data_ptr(), sc.data_ptr(), wq.shape[0], wq.shape[1] * kmul) for wq, sc in mats])
         self.x = (_vp * n)(*[x.data_ptr() for x in xs])
         self.y = (_vp * n)(*[y.data_ptr() for y in ys])
 
     def run(self):
-        _check(lib().bitrl_w8a8_forward_multi(self.count, self.mats, self.x, self.y, self.M, self.out_dtype, _stream()),
-               "bitrl_w8a8_forward_multi")
+        fn = lib().bitrl_w4a8_forward_multi if self.int4 else lib().bitrl_w8a8_forward_multi
+        _check(fn(self.count, self.mats, self.x, self.y, self.M, self.out_dtype, _stream()),
+               "bitrl_w4a8_forward_multi" if self.int4 else "bitrl_w8a8_forward_multi")
         return self.keep[2]
 
 

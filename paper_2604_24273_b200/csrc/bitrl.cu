@@ -668,7 +668,7 @@ bitrl_status bitrl_w8a8_forward_multi(int32_t count, const bitrl_w8_matrix_t* ma
   }
   bitrl_status s = check_arch();
   if (s != BITRL_OK) return s;
-  return launch_gemv8_multi(count, w, x, y, M, out_dtype, static_cast<cudaStream_t>(stream));
+  return launch_gemv8_multi(count, w, x, y, M, out_dtype, false, static_cast<cudaStream_t>(stream));
 }
 
 // ---- W4A8 layer (INT4 critic) -----------------------------------------------------------------------------------
@@ -794,6 +794,23 @@ bitrl_status bitrl_bitlinear5_forward_multi(int32_t count, const bitrl_linear5_t
   bitrl_status s = check_arch();
   if (s != BITRL_OK) return s;
   return launch_gemv5_multi(count, lins, x, y, M, out_dtype, static_cast<cudaStream_t>(stream));
+}
+
+bitrl_status bitrl_w4a8_forward_multi(int32_t count, const bitrl_w4_matrix_t* mats, const void* const* x, void* const* y,
+                                      int32_t M, int32_t out_dtype, void* stream) {
+  if (!mats || !x || !y) return BITRL_ERR_NULL;
+  if (count < 1 || count > BITRL_MULTI_MAX_JOBS || M < 1 || M > BITRL_W8_MULTI_MAX_M) return BITRL_ERR_SHAPE;
+  if (out_dtype != BITRL_OUT_F32 && out_dtype != BITRL_OUT_BF16) return BITRL_ERR_DTYPE;
+  W8Matrix w[BITRL_MULTI_MAX_JOBS];
+  for (int i = 0; i < count; ++i) {
+    if (!mats[i].packed || !mats[i].scale || !x[i] || !y[i]) return BITRL_ERR_NULL;
+    if (!shape_ok(mats[i].N, mats[i].K) || mats[i].K > 32768) return BITRL_ERR_SHAPE;
+    if (!aligned16(mats[i].packed) || !aligned16(x[i]) || !aligned16(y[i])) return BITRL_ERR_ALIGN;
+    w[i] = W8Matrix{reinterpret_cast<const int8_t*>(mats[i].packed), mats[i].scale, mats[i].N, mats[i].K};
+  }
+  bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  return launch_gemv8_multi(count, w, x, y, M, out_dtype, true, static_cast<cudaStream_t>(stream));
 }
 
 // ---- self-test of the bounded-wait / status-word path ----

@@ -1,13 +1,16 @@
-// Grouped streaming kernel of the W8A8 layer (the higher-precision critic of Table IV): several independent layers with
-// M <= 2 tokens in ONE launch, int8 weights read once at HBM speed.
+// Grouped streaming kernel of the W8A8 and W4A8 layers (the higher-precision critics of Table IV): several independent
+// layers with M <= 2 tokens in ONE launch, the int8 (or packed int4) weights read once at HBM speed.
 //
 // A single decode-size launch of this layer (35 MB at most) spends a third of its time ramping up and quantizing the
 // activations; a critic backbone evaluated for one state per step is a sweep over many such matrices.  As in the
 // ternary path the sweep is one persistent kernel: one CTA per SM, a producer thread that streams the row-major weights
 // in slots of R whole rows (R * K <= 32 KB, one bulk copy and one mbarrier per slot) through a ring of six slots, and
-// sixteen consumer warps.  Nothing is decoded: a warp owns whole rows (global row index mod 16), its lanes walk a row in
-// 16-byte steps (conflict-free in shared memory), dp4a signed x signed, one shuffle tree per row.  The work list is
-// every job's rows in slot units, split into contiguous byte-balanced ranges, two per CTA.
+// sixteen consumer warps.  A warp owns whole rows (global row index mod 16), its lanes walk a row in 16-byte steps
+// (conflict-free in shared memory) and feed dp4a; one shuffle tree per row.  int8 weights are used as they are
+// (signed x signed); int4 weights are two biased codes (q + 8) per byte, split into their nibble planes by two masks
+// (the high plane stays at its bit position and is scaled back by an exact shift once per row) and multiplied as
+// unsigned bytes with activations stored even-k / odd-k de-interleaved, the bias repaid as 8 * sum_k x_q.  The work
+// list is every job's rows in slot units, split into contiguous byte-balanced ranges, two per CTA.
 #pragma once
 
 #include <algorithm>
@@ -16,6 +19,7 @@
 #include "common.cuh"
 #include "gemm_w8.cuh"
 #include "gemv_multi.cuh"
+#include "w4.cuh"
 #include "ptx.cuh"
 
 namespace bitrl {
@@ -32,7 +36,8 @@ struct Gv8Job {
   const unsigned short* x;
   void* y;
   int N, K;
-  int rows_per_slot;  // R = floor(32 KB / K), at least 1
+  int row_bytes;      // K for int8 weights, K / 2 for packed int4
+  int rows_per_slot;  // R = floor(32 KB / row_bytes), at least 1
   int unit_begin;     // index of this job's first slot unit in the global work list
 };
 
@@ -42,7 +47,7 @@ struct Gv8mArgs {
   int njobs, M, out_dtype, kmax;
 };
 
-template <int MT>
+template <int MT, bool W4>
 __global__ void __launch_bounds__(GV8M_THREADS, 1) gemv8_multi_kernel(const __grid_constant__ Gv8mArgs a) {
   extern __shared__ __align__(128) unsigned char gv8m_smem[];
   const uint32_t ring = ptx::smem_u32(gv8m_smem);
@@ -52,6 +57,8 @@ __global__ void __launch_bounds__(GV8M_THREADS, 1) gemv8_multi_kernel(const __gr
   const uint32_t bar_empty = bar_full + 8 * GV8M_DEPTH;    // [DEPTH]
   float* sc_s = reinterpret_cast<float*>(tail + 16 * GV8M_DEPTH);  // [MT] a_m / 127
   float* redf = sc_s + MT;                                         // [CONSUMERS]
+  int* redi = reinterpret_cast<int*>(redf + GV8M_CONSUMERS);       // [CONSUMERS]
+  int* rs_s = redi + GV8M_CONSUMERS;                               // [MT] sum_k x_q (int4 weights only)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int u_begin = a.seg[blockIdx.x][0], u_mid = a.seg[blockIdx.x][1], u_resume = a.seg[blockIdx.x][2],
@@ -78,10 +85,10 @@ __global__ void __launch_bounds__(GV8M_THREADS, 1) gemv8_multi_kernel(const __gr
         const Gv8Job& job = a.jobs[j];
         const int row0 = (u - job.unit_begin) * job.rows_per_slot;
         const int rows = min(job.rows_per_slot, job.N - row0);
-        const uint32_t bytes = static_cast<uint32_t>(rows) * job.K;
+        const uint32_t bytes = static_cast<uint32_t>(rows) * job.row_bytes;
         if (!ptx::mbar_wait(bar_empty + 8 * s, ph ^ 1u)) { report_timeout(GV8M_WAIT_EMPTY); ok = false; break; }
         ptx::mbar_arrive_expect_tx(bar_full + 8 * s, bytes);
-        ptx::bulk_g2s(ring + s * GV8M_SLOT_BYTES, job.wq + static_cast<size_t>(row0) * job.K, bytes, bar_full + 8 * s);
+        ptx::bulk_g2s(ring + s * GV8M_SLOT_BYTES, job.wq + static_cast<size_t>(row0) * job.row_bytes, bytes, bar_full + 8 * s);
         if (++s == GV8M_DEPTH) { s = 0; ph ^= 1u; }
       }
     }
@@ -106,7 +113,7 @@ __global__ void __launch_bounds__(GV8M_THREADS, 1) gemv8_multi_kernel(const __gr
           uint2* dst = reinterpret_cast<uint2*>(xq_s + m * K);
           if (m >= a.M) {
             for (int i = threadIdx.x; i < nvec8; i += NTH) dst[i] = make_uint2(0u, 0u);
-            if (threadIdx.x == 0) sc_s[m] = 0.0f;
+            if (threadIdx.x == 0) { sc_s[m] = 0.0f; rs_s[m] = 0; }
             continue;
           }
           const uint4* xr = reinterpret_cast<const uint4*>(job.x + static_cast<size_t>(m) * K);
@@ -119,6 +126,7 @@ __global__ void __launch_bounds__(GV8M_THREADS, 1) gemv8_multi_kernel(const __gr
           for (int i = 0; i < GV8M_CONSUMERS; ++i) mx = fmaxf(mx, redf[i]);
           const float amax = fmaxf(mx, 1e-5f);
           const float inv = __fdiv_rn(127.0f, amax);
+          int rs = 0;
           for (int i = threadIdx.x; i < nvec8; i += NTH) {
             const uint4 raw = xr[i];
             const uint32_t rwd[4] = {raw.x, raw.y, raw.z, raw.w};
@@ -131,10 +139,26 @@ __global__ void __launch_bounds__(GV8M_THREADS, 1) gemv8_multi_kernel(const __gr
             uint2 wd;
             wd.x = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | (static_cast<uint32_t>(q[3]) << 24);
             wd.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | (static_cast<uint32_t>(q[7]) << 24);
+            if (W4) {  // even k | odd k of every eight: the order the two nibble planes of a weight word come out in
+              rs += q[0] + q[1] + q[2] + q[3] + q[4] + q[5] + q[6] + q[7];
+              wd = make_uint2(__byte_perm(wd.x, wd.y, 0x6420), __byte_perm(wd.x, wd.y, 0x7531));
+            }
             dst[i] = wd;
           }
+          if (W4) {
+            rs = warp_sum_i(rs);
+            if (lane == 0) redi[warp] = rs;
+          }
           asm volatile("bar.sync 2, %0;" ::"n"(GV8M_CONSUMERS * 32) : "memory");  // redf is reused by the next token
-          if (threadIdx.x == 0) sc_s[m] = __fdiv_rn(amax, 127.0f);
+          if (threadIdx.x == 0) {
+            sc_s[m] = __fdiv_rn(amax, 127.0f);
+            int t = 0;
+            if (W4) {
+#pragma unroll
+              for (int i = 0; i < GV8M_CONSUMERS; ++i) t += redi[i];
+            }
+            rs_s[m] = t;
+          }
         }
         asm volatile("bar.sync 2, %0;" ::"n"(GV8M_CONSUMERS * 32) : "memory");
         cached_x = job.x;
@@ -147,30 +171,44 @@ __global__ void __launch_bounds__(GV8M_THREADS, 1) gemv8_multi_kernel(const __gr
       const float wscale = *job.scale;
       if (ok && !ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(GV8M_WAIT_FULL); ok = false; }
       if (ok) {
-        const int nvec16 = K >> 4;
+        const int nvec16 = job.row_bytes >> 4;  // 16-byte pieces of a row: 16 int8 or 32 int4 weights each
         for (int r = (warp - row0) & (GV8M_CONSUMERS - 1); r < rows; r += GV8M_CONSUMERS) {
-          const uint32_t wrow = ring + s * GV8M_SLOT_BYTES + static_cast<uint32_t>(r) * K;
-          int acc[MT];
+          const uint32_t wrow = ring + s * GV8M_SLOT_BYTES + static_cast<uint32_t>(r) * job.row_bytes;
+          int acc[MT], acc_hi[MT];  // acc_hi: the high-nibble plane left at its bit position, i.e. 16 times its share
 #pragma unroll
-          for (int m = 0; m < MT; ++m) acc[m] = 0;
+          for (int m = 0; m < MT; ++m) acc[m] = acc_hi[m] = 0;
 #pragma unroll 4
           for (int i = lane; i < nvec16; i += 32) {
             const uint4 wv = ptx::lds128(wrow + 16 * i);
 #pragma unroll
             for (int m = 0; m < MT; ++m) {
-              const uint4 xv = *reinterpret_cast<const uint4*>(xq_s + m * K + 16 * i);
-              acc[m] = dp4a_s8s8(wv.x, xv.x, acc[m]);
-              acc[m] = dp4a_s8s8(wv.y, xv.y, acc[m]);
-              acc[m] = dp4a_s8s8(wv.z, xv.z, acc[m]);
-              acc[m] = dp4a_s8s8(wv.w, xv.w, acc[m]);
+              if (W4) {
+                // word p of the piece holds k = 32 i + 8 p .. + 7; its activations are the words 2p (even k), 2p + 1 (odd k)
+                const uint4 xa = *reinterpret_cast<const uint4*>(xq_s + m * K + 32 * i);
+                const uint4 xb = *reinterpret_cast<const uint4*>(xq_s + m * K + 32 * i + 16);
+                const uint32_t xe[4] = {xa.x, xa.z, xb.x, xb.z}, xo[4] = {xa.y, xa.w, xb.y, xb.w};
+                const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+                for (int p = 0; p < 4; ++p) {
+                  acc[m] = dp4a_u8s8(ww[p] & 0x0f0f0f0fu, static_cast<int>(xe[p]), acc[m]);
+                  acc_hi[m] = dp4a_u8s8(ww[p] & 0xf0f0f0f0u, static_cast<int>(xo[p]), acc_hi[m]);
+                }
+              } else {
+                const uint4 xv = *reinterpret_cast<const uint4*>(xq_s + m * K + 16 * i);
+                acc[m] = dp4a_s8s8(wv.x, xv.x, acc[m]);
+                acc[m] = dp4a_s8s8(wv.y, xv.y, acc[m]);
+                acc[m] = dp4a_s8s8(wv.z, xv.z, acc[m]);
+                acc[m] = dp4a_s8s8(wv.w, xv.w, acc[m]);
+              }
             }
           }
 #pragma unroll
-          for (int m = 0; m < MT; ++m) acc[m] = warp_sum_i(acc[m]);
+          for (int m = 0; m < MT; ++m) acc[m] = warp_sum_i(acc[m] + (acc_hi[m] >> 4));  // exact: a multiple of 16
           if (lane == 0) {
 #pragma unroll
             for (int m = 0; m < MT; ++m) {
               if (m < a.M) {
+                if (W4) acc[m] -= 8 * rs_s[m];
                 const float yv = __fmul_rn(static_cast<float>(acc[m]), __fmul_rn(wscale, sc_s[m]));
                 const size_t o = static_cast<size_t>(m) * job.N + row0 + r;
                 if (a.out_dtype == BITRL_OUT_F32) static_cast<float*>(job.y)[o] = yv;
@@ -188,7 +226,7 @@ __global__ void __launch_bounds__(GV8M_THREADS, 1) gemv8_multi_kernel(const __gr
 }
 
 struct W8Matrix {
-  const int8_t* wq;
+  const int8_t* wq;   // int8 [N,K], or packed int4 [N,K/2] (as bytes)
   const float* scale;
   int32_t N, K;
 };
@@ -198,17 +236,18 @@ inline bool gemv8_multi_fits(int M, int kmax) {
          kmax <= GV8M_SLOT_BYTES;
 }
 
-template <int MT>
+template <int MT, bool W4>
 bitrl_status launch_gemv8_multi_t(const Gv8mArgs& a, int grid, size_t smem, cudaStream_t st) {
-  BITRL_CUDA(cudaFuncSetAttribute(gemv8_multi_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  BITRL_CUDA(cudaFuncSetAttribute(gemv8_multi_kernel<MT, W4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   static_cast<int>(smem)));
-  BITRL_CUDA(launch_pdl(gemv8_multi_kernel<MT>, dim3(grid), dim3(GV8M_THREADS), smem, st, a));
+  BITRL_CUDA(launch_pdl(gemv8_multi_kernel<MT, W4>, dim3(grid), dim3(GV8M_THREADS), smem, st, a));
   count_launch(1);
   return BITRL_OK;
 }
 
+// int4 = false: w[i].wq is int8 [N,K]; true: packed int4 [N,K/2].
 bitrl_status launch_gemv8_multi(int count, const W8Matrix* w, const void* const* x, void* const* y, int M, int out_dtype,
-                                cudaStream_t st) {
+                                bool int4, cudaStream_t st) {
   static thread_local Gv8mArgs a;
   int kmax = 0, units = 0;
   long long pieces = 0;  // in 1 KB, for the byte balance
@@ -219,12 +258,14 @@ bitrl_status launch_gemv8_multi(int count, const W8Matrix* w, const void* const*
   sz.clear();
   for (int i = 0; i < count; ++i) {
     const W8Matrix& m = w[order[i]];
-    const int R = std::max(1, GV8M_SLOT_BYTES / m.K);
-    a.jobs[i] = Gv8Job{m.wq, m.scale, static_cast<const unsigned short*>(x[order[i]]), y[order[i]], m.N, m.K, R, units};
+    const int row_bytes = int4 ? m.K / 2 : m.K;
+    const int R = std::max(1, GV8M_SLOT_BYTES / row_bytes);
+    a.jobs[i] = Gv8Job{m.wq, m.scale, static_cast<const unsigned short*>(x[order[i]]), y[order[i]], m.N, m.K, row_bytes, R,
+                       units};
     const int nslots = (m.N + R - 1) / R;
     for (int u = 0; u < nslots; ++u) {
       const int rows = std::min(R, m.N - u * R);
-      const int kb = (rows * m.K + 1023) / 1024;
+      const int kb = (rows * row_bytes + 1023) / 1024;
       sz.push_back(kb);
       pieces += kb;
     }
@@ -241,7 +282,8 @@ bitrl_status launch_gemv8_multi(int count, const W8Matrix* w, const void* const*
   a.out_dtype = out_dtype;
   a.kmax = kmax;
   const size_t smem = static_cast<size_t>(GV8M_DEPTH) * GV8M_SLOT_BYTES + static_cast<size_t>(M) * kmax + 1024;
-  return M == 1 ? launch_gemv8_multi_t<1>(a, grid, smem, st) : launch_gemv8_multi_t<2>(a, grid, smem, st);
+  if (int4) return M == 1 ? launch_gemv8_multi_t<1, true>(a, grid, smem, st) : launch_gemv8_multi_t<2, true>(a, grid, smem, st);
+  return M == 1 ? launch_gemv8_multi_t<1, false>(a, grid, smem, st) : launch_gemv8_multi_t<2, false>(a, grid, smem, st);
 }
 
 }  // namespace bitrl

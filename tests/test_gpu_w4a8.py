@@ -66,6 +66,34 @@ def test_w4a8_full(oracle_mod, B, M, K, N, seed, out_dtype):
         assert np.array_equal(yb, ref["ybf16"]) and torch.equal(y, y2)
 
 
+@pytest.mark.parametrize("M,out_dtype", [(1, 1), (2, 0), (2, 1)])
+def test_w4a8_forward_multi_matches_oracle_and_single_calls(oracle_mod, B, M, out_dtype):
+    """Several independent W4A8 layers in one launch: bit-identical to the oracle and to separate calls."""
+    specs = [(384, 256, 9500), (128, 640, 9501), (2560, 2560, 9502), (384, 256, 9500), (2560, 6912, 9504)]
+    xs_cpu = {K: inputs.activations(M, K, 9900 + K + M) for K in {k for _, k, _ in specs}}
+    xs_gpu = {K: v.cuda() for K, v in xs_cpu.items()}
+    mats, xs, ys, refs = [], [], [], []
+    dt = torch.float32 if out_dtype == 0 else torch.bfloat16
+    for N, K, seed in specs:
+        Wq, scale, packed_gpu, scale_gpu = weights(oracle_mod, B, N, K, seed)
+        mats.append((packed_gpu, scale_gpu))
+        xs.append(xs_gpu[K])
+        ys.append(torch.full((M, N), 7.0, dtype=dt, device="cuda"))
+        refs.append(oracle_mod.bitlinear(inputs.bf16_bits(xs_cpu[K]), Wq, scale))
+    call = B.W8MultiCall(mats, xs, ys, out_dtype, int4=True)
+    call.run()
+    call.run()
+    B.poll_status()
+    for (packed_gpu, scale_gpu), x, y, ref in zip(mats, xs, ys, refs):
+        assert torch.equal(B.w4a8_forward(packed_gpu, scale_gpu, x, out_dtype), y)
+        if out_dtype == 0:
+            assert np.array_equal(y.cpu().numpy(), ref["y32"])
+        else:
+            yb = inputs.bf16_bits(y.cpu())
+            assert np.array_equal(yb, ref["ybf16"])
+            assert rel_err(bits_to_f64(yb), ref["y64"]) <= 8e-3
+
+
 def test_w4a8_argument_errors(oracle_mod, B):
     L = B.lib()
     Wq, scale, packed_gpu, scale_gpu = weights(oracle_mod, B, 384, 256, 9500)
