@@ -103,11 +103,24 @@ BITRL_API bitrl_status bitrl_quant_act(const void* x, int32_t M, int32_t K, int8
  * x: dev bf16 [M,K]; y: dev [M,N] fp32 (BITRL_OUT_F32) or bf16 (BITRL_OUT_BF16).  K, N must equal the
  * handle's.  M <= BITRL_GEMV_MAX_M: one streaming kernel (quantization in its prologue, rescale in its
  * epilogue; no workspace needed).  Larger M: quantization kernel into the workspace, then the tcgen05 GEMM.
- * workspace: dev, >= bitrl_workspace_bytes(M,K,N) (0 for M <= 16, then NULL is accepted).  Up to M = 512 it also
- * holds M*N int32 of scratch: when a launch has too few output tiles to occupy the SMs, K is split across them, the
- * exact int32 partial sums meet in that scratch (integer atomics: order-free, deterministic) and a finishing kernel
- * applies the rescale.  The results are the same bits either way. */
+ * workspace: dev, >= bitrl_workspace_bytes(M,K,N) (0 for M <= 16, then NULL is accepted).
+ * When a launch has too few output tiles to occupy the SMs, K is split across them.  Narrow token tiles (<= 128
+ * tokens) do that inside one launch: the CTAs of a thread-block cluster take the k ranges of one tile and exchange
+ * their exact int32 partial sums through distributed shared memory.  Otherwise, up to M = 512, the workspace also
+ * holds M*N int32 of scratch where the partial sums meet (integer atomics: order-free, deterministic) and a
+ * finishing kernel applies the rescale.  The results are the same bits in every form. */
 BITRL_API size_t bitrl_workspace_bytes(int32_t M, int32_t K, int32_t N);
+/* Which kernel form the launcher takes for an [M,K] x [N,K]^T product with M > BITRL_GEMV_MAX_M on the current device
+ * (a query for tests and diagnostics; launches nothing).  tok: tokens per tile (64 ... 256).  splits: k ranges per tile.
+ * kind: BITRL_GEMM_SINGLE (one CTA per tile, splits = 1), BITRL_GEMM_SPLIT_SCRATCH, BITRL_GEMM_SPLIT_CLUSTER or
+ * BITRL_GEMM_PAIRED (256-row tiles on CTA pairs).  with_workspace != 0: the caller would pass the workspace above.
+ * Any of the three output pointers may be NULL.  BITRL_ERR_SHAPE unless N, K are multiples of 128 and M >= 1. */
+#define BITRL_GEMM_SINGLE 0
+#define BITRL_GEMM_SPLIT_SCRATCH 1
+#define BITRL_GEMM_SPLIT_CLUSTER 2
+#define BITRL_GEMM_PAIRED 3
+BITRL_API bitrl_status bitrl_gemm_plan(int32_t M, int32_t K, int32_t N, int32_t with_workspace, int32_t* tok,
+                                       int32_t* splits, int32_t* kind);
 BITRL_API bitrl_status bitrl_bitlinear_forward(const bitrl_linear_t* w, const void* x, int32_t M, int32_t K, int32_t N,
                                      void* y, int32_t out_dtype, void* workspace, size_t workspace_bytes,
                                      void* stream);

@@ -94,6 +94,7 @@ EXPORTS = {
     "bitrl_last_cuda_error": (_i32, []),
     "bitrl_status_string": (ctypes.c_char_p, [_i32]),
     "bitrl_launch_count": (ctypes.c_uint64, []),
+    "bitrl_gemm_plan": (_i32, [_i32, _i32, _i32, _i32, ctypes.POINTER(_i32), ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
 }
 
 
@@ -145,6 +146,17 @@ def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
 
 def launch_count() -> int:
     return int(lib().bitrl_launch_count())
+
+
+GEMM_SINGLE, GEMM_SPLIT_SCRATCH, GEMM_SPLIT_CLUSTER, GEMM_PAIRED = 0, 1, 2, 3
+
+
+def gemm_plan(M: int, K: int, N: int, with_workspace: bool = True):
+    """(tokens per tile, k ranges per tile, kind) the launcher takes for this product on the current device."""
+    tok, splits, kind = _i32(), _i32(), _i32()
+    _check(lib().bitrl_gemm_plan(M, K, N, int(with_workspace), ctypes.byref(tok), ctypes.byref(splits),
+                                 ctypes.byref(kind)), "bitrl_gemm_plan")
+    return tok.value, splits.value, kind.value
 
 
 def poll_status() -> None:

@@ -39,6 +39,17 @@ int gemm_pair_mode() {
   return v;
 }
 
+// BITRL_GEMM_CLSK=0 turns the cluster split-K GEMM off (split launches then go through scratch and a finishing kernel);
+// a value of 2 ... 8 makes every launch that can take a cluster of that size take it (tuning runs).
+int gemm_clsk_mode() {
+  static int v = -2;
+  if (v == -2) {
+    const char* e = getenv("BITRL_GEMM_CLSK");
+    v = !e ? -1 : atoi(e);
+  }
+  return v;
+}
+
 // BITRL_GEMM_TOK=<64|128|192|224|256> overrides the launcher's choice of token-tile width (for tuning runs).
 int gemm_forced_tok() {
   static int v = -1;
@@ -857,6 +868,20 @@ bitrl_status bitrl_poll_status(void* stream) {
 int32_t bitrl_last_timeout_stage(void) { return g_last_stage.load(); }
 int32_t bitrl_last_cuda_error(void) { return g_last_cuda.load(); }
 uint64_t bitrl_launch_count(void) { return g_launches.load(); }
+
+bitrl_status bitrl_gemm_plan(int32_t M, int32_t K, int32_t N, int32_t with_workspace, int32_t* tok, int32_t* splits,
+                             int32_t* kind) {
+  if (M < 1 || K < 128 || N < 128 || K % 128 != 0 || N % 128 != 0) return BITRL_ERR_SHAPE;
+  const bitrl_status s = check_arch();
+  if (s != BITRL_OK) return s;
+  const GemmPlan p = gemm_plan(N, K, M, with_workspace != 0);
+  if (tok) *tok = p.tok;
+  if (splits) *splits = p.splits;
+  if (kind)
+    *kind = p.pair ? BITRL_GEMM_PAIRED
+                   : p.splits == 1 ? BITRL_GEMM_SINGLE : p.clsk ? BITRL_GEMM_SPLIT_CLUSTER : BITRL_GEMM_SPLIT_SCRATCH;
+  return BITRL_OK;
+}
 
 const char* bitrl_status_string(bitrl_status s) {
   switch (s) {

@@ -75,21 +75,33 @@ struct GemmArgs {
   int32_t* part;
 };
 
+// Shared memory that the cluster split-K variant sets aside for received partial sums (4 KB per unit of 8 token columns).
+__host__ __device__ constexpr uint32_t gemm_clsk_recv_bytes(int tok) { return tok <= 64 ? 49152u : 65536u; }
+
 // PAIR: two CTAs of a cluster work on one 256-row x TOK-token tile with tcgen05.mma.cta_group::2.  CTA rank r expands
 // weight rows [256 t + 128 r, +128) into its own tensor memory, fetches tokens [TOK/2 * r, +TOK/2) of the tile into its
 // own shared memory and drains its own 128 x TOK slice of the accumulator; rank 0 issues the MMAs.  Per SM this halves
 // the B-operand traffic through shared memory, the binding resource of the single-CTA kernel.  The barriers that gate
 // the MMA (x_full, tmem_empty) are rank 0's and collect the arrivals of both CTAs; the barriers that the MMA's
 // completion releases (x_empty, tmem_full) exist in both CTAs and are reached by one multicast commit.
-template <int GM_TOK, bool A_TMEM, bool PAIR = false>
+//
+// CLSK (cluster split-K, for launches with few tiles): the a.splits CTAs of a cluster take the k ranges of ONE tile, one
+// item per CTA.  When its main loop is done a CTA sends, through distributed shared memory, every peer the raw int32
+// partial sums of the token columns that peer owns (columns are dealt in units of 8, unit range [r U / S, (r+1) U / S)
+// to rank r); after one cluster barrier each CTA adds what it received to its own partial sums and applies the
+// epilogue to its columns.  Integer sums: exact and independent of the order, so the result equals the unsplit one.
+template <int GM_TOK, bool A_TMEM, bool PAIR = false, bool CLSK = false>
 __global__ void __launch_bounds__(GM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   static_assert(!PAIR || A_TMEM, "the paired kernel keeps its weights in tensor memory");
   static_assert(!PAIR || GM_TOK % 16 == 0, "each CTA holds TOK/2 tokens in whole 8-row swizzle groups");
+  static_assert(!CLSK || (A_TMEM && !PAIR && GM_TOK <= 128), "cluster split-K: narrow single-CTA tiles, weights in tensor memory");
   constexpr uint32_t GM_X_BYTES = (PAIR ? GM_TOK / 2 : GM_TOK) * GM_BK;  // this CTA's part of a token tile
   // x_q ring: 128 KB, plus the 48 KB of the shared-memory weight ring when the weights go through tensor memory
-  // (4 stages at 256 tokens, 6 at 224, 7 at 192, 11 at 128, 16 at 64).
-  constexpr uint32_t GM_X_RING = A_TMEM ? GM_OFF_P - GM_OFF_X : GM_X_RING_BYTES;
+  // (4 stages at 256 tokens, 6 at 224, 7 at 192, 11 at 128, 16 at 64).  The cluster split-K variant takes the end of
+  // that area for the partial sums it receives from its peers.
+  constexpr uint32_t GM_RECV = CLSK ? gemm_clsk_recv_bytes(GM_TOK) : 0u;
+  constexpr uint32_t GM_X_RING = A_TMEM ? GM_OFF_P - GM_OFF_X - GM_RECV : GM_X_RING_BYTES;
   constexpr uint32_t GM_XS = GM_X_RING / GM_X_BYTES < GM_XS_MAX ? GM_X_RING / GM_X_BYTES : GM_XS_MAX;
   static_assert(GM_TOK % 32 == 0 && GM_TOK >= 64 && GM_TOK <= GM_TOK_MAX && GM_XS <= GM_XS_MAX, "token tile");
   // With the A operand in tensor memory the two accumulators sit at columns [0,TOK) and [256,256+TOK).
@@ -99,7 +111,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
 #define GM_WSK_CAP 12
 #endif
   constexpr uint32_t WSK_FREE = 2 * ((256 - GM_TOK) / 32);  // every free 32-column piece of tensor memory is a slot
-  constexpr uint32_t WSK = !A_TMEM ? GM_WS : (WSK_FREE < GM_WSK_CAP ? WSK_FREE : GM_WSK_CAP);
+  constexpr uint32_t WSK_CAP = GM_WSK_CAP < GM_XS - 1 ? GM_WSK_CAP : GM_XS - 1;
+  constexpr uint32_t WSK = !A_TMEM ? GM_WS : (WSK_FREE < WSK_CAP ? WSK_FREE : WSK_CAP);
   static_assert(!A_TMEM || (GM_TOK <= 224 && WSK >= 2), "tensor-memory column budget");
   static_assert(WSK < GM_XS, "the expanders watch the x_q ring WSK steps behind; a watched barrier must not flip twice");
   auto a_slot = [](uint32_t slot) { return (slot & 1u) * 256u + GM_TOK + 32u * (slot >> 1); };
@@ -127,7 +140,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   const int kblocks = a.K / GM_BK;
   const int items = a.tiles_total * a.splits;
   // PAIR: both CTAs of a cluster walk the same items (tiles_n then counts 256-row tiles); rank selects the halves.
-  const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;
+  const uint32_t rank = (PAIR || CLSK) ? ptx::cluster_ctarank() : 0u;  // CLSK: = the item's k range (clusters are consecutive CTAs)
+  const uint32_t recv_base = base + GM_OFF_P - GM_RECV;
   const uint32_t failed_peer = PAIR ? ptx::mapa_u32(failed_addr, rank ^ 1u) : 0u;
   auto wait = [&](uint32_t bar, uint32_t parity) { return ptx::mbar_wait_abortable(bar, parity, failed_addr); };
   auto give_up = [&](int stage) {
@@ -172,7 +186,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
-  if (PAIR) ptx::cluster_sync_all();  // the peer's barriers are initialised before anything is sent to them
+  // the peer's barriers are initialised (PAIR) / every CTA of the cluster has started (CLSK) before anything is sent to it
+  if (PAIR || CLSK) ptx::cluster_sync_all();
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   pdl_enter();  // barriers and tensor memory are set up; inputs of the preceding kernel are read only from here on
@@ -224,7 +239,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     // ------------------------------------------------------------------ MMA issuer
     // The whole warp walks the loop (waits included) and one elected lane issues: with uniform control flow the
     // descriptors and addresses stay in uniform registers, which is what the MMA instruction takes its operands from.
-    if (rank == 0) {
+    if (!PAIR || rank == 0) {
       const uint32_t idesc = ptx::idesc_i8(PAIR ? 2 * GM_ROWS : GM_ROWS, GM_TOK, /*a_signed=*/false, /*b_signed=*/true);
       uint32_t lt = 0;
       uint32_t xs = 0, xph = 0, ws = 0;  // ring slots and phase, advanced without divisions
@@ -378,6 +393,101 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     const bool f32 = a.out_dtype == BITRL_OUT_F32;
     uint32_t lt = 0;
     bool ok = true;
+    if constexpr (CLSK) {
+      // One item per CTA.  These four warps are idle during the main loop, so everything the epilogue reads from global
+      // memory is requested first: the per-token scales and row sums go to shared memory, the residual values of the
+      // first unit of this CTA's columns to registers (the later units' are requested one unit ahead).
+      const int tile = static_cast<int>(blockIdx.x) / a.splits;
+      const int tn = tile % a.tiles_n, tm = tile / a.tiles_n;
+      const int S = a.splits;
+      const int tok0 = tm * GM_TOK, tok_hi = min(GM_TOK, a.M - tok0);
+      const int U = (tok_hi + 7) >> 3;  // units of 8 token columns that hold tokens
+      const int own_max = (U + S - 1) / S;
+      const int own_lo = static_cast<int>(rank) * U / S, own_hi = (static_cast<int>(rank) + 1) * U / S;
+      const int row = q * 32 + lane;  // weight row of the tile = tensor-memory lane
+      const int n = tn * GM_ROWS + row;
+      const uint32_t sc_addr = base + GM_OFF_TOK, rs_addr = base + GM_OFF_TOK + 2 * GM_TOK_MAX * 4;
+      for (int j = ep; j < GM_TOK; j += 128) {
+        const int tok = tok0 + j;
+        ptx::sts32(sc_addr + 4 * j, __float_as_uint(tok < a.M ? out_scale(gamma, a.absmax[tok]) : 0.0f));
+        ptx::sts32(rs_addr + 4 * j, static_cast<uint32_t>(tok < a.M ? a.rowsum[tok] : 0));
+      }
+      const bool use_res = a.residual && !f32;
+      auto load_res = [&](int u, unsigned short (&r)[8]) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int col = u * 8 + j;
+          r[j] = (use_res && col < tok_hi) ? a.residual[static_cast<size_t>(tok0 + col) * a.N + n] : static_cast<unsigned short>(0);
+        }
+      };
+      unsigned short rcur[8] = {}, rnxt[8] = {};
+      if (own_lo < own_hi) load_res(own_lo, rcur);
+      // (the named barrier also publishes the scales among the four warps)
+      const bool got = ptx::bar_red_and(1, 128, wait(bar_tmem_full, 0u));
+      if (!got) {
+        if (ep == 0) give_up(GM_WAIT_TMEM_FULL);
+      } else {
+        // Send every peer the partial sums of its token columns: lane = weight row, so the 32 lanes of a warp store 128
+        // consecutive bytes of the peer's receive area [sender slot][unit][column of the unit][row].
+        ptx::tc_fence_after_sync();
+        for (int i = 1; i < S; ++i) {
+          const int p = (static_cast<int>(rank) + i) % S;  // start with the next rank: spreads the traffic
+          const int u_lo = p * U / S, u_hi = (p + 1) * U / S;
+          const int slot = static_cast<int>(rank) < p ? static_cast<int>(rank) : static_cast<int>(rank) - 1;
+          const uint32_t dst = ptx::mapa_u32(recv_base + static_cast<uint32_t>(slot * own_max) * 4096u +
+                                                 static_cast<uint32_t>(row) * 4u, static_cast<uint32_t>(p));
+          for (int u = u_lo; u < u_hi; ++u) {
+            uint32_t v[8];
+            ptx::tmem_ld_32x32b_x8(tmem_base + static_cast<uint32_t>(u * 8) + (static_cast<uint32_t>(q * 32) << 16), v);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) ptx::sts32_cluster(dst + static_cast<uint32_t>((u - u_lo) * 8 + j) * 512u, v[j]);
+          }
+        }
+      }
+      // Every partial sum has arrived once all threads of the cluster have passed this barrier (release / acquire at
+      // cluster scope; the other warps take part from the teardown).  Nobody writes to a peer after it.
+      ptx::cluster_sync_all();
+      if (got && !*failed) {
+        // own partial sums + the S - 1 received ones, then the usual epilogue on this CTA's token columns
+        for (int u = own_lo; u < own_hi; ++u) {
+          if (u + 1 < own_hi) load_res(u + 1, rnxt);
+          uint32_t v[8];
+          ptx::tmem_ld_32x32b_x8(tmem_base + static_cast<uint32_t>(u * 8) + (static_cast<uint32_t>(q * 32) << 16), v);
+          ptx::tmem_ld_wait();
+          for (int sl = 0; sl < S - 1; ++sl) {
+            const uint32_t src = recv_base + static_cast<uint32_t>((sl * own_max + (u - own_lo)) * 8) * 512u +
+                                 static_cast<uint32_t>(row) * 4u;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] += ptx::lds32(src + static_cast<uint32_t>(j) * 512u);
+          }
+          const uint4 rsa = ptx::lds128(rs_addr + u * 32), rsb = ptx::lds128(rs_addr + u * 32 + 16);
+          const uint4 sca = ptx::lds128(sc_addr + u * 32), scb = ptx::lds128(sc_addr + u * 32 + 16);
+          const uint32_t rsv[8] = {rsa.x, rsa.y, rsa.z, rsa.w, rsb.x, rsb.y, rsb.z, rsb.w};
+          const uint32_t scv[8] = {sca.x, sca.y, sca.z, sca.w, scb.x, scb.y, scb.z, scb.w};
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int col = u * 8 + j;
+            if (col < tok_hi) {
+              const size_t off = static_cast<size_t>(tok0 + col) * a.N + n;
+              const int acc = static_cast<int>(v[j] - rsv[j]);
+              if (a.acc_out) a.acc_out[off] = acc;
+              const float yv = __fmul_rn(static_cast<float>(acc), __uint_as_float(scv[j]));
+              if (f32) {
+                static_cast<float*>(a.y)[off] = yv;
+              } else {
+                unsigned short b = float_to_bf16_bits(yv);
+                if (a.residual) b = float_to_bf16_bits(__fadd_rn(bf16_bits_to_float(rcur[j]), bf16_bits_to_float(b)));
+                static_cast<unsigned short*>(a.y)[off] = b;
+              }
+            }
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) rcur[j] = rnxt[j];
+        }
+      }
+      (void)lt; (void)ok; (void)stage; (void)ew;
+    } else
     for (int item = item0; ok && item < items; item += item_step, ++lt) {
       const int tile = item / a.splits;
       const int tn = PAIR ? 2 * (tile % a.tiles_n) + static_cast<int>(rank) : tile % a.tiles_n, tm = tile / a.tiles_n;
@@ -502,13 +612,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   // ---- teardown: every role leaves through here, also after a timeout ----
   __syncwarp();
   ptx::tc_fence_before_sync();
+  if constexpr (CLSK) {
+    // the cluster barrier of the exchange: the epilogue warps pass it inside their role, everyone else here
+    if (warp < GM_EPI_WARP0 || warp >= GM_EXPAND2_WARP0) ptx::cluster_sync_all();
+  }
   __syncthreads();
   if (PAIR) ptx::cluster_sync_all();  // neither CTA leaves (or frees tensor memory) while the other may still reach it
   if (*failed) {
     // Failure path only: a role gave up, so copies and MMAs that nobody waited for may still be in flight.  The MMA
     // issuer waits (bounded) for its MMAs, then every thread lets about a millisecond pass, far longer than any copy
     // takes, before shared and tensor memory are given back.
-    if (warp == 1 && rank == 0) {
+    if (warp == 1 && (!PAIR || rank == 0)) {
       if (ptx::elect_one()) {
         if (PAIR) ptx::mma_commit_pair(bar_drain, 1);
         else ptx::mma_commit(bar_drain);
@@ -548,6 +662,7 @@ inline encode_tiled_fn get_encode_tiled() {
 int sm_count();
 bool gemm_a_in_tmem();
 int gemm_pair_mode();     // BITRL_GEMM_PAIR: 1 = paired CTAs wherever the shape allows, 0 = never, unset = launcher's choice
+int gemm_clsk_mode();     // BITRL_GEMM_CLSK: 0 = no cluster split-K (the scratch + finishing-kernel form is used instead)
 int gemm_forced_tok();    // 0, or the token-tile width forced through BITRL_GEMM_TOK (64, 128, 192, 224, 256)  // expanded weights through tensor memory (default) or through shared memory
 
 // Second kernel of a split-K launch: y = (part - rowsum) * gamma * a_m / 127 (+ residual), 8 outputs per thread.
@@ -648,20 +763,61 @@ inline int gemm_pair_max_clusters(int tok) {
   return gemm_pair_mode() == 1 ? sm_count() / 2 : 0;
 }
 
+inline void (*gemm_clsk_kernel(int tok))(const CUtensorMap, const GemmArgs) {
+  return tok == 128 ? gemm_i8_kernel<128, true, false, true> : gemm_i8_kernel<64, true, false, true>;
+}
+
+// Clusters of `S` CTAs of the cluster split-K kernel that can be resident at once (0: this size cannot be launched).
+inline int gemm_clsk_max_clusters(int tok, int S) {
+  static int cached[64][2][9] = {};
+  int dev = 0;
+  if (S < 2 || S > 8 || cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  int& c = cached[dev][tok == 128 ? 1 : 0][S];
+  if (c == 0) {
+    void (*k)(const CUtensorMap, const GemmArgs) = gemm_clsk_kernel(tok);
+    int n = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(S * 32);
+    cfg.blockDim = dim3(GM_THREADS);
+    cfg.dynamicSmemBytes = GM_SMEM_BYTES;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = S;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM_BYTES) != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&n, k, &cfg) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      n = -1;
+    }
+    c = n;
+  }
+  if (c > 0) return c;
+  // The query can fail under a profiler.  The grid is a static partition and a CTA waits only for the peers of its own
+  // cluster, so an optimistic count merely queues clusters; sizes that may not exist at all are not offered then.
+  return (S == 2 || S == 4 || S == 8) ? sm_count() / S : 0;
+}
+
 // Largest M for which a split-K workspace (M*N int32) is offered.
 constexpr int GM_SPLITK_MAX_M = 512;
 
-// splitk_ws: nullptr, or M*N int32 of scratch that allows split-K when the launch has too few tiles to fill the SMs.
-bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax, const int32_t* rowsum, int M,
-                         void* y, int out_dtype, const void* residual, int32_t* acc_out, cudaStream_t st,
-                         int32_t* splitk_ws) {
-  encode_tiled_fn encode = get_encode_tiled();
-  if (!encode) return cuda_fail(cudaErrorSymbolNotFound);
+// What the launcher does with an [M, K] x [N, K] product on the current device.
+struct GemmPlan {
+  int tok, splits;    // token-tile width; k ranges per tile
+  bool clsk, pair;    // splits > 1 reduced inside a cluster (else through scratch); 256-row tiles on CTA pairs
+  int pair_clusters;  // persistent grid of the paired kernel
+};
+
+// have_ws: the caller offers M*N int32 of scratch (the scratch form of split-K needs it).
+inline GemmPlan gemm_plan(int N, int K, int M, bool have_ws) {
   // Token-tile width and split count: fewest "waves x k blocks per item x time per k block" over the SMs.
   const int sms = sm_count();
-  const int tiles_n = w->N / GM_ROWS;
-  const int kblocks = w->K / GM_BK;
+  const int tiles_n = N / GM_ROWS;
+  const int kblocks = K / GM_BK;
   int tok = 256, splits = 1;
+  bool clsk = false;  // split over the CTAs of a cluster (reduced through distributed shared memory) or through scratch
   long long best = -1;
   {
     const int cand[5] = {256, 224, 192, 128, 64};
@@ -669,18 +825,34 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
       if (cand[i] == 224 && !gemm_a_in_tmem()) continue;
       const long long tiles = static_cast<long long>(tiles_n) * ((M + cand[i] - 1) / cand[i]);
       const long long per_kb = gemm_kb_ns(cand[i], false);
-      const int smax = (splitk_ws && M <= GM_SPLITK_MAX_M && tiles * 2 <= sms) ? static_cast<int>(sms / tiles) : 1;
+      const int smax = (have_ws && M <= GM_SPLITK_MAX_M && tiles * 2 <= sms) ? static_cast<int>(sms / tiles) : 1;
       for (int sp = 1; sp <= smax && sp <= kblocks; ++sp) {
         const int kps = (kblocks + sp - 1) / sp;
         if ((kblocks + kps - 1) / kps != sp) continue;  // this count would leave an empty split
         const long long waves = (tiles * sp + sms - 1) / sms;
         // a split launch pays for clearing the scratch and for the finishing kernel (about 5 us in a chain of dependent launches)
         const long long cost = waves * kps * per_kb + (sp > 1 ? 5000 : 0);
-        if (best < 0 || cost <= best) { best = cost; tok = cand[i]; splits = sp; }  // ties go to the narrower tile
+        if (best < 0 || cost <= best) { best = cost; tok = cand[i]; splits = sp; clsk = false; }  // ties go to the narrower tile
+      }
+      // Cluster split-K needs no scratch and no further launch.  Measured against the unsplit kernel (M = 32 ... 256 on
+      // the block shapes) a wave of clusters costs 1.5 - 2.5 us more than its k blocks: the cluster launch (growing with
+      // the number of clusters), two cluster barriers and the exchange (growing with the cluster size).
+      if (cand[i] <= 128 && tiles * 2 <= sms && gemm_clsk_mode() != 0 && gemm_a_in_tmem()) {
+        for (int sp = 2; sp <= 8 && sp <= kblocks; ++sp) {
+          const int kps = (kblocks + sp - 1) / sp;
+          if ((kblocks + kps - 1) / kps != sp) continue;
+          const int units = cand[i] / 8;
+          if (static_cast<uint32_t>((sp - 1) * ((units + sp - 1) / sp)) * 4096u > gemm_clsk_recv_bytes(cand[i])) continue;
+          const int clusters = gemm_clsk_max_clusters(cand[i], sp);
+          if (clusters <= 0) continue;
+          long long cost = ((tiles + clusters - 1) / clusters) * (kps * per_kb + 1500 + 150 * sp + 15 * tiles);
+          if (gemm_clsk_mode() == sp) cost = 0;  // forced size (tuning knob); the narrowest tile that allows it wins
+          if (cost <= best) { best = cost; tok = cand[i]; splits = sp; clsk = true; }
+        }
       }
     }
   }
-  if (const int forced = gemm_forced_tok()) { tok = forced; splits = 1; }  // tuning knob, see bitrl.cu
+  if (const int forced = gemm_forced_tok()) { tok = forced; splits = 1; clsk = false; }  // tuning knob, see bitrl.cu
   // CTA pairs (256-row tiles): for launches with many tiles, an even number of 128-row tiles and weights in tensor memory.
   bool pair = false;
   int pair_clusters = 0;
@@ -708,6 +880,22 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
       if (pair_clusters > 0) { pair = true; tok = ptok; }
     }
   }
+  return GemmPlan{tok, splits, clsk, pair, pair_clusters};
+}
+
+// splitk_ws: nullptr, or M*N int32 of scratch that allows the scratch form of split-K when the launch has too few
+// tiles to fill the SMs and the cluster form does not apply.
+bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax, const int32_t* rowsum, int M,
+                         void* y, int out_dtype, const void* residual, int32_t* acc_out, cudaStream_t st,
+                         int32_t* splitk_ws) {
+  encode_tiled_fn encode = get_encode_tiled();
+  if (!encode) return cuda_fail(cudaErrorSymbolNotFound);
+  const GemmPlan plan = gemm_plan(w->N, w->K, M, splitk_ws != nullptr);
+  const int sms = sm_count();
+  const int tiles_n = w->N / GM_ROWS;
+  const int kblocks = w->K / GM_BK;
+  const int tok = plan.tok, splits = plan.splits, pair_clusters = plan.pair_clusters;
+  const bool clsk = plan.clsk, pair = plan.pair;
   CUtensorMap tmap;
   const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(w->K), static_cast<cuuint64_t>(M)};
   const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(w->K)};
@@ -718,6 +906,29 @@ bitrl_status launch_gemm(const Linear* w, const int8_t* xq, const float* absmax,
                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return cuda_fail(cudaErrorInvalidValue);
 
+  if (clsk) {
+    GemmArgs a{w->tiles, w->gamma, absmax, rowsum, M, w->N, w->K, y, out_dtype, static_cast<const unsigned short*>(residual),
+               acc_out, tiles_n, tiles_n * ((M + tok - 1) / tok), splits, (kblocks + splits - 1) / splits, nullptr};
+    void (*ck)(const CUtensorMap, const GemmArgs) = gemm_clsk_kernel(tok);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(a.tiles_total * splits));  // cluster c = tile c, rank = k range
+    cfg.blockDim = dim3(GM_THREADS);
+    cfg.dynamicSmemBytes = GM_SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(splits);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    BITRL_CUDA(cudaFuncSetAttribute(ck, cudaFuncAttributeMaxDynamicSharedMemorySize, GM_SMEM_BYTES));
+    BITRL_CUDA(cudaLaunchKernelEx(&cfg, ck, tmap, a));
+    count_launch(1);
+    return BITRL_OK;
+  }
   const bool split = splits > 1;
   GemmArgs a{w->tiles, w->gamma, absmax, rowsum, M, w->N, w->K, y, out_dtype,
              split ? nullptr : static_cast<const unsigned short*>(residual), split ? nullptr : acc_out, tiles_n, 0,
