@@ -241,13 +241,14 @@ def _out(M, N, out_dtype, device):
 
 
 def bitlinear_forward(w: Linear, x: torch.Tensor, out_dtype: int = OUT_BF16, y: torch.Tensor | None = None,
-                      workspace: torch.Tensor | None = None) -> torch.Tensor:
-    """y = BitLinear(x): x CUDA bf16 [M,K] -> y [M,N]."""
+                      workspace: torch.Tensor | None = None, streaming: bool = False) -> torch.Tensor:
+    """y = BitLinear(x): x CUDA bf16 [M,K] -> y [M,N].  ``streaming`` (M <= GEMV_MAX_M): pass no workspace, so that
+    the streaming kernel serves the call whatever M is."""
     _dev(x, torch.bfloat16, "x")
     M, K = x.shape
     if y is None:
         y = _out(M, w.N, out_dtype, x.device)
-    need = workspace_bytes(M, K, w.N)
+    need = 0 if streaming else workspace_bytes(M, K, w.N)
     if workspace is None and need:
         workspace = torch.empty((need,), dtype=torch.uint8, device=x.device)
     nbytes = 0 if workspace is None else workspace.numel()
@@ -332,15 +333,15 @@ class MultiCall5(MultiCall):
         return self.keep[2]
 
 
-def bitlinear_forward_debug(w: Linear, x: torch.Tensor, out_dtype: int = OUT_BF16):
-    """Returns (y, x_q int8 [M,K], absmax fp32 [M], acc int32 [M,N])."""
+def bitlinear_forward_debug(w: Linear, x: torch.Tensor, out_dtype: int = OUT_BF16, streaming: bool = False):
+    """Returns (y, x_q int8 [M,K], absmax fp32 [M], acc int32 [M,N]).  ``streaming``: as in bitlinear_forward."""
     _dev(x, torch.bfloat16, "x")
     M, K = x.shape
     y = _out(M, w.N, out_dtype, x.device)
     xq = torch.empty((M, K), dtype=torch.int8, device=x.device)
     a = torch.empty((M,), dtype=torch.float32, device=x.device)
     acc = torch.empty((M, w.N), dtype=torch.int32, device=x.device)
-    need = workspace_bytes(M, K, w.N)
+    need = 0 if streaming else workspace_bytes(M, K, w.N)
     ws = torch.empty((max(need, 16),), dtype=torch.uint8, device=x.device)
     _check(lib().bitrl_bitlinear_forward_debug(w.handle, _ptr(x), M, K, w.N, _ptr(y), out_dtype, _ptr(ws), ws.numel(),
                                                _ptr(xq), _ptr(a), _ptr(acc), _stream()),

@@ -61,6 +61,19 @@ int gemm_forced_tok() {
   return v;
 }
 
+// Largest M that a call with pre-quantized activations gives to the streaming kernel; above it the tensor-core GEMM
+// (with its cluster split-K) is faster.  BITRL_GEMV_Q_MAX_M=<1..16> overrides it (tuning runs).
+constexpr int GEMV_Q_MAX_M_DEFAULT = 4;
+int gemv_q_max_m() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("BITRL_GEMV_Q_MAX_M");
+    const int t = e ? atoi(e) : 0;
+    v = (t >= 1 && t <= BITRL_GEMV_MAX_M) ? t : GEMV_Q_MAX_M_DEFAULT;
+  }
+  return v;
+}
+
 int sm_count() {
   static int cached[64] = {0};
   int dev = 0;
@@ -256,9 +269,13 @@ bitrl_status bitrl_quant_act(const void* x, int32_t M, int32_t K, int8_t* xq, fl
   return launch_quant_act(x, M, K, xq, absmax, rowsum, static_cast<cudaStream_t>(stream));
 }
 
+// Whole-layer calls: up to this M the streaming kernel (quantization in its prologue) is the faster form; from there to
+// BITRL_GEMV_MAX_M it still serves callers that pass no workspace, but quantizer + tensor-core GEMM is 2-3 x faster.
+constexpr int FWD_GEMV_PREFERRED_MAX_M = 8;
+
 size_t bitrl_workspace_bytes(int32_t M, int32_t K, int32_t N) {
   if (M < 1 || K < 1 || N < 1) return 0;
-  if (gemv_fits(M, K)) return 0;
+  if (M <= FWD_GEMV_PREFERRED_MAX_M && gemv_fits(M, K)) return 0;
   return carve_fwd(nullptr, M, K, N).bytes;
 }
 
@@ -272,9 +289,9 @@ static bitrl_status forward_impl(const bitrl_linear_t* w, const void* x, int32_t
   bitrl_status s = check_arch();
   if (s != BITRL_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (gemv_fits(M, K))
-    return launch_gemv(&w->l, x, nullptr, nullptr, M, y, out_dtype, nullptr, xq_out, absmax_out, acc_out, st);
   const size_t need = carve_fwd(nullptr, M, K, N).bytes;
+  if (gemv_fits(M, K) && (M <= FWD_GEMV_PREFERRED_MAX_M || !workspace || workspace_bytes < need))
+    return launch_gemv(&w->l, x, nullptr, nullptr, M, y, out_dtype, nullptr, xq_out, absmax_out, acc_out, st);
   if (!workspace || workspace_bytes < need) return BITRL_ERR_WORKSPACE;
   if (!aligned16(workspace)) return BITRL_ERR_ALIGN;
   FwdWs f = carve_fwd(workspace, M, K, N);
@@ -332,7 +349,7 @@ bitrl_status bitrl_bitlinear_forward_q(const bitrl_linear_t* w, const int8_t* xq
   bitrl_status s = check_arch();
   if (s != BITRL_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (gemv_fits(M, w->l.K))
+  if (M <= gemv_q_max_m() && gemv_fits(M, w->l.K))
     return launch_gemv(&w->l, nullptr, xq, absmax, M, y, out_dtype, residual, nullptr, nullptr, acc_out, st);
   return launch_gemm(&w->l, xq, absmax, rowsum, M, y, out_dtype, residual, acc_out, st);
 }
@@ -461,7 +478,7 @@ bitrl_status encoder_run(const bitrl_encoder_t* enc, const void* h_in, int32_t T
     BITRL_CUDA(cudaMemcpyAsync(h_out, h_in, static_cast<size_t>(T) * d * 2, cudaMemcpyDeviceToDevice, st));
   if (max_state_len > 0 && (s = launch_rope_table(w.rope, max_state_len, enc->head_dim, theta, st)) != BITRL_OK) return s;
   auto linear = [&](const bitrl_linear* lin, void* y, const void* residual) -> bitrl_status {
-    if (gemv_fits(T, lin->l.K))
+    if (T <= gemv_q_max_m() && gemv_fits(T, lin->l.K))
       return launch_gemv(&lin->l, nullptr, w.xq, w.absmax, T, y, BITRL_OUT_BF16, residual, nullptr, nullptr, nullptr, st);
     return launch_gemm(&lin->l, w.xq, w.absmax, w.rowsum, T, y, BITRL_OUT_BF16, residual, nullptr, st, w.splitk);
   };

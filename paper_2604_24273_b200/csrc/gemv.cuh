@@ -263,6 +263,8 @@ bitrl_status launch_gemv_t(const GemvArgs& a, cudaStream_t st) {
   return BITRL_OK;
 }
 
+int gemv_q_max_m();
+
 // Shared-memory budget of the streaming kernel: MT*K bytes of codes must fit beside the static arrays.
 inline bool gemv_fits(int M, int K) {
   int mt = 1;

@@ -101,14 +101,14 @@ def test_quant_act_bitexact(oracle_mod, B, M, K, seed):
 
 # ------------------------------------------------------------------------------------- a1..a3, whole layer
 
-def check_layer(oracle_mod, B, M, K, N, wseed, xseed, out_dtype, outliers=True):
+def check_layer(oracle_mod, B, M, K, N, wseed, xseed, out_dtype, outliers=True, streaming=False):
     W, Wq, g, _, gamma_gpu, lin = layer(oracle_mod, B, N, K, wseed)
     assert np.float32(gamma_gpu.cpu().numpy()[0]) == g
     x = inputs.activations(M, K, xseed, outliers=outliers)
     ref = oracle_mod.bitlinear(inputs.bf16_bits(x), Wq, g)
     xg = x.cuda()
-    y, xq, a, acc = B.bitlinear_forward_debug(lin, xg, out_dtype)
-    y2 = B.bitlinear_forward(lin, xg, out_dtype)
+    y, xq, a, acc = B.bitlinear_forward_debug(lin, xg, out_dtype, streaming=streaming)
+    y2 = B.bitlinear_forward(lin, xg, out_dtype, streaming=streaming)
     B.poll_status()
     assert np.array_equal(xq.cpu().numpy(), ref["xq"])
     assert np.array_equal(a.cpu().numpy(), ref["absmax"])
@@ -132,7 +132,10 @@ def test_config1_single_token_fp32(oracle_mod, B):
 @pytest.mark.parametrize("M", [1, 2, 3, 8, 13, 16])
 @pytest.mark.parametrize("K,N,wseed", [(2560, 3840, 1001), (6912, 2560, 1004), (384, 256, 5), (128, 128, 6)])
 def test_gemv_decode_shapes(oracle_mod, B, M, K, N, wseed):
+    """With a workspace (M > 8 then takes quantizer + tensor-core GEMM) and without (the streaming kernel for every M)."""
     check_layer(oracle_mod, B, M, K, N, wseed, 2000 + M, 1)
+    check_layer(oracle_mod, B, M, K, N, wseed, 2000 + M, 1, streaming=True)
+    check_layer(oracle_mod, B, M, K, N, wseed, 2000 + M, 0, streaming=True)
 
 
 @pytest.mark.parametrize("K,N,wseed", [(2560, 2560, 1002), (2560, 13824, 1003)])
@@ -206,8 +209,24 @@ def test_gemm_paired_ctas_forced(B):
     assert "paired-CTA GEMM parity ok" in r.stdout
 
 
+def test_forward_q_streaming_kernel_forced(B):
+    """Pre-quantized calls with 5 <= M <= 16 go to the tensor-core GEMM by default; a child process with
+    BITRL_GEMV_Q_MAX_M=16 (the knob is read once per process) keeps the streaming kernel's form of them checked."""
+    import os
+    import subprocess
+    import sys
+    from pathlib import Path
+
+    root = Path(__file__).resolve().parent.parent
+    env = dict(os.environ, BITRL_GEMV_Q_MAX_M="16", PYTHONPATH=str(root))
+    r = subprocess.run([sys.executable, str(root / "tests" / "gemv_q_child.py")], env=env, cwd=str(root),
+                       capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+    assert "streaming forward_q parity ok" in r.stdout
+
+
 def test_forward_q_with_residual(oracle_mod, B):
-    for M in (4, 130):
+    for M in (4, 6, 16, 130):
         K, N = 256, 384
         W, Wq, g, _, _, lin = layer(oracle_mod, B, N, K, 7)
         x = inputs.activations(M, K, 2500)
