@@ -190,11 +190,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   if (PAIR || CLSK) ptx::cluster_sync_all();
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_enter();  // barriers and tensor memory are set up; inputs of the preceding kernel are read only from here on
+  // Barriers and tensor memory are set up: the next kernel in the stream may start its own set-up.  Only the roles that
+  // touch what the preceding kernel wrote (the x_q producer; the epilogue: scales, row sums, residual, outputs) wait for
+  // it; the packed weights are constant, so their copies, the expansion into tensor memory and everything else that
+  // does not need x_q start while the predecessor is still draining.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == 0) {
     // ------------------------------------------------------------------ X producer
     if (lane == 0) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       uint32_t it = 0;
       bool ok = true;
       for (int item = item0; ok && item < items; item += item_step) {
@@ -385,6 +390,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     }
   } else {
     // ------------------------------------------------------------------ epilogue
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int q = warp & 3;                           // TMEM lane quarter this warp may read
     const int ep = threadIdx.x - GM_EPI_WARP0 * 32;   // 0..127
     const int ew = warp - GM_EPI_WARP0;               // staging buffer index
