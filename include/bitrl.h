@@ -259,9 +259,11 @@ BITRL_API bitrl_status bitrl_ppo_loss(const float* logits, const int32_t* action
  * with round-to-nearest-even.
  * bitrl_w8_quantize: W dev fp32 [N,K] -> wq dev int8 [N,K] (row-major, the format the forward call reads) and
  * scale: dev fp32 [2] - scale[0] receives the scale, scale[1] is scratch of the call.
- * bitrl_w8a8_forward: x dev bf16 [M,K], y dev [M,N] fp32 or bf16.  M <= BITRL_GEMV_MAX_M: one streaming kernel
- * (quantization in its prologue, dp4a, no workspace); larger M: quantization kernel, then a tcgen05 GEMM with both
- * operands straight from TMA tiles.  workspace: dev, >= bitrl_w8a8_workspace_bytes(M, K) (0 for M <= 16, NULL accepted).
+ * bitrl_w8a8_forward: x dev bf16 [M,K], y dev [M,N] fp32 or bf16.  M <= 4: one streaming kernel (quantization in its
+ * prologue, dp4a, no workspace); larger M: quantization kernel, then a tcgen05 GEMM with both operands straight from
+ * TMA tiles.  workspace: dev, >= bitrl_w8a8_workspace_bytes(M, K) (0 for M <= 4, NULL accepted).  For
+ * 5 <= M <= BITRL_GEMV_MAX_M the workspace is optional: without it (NULL or too small) the streaming kernel serves the
+ * call, 1.2-3 x slower.  Same bits either way.
  * The _debug variant also writes xq_out dev int8 [M,K], absmax_out dev fp32 [M], acc_out dev int32 [M,N] (any may be NULL). */
 BITRL_API bitrl_status bitrl_w8_quantize(const float* W, int32_t N, int32_t K, int8_t* wq, float* scale, void* stream);
 BITRL_API size_t bitrl_w8a8_workspace_bytes(int32_t M, int32_t K);
@@ -292,8 +294,9 @@ BITRL_API bitrl_status bitrl_w8a8_forward_multi(int32_t count, const bitrl_w8_ma
  * Same reading with 7 in place of 127:  a = max(max|W|, 1e-20),  W_q = clip(rint(W * (7 / a)), -8, 7),  scale = a / 7,
  * acc and y as for W8A8.  packed: dev uint8 [N, K/2], byte j of row n = (W_q[n,2j] + 8) | (W_q[n,2j+1] + 8) << 4.
  * bitrl_w4_quantize: W dev fp32 [N,K] -> packed and scale (dev fp32 [2]: scale[0] the result, scale[1] scratch).
- * bitrl_w4a8_forward: M <= BITRL_GEMV_MAX_M streams the packed bytes once (dp4a; no workspace); larger M expands the
- * codes to int8 in the workspace and runs the W8A8 GEMM on them.  workspace >= bitrl_w4a8_workspace_bytes(M, K, N). */
+ * bitrl_w4a8_forward: M <= 4 streams the packed bytes once (dp4a; no workspace); larger M expands the codes to int8 in
+ * the workspace and runs the W8A8 GEMM on them.  workspace >= bitrl_w4a8_workspace_bytes(M, K, N) (0 for M <= 4); for
+ * 5 <= M <= BITRL_GEMV_MAX_M it is optional, as for bitrl_w8a8_forward. */
 BITRL_API bitrl_status bitrl_w4_quantize(const float* W, int32_t N, int32_t K, uint8_t* packed, float* scale, void* stream);
 BITRL_API size_t bitrl_w4a8_workspace_bytes(int32_t M, int32_t K, int32_t N);
 BITRL_API bitrl_status bitrl_w4a8_forward(const uint8_t* packed, const float* scale, const void* x, int32_t M, int32_t K,

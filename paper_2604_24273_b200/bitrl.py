@@ -455,8 +455,9 @@ def w8_quantize(W: torch.Tensor):
 
 
 def w8a8_forward(wq: torch.Tensor, scale: torch.Tensor, x: torch.Tensor, out_dtype: int = OUT_BF16, debug: bool = False,
-                 y: torch.Tensor | None = None, workspace: torch.Tensor | None = None):
-    """y = W8A8(x).  With debug=True returns (y, x_q, absmax, acc)."""
+                 y: torch.Tensor | None = None, workspace: torch.Tensor | None = None, streaming: bool = False):
+    """y = W8A8(x).  With debug=True returns (y, x_q, absmax, acc).  ``streaming`` (M <= GEMV_MAX_M): pass a workspace too
+    small for the GEMM form, so that the streaming kernel serves the call whatever M is."""
     _dev(wq, torch.int8, "wq")
     _dev(scale, torch.float32, "scale")
     _dev(x, torch.bfloat16, "x")
@@ -465,7 +466,8 @@ def w8a8_forward(wq: torch.Tensor, scale: torch.Tensor, x: torch.Tensor, out_dty
     if y is None:
         y = _out(M, N, out_dtype, x.device)
     if workspace is None:
-        workspace = torch.empty((max(int(lib().bitrl_w8a8_workspace_bytes(M, K)), 16),), dtype=torch.uint8, device=x.device)
+        need = 0 if streaming else int(lib().bitrl_w8a8_workspace_bytes(M, K))
+        workspace = torch.empty((max(need, 16),), dtype=torch.uint8, device=x.device)
     if not debug:
         _check(lib().bitrl_w8a8_forward(_ptr(wq), _ptr(scale), _ptr(x), M, K, N, _ptr(y), out_dtype, _ptr(workspace),
                                         workspace.numel(), _stream()), "bitrl_w8a8_forward")
@@ -523,8 +525,9 @@ def w4_quantize(W: torch.Tensor):
 
 
 def w4a8_forward(packed: torch.Tensor, scale: torch.Tensor, x: torch.Tensor, out_dtype: int = OUT_BF16,
-                 debug: bool = False, y: torch.Tensor | None = None, workspace: torch.Tensor | None = None):
-    """y = W4A8(x).  With debug=True returns (y, x_q, absmax, acc)."""
+                 debug: bool = False, y: torch.Tensor | None = None, workspace: torch.Tensor | None = None,
+                 streaming: bool = False):
+    """y = W4A8(x).  With debug=True returns (y, x_q, absmax, acc).  ``streaming``: as in w8a8_forward."""
     _dev(packed, torch.uint8, "packed")
     _dev(scale, torch.float32, "scale")
     _dev(x, torch.bfloat16, "x")
@@ -533,7 +536,8 @@ def w4a8_forward(packed: torch.Tensor, scale: torch.Tensor, x: torch.Tensor, out
     if y is None:
         y = _out(M, N, out_dtype, x.device)
     if workspace is None:
-        workspace = torch.empty((max(int(lib().bitrl_w4a8_workspace_bytes(M, K, N)), 16),), dtype=torch.uint8, device=x.device)
+        need = 0 if streaming else int(lib().bitrl_w4a8_workspace_bytes(M, K, N))
+        workspace = torch.empty((max(need, 16),), dtype=torch.uint8, device=x.device)
     if not debug:
         _check(lib().bitrl_w4a8_forward(_ptr(packed), _ptr(scale), _ptr(x), M, K, N, _ptr(y), out_dtype, _ptr(workspace),
                                         workspace.numel(), _stream()), "bitrl_w4a8_forward")

@@ -47,12 +47,19 @@ def weights(oracle_mod, B, N, K, seed):
 
 @pytest.mark.parametrize("M", [1, 2, 3, 8, 13, 16, 17, 64, 300])
 @pytest.mark.parametrize("K,N,seed,out_dtype", [(256, 384, 9500, 1), (640, 128, 9501, 0), (2560, 2560, 9502, 1)])
-def test_w4a8_full(oracle_mod, B, M, K, N, seed, out_dtype):
+@pytest.mark.parametrize("streaming", [False, True])
+def test_w4a8_full(oracle_mod, B, M, K, N, seed, out_dtype, streaming):
+    """streaming: without a workspace, so that the streaming kernel also serves 5 <= M <= 16 (with one, those take the
+    quantizer + expansion + tensor-core GEMM)."""
+    if streaming and not 4 < M <= 16:
+        pytest.skip("same path as without the flag")
     Wq, scale, packed_gpu, scale_gpu = weights(oracle_mod, B, N, K, seed)
     x = inputs.activations(M, K, 9600 + M)
     ref = oracle_mod.bitlinear(inputs.bf16_bits(x), Wq, scale)
-    y, xq, a, acc = B.w4a8_forward(packed_gpu, scale_gpu, x.cuda(), out_dtype, debug=True)
-    y2 = B.w4a8_forward(packed_gpu, scale_gpu, x.cuda(), out_dtype)
+    n0 = B.launch_count()
+    y, xq, a, acc = B.w4a8_forward(packed_gpu, scale_gpu, x.cuda(), out_dtype, debug=True, streaming=streaming)
+    assert (B.launch_count() - n0 == 1) == (M <= 4 or streaming)
+    y2 = B.w4a8_forward(packed_gpu, scale_gpu, x.cuda(), out_dtype, streaming=streaming)
     B.poll_status()
     assert np.array_equal(xq.cpu().numpy(), ref["xq"])
     assert np.array_equal(a.cpu().numpy(), ref["absmax"])

@@ -48,12 +48,19 @@ def weights(oracle_mod, B, N, K, seed):
 
 @pytest.mark.parametrize("M", [1, 2, 3, 8, 13, 16, 17, 64, 300, 513])
 @pytest.mark.parametrize("K,N,seed,out_dtype", [(256, 384, 9200, 1), (640, 128, 9201, 0), (2560, 2560, 9202, 1)])
-def test_w8a8_full(oracle_mod, B, M, K, N, seed, out_dtype):
+@pytest.mark.parametrize("streaming", [False, True])
+def test_w8a8_full(oracle_mod, B, M, K, N, seed, out_dtype, streaming):
+    """streaming: without a workspace, so that the streaming kernel also serves 5 <= M <= 16 (with one, those take the
+    quantizer + tensor-core GEMM)."""
+    if streaming and not 4 < M <= 16:
+        pytest.skip("same path as without the flag")
     Wq, scale, wq_gpu, scale_gpu = weights(oracle_mod, B, N, K, seed)
     x = inputs.activations(M, K, 9300 + M)
     ref = oracle_mod.bitlinear(inputs.bf16_bits(x), Wq, scale)
-    y, xq, a, acc = B.w8a8_forward(wq_gpu, scale_gpu, x.cuda(), out_dtype, debug=True)
-    y2 = B.w8a8_forward(wq_gpu, scale_gpu, x.cuda(), out_dtype)
+    n0 = B.launch_count()
+    y, xq, a, acc = B.w8a8_forward(wq_gpu, scale_gpu, x.cuda(), out_dtype, debug=True, streaming=streaming)
+    assert (B.launch_count() - n0 == 1) == (M <= 4 or streaming)
+    y2 = B.w8a8_forward(wq_gpu, scale_gpu, x.cuda(), out_dtype, streaming=streaming)
     B.poll_status()
     assert np.array_equal(xq.cpu().numpy(), ref["xq"])
     assert np.array_equal(a.cpu().numpy(), ref["absmax"])
@@ -72,7 +79,7 @@ def test_w8a8_full(oracle_mod, B, M, K, N, seed, out_dtype):
 def test_w8a8_paired_cta_shapes_full(oracle_mod, B, M, K, N, seed, out_dtype):
     """M >= 2048 with an even number of 128-row tiles: the paired-CTA kernel (tcgen05 cta_group::2); ragged token counts,
     one and several k blocks, every stage against the oracle."""
-    test_w8a8_full(oracle_mod, B, M, K, N, seed, out_dtype)
+    test_w8a8_full(oracle_mod, B, M, K, N, seed, out_dtype, False)
 
 
 def test_w8a8_m4096_sampled(oracle_mod, B):
