@@ -22,6 +22,7 @@
 
 #include <cuda.h>
 
+#include "clsk.cuh"
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -75,9 +76,6 @@ struct GemmArgs {
   int32_t* part;
 };
 
-// Shared memory that the cluster split-K variant sets aside for received partial sums (4 KB per unit of 8 token columns).
-__host__ __device__ constexpr uint32_t gemm_clsk_recv_bytes(int tok) { return tok <= 64 ? 49152u : 65536u; }
-
 // PAIR: two CTAs of a cluster work on one 256-row x TOK-token tile with tcgen05.mma.cta_group::2.  CTA rank r expands
 // weight rows [256 t + 128 r, +128) into its own tensor memory, fetches tokens [TOK/2 * r, +TOK/2) of the tile into its
 // own shared memory and drains its own 128 x TOK slice of the accumulator; rank 0 issues the MMAs.  Per SM this halves
@@ -100,7 +98,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
   // x_q ring: 128 KB, plus the 48 KB of the shared-memory weight ring when the weights go through tensor memory
   // (4 stages at 256 tokens, 6 at 224, 7 at 192, 11 at 128, 16 at 64).  The cluster split-K variant takes the end of
   // that area for the partial sums it receives from its peers.
-  constexpr uint32_t GM_RECV = CLSK ? gemm_clsk_recv_bytes(GM_TOK) : 0u;
+  constexpr uint32_t GM_RECV = CLSK ? clsk_recv_bytes(GM_TOK) : 0u;
   constexpr uint32_t GM_X_RING = A_TMEM ? GM_OFF_P - GM_OFF_X - GM_RECV : GM_X_RING_BYTES;
   constexpr uint32_t GM_XS = GM_X_RING / GM_X_BYTES < GM_XS_MAX ? GM_X_RING / GM_X_BYTES : GM_XS_MAX;
   static_assert(GM_TOK % 32 == 0 && GM_TOK >= 64 && GM_TOK <= GM_TOK_MAX && GM_XS <= GM_XS_MAX, "token tile");
@@ -400,99 +398,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmArgs a) {
     uint32_t lt = 0;
     bool ok = true;
     if constexpr (CLSK) {
-      // One item per CTA.  These four warps are idle during the main loop, so everything the epilogue reads from global
-      // memory is requested first: the per-token scales and row sums go to shared memory, the residual values of the
-      // first unit of this CTA's columns to registers (the later units' are requested one unit ahead).
+      // One item per CTA: exchange of the partial sums inside the cluster, then the epilogue on this CTA's columns.
       const int tile = static_cast<int>(blockIdx.x) / a.splits;
-      const int tn = tile % a.tiles_n, tm = tile / a.tiles_n;
-      const int S = a.splits;
-      const int tok0 = tm * GM_TOK, tok_hi = min(GM_TOK, a.M - tok0);
-      const int U = (tok_hi + 7) >> 3;  // units of 8 token columns that hold tokens
-      const int own_max = (U + S - 1) / S;
-      const int own_lo = static_cast<int>(rank) * U / S, own_hi = (static_cast<int>(rank) + 1) * U / S;
-      const int row = q * 32 + lane;  // weight row of the tile = tensor-memory lane
-      const int n = tn * GM_ROWS + row;
-      const uint32_t sc_addr = base + GM_OFF_TOK, rs_addr = base + GM_OFF_TOK + 2 * GM_TOK_MAX * 4;
-      for (int j = ep; j < GM_TOK; j += 128) {
-        const int tok = tok0 + j;
-        ptx::sts32(sc_addr + 4 * j, __float_as_uint(tok < a.M ? out_scale(gamma, a.absmax[tok]) : 0.0f));
-        ptx::sts32(rs_addr + 4 * j, static_cast<uint32_t>(tok < a.M ? a.rowsum[tok] : 0));
-      }
-      const bool use_res = a.residual && !f32;
-      auto load_res = [&](int u, unsigned short (&r)[8]) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int col = u * 8 + j;
-          r[j] = (use_res && col < tok_hi) ? a.residual[static_cast<size_t>(tok0 + col) * a.N + n] : static_cast<unsigned short>(0);
-        }
-      };
-      unsigned short rcur[8] = {}, rnxt[8] = {};
-      if (own_lo < own_hi) load_res(own_lo, rcur);
-      // (the named barrier also publishes the scales among the four warps)
-      const bool got = ptx::bar_red_and(1, 128, wait(bar_tmem_full, 0u));
-      if (!got) {
-        if (ep == 0) give_up(GM_WAIT_TMEM_FULL);
-      } else {
-        // Send every peer the partial sums of its token columns: lane = weight row, so the 32 lanes of a warp store 128
-        // consecutive bytes of the peer's receive area [sender slot][unit][column of the unit][row].
-        ptx::tc_fence_after_sync();
-        for (int i = 1; i < S; ++i) {
-          const int p = (static_cast<int>(rank) + i) % S;  // start with the next rank: spreads the traffic
-          const int u_lo = p * U / S, u_hi = (p + 1) * U / S;
-          const int slot = static_cast<int>(rank) < p ? static_cast<int>(rank) : static_cast<int>(rank) - 1;
-          const uint32_t dst = ptx::mapa_u32(recv_base + static_cast<uint32_t>(slot * own_max) * 4096u +
-                                                 static_cast<uint32_t>(row) * 4u, static_cast<uint32_t>(p));
-          for (int u = u_lo; u < u_hi; ++u) {
-            uint32_t v[8];
-            ptx::tmem_ld_32x32b_x8(tmem_base + static_cast<uint32_t>(u * 8) + (static_cast<uint32_t>(q * 32) << 16), v);
-            ptx::tmem_ld_wait();
-#pragma unroll
-            for (int j = 0; j < 8; ++j) ptx::sts32_cluster(dst + static_cast<uint32_t>((u - u_lo) * 8 + j) * 512u, v[j]);
-          }
-        }
-      }
-      // Every partial sum has arrived once all threads of the cluster have passed this barrier (release / acquire at
-      // cluster scope; the other warps take part from the teardown).  Nobody writes to a peer after it.
-      ptx::cluster_sync_all();
-      if (got && !*failed) {
-        // own partial sums + the S - 1 received ones, then the usual epilogue on this CTA's token columns
-        for (int u = own_lo; u < own_hi; ++u) {
-          if (u + 1 < own_hi) load_res(u + 1, rnxt);
-          uint32_t v[8];
-          ptx::tmem_ld_32x32b_x8(tmem_base + static_cast<uint32_t>(u * 8) + (static_cast<uint32_t>(q * 32) << 16), v);
-          ptx::tmem_ld_wait();
-          for (int sl = 0; sl < S - 1; ++sl) {
-            const uint32_t src = recv_base + static_cast<uint32_t>((sl * own_max + (u - own_lo)) * 8) * 512u +
-                                 static_cast<uint32_t>(row) * 4u;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) v[j] += ptx::lds32(src + static_cast<uint32_t>(j) * 512u);
-          }
-          const uint4 rsa = ptx::lds128(rs_addr + u * 32), rsb = ptx::lds128(rs_addr + u * 32 + 16);
-          const uint4 sca = ptx::lds128(sc_addr + u * 32), scb = ptx::lds128(sc_addr + u * 32 + 16);
-          const uint32_t rsv[8] = {rsa.x, rsa.y, rsa.z, rsa.w, rsb.x, rsb.y, rsb.z, rsb.w};
-          const uint32_t scv[8] = {sca.x, sca.y, sca.z, sca.w, scb.x, scb.y, scb.z, scb.w};
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int col = u * 8 + j;
-            if (col < tok_hi) {
-              const size_t off = static_cast<size_t>(tok0 + col) * a.N + n;
-              const int acc = static_cast<int>(v[j] - rsv[j]);
-              if (a.acc_out) a.acc_out[off] = acc;
-              const float yv = __fmul_rn(static_cast<float>(acc), __uint_as_float(scv[j]));
-              if (f32) {
-                static_cast<float*>(a.y)[off] = yv;
-              } else {
-                unsigned short b = float_to_bf16_bits(yv);
-                if (a.residual) b = float_to_bf16_bits(__fadd_rn(bf16_bits_to_float(rcur[j]), bf16_bits_to_float(b)));
-                static_cast<unsigned short*>(a.y)[off] = b;
-              }
-            }
-          }
-#pragma unroll
-          for (int j = 0; j < 8; ++j) rcur[j] = rnxt[j];
-        }
-      }
-      (void)lt; (void)ok; (void)stage; (void)ew;
+      const ClskArgs c{tmem_base, recv_base, base + GM_OFF_TOK, base + GM_OFF_TOK + 2 * GM_TOK_MAX * 4, rank, a.splits,
+                       tile % a.tiles_n, tile / a.tiles_n, a.M, a.N, gamma, a.absmax, a.rowsum, a.y, a.out_dtype,
+                       a.residual, a.acc_out, failed};
+      if (!clsk_exchange_epilogue<GM_TOK>(c, q, lane, ep, [&] { return wait(bar_tmem_full, 0u); }) && ep == 0)
+        give_up(GM_WAIT_TMEM_FULL);
+      (void)lt; (void)ok; (void)stage; (void)ew; (void)f32;
     } else
     for (int item = item0; ok && item < items; item += item_step, ++lt) {
       const int tile = item / a.splits;
@@ -847,8 +760,7 @@ inline GemmPlan gemm_plan(int N, int K, int M, bool have_ws) {
         for (int sp = 2; sp <= 8 && sp <= kblocks; ++sp) {
           const int kps = (kblocks + sp - 1) / sp;
           if ((kblocks + kps - 1) / kps != sp) continue;
-          const int units = cand[i] / 8;
-          if (static_cast<uint32_t>((sp - 1) * ((units + sp - 1) / sp)) * 4096u > gemm_clsk_recv_bytes(cand[i])) continue;
+          if (!clsk_fits(cand[i], sp)) continue;
           const int clusters = gemm_clsk_max_clusters(cand[i], sp);
           if (clusters <= 0) continue;
           long long cost = ((tiles + clusters - 1) / clusters) * (kps * per_kb + 1500 + 150 * sp + 15 * tiles);

@@ -15,6 +15,7 @@
 
 #include <cuda.h>
 
+#include "clsk.cuh"
 #include "common.cuh"
 #include "gemm.cuh"
 #include "gemv.cuh"
@@ -46,6 +47,7 @@ struct Gemm8Args {
   const unsigned short* residual;
   int32_t* acc_out;
   int tiles_n, tiles_total;
+  int splits, kb_per_split;  // cluster split-K (CLSK below): k ranges per tile; 1 and K/128 otherwise
 };
 
 // PAIR: two CTAs of a cluster work on one 256-row x TOK-token tile with tcgen05.mma.cta_group::2, as in the ternary
@@ -53,12 +55,17 @@ struct Gemm8Args {
 // shared memory (completion counted on rank 0's barrier) and drains its own 128 x TOK slice of the accumulator;
 // rank 0 issues the MMAs and releases the stage in both CTAs with one multicast commit.  Per SM the B tile is halved,
 // and shared-memory traffic is what binds this kernel.
-template <int TOK, bool PAIR = false>
+//
+// CLSK (launches with few tiles): the a.splits CTAs of a cluster take the k ranges of ONE tile, one item per CTA, and
+// exchange their int32 partial sums through distributed shared memory (clsk.cuh); the receive area is the end of the ring.
+template <int TOK, bool PAIR = false, bool CLSK = false>
 __global__ void __launch_bounds__(G8_THREADS, 1)
 gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, const Gemm8Args a) {
+  static_assert(!CLSK || (!PAIR && TOK <= 128), "cluster split-K: narrow single-CTA tiles");
   constexpr uint32_t X_BYTES = (PAIR ? TOK / 2 : TOK) * 128;
   constexpr uint32_t STAGE = X_BYTES + G8_W_BYTES;
-  constexpr uint32_t NS = G8_RING_BYTES / STAGE < G8_MAX_STAGES ? G8_RING_BYTES / STAGE : G8_MAX_STAGES;
+  constexpr uint32_t RECV = CLSK ? clsk_recv_bytes(TOK) : 0u;
+  constexpr uint32_t NS = (G8_RING_BYTES - RECV) / STAGE < G8_MAX_STAGES ? (G8_RING_BYTES - RECV) / STAGE : G8_MAX_STAGES;
   static_assert(TOK % 32 == 0 && TOK >= 64 && TOK <= 256, "token tile");
   extern __shared__ unsigned char g8_smem_raw[];
   const uint32_t raw_addr = ptx::smem_u32(g8_smem_raw);
@@ -76,9 +83,12 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kblocks = a.K / 128;
-  const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;
-  const int tile0 = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
-  const int tile_step = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
+  const uint32_t rank = (PAIR || CLSK) ? ptx::cluster_ctarank() : 0u;  // CLSK: = the k range (clusters are consecutive CTAs)
+  const int tile0 = CLSK ? static_cast<int>(blockIdx.x) / a.splits
+                         : PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+  const int tile_step = CLSK ? a.tiles_total : PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
+  const int kb0 = CLSK ? static_cast<int>(rank) * a.kb_per_split : 0;
+  const int kb1 = CLSK ? min(kblocks, kb0 + a.kb_per_split) : kblocks;
   const uint32_t full_lead = PAIR ? ptx::mapa_u32(bar_full, 0) : bar_full;  // rank 0's barriers as seen from either CTA
   const uint32_t tmem_empty_lead = PAIR ? ptx::mapa_u32(bar_tmem_empty, 0) : bar_tmem_empty;
   const uint32_t failed_peer = PAIR ? ptx::mapa_u32(failed_addr, rank ^ 1u) : 0u;
@@ -112,7 +122,8 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
-  if (PAIR) ptx::cluster_sync_all();  // the peer's barriers are initialised before anything is sent to them
+  // the peer's barriers are initialised (PAIR) / every CTA of the cluster has started (CLSK) before anything is sent to it
+  if (PAIR || CLSK) ptx::cluster_sync_all();
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   pdl_enter();
@@ -124,7 +135,7 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       bool ok = true;
       for (int tile = tile0; ok && tile < a.tiles_total; tile += tile_step) {
         const int tn = PAIR ? 2 * (tile % a.tiles_n) + static_cast<int>(rank) : tile % a.tiles_n, tm = tile / a.tiles_n;
-        for (int kb = 0; kb < kblocks; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!wait(bar_empty + 8 * s, ph ^ 1u)) { give_up(G8_WAIT_EMPTY); ok = false; break; }
           if (PAIR) {
             // Rank 0 announces the bytes of both CTAs' stages on its barrier; each CTA's copies report there.
@@ -146,7 +157,7 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     // ------------------------------------------------------------------ MMA issuer
     // The whole warp walks the loop and one elected lane issues: uniform control flow keeps the descriptors in
     // uniform registers, from which the MMA instruction takes its operands.
-    if (rank == 0) {
+    if (!PAIR || rank == 0) {
       const uint32_t idesc = ptx::idesc_i8(PAIR ? 256 : 128, TOK, /*a_signed=*/true, /*b_signed=*/true);
       uint32_t s = 0, ph = 0, lt = 0;
       bool ok = true;
@@ -159,7 +170,7 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         }
         const uint32_t d_tmem = tmem_base + buf * 256;
         ptx::tc_fence_after_sync();
-        for (int kb = 0; kb < kblocks; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!__any_sync(0xffffffffu, wait(bar_full + 8 * s, ph))) {
             if (lane == 0) give_up(G8_WAIT_FULL);
             ok = false;
@@ -171,12 +182,12 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
             if (PAIR) {
 #pragma unroll
               for (int k4 = 0; k4 < 4; ++k4)
-                ptx::mma_i8_ss_pair(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+                ptx::mma_i8_ss_pair(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb != kb0 || k4 != 0) ? 1u : 0u);
               ptx::mma_commit_pair(bar_empty + 8 * s, 3);  // frees the stage in both CTAs
             } else {
 #pragma unroll
               for (int k4 = 0; k4 < 4; ++k4)
-                ptx::mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+                ptx::mma_i8_ss(d_tmem, adesc + 2 * k4, bdesc + 2 * k4, idesc, (kb != kb0 || k4 != 0) ? 1u : 0u);
               ptx::mma_commit(bar_empty + 8 * s);
             }
           }
@@ -200,6 +211,15 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     const bool f32 = a.out_dtype == BITRL_OUT_F32;
     uint32_t lt = 0;
     bool ok = true;
+    if constexpr (CLSK) {
+      // One item per CTA: exchange of the partial sums inside the cluster, then the epilogue on this CTA's columns.
+      const ClskArgs c{tmem_base, base + G8_RING_BYTES - RECV, base + G8_OFF_TOK, base + G8_OFF_TOK + 256 * 4, rank,
+                       a.splits, tile0 % a.tiles_n, tile0 / a.tiles_n, a.M, a.N, wscale, a.absmax, nullptr, a.y,
+                       a.out_dtype, a.residual, a.acc_out, failed};
+      if (!clsk_exchange_epilogue<TOK>(c, q, lane, ep, [&] { return wait(bar_tmem_full, 0u); }) && ep == 0)
+        give_up(G8_WAIT_TMEM_FULL);
+      (void)lt; (void)ok; (void)stage; (void)ew; (void)f32;
+    } else
     for (int tile = tile0; ok && tile < a.tiles_total; tile += tile_step, ++lt) {
       const int tn = PAIR ? 2 * (tile % a.tiles_n) + static_cast<int>(rank) : tile % a.tiles_n, tm = tile / a.tiles_n;
       const uint32_t buf = lt & 1u;
@@ -304,12 +324,16 @@ gemm_w8_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   // ---- teardown: every role leaves through here, also after a timeout ----
   __syncwarp();
   ptx::tc_fence_before_sync();
+  if constexpr (CLSK) {
+    // the cluster barrier of the exchange: the epilogue warps pass it inside their role, the other two warps here
+    if (warp < G8_EPI_WARP0) ptx::cluster_sync_all();
+  }
   __syncthreads();
   if (PAIR) ptx::cluster_sync_all();  // neither CTA leaves (or frees tensor memory) while the other may still reach it
   if (*failed) {
     // Failure path only: copies and MMAs that nobody waited for may still be in flight.  The MMA issuer waits (bounded)
     // for its MMAs, then every thread lets about a millisecond pass before shared and tensor memory are given back.
-    if (warp == 1 && rank == 0) {
+    if (warp == 1 && (!PAIR || rank == 0)) {
       if (ptx::elect_one()) {
         if (PAIR) ptx::mma_commit_pair(bar_drain, 1);
         else ptx::mma_commit(bar_drain);
@@ -365,6 +389,41 @@ inline int gemm_w8_pair_max_clusters(int tok) {
   // one cluster per SM pair: the grid is a static partition of the tiles, CTAs wait only on their own cluster peer, so
   // a grid larger than what is resident at once is merely queued.
   return gemm_pair_mode() == 1 ? sm_count() / 2 : 0;
+}
+
+inline void (*gemm_w8_clsk_kernel(int tok))(const CUtensorMap, const CUtensorMap, const Gemm8Args) {
+  return tok == 128 ? gemm_w8_kernel<128, false, true> : gemm_w8_kernel<64, false, true>;
+}
+
+// Clusters of `S` CTAs of the cluster split-K kernel that can be resident at once (0: this size cannot be launched).
+inline int gemm_w8_clsk_max_clusters(int tok, int S) {
+  static int cached[64][2][9] = {};
+  int dev = 0;
+  if (S < 2 || S > 8 || cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  int& c = cached[dev][tok == 128 ? 1 : 0][S];
+  if (c == 0) {
+    void (*k)(const CUtensorMap, const CUtensorMap, const Gemm8Args) = gemm_w8_clsk_kernel(tok);
+    int n = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(S * 32);
+    cfg.blockDim = dim3(G8_THREADS);
+    cfg.dynamicSmemBytes = G8_SMEM_BYTES;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = S;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, G8_SMEM_BYTES) != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&n, k, &cfg) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      n = -1;
+    }
+    c = n;
+  }
+  if (c > 0) return c;
+  return (S == 2 || S == 4 || S == 8) ? sm_count() / S : 0;  // the query can fail under a profiler (see gemm.cuh)
 }
 
 // ---- M <= 16: streaming kernel ----------------------------------------------------------------------------------
@@ -594,7 +653,8 @@ bitrl_status launch_gemm_w8(const int8_t* wq, const float* scale, int N, int K, 
   if (!encode) return cuda_fail(cudaErrorSymbolNotFound);
   const int sms = sm_count();
   const int tiles_n = N / 128;
-  int tok = 256;
+  int tok = 256, splits = 1;
+  const int kblocks = K / 128;
   {
     long long best = -1;
     const int cand[5] = {256, 224, 192, 128, 64};
@@ -604,11 +664,30 @@ bitrl_status launch_gemm_w8(const int8_t* wq, const float* scale, int N, int K, 
       const long long cost = waves * (2 * cand[i] > 300 ? 2 * cand[i] : 300);  // tensor time per k block, floor for small tiles
       if (best < 0 || cost <= best) { best = cost; tok = cand[i]; }
     }
+    // Few tiles and a long K: k ranges over the CTAs of a cluster, as in the ternary GEMM (same cost model, in ns:
+    // 0.9 ns per unit of the cost above; a wave of clusters pays 2 + 0.15 S + 0.015 tiles us on top of its k blocks:
+    // at M = 64, 2560 -> 6912, two k ranges measured 10.9 us against 9.6 us unsplit, so the fixed part is larger here).
+    if (gemm_clsk_mode() != 0) {
+      long long best_ns = best * kblocks * 9 / 10;
+      for (int i = 3; i < 5; ++i) {
+        const long long tiles = static_cast<long long>(tiles_n) * ((M + cand[i] - 1) / cand[i]);
+        if (tiles * 2 > sms) continue;
+        for (int sp = 2; sp <= 8 && sp <= kblocks; ++sp) {
+          const int kps = (kblocks + sp - 1) / sp;
+          if ((kblocks + kps - 1) / kps != sp || !clsk_fits(cand[i], sp)) continue;
+          const int clusters = gemm_w8_clsk_max_clusters(cand[i], sp);
+          if (clusters <= 0) continue;
+          long long cost = ((tiles + clusters - 1) / clusters) * (kps * 270LL + 2000 + 150 * sp + 15 * tiles);
+          if (gemm_clsk_mode() == sp) cost = 0;  // forced size (tuning knob)
+          if (cost <= best_ns) { best_ns = cost; tok = cand[i]; splits = sp; }
+        }
+      }
+    }
   }
   // Paired CTAs for large launches (same knob as the ternary GEMM): widest tile that fills whole waves of clusters.
   bool pair = false;
   int pair_clusters = 0;
-  if (gemm_pair_mode() != 0 && tiles_n % 2 == 0 && M >= G8_PAIR_MIN_M) {
+  if (gemm_pair_mode() != 0 && tiles_n % 2 == 0 && M >= G8_PAIR_MIN_M && splits == 1) {
     long long best = -1;
     int ptok = 0;
     const int cand[3] = {256, 192, 128};
@@ -646,7 +725,30 @@ bitrl_status launch_gemm_w8(const int8_t* wq, const float* scale, int N, int K, 
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cuda_fail(cudaErrorInvalidValue);
   }
-  Gemm8Args a{scale, absmax, M, N, K, y, out_dtype, static_cast<const unsigned short*>(residual), acc_out, tiles_n, 0};
+  Gemm8Args a{scale, absmax, M, N, K, y, out_dtype, static_cast<const unsigned short*>(residual), acc_out, tiles_n, 0,
+              splits, (kblocks + splits - 1) / splits};
+  if (splits > 1) {
+    a.tiles_total = tiles_n * ((M + tok - 1) / tok);
+    void (*ck)(const CUtensorMap, const CUtensorMap, const Gemm8Args) = gemm_w8_clsk_kernel(tok);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(a.tiles_total * splits));  // cluster c = tile c, rank = k range
+    cfg.blockDim = dim3(G8_THREADS);
+    cfg.dynamicSmemBytes = G8_SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(splits);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    BITRL_CUDA(cudaFuncSetAttribute(ck, cudaFuncAttributeMaxDynamicSharedMemorySize, G8_SMEM_BYTES));
+    BITRL_CUDA(cudaLaunchKernelEx(&cfg, ck, tmx, tmw, a));
+    count_launch(1);
+    return BITRL_OK;
+  }
   if (pair) {
     a.tiles_n = tiles_n / 2;
     a.tiles_total = a.tiles_n * ((M + tok - 1) / tok);

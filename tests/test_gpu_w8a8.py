@@ -82,6 +82,19 @@ def test_w8a8_paired_cta_shapes_full(oracle_mod, B, M, K, N, seed, out_dtype):
     test_w8a8_full(oracle_mod, B, M, K, N, seed, out_dtype, False)
 
 
+@pytest.mark.parametrize("M,K,N,seed,out_dtype", [(17, 6912, 256, 9220, 1), (64, 6912, 2560, 9221, 1), (100, 640, 128, 9222, 0),
+                                                   (200, 2560, 256, 9223, 1), (256, 6912, 2560, 9221, 0)])
+def test_w8a8_cluster_split_shapes_full(oracle_mod, B, M, K, N, seed, out_dtype):
+    """Few tiles and a long K: the k ranges of a tile go to the CTAs of a cluster (partial sums exchanged through
+    distributed shared memory); one launch after the quantizer, every stage against the oracle."""
+    x = inputs.activations(M, K, 9300 + M).cuda()
+    Wq, scale, wq_gpu, scale_gpu = weights(oracle_mod, B, N, K, seed)
+    n0 = B.launch_count()
+    B.w8a8_forward(wq_gpu, scale_gpu, x, out_dtype)
+    assert B.launch_count() - n0 == 2
+    test_w8a8_full(oracle_mod, B, M, K, N, seed, out_dtype, False)
+
+
 def test_w8a8_m4096_sampled(oracle_mod, B):
     """The batched-state shape at full size (M = 4096, 2560 -> 6912): sampled outputs one by one."""
     K, N, M = 2560, 6912, 4096
