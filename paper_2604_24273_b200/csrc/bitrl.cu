@@ -646,10 +646,20 @@ bitrl_status bitrl_w8_quantize(const float* W, int32_t N, int32_t K, int8_t* wq,
 // Critic layers: up to this M the streaming kernels are the faster form; from there to BITRL_GEMV_MAX_M they still serve
 // callers that pass no workspace, but quantizer (+ expansion) + tensor-core GEMM is 1.2-3 x faster (measured at M = 8, 12, 16).
 constexpr int W8_GEMV_PREFERRED_MAX_M = 4;
+// ... and only for rows of up to this many weights: a warp of the streaming kernels walks whole rows, so long rows of a
+// matrix with few rows leave it little memory parallelism (6912 -> 2560 at M = 1: 11.6 us streaming, 8.9 us through the
+// GEMM and its cluster split-K; 2560 -> 6912: 6.1 against 9.0 us).
+constexpr int W8_GEMV_PREFERRED_MAX_K = 4096;
+static bool w8_streaming_preferred(int M, int K) {
+  return M <= W8_GEMV_PREFERRED_MAX_M && K <= W8_GEMV_PREFERRED_MAX_K && gemv_w8_fits(M, K);
+}
+// The INT4 layer's GEMM form has a third launch (the expansion to int8), so its streaming kernel keeps long rows too
+// (6912 -> 2560 at M = 1: 10.5 us streaming, 12.9 us through expansion + GEMM).
+static bool w4_streaming_preferred(int M, int K) { return M <= W8_GEMV_PREFERRED_MAX_M && gemv_w8_fits(M, K); }
 
 size_t bitrl_w8a8_workspace_bytes(int32_t M, int32_t K) {
   if (M < 1 || K < 1) return 0;
-  if (M <= W8_GEMV_PREFERRED_MAX_M && gemv_w8_fits(M, K)) return 0;
+  if (w8_streaming_preferred(M, K)) return 0;
   return align_up(static_cast<size_t>(M) * K, 256) + align_up(static_cast<size_t>(M) * 4, 256);
 }
 
@@ -664,7 +674,7 @@ static bitrl_status w8a8_impl(const int8_t* wq, const float* scale, const void* 
   if (s != BITRL_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (gemv_w8_fits(M, K) &&
-      (M <= W8_GEMV_PREFERRED_MAX_M || !workspace || workspace_bytes < bitrl_w8a8_workspace_bytes(M, K)))
+      (w8_streaming_preferred(M, K) || !workspace || workspace_bytes < bitrl_w8a8_workspace_bytes(M, K)))
     return launch_gemv_w8(wq, scale, N, K, x, M, y, out_dtype, xq_out, absmax_out, acc_out, st);
   if (!workspace || workspace_bytes < bitrl_w8a8_workspace_bytes(M, K)) return BITRL_ERR_WORKSPACE;
   int8_t* xq = static_cast<int8_t*>(workspace);
@@ -717,7 +727,7 @@ bitrl_status bitrl_w4_quantize(const float* W, int32_t N, int32_t K, uint8_t* pa
 
 size_t bitrl_w4a8_workspace_bytes(int32_t M, int32_t K, int32_t N) {
   if (M < 1 || K < 1 || N < 1) return 0;
-  if (M <= W8_GEMV_PREFERRED_MAX_M && gemv_w8_fits(M, K)) return 0;
+  if (w4_streaming_preferred(M, K)) return 0;
   return bitrl_w8a8_workspace_bytes(M, K) + align_up(static_cast<size_t>(N) * K, 256);
 }
 
@@ -732,7 +742,7 @@ static bitrl_status w4a8_impl(const uint8_t* packed, const float* scale, const v
   if (s != BITRL_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (gemv_w8_fits(M, K) &&
-      (M <= W8_GEMV_PREFERRED_MAX_M || !workspace || workspace_bytes < bitrl_w4a8_workspace_bytes(M, K, N)))
+      (w4_streaming_preferred(M, K) || !workspace || workspace_bytes < bitrl_w4a8_workspace_bytes(M, K, N)))
     return launch_gemv_w4(packed, scale, N, K, x, M, y, out_dtype, xq_out, absmax_out, acc_out, st);
   if (!workspace || workspace_bytes < bitrl_w4a8_workspace_bytes(M, K, N)) return BITRL_ERR_WORKSPACE;
   unsigned char* b = static_cast<unsigned char*>(workspace);

@@ -450,7 +450,7 @@ __device__ __forceinline__ int dp4a_s8s8(uint32_t a, uint32_t b, int acc) {
   return d;
 }
 
-template <int MT>
+template <int MT, int R>
 __global__ void __launch_bounds__(GV8_THREADS) gemv_w8_kernel(Gemv8Args a) {
   extern __shared__ __align__(16) unsigned char gv8_smem[];
   int8_t* xq_s = reinterpret_cast<int8_t*>(gv8_smem);               // [MT][K]
@@ -459,8 +459,8 @@ __global__ void __launch_bounds__(GV8_THREADS) gemv_w8_kernel(Gemv8Args a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int K = a.K, nvec8 = K >> 3, nvec16 = K >> 4;
   // A warp streams R rows at a time (N is a multiple of 128): R times as many loads in flight per lane, and every
-  // 16-byte piece of the activations read from shared memory serves R rows.
-  constexpr int R = MT <= 4 ? 4 : 2;
+  // 16-byte piece of the activations read from shared memory serves R rows.  The launcher takes fewer rows per warp
+  // when the matrix has too few rows to give every SM a CTA otherwise.
   constexpr int PRE = 2;  // 16-byte steps of the first row group requested before anything else
   const int n_first = (blockIdx.x * (GV8_THREADS / 32) + warp) * R;
   // The weights depend neither on the activations nor on the preceding kernel: the first loads of this warp's first
@@ -583,16 +583,33 @@ __global__ void __launch_bounds__(GV8_THREADS) gemv_w8_kernel(Gemv8Args a) {
   }
 }
 
-template <int MT>
-bitrl_status launch_gemv_w8_t(const Gemv8Args& a, cudaStream_t st) {
+template <int MT, int R>
+bitrl_status launch_gemv_w8_tr(const Gemv8Args& a, cudaStream_t st) {
   const size_t smem = static_cast<size_t>(MT) * a.K + MT * sizeof(float) + 16;
-  BITRL_CUDA(cudaFuncSetAttribute(gemv_w8_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  BITRL_CUDA(cudaFuncSetAttribute(gemv_w8_kernel<MT, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   int grid = sm_count() * (smem <= 100 * 1024 ? 2 : 1);
-  const int row_groups = (a.N + GV8_THREADS / 8 - 1) / (GV8_THREADS / 8);  // at most four rows per warp and step
+  const int rows_per_cta = (GV8_THREADS / 32) * R;
+  const int row_groups = (a.N + rows_per_cta - 1) / rows_per_cta;
   if (grid > row_groups) grid = row_groups;
-  BITRL_CUDA(launch_pdl(gemv_w8_kernel<MT>, dim3(grid), dim3(GV8_THREADS), smem, st, a));
+  BITRL_CUDA(launch_pdl(gemv_w8_kernel<MT, R>, dim3(grid), dim3(GV8_THREADS), smem, st, a));
   count_launch(1);
   return BITRL_OK;
+}
+
+template <int MT>
+bitrl_status launch_gemv_w8_t(const Gemv8Args& a, cudaStream_t st) {
+  // Four rows per warp (two for the wide token counts).  For one or two tokens fewer rows per warp when four would leave
+  // SMs without a CTA (N = 2560: 80 CTAs of 32 rows; 6912 -> 2560 at M = 1: 14.6 -> 11.6 us); from four tokens on the
+  // activation reads from shared memory that fewer rows share cost more than the idle SMs (M = 4: 14.9 -> 15.6 us).
+  constexpr int RMAX = MT <= 4 ? 4 : 2;
+  if constexpr (MT <= 2) {
+    const int ctas_wanted = sm_count();
+    if (a.N / ((GV8_THREADS / 32) * 4) >= ctas_wanted) return launch_gemv_w8_tr<MT, 4>(a, st);
+    if (a.N / ((GV8_THREADS / 32) * 2) >= ctas_wanted) return launch_gemv_w8_tr<MT, 2>(a, st);
+    return launch_gemv_w8_tr<MT, 1>(a, st);
+  } else {
+    return launch_gemv_w8_tr<MT, RMAX>(a, st);
+  }
 }
 
 inline bool gemv_w8_fits(int M, int K) { return M <= BITRL_GEMV_MAX_M && static_cast<size_t>(16) * K <= 200 * 1024; }

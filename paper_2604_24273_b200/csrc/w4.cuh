@@ -26,7 +26,7 @@ struct Gemv4Args {
 
 // The activations are quantized once per CTA into shared memory with the even and the odd k of every group of eight
 // in separate words, which is the order the two nibble planes of a weight word come out in.
-template <int MT>
+template <int MT, int R>
 __global__ void __launch_bounds__(GV8_THREADS) gemv_w4_kernel(Gemv4Args a) {
   extern __shared__ __align__(16) unsigned char gv4_smem[];
   int8_t* xq_s = reinterpret_cast<int8_t*>(gv4_smem);           // [MT][K], de-interleaved per 8 k
@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(GV8_THREADS) gemv_w4_kernel(Gemv4Args a) {
 
   const float wscale = *a.scale;
   const int nvec16 = K >> 5;  // 16-byte pieces of a packed row (32 weights each)
-  constexpr int R = MT <= 4 ? 4 : 2;
+  // R rows per warp at a time; the launcher takes fewer when the matrix has too few rows to give every SM a CTA.
   for (int n0 = (blockIdx.x * (GV8_THREADS / 32) + warp) * R; n0 < a.N; n0 += gridDim.x * (GV8_THREADS / 32) * R) {
     const uint4* wr = reinterpret_cast<const uint4*>(a.packed + static_cast<size_t>(n0) * (K >> 1));
     int acc[R][MT];
@@ -129,16 +129,31 @@ __global__ void __launch_bounds__(GV8_THREADS) gemv_w4_kernel(Gemv4Args a) {
   }
 }
 
-template <int MT>
-bitrl_status launch_gemv_w4_t(const Gemv4Args& a, cudaStream_t st) {
+template <int MT, int R>
+bitrl_status launch_gemv_w4_tr(const Gemv4Args& a, cudaStream_t st) {
   const size_t smem = static_cast<size_t>(MT) * a.K + 2 * MT * sizeof(float) + 16;
-  BITRL_CUDA(cudaFuncSetAttribute(gemv_w4_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  BITRL_CUDA(cudaFuncSetAttribute(gemv_w4_kernel<MT, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   int grid = sm_count() * (smem <= 100 * 1024 ? 2 : 1);
-  const int row_groups = (a.N + GV8_THREADS / 8 - 1) / (GV8_THREADS / 8);
+  const int rows_per_cta = (GV8_THREADS / 32) * R;
+  const int row_groups = (a.N + rows_per_cta - 1) / rows_per_cta;
   if (grid > row_groups) grid = row_groups;
-  BITRL_CUDA(launch_pdl(gemv_w4_kernel<MT>, dim3(grid), dim3(GV8_THREADS), smem, st, a));
+  BITRL_CUDA(launch_pdl(gemv_w4_kernel<MT, R>, dim3(grid), dim3(GV8_THREADS), smem, st, a));
   count_launch(1);
   return BITRL_OK;
+}
+
+template <int MT>
+bitrl_status launch_gemv_w4_t(const Gemv4Args& a, cudaStream_t st) {
+  // as for the int8 streaming kernel: at one token, fewer rows per warp when four would leave SMs without a CTA
+  constexpr int RMAX = MT <= 4 ? 4 : 2;
+  if constexpr (MT == 1) {
+    const int ctas_wanted = sm_count();
+    if (a.N / ((GV8_THREADS / 32) * 4) >= ctas_wanted) return launch_gemv_w4_tr<MT, 4>(a, st);
+    if (a.N / ((GV8_THREADS / 32) * 2) >= ctas_wanted) return launch_gemv_w4_tr<MT, 2>(a, st);
+    return launch_gemv_w4_tr<MT, 1>(a, st);
+  } else {
+    return launch_gemv_w4_tr<MT, RMAX>(a, st);
+  }
 }
 
 bitrl_status launch_gemv_w4(const uint8_t* packed, const float* scale, int N, int K, const void* x, int M, void* y,

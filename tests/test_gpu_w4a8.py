@@ -73,6 +73,22 @@ def test_w4a8_full(oracle_mod, B, M, K, N, seed, out_dtype, streaming):
         assert np.array_equal(yb, ref["ybf16"]) and torch.equal(y, y2)
 
 
+@pytest.mark.parametrize("M", [1, 2, 4])
+def test_w4a8_long_rows_both_forms(oracle_mod, B, M):
+    """K = 6912 with few rows: the streaming kernel with one (M = 1) or four rows per warp, with and without a workspace."""
+    K, N = 6912, 256
+    Wq, scale, packed_gpu, scale_gpu = weights(oracle_mod, B, N, K, 9520)
+    x = inputs.activations(M, K, 9650 + M)
+    ref = oracle_mod.bitlinear(inputs.bf16_bits(x), Wq, scale)
+    for streaming in (False, True):
+        n0 = B.launch_count()
+        y, xq, a, acc = B.w4a8_forward(packed_gpu, scale_gpu, x.cuda(), B.OUT_BF16, debug=True, streaming=streaming)
+        assert B.launch_count() - n0 == 1
+        B.poll_status()
+        assert np.array_equal(xq.cpu().numpy(), ref["xq"]) and np.array_equal(acc.cpu().numpy(), ref["acc"])
+        assert np.array_equal(inputs.bf16_bits(y.cpu()), ref["ybf16"])
+
+
 @pytest.mark.parametrize("M,out_dtype", [(1, 1), (2, 0), (2, 1)])
 def test_w4a8_forward_multi_matches_oracle_and_single_calls(oracle_mod, B, M, out_dtype):
     """Several independent W4A8 layers in one launch: bit-identical to the oracle and to separate calls."""

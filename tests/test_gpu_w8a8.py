@@ -95,6 +95,23 @@ def test_w8a8_cluster_split_shapes_full(oracle_mod, B, M, K, N, seed, out_dtype)
     test_w8a8_full(oracle_mod, B, M, K, N, seed, out_dtype, False)
 
 
+@pytest.mark.parametrize("M", [1, 2, 4])
+def test_w8a8_long_rows_both_forms(oracle_mod, B, M):
+    """K = 6912 > 4096: with a workspace even M <= 4 takes quantizer + GEMM (cluster split-K); without one the streaming
+    kernel (one, two or four rows per warp).  Same bits, both equal to the oracle."""
+    K, N = 6912, 2560
+    Wq, scale, wq_gpu, scale_gpu = weights(oracle_mod, B, N, K, 9221)
+    x = inputs.activations(M, K, 9350 + M)
+    ref = oracle_mod.bitlinear(inputs.bf16_bits(x), Wq, scale)
+    for streaming in (False, True):
+        n0 = B.launch_count()
+        y, xq, a, acc = B.w8a8_forward(wq_gpu, scale_gpu, x.cuda(), B.OUT_BF16, debug=True, streaming=streaming)
+        assert B.launch_count() - n0 == (1 if streaming else 2)
+        B.poll_status()
+        assert np.array_equal(xq.cpu().numpy(), ref["xq"]) and np.array_equal(acc.cpu().numpy(), ref["acc"])
+        assert np.array_equal(inputs.bf16_bits(y.cpu()), ref["ybf16"])
+
+
 def test_w8a8_m4096_sampled(oracle_mod, B):
     """The batched-state shape at full size (M = 4096, 2560 -> 6912): sampled outputs one by one."""
     K, N, M = 2560, 6912, 4096
