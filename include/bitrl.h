@@ -259,11 +259,12 @@ BITRL_API bitrl_status bitrl_ppo_loss(const float* logits, const int32_t* action
  * with round-to-nearest-even.
  * bitrl_w8_quantize: W dev fp32 [N,K] -> wq dev int8 [N,K] (row-major, the format the forward call reads) and
  * scale: dev fp32 [2] - scale[0] receives the scale, scale[1] is scratch of the call.
- * bitrl_w8a8_forward: x dev bf16 [M,K], y dev [M,N] fp32 or bf16.  M <= 4: one streaming kernel (quantization in its
- * prologue, dp4a, no workspace); larger M: quantization kernel, then a tcgen05 GEMM with both operands straight from
- * TMA tiles.  workspace: dev, >= bitrl_w8a8_workspace_bytes(M, K) (0 for M <= 4, NULL accepted).  For
- * 5 <= M <= BITRL_GEMV_MAX_M the workspace is optional: without it (NULL or too small) the streaming kernel serves the
- * call, 1.2-3 x slower.  Same bits either way.
+ * bitrl_w8a8_forward: x dev bf16 [M,K], y dev [M,N] fp32 or bf16.  M <= 4 and K <= 4096: one streaming kernel
+ * (quantization in its prologue, dp4a, no workspace); otherwise: quantization kernel, then a tcgen05 GEMM with both
+ * operands straight from TMA tiles (split over the CTAs of a cluster along K when the tiles are few).
+ * workspace: dev, >= bitrl_w8a8_workspace_bytes(M, K) (0 where the streaming kernel is preferred, NULL accepted).  For
+ * every M <= BITRL_GEMV_MAX_M the workspace is optional: without it (NULL or too small) the streaming kernel serves the
+ * call, 1.2-3 x slower where it is not the preferred form.  Same bits either way.
  * The _debug variant also writes xq_out dev int8 [M,K], absmax_out dev fp32 [M], acc_out dev int32 [M,N] (any may be NULL). */
 BITRL_API bitrl_status bitrl_w8_quantize(const float* W, int32_t N, int32_t K, int8_t* wq, float* scale, void* stream);
 BITRL_API size_t bitrl_w8a8_workspace_bytes(int32_t M, int32_t K);
