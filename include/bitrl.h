@@ -101,10 +101,10 @@ BITRL_API bitrl_status bitrl_quant_act(const void* x, int32_t M, int32_t K, int8
 
 /* ---- a1..a3: the whole layer  y = BitLinear(x) --------------------------------------------------------
  * x: dev bf16 [M,K]; y: dev [M,N] fp32 (BITRL_OUT_F32) or bf16 (BITRL_OUT_BF16).  K, N must equal the
- * handle's.  M <= 8: one streaming kernel (quantization in its prologue, rescale in its epilogue; no workspace
- * needed).  Larger M: quantization kernel into the workspace, then the tcgen05 GEMM.  For 9 <= M <= BITRL_GEMV_MAX_M
- * the workspace is optional: without it (NULL, or too small) the streaming kernel serves the call, 2-3 x slower.
- * workspace: dev, >= bitrl_workspace_bytes(M,K,N) (0 for M <= 8, then NULL is accepted).  The results are the same
+ * handle's.  M <= 4: one streaming kernel (quantization in its prologue, rescale in its epilogue; no workspace
+ * needed).  Larger M: quantization kernel into the workspace, then the tcgen05 GEMM.  For 5 <= M <= BITRL_GEMV_MAX_M
+ * the workspace is optional: without it (NULL, or too small) the streaming kernel serves the call, 1.4-3 x slower.
+ * workspace: dev, >= bitrl_workspace_bytes(M,K,N) (0 for M <= 4, then NULL is accepted).  The results are the same
  * bits whichever kernel runs.
  * When a launch has too few output tiles to occupy the SMs, K is split across them.  Narrow token tiles (<= 128
  * tokens) do that inside one launch: the CTAs of a thread-block cluster take the k ranges of one tile and exchange

@@ -270,8 +270,9 @@ bitrl_status bitrl_quant_act(const void* x, int32_t M, int32_t K, int8_t* xq, fl
 }
 
 // Whole-layer calls: up to this M the streaming kernel (quantization in its prologue) is the faster form; from there to
-// BITRL_GEMV_MAX_M it still serves callers that pass no workspace, but quantizer + tensor-core GEMM is 2-3 x faster.
-constexpr int FWD_GEMV_PREFERRED_MAX_M = 8;
+// BITRL_GEMV_MAX_M it still serves callers that pass no workspace, but quantizer + tensor-core GEMM is faster (a block's
+// four layers at M = 8: 31 against 44 us; at M = 16: 2-3 x).
+constexpr int FWD_GEMV_PREFERRED_MAX_M = 4;
 
 size_t bitrl_workspace_bytes(int32_t M, int32_t K, int32_t N) {
   if (M < 1 || K < 1 || N < 1) return 0;

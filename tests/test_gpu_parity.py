@@ -132,7 +132,7 @@ def test_config1_single_token_fp32(oracle_mod, B):
 @pytest.mark.parametrize("M", [1, 2, 3, 8, 13, 16])
 @pytest.mark.parametrize("K,N,wseed", [(2560, 3840, 1001), (6912, 2560, 1004), (384, 256, 5), (128, 128, 6)])
 def test_gemv_decode_shapes(oracle_mod, B, M, K, N, wseed):
-    """With a workspace (M > 8 then takes quantizer + tensor-core GEMM) and without (the streaming kernel for every M)."""
+    """With a workspace (M > 4 then takes quantizer + tensor-core GEMM) and without (the streaming kernel for every M)."""
     check_layer(oracle_mod, B, M, K, N, wseed, 2000 + M, 1)
     check_layer(oracle_mod, B, M, K, N, wseed, 2000 + M, 1, streaming=True)
     check_layer(oracle_mod, B, M, K, N, wseed, 2000 + M, 0, streaming=True)
