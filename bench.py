@@ -440,7 +440,7 @@ def run_ours(args):
                        "us_per_launch": msc * 1e3 / (args.steps * lc)}
         del gc
         _, _, step8, chain8 = decode_setup(8)
-        for label, fn in (("sweep_m8_grouped", step8), ("chain_m8_one_launch_per_matrix", chain8)):
+        for label, fn in (("sweep_m8_grouped", step8), ("chain_m8_one_call_per_matrix", chain8)):
             g8, l8 = capture(fn)
             ms8 = time_graph(g8, args.steps, args.warmup, 1)
             gb8 = bytes_step * args.steps / (ms8 * 1e-3) / 1e9
