@@ -5,10 +5,12 @@ import numpy as np
 from paper_2604_24273_b200 import inputs
 
 # (M, K, N, out_dtype): one and several token tiles, ragged tails, fewer 8-token units than k ranges (M = 17),
-# k-block counts that leave uneven ranges (K = 640, 6912), both output types
+# k-block counts that leave uneven ranges (K = 640, 6912), many token tiles of one weight tile (M = 1000, 2000),
+# both output types
 CASES = [(17, 6912, 256, 1), (33, 2560, 128, 0), (40, 1024, 128, 1), (64, 1024, 256, 1), (64, 6912, 2560, 1),
          (64, 2560, 6912, 1), (100, 640, 128, 0), (128, 6912, 384, 1), (200, 2560, 256, 1), (256, 6912, 2560, 1),
-         (257, 3840, 128, 0), (300, 6912, 128, 1), (32, 6912, 2560, 1), (32, 2560, 3840, 1)]
+         (257, 3840, 128, 0), (300, 6912, 128, 1), (32, 6912, 2560, 1), (32, 2560, 3840, 1), (2000, 2560, 128, 1),
+         (1000, 640, 256, 0)]
 
 
 def check_case(O, B, M, K, N, out_dtype, wseed=8100):
