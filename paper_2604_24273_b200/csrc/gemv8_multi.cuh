@@ -9,7 +9,8 @@
 // (conflict-free in shared memory) and feed dp4a; one shuffle tree per row.  int8 weights are used as they are
 // (signed x signed); int4 weights are two biased codes (q + 8) per byte, split into their nibble planes by two masks
 // (the high plane stays at its bit position and is scaled back by an exact shift once per row) and multiplied as
-// unsigned bytes with activations stored even-k / odd-k de-interleaved, the bias repaid as 8 * sum_k x_q.  The work
+// unsigned bytes with activations stored as an even-k and an odd-k plane, the bias repaid as 8 * sum_k x_q; at one token
+// a warp takes two of the (half as long) int4 rows at a time, one per half-warp.  The work
 // list is every job's rows in slot units, split into contiguous byte-balanced ranges, two per CTA.
 #pragma once
 
@@ -139,11 +140,18 @@ __global__ void __launch_bounds__(GV8M_THREADS, 1) gemv8_multi_kernel(const __gr
             uint2 wd;
             wd.x = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | (static_cast<uint32_t>(q[3]) << 24);
             wd.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | (static_cast<uint32_t>(q[7]) << 24);
-            if (W4) {  // even k | odd k of every eight: the order the two nibble planes of a weight word come out in
+            if (W4) {
+              // The even k and the odd k of every eight, the order the two nibble planes of a weight word come out in, go
+              // to two planes of K/2 bytes each: a lane then reads 16 contiguous bytes of either plane per step and the
+              // lanes of a warp read consecutive 16-byte pieces (one plane with both halves side by side made every
+              // activation load a two-way bank conflict).
               rs += q[0] + q[1] + q[2] + q[3] + q[4] + q[5] + q[6] + q[7];
-              wd = make_uint2(__byte_perm(wd.x, wd.y, 0x6420), __byte_perm(wd.x, wd.y, 0x7531));
+              uint32_t* plane = reinterpret_cast<uint32_t*>(xq_s + m * K);
+              plane[i] = __byte_perm(wd.x, wd.y, 0x6420);
+              plane[(K >> 3) + i] = __byte_perm(wd.x, wd.y, 0x7531);
+            } else {
+              dst[i] = wd;
             }
-            dst[i] = wd;
           }
           if (W4) {
             rs = warp_sum_i(rs);
@@ -172,6 +180,40 @@ __global__ void __launch_bounds__(GV8M_THREADS, 1) gemv8_multi_kernel(const __gr
       if (ok && !ptx::mbar_wait(bar_full + 8 * s, ph)) { report_timeout(GV8M_WAIT_FULL); ok = false; }
       if (ok) {
         const int nvec16 = job.row_bytes >> 4;  // 16-byte pieces of a row: 16 int8 or 32 int4 weights each
+        if constexpr (W4 && MT == 1) {
+          // int4 rows are half as long, so the reduction and the epilogue of a row weigh twice as much: a warp takes
+          // two rows at a time, one per half-warp (16 lanes walk a row; one four-step shuffle tree serves both rows).
+          const int hl = lane & 15, hr = lane >> 4;
+          for (int r2 = ((warp - (row0 >> 1)) & (GV8M_CONSUMERS - 1)) * 2; r2 < rows; r2 += 2 * GV8M_CONSUMERS) {
+            const int r = r2 + hr;
+            const bool live = r < rows;
+            const uint32_t wrow = ring + s * GV8M_SLOT_BYTES + static_cast<uint32_t>(live ? r : r2) * job.row_bytes;
+            int acc = 0, acc_hi = 0;
+#pragma unroll 5
+            for (int i = hl; i < nvec16; i += 16) {
+              const uint4 wv = ptx::lds128(wrow + 16 * i);
+              const uint4 xa = *reinterpret_cast<const uint4*>(xq_s + 16 * i);
+              const uint4 xb = *reinterpret_cast<const uint4*>(xq_s + (K >> 1) + 16 * i);
+              const uint32_t xe[4] = {xa.x, xa.y, xa.z, xa.w}, xo[4] = {xb.x, xb.y, xb.z, xb.w};
+              const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+              for (int p = 0; p < 4; ++p) {
+                acc = dp4a_u8s8(ww[p] & 0x0f0f0f0fu, static_cast<int>(xe[p]), acc);
+                acc_hi = dp4a_u8s8(ww[p] & 0xf0f0f0f0u, static_cast<int>(xo[p]), acc_hi);
+              }
+            }
+            acc += acc_hi >> 4;  // exact: a multiple of 16
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            if (hl == 0 && live) {
+              acc -= 8 * rs_s[0];
+              const float yv = __fmul_rn(static_cast<float>(acc), __fmul_rn(wscale, sc_s[0]));
+              const size_t o = static_cast<size_t>(row0 + r);
+              if (a.out_dtype == BITRL_OUT_F32) static_cast<float*>(job.y)[o] = yv;
+              else static_cast<unsigned short*>(job.y)[o] = float_to_bf16_bits(yv);
+            }
+          }
+        } else
         for (int r = (warp - row0) & (GV8M_CONSUMERS - 1); r < rows; r += GV8M_CONSUMERS) {
           const uint32_t wrow = ring + s * GV8M_SLOT_BYTES + static_cast<uint32_t>(r) * job.row_bytes;
           int acc[MT], acc_hi[MT];  // acc_hi: the high-nibble plane left at its bit position, i.e. 16 times its share
@@ -183,10 +225,11 @@ __global__ void __launch_bounds__(GV8M_THREADS, 1) gemv8_multi_kernel(const __gr
 #pragma unroll
             for (int m = 0; m < MT; ++m) {
               if (W4) {
-                // word p of the piece holds k = 32 i + 8 p .. + 7; its activations are the words 2p (even k), 2p + 1 (odd k)
-                const uint4 xa = *reinterpret_cast<const uint4*>(xq_s + m * K + 32 * i);
-                const uint4 xb = *reinterpret_cast<const uint4*>(xq_s + m * K + 32 * i + 16);
-                const uint32_t xe[4] = {xa.x, xa.z, xb.x, xb.z}, xo[4] = {xa.y, xa.w, xb.y, xb.w};
+                // word p of the piece holds k = 32 i + 8 p .. + 7; its activations are word 4 i + p of the even-k plane
+                // and of the odd-k plane
+                const uint4 xa = *reinterpret_cast<const uint4*>(xq_s + m * K + 16 * i);
+                const uint4 xb = *reinterpret_cast<const uint4*>(xq_s + m * K + (K >> 1) + 16 * i);
+                const uint32_t xe[4] = {xa.x, xa.y, xa.z, xa.w}, xo[4] = {xb.x, xb.y, xb.z, xb.w};
                 const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
 #pragma unroll
                 for (int p = 0; p < 4; ++p) {

@@ -29,7 +29,7 @@ struct Gemv4Args {
 template <int MT, int R>
 __global__ void __launch_bounds__(GV8_THREADS) gemv_w4_kernel(Gemv4Args a) {
   extern __shared__ __align__(16) unsigned char gv4_smem[];
-  int8_t* xq_s = reinterpret_cast<int8_t*>(gv4_smem);           // [MT][K], de-interleaved per 8 k
+  int8_t* xq_s = reinterpret_cast<int8_t*>(gv4_smem);           // [MT][K]: per token an even-k plane and an odd-k plane of K/2 bytes
   float* sc_s = reinterpret_cast<float*>(gv4_smem + MT * a.K);  // [MT] a_m / 127
   int* rs_s = reinterpret_cast<int*>(sc_s + MT);                // [MT] sum_k x_q
   pdl_enter();
@@ -64,7 +64,11 @@ __global__ void __launch_bounds__(GV8_THREADS) gemv_w4_kernel(Gemv4Args a) {
       wd.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | (static_cast<uint32_t>(q[7]) << 24);
       rs += q[0] + q[1] + q[2] + q[3] + q[4] + q[5] + q[6] + q[7];
       if (tap) tap[i] = wd;
-      dst[i] = make_uint2(__byte_perm(wd.x, wd.y, 0x6420), __byte_perm(wd.x, wd.y, 0x7531));  // even k | odd k
+      // even k and odd k of every eight into two planes of K/2 bytes: the lanes of a warp then read consecutive 16-byte
+      // pieces of either plane (side by side in one plane, every activation load was a two-way bank conflict)
+      uint32_t* plane = reinterpret_cast<uint32_t*>(xq_s + m * K);
+      plane[i] = __byte_perm(wd.x, wd.y, 0x6420);
+      plane[(K >> 3) + i] = __byte_perm(wd.x, wd.y, 0x7531);
     }
     rs = warp_sum_i(rs);
     if (lane == 0) {
@@ -92,10 +96,10 @@ __global__ void __launch_bounds__(GV8_THREADS) gemv_w4_kernel(Gemv4Args a) {
       for (int r = 0; r < R; ++r) wv[r] = wr[static_cast<size_t>(r) * nvec16 + i];
 #pragma unroll
       for (int m = 0; m < MT; ++m) {
-        // word p of the piece holds k = 32 i + 8 p .. + 7; its activations are the words 2p (even k) and 2p + 1 (odd k)
-        const uint4 xa = *reinterpret_cast<const uint4*>(xq_s + m * K + 32 * i);
-        const uint4 xb = *reinterpret_cast<const uint4*>(xq_s + m * K + 32 * i + 16);
-        const uint32_t xe[4] = {xa.x, xa.z, xb.x, xb.z}, xo[4] = {xa.y, xa.w, xb.y, xb.w};
+        // word p of the piece holds k = 32 i + 8 p .. + 7; its activations are word 4 i + p of the even-k and odd-k planes
+        const uint4 xa = *reinterpret_cast<const uint4*>(xq_s + m * K + 16 * i);
+        const uint4 xb = *reinterpret_cast<const uint4*>(xq_s + m * K + (K >> 1) + 16 * i);
+        const uint32_t xe[4] = {xa.x, xa.y, xa.z, xa.w}, xo[4] = {xb.x, xb.y, xb.z, xb.w};
 #pragma unroll
         for (int r = 0; r < R; ++r) {
           const uint32_t ww[4] = {wv[r].x, wv[r].y, wv[r].z, wv[r].w};
