@@ -65,3 +65,36 @@ def test_scratch_split_form_still_exact(B):
                        capture_output=True, text=True, timeout=900)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
     assert "scratch split-K parity ok" in r.stdout
+
+
+def test_random_shapes_sampled_rows(oracle_mod, B):
+    """40 seeded random (M, K, N) over the range where the launcher switches between the unsplit, cluster and scratch
+    forms: int32 sums of 12 sampled token rows per case against the oracle, and two runs bit-identical (the exchange
+    inside a cluster must not depend on which CTA finishes first)."""
+    import random
+
+    import numpy as np
+
+    from paper_2604_24273_b200 import inputs
+
+    rnd = random.Random(20240607)
+    layers, kinds = {}, set()
+    for case in range(40):
+        K = rnd.choice([640, 1024, 2560, 3840, 6912])
+        N = rnd.choice([128, 256, 384, 2560])
+        M = rnd.choice([5, 9, 17, 31, 33, 40, 63, 65, 100, 127, 129, 200, 256, 300, 511, 700, 1000])
+        if (N, K) not in layers:
+            W = inputs.master_weights(N, K, 8800 + N + K)
+            layers[(N, K)] = (oracle_mod.ternarize(W.numpy())[0], B.Linear.from_master(W.cuda()))
+        Wq, lin = layers[(N, K)]
+        x = inputs.activations(M, K, 8900 + case)
+        res = inputs.activations(M, N, 9000 + case, outliers=False).cuda()
+        xq, a, rs = B.quant_act(x.cuda())
+        y1, acc1 = B.bitlinear_forward_q(lin, xq, a, rs, B.OUT_BF16, residual=res, want_acc=True)
+        y2, acc2 = B.bitlinear_forward_q(lin, xq, a, rs, B.OUT_BF16, residual=res, want_acc=True)
+        B.poll_status()
+        assert torch.equal(acc1, acc2) and torch.equal(y1, y2), (M, K, N)
+        rows = np.unique(np.concatenate([[0, M - 1], np.random.default_rng(case).integers(0, M, 10)]))
+        assert np.array_equal(acc1.cpu().numpy()[rows], oracle_mod.contract(xq.cpu().numpy()[rows], Wq)), (M, K, N)
+        kinds.add(B.gemm_plan(M, K, N)[2])
+    assert B.GEMM_SPLIT_CLUSTER in kinds and B.GEMM_SINGLE in kinds
