@@ -459,6 +459,28 @@ def run_ours(args):
                                                       "frac_of_hbm_peak": gb8k / peaks["hbm_gbs"]}
                 del g8k
 
+    if rank == 0 and "pack" in sections:
+        # a0, the offline step: absmean scale + ternarize + pack of the block's largest matrix (fp32 master weights, 141.6 MB;
+        # three matrices in turn so that nothing is left in L2).  Algorithmic bytes: W read once, packed codes written.
+        Np, Kp = 13824, 2560
+        gen0 = torch.Generator(device="cuda")
+        gen0.manual_seed(4242)
+        Wm = [torch.randn(Np, Kp, generator=gen0, device="cuda", dtype=torch.float32) * inputs.SIGMA_W for _ in range(3)]
+        pk = torch.empty((Np, Kp // 4), dtype=torch.uint8, device=dev)
+        gm = torch.empty((1,), dtype=torch.float32, device=dev)
+
+        def pack3():
+            for W_ in Wm:
+                bitrl.pack_ternary_static(W_, pk, gm)
+
+        gp, lp = capture(pack3)
+        usp = time_graph(gp, sub_steps, args.warmup, 1) * 1e3 / (sub_steps * 3)
+        alg = Np * Kp * 4.25
+        extra["pack_ternary_13824x2560"] = {"us": usp, "GBps_algorithmic": alg / (usp * 1e-6) / 1e9,
+                                            "frac_of_hbm_peak": alg / (usp * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                                            "passes_over_W": 2, "launches": lp / 3}
+        del gp, Wm, pk, gm
+
     if rank == 0 and "pack5" in sections:
         # the same M = 1 sweep on the five-weights-per-byte format (1.6 bits per weight, lookup-table decode): judged on
         # microseconds per sweep against the 2-bit kernel's, and on GB/s of its own (smaller) packed bytes
@@ -816,7 +838,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=FULL_LAYERS, help="blocks in the backbone (30 = full model)")
-    ap.add_argument("--sections", default="decode8,pack5,gemm,critic,encoder,cpu",
+    ap.add_argument("--sections", default="decode8,pack,pack5,gemm,critic,encoder,cpu",
                     help="secondary measurements besides the M=1 headline (comma list; empty = none)")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:

@@ -36,14 +36,21 @@ __global__ void __launch_bounds__(ABSSUM_THREADS) abssum_partial_kernel(const fl
   if (threadIdx.x == 0) partial[blockIdx.x] = red[0];
 }
 
-// Stage 2: one thread adds the partials in index order and rounds S/count to fp32 once.
-__global__ void abssum_final_kernel(const double* __restrict__ partial, int nparts, long long count,
-                                    float* __restrict__ gamma) {
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
-    double s = 0.0;
-    for (int i = 0; i < nparts; ++i) s += partial[i];
-    *gamma = static_cast<float>(s / static_cast<double>(count));
+// Stage 2 (one CTA): thread t adds partials t, t + 256, ... in that order, a shared-memory tree adds the 256 sums (a
+// fixed order, so gamma is reproducible), and S/count is rounded to fp32 once.  One thread adding up to 1024 partials in a
+// row, as this kernel first did, was a chain of dependent loads and fp64 adds: 30 us, longer than either pass over W.
+__global__ void __launch_bounds__(ABSSUM_THREADS) abssum_final_kernel(const double* __restrict__ partial, int nparts,
+                                                                      long long count, float* __restrict__ gamma) {
+  __shared__ double red[ABSSUM_THREADS];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < nparts; i += ABSSUM_THREADS) s += partial[i];
+  red[threadIdx.x] = s;
+  __syncthreads();
+  for (int o = ABSSUM_THREADS / 2; o > 0; o >>= 1) {
+    if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+    __syncthreads();
   }
+  if (threadIdx.x == 0) *gamma = static_cast<float>(red[0] / static_cast<double>(count));
 }
 
 // Each thread turns 16 consecutive weights of a row into one canonical 32-bit word (4 bytes, k ascending,
@@ -109,7 +116,7 @@ bitrl_status launch_pack(const float* W, int N, int K, uint8_t* packed, float* g
   chunk = (chunk + 3) & ~3LL;
   double* partial = static_cast<double*>(ws);
   abssum_partial_kernel<<<nb, ABSSUM_THREADS, 0, st>>>(W, count, chunk, partial);
-  abssum_final_kernel<<<1, 32, 0, st>>>(partial, nb, count, gamma);
+  abssum_final_kernel<<<1, ABSSUM_THREADS, 0, st>>>(partial, nb, count, gamma);
   const long long nwords = count / 16;
   ternarize_pack_kernel<<<static_cast<unsigned>((nwords + 255) / 256), 256, 0, st>>>(
       W, nwords, gamma, reinterpret_cast<uint32_t*>(packed));
