@@ -582,3 +582,21 @@ def test_zero_and_tiny_token_rows(oracle_mod, B, M):
     B.poll_status()
     check_producer(oracle_mod, xq2, a2, rs2, u, oracle_mod.rmsnorm_bf16(inputs.bf16_bits(x)))
     assert not xq2[0].any() and rs2[0].item() == 0
+
+
+def test_packed_weight_file_round_trip_on_device(oracle_mod, B, tmp_path):
+    """Packed bytes and gamma saved to the flat file and loaded back give a layer with bit-identical outputs."""
+    from paper_2604_24273_b200 import weights_io
+
+    N, K, M = 384, 640, 40
+    W = inputs.master_weights(N, K, 9900)
+    packed, gamma = B.pack_ternary(W.cuda())
+    f = tmp_path / "layer.bitrl"
+    weights_io.save_packed(f, packed.cpu().numpy(), gamma.cpu().numpy(), N, K)
+    p2, g2, n2, k2 = weights_io.load_packed(f)
+    assert np.array_equal(p2, oracle_mod.pack(oracle_mod.ternarize(W.numpy(), gamma=g2)[0]))
+    lin_a = B.Linear(packed, gamma, N, K)
+    lin_b = B.Linear(torch.from_numpy(p2).cuda(), torch.tensor([g2], dtype=torch.float32, device="cuda"), n2, k2)
+    x = inputs.activations(M, K, 9901).cuda()
+    assert torch.equal(B.bitlinear_forward(lin_a, x), B.bitlinear_forward(lin_b, x))
+    B.poll_status()
