@@ -176,6 +176,14 @@ def capture(fn):
     return g, launches
 
 
+def gemm_kernel_name(bitrl, M, K, N):
+    """The form of the tensor-core kernel the launcher takes for this shape, as the library reports it."""
+    tok, splits, kind = bitrl.gemm_plan(M, K, N)
+    form = {bitrl.GEMM_SINGLE: "single CTAs", bitrl.GEMM_SPLIT_SCRATCH: f"split-K x{splits} through scratch",
+            bitrl.GEMM_SPLIT_CLUSTER: f"split-K x{splits} inside a cluster", bitrl.GEMM_PAIRED: "CTA pairs (cta_group::2)"}[kind]
+    return f"gemm_i8_kernel<TOK={tok}>, {form}"
+
+
 def build_backbone(bitrl, n_layers, seed=5000):
     """Blocks of ternary weights.  Master weights are drawn on the GPU (N(0, 0.02), seeded per matrix) to keep
     set-up short, packed by the library and dropped; only the packed handles stay (17.4 MB per block)."""
@@ -546,7 +554,7 @@ def run_ours(args):
             gemm_roofline.append({
                 "shape": f"M=4096 K={K} N={N}", "bound": "tensor", "unit": "TOPS", "peak": i8_peak,
                 "peak_source": f"2 x bf16 burst, of {peak_src}",
-                "kernel": "gemm_i8_kernel<224,true,true>" if N == 6912 else "gemm_i8_kernel<192,true,true>",
+                "kernel": gemm_kernel_name(bitrl, M, K, N),
                 "us": res["gemm_kernel"]["us"], "achieved": res["gemm_kernel"]["TOPS"],
                 "frac": res["gemm_kernel"]["frac_of_int8_peak"], "frac_of_nominal_4500": res["gemm_kernel"]["frac_of_nominal_4500"],
                 "layer_us": res["layer"]["us"], "layer_achieved": res["layer"]["TOPS"],
@@ -670,6 +678,7 @@ def run_ours(args):
                 ms = time_graph(g, sub_steps, args.warmup, 1)
                 us = ms * 1e3 / (sub_steps * reps)
                 extra[f"layer_m{M}_k{K}_n{N}"] = {"us": us, "TOPS": 2.0 * M * N * K / (us * 1e-6) / 1e12,
+                                                  "kernel": gemm_kernel_name(bitrl, M, K, N),
                                                   "packed_GBps": N * K / 4 / (us * 1e-6) / 1e9,
                                                   "launches_per_layer": lc / reps}
                 del g, xs, y, ws
